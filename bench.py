@@ -1,0 +1,359 @@
+#!/usr/bin/env python
+"""Benchmark of the LCA prefill hot path (condense + condensed attention) on B200.
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--config mla_128k] [--impl ours|reference]
+
+One "step" = one pass of the whole hot path over one synthetic sequence of the chosen
+configuration: lca_condense (summary query, group scores, softmax, pooling, anchors, local
+window) followed by lca_prefill_attention.  Inputs are resident in HBM for `value`; the `e2e`
+figure repeats the step from pinned host buffers with the host<->device copies inside the timed
+region.  With N > 1 every rank runs an independent replica (the path has no exchange step):
+value = N * tokens / max-over-ranks time.
+
+--impl reference times the CPU oracle (fp64, OpenMP) on a bounded sample of the same workload.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import subprocess
+import sys
+import threading
+import time
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+import numpy as np
+import torch
+
+from paper_2604_12452_b200 import inputs as I
+
+METRIC = "lca_prefill_tokens_per_s"
+UNIT = "tokens/s"
+
+
+# ---------------------------------------------------------------------------- work counts
+def key_visits(L: int, g: int, w: int) -> int:
+    """sum over query positions of (representatives + local tokens) it attends to."""
+    t = np.arange(1, L + 1, dtype=np.int64)
+    mt = np.where(t < w + g, 0, (t - w) // g)
+    return int((mt + (t - mt * g)).sum())
+
+
+def attention_flops(cfg) -> float:
+    dk = cfg.d_sem + cfg.d_pos if cfg.variant == "mla" else cfg.d_sem
+    return float(key_visits(cfg.seq_len, cfg.group_size, cfg.window)) * cfg.n_q_heads * 2.0 * (dk + cfg.d_sem) * cfg.batch
+
+
+def condense_bytes(cfg) -> float:
+    """Algorithmic HBM bytes of lca_condense: history rows read once, query tail read once,
+    representatives + anchors written, local window read and written."""
+    L, g, w = cfg.seq_len, cfg.group_size, cfg.window
+    m = 0 if L < w + g else (L - w) // g
+    k = L - m * g
+    d_pos = cfg.d_pos if cfg.variant == "mla" else cfg.d_sem
+    row = (cfg.d_sem + d_pos) * 2 * cfg.n_kv_heads
+    qrow = ((cfg.d_sem + cfg.d_pos) if cfg.variant == "mla" else cfg.d_sem) * 2 * cfg.n_q_heads
+    return float(cfg.batch) * (m * g * row + min(g, L) * qrow + m * row + 4 * m * cfg.n_kv_heads + 2 * k * row)
+
+
+def measured_peaks():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(path):
+        with open(path) as f:
+            d = json.load(f)
+        return dict(hbm_gbs=d["hbm_gbs"], tflops_burst=d["bf16_tflops"], tflops_sustained=d["bf16_tflops_sustained"],
+                    source="measured")
+    return dict(hbm_gbs=6650.0, tflops_burst=1590.0, tflops_sustained=1400.0, source="fallback")
+
+
+# ---------------------------------------------------------------------------------- clocks
+class ClockSampler:
+    """Samples nvidia-smi clocks / throttle reasons of one GPU while the timed region runs."""
+    FIELDS = ("clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.hw_slowdown,"
+              "clocks_event_reasons.hw_thermal_slowdown,clocks_event_reasons.sw_thermal_slowdown,"
+              "clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, index: int):
+        self.index = index
+        self.proc = None
+        self.lines = []
+
+    def start(self):
+        try:
+            self.proc = subprocess.Popen(
+                ["nvidia-smi", "-i", str(self.index), f"--query-gpu={self.FIELDS}", "--format=csv,noheader,nounits",
+                 "-lms", "200"], stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
+            self.thread = threading.Thread(target=self._read, daemon=True)
+            self.thread.start()
+        except Exception:
+            self.proc = None
+
+    def _read(self):
+        for ln in self.proc.stdout:
+            self.lines.append(ln.strip())
+
+    def stop(self):
+        if self.proc is None:
+            return dict(sm_mhz=None, sm_max_mhz=None, reasons=["nvidia-smi unavailable"])
+        self.proc.terminate()
+        try:
+            self.proc.wait(timeout=5)
+        except Exception:
+            self.proc.kill()
+        sm, mx, reasons = [], [], set()
+        names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
+        for ln in self.lines:
+            parts = [x.strip() for x in ln.split(",")]
+            if len(parts) < 7:
+                continue
+            try:
+                sm.append(float(parts[0]))
+                mx.append(float(parts[1]))
+            except ValueError:
+                continue
+            for nm, val in zip(names, parts[3:7]):
+                if val.lower().startswith("active"):
+                    reasons.add(nm)
+        return dict(sm_mhz=float(np.median(sm)) if sm else None, sm_max_mhz=max(mx) if mx else None,
+                    reasons=sorted(reasons), samples=len(sm))
+
+
+# ----------------------------------------------------------------------------- CPU oracle
+def oracle_sample(cfg, inp_cpu_small, n_rows: int, n_heads: int, seed: int = 0):
+    """Time the oracle on a bounded sample: condensation of the whole sequence plus `n_rows`
+    stratified query rows x `n_heads` heads.  Returns (tokens_per_s_estimate, description, threads)."""
+    from oracle import lca_oracle as O
+    from tests import helpers as Hh
+    L, g, w, H = cfg.seq_len, cfg.group_size, cfg.window, cfg.n_q_heads
+    rows = Hh.sample_positions(L, g, w, n_uniform=max(0, n_rows - 18), seed=seed)[:max(n_rows, 1)]
+    heads = np.arange(min(n_heads, H))
+    t0 = time.perf_counter()
+    ref = Hh.oracle_mla(inp_cpu_small, g, w, cfg.softmax_scale, rows=None)
+    t_cond = time.perf_counter() - t0
+    cond = ref["cond"]
+    m = cond["m"]
+    ckv = O.torch_bf16_to_f64(inp_cpu_small["ckv"])
+    kr = O.torch_bf16_to_f64(inp_cpu_small["kr"])
+    rep_sem = O.bits_to_f64(cond["cache_sem_bits"][:m])
+    rep_pos = O.bits_to_f64(cond["cache_pos_bits"][:m])
+    qs = O.torch_bf16_to_f64(inp_cpu_small["q_sem_rows"][:len(rows)][:, heads])
+    qp = O.torch_bf16_to_f64(inp_cpu_small["q_pos_rows"][:len(rows)][:, heads])
+    t0 = time.perf_counter()
+    O.mla_prefill_rows(qs, qp, rows, ckv, kr, rep_sem if m else None, rep_pos if m else None, g, w,
+                       float(np.float32(cfg.softmax_scale)))
+    t_rows = time.perf_counter() - t0
+    mt = np.where(rows + 1 < w + g, 0, (rows + 1 - w) // g)
+    sampled_visits = float((mt + (rows + 1 - mt * g)).sum()) * len(heads)
+    total_visits = float(key_visits(L, g, w)) * H
+    est_total = t_cond + t_rows * total_visits / max(sampled_visits, 1.0)
+    desc = (f"condense of all {L} tokens ({t_cond:.2f}s) + {len(rows)} stratified query rows x {len(heads)} heads "
+            f"({t_rows:.2f}s), scaled by visited (query,key,head) triples {sampled_visits:.3g}/{total_visits:.3g}")
+    return L * cfg.batch / est_total, desc, O.num_threads(), dict(rows=rows, heads=heads)
+
+
+def gather_oracle_inputs(cfg, inp, n_rows, seed=0):
+    """CPU copies of what the oracle sample needs (the K/V streams and the sampled query rows)."""
+    from tests import helpers as Hh
+    L, g, w = cfg.seq_len, cfg.group_size, cfg.window
+    rows = Hh.sample_positions(L, g, w, n_uniform=max(0, n_rows - 18), seed=seed)[:max(n_rows, 1)]
+    idx = torch.from_numpy(rows).to(inp["q_sem"].device)
+    return dict(ckv=inp["ckv"].cpu(), kr=inp["kr"].cpu(), q_sem=inp["q_sem"][L - g:].cpu(), q_pos=inp["q_pos"][L - g:].cpu(),
+                q_sem_rows=inp["q_sem"][idx].cpu(), q_pos_rows=inp["q_pos"][idx].cpu())
+
+
+# -------------------------------------------------------------------------------- main arms
+def run_reference(args, cfg, rank, world):
+    if rank != 0:
+        return
+    dev = "cuda:0" if torch.cuda.is_available() else "cpu"
+    inp = I.make_mla_inputs(cfg, dev) if cfg.seq_len * cfg.n_q_heads * 576 * 2 < 8e9 or dev != "cpu" else None
+    small = gather_oracle_inputs(cfg, inp, args.ref_rows)
+    del inp
+    times, vals = [], []
+    desc, threads = "", 1
+    for it in range(args.warmup + args.steps):
+        t0 = time.perf_counter()
+        v, desc, threads, _ = oracle_sample(cfg, small, args.ref_rows, args.ref_heads)
+        if it >= args.warmup:
+            times.append(time.perf_counter() - t0)
+            vals.append(v)
+    value = float(np.mean(vals))
+    line = dict(impl="reference", metric=METRIC, value=value, unit=UNIT, n_gpus=args.gpus, steps=args.steps,
+                warmup=args.warmup, ms_per_step=1e3 * cfg.seq_len * cfg.batch / value, higher_is_better=True,
+                scaling="weak", vs_baseline=None, dtype="f64", data="synthetic",
+                config=workload_config(cfg, args.gpus),
+                cpu_baseline=dict(value=value, unit=UNIT, cores=threads, kind="oracle", sample=desc),
+                e2e=dict(value=value, unit=UNIT, h2d_bytes_per_step=0, d2h_bytes_per_step=0),
+                sample_wall_s=float(np.mean(times)))
+    print(json.dumps(line))
+
+
+def workload_config(cfg, n_gpus):
+    return dict(workload=f"{cfg.name}: one {cfg.variant.upper()} layer, batch {cfg.batch}, L={cfg.seq_len}, "
+                         f"H={cfg.n_q_heads}, d_sem={cfg.d_sem}, d_pos={cfg.d_pos}, g={cfg.group_size}, w={cfg.window}, causal",
+                seq_len=cfg.seq_len, n_q_heads=cfg.n_q_heads, group_size=cfg.group_size, window=cfg.window,
+                parallelism=f"replicas x{n_gpus}" if n_gpus > 1 else "single GPU",
+                l2_policy="inputs (>= 19 GB of queries per step) exceed the 126 MB L2; no flush needed")
+
+
+def run_ours(args, cfg, rank, world, local_rank):
+    from paper_2604_12452_b200 import build
+    build.build()
+    from paper_2604_12452_b200 import binding as B
+    torch.cuda.set_device(local_rank)
+    dev = f"cuda:{local_rank}"
+    dist = None
+    if world > 1:
+        import torch.distributed as dist_mod
+        dist = dist_mod
+        dist.init_process_group("nccl", device_id=torch.device(dev))
+
+    def barrier():
+        if dist is not None:
+            dist.barrier()
+        torch.cuda.synchronize()
+
+    L, g = cfg.seq_len, cfg.group_size
+    inp = I.make_mla_inputs(cfg, dev)
+    p = B.params_from_config(cfg, batch=1)
+    m, k = B.lca_partition(p)
+    out = torch.empty((1, L, cfg.n_q_heads, cfg.d_sem), dtype=torch.bfloat16, device=dev)
+    cache = dict(cache_sem=torch.empty((1, m + k, 1, cfg.d_sem), dtype=torch.bfloat16, device=dev),
+                 cache_pos=torch.empty((1, m + k, 1, cfg.d_pos), dtype=torch.bfloat16, device=dev),
+                 anchor_idx=torch.empty((1, max(m, 1), 1), dtype=torch.int32, device=dev))
+    ws_c = B.workspace(p, B.LCA_WS_CONDENSE, dev)
+    ws_a = B.workspace(p, B.LCA_WS_PREFILL, dev)
+    q_tail_sem, q_tail_pos = inp["q_sem"][L - g:], inp["q_pos"][L - g:]
+
+    def step(ev=None):
+        if ev:
+            ev[0].record()
+        B.condense(p, q_tail_sem, q_tail_pos, inp["ckv"], inp["kr"], out=cache, ws=ws_c)
+        if ev:
+            ev[1].record()
+        B.prefill_attention(p, inp["q_sem"], inp["q_pos"], inp["ckv"], inp["kr"], cache["cache_sem"],
+                            cache["cache_pos"], out=out, ws=ws_a)
+        if ev:
+            ev[2].record()
+
+    for _ in range(args.warmup):
+        step()
+    barrier()
+    sampler = ClockSampler(local_rank)
+    sampler.start()
+    evs = [[torch.cuda.Event(enable_timing=True) for _ in range(3)] for _ in range(args.steps)]
+    launches0 = B.lca_launch_count()
+    barrier()
+    for i in range(args.steps):
+        step(evs[i])
+    barrier()
+    launches = B.lca_launch_count() - launches0
+    clocks = sampler.stop()
+    total_ms = evs[0][0].elapsed_time(evs[-1][2])
+    t_cond = float(np.mean([e[0].elapsed_time(e[1]) for e in evs]))
+    t_attn = float(np.mean([e[1].elapsed_time(e[2]) for e in evs]))
+    status = B.lca_last_device_status()
+    if status != 0:
+        raise RuntimeError(f"device status {status}: {B.lca_status_string(status)}")
+    tmax = torch.tensor([total_ms], device=dev, dtype=torch.float64)
+    if dist is not None:
+        dist.all_reduce(tmax, op=dist.ReduceOp.MAX)
+    total_ms = float(tmax.item())
+    ms_per_step = total_ms / args.steps
+    value = world * L * cfg.batch / (ms_per_step * 1e-3)
+
+    # ---- end to end: pinned host buffers, H2D of the step's inputs and D2H of its output inside the timing
+    e2e = None
+    if not args.no_e2e:
+        try:
+            host = {kname: torch.empty(v.shape, dtype=v.dtype, pin_memory=True).copy_(v) for kname, v in inp.items()}
+            host_out = torch.empty(out.shape, dtype=out.dtype, pin_memory=True)
+            n_e2e = max(1, min(args.steps, args.e2e_steps))
+            h2d = sum(v.numel() * v.element_size() for v in host.values())
+            d2h = host_out.numel() * host_out.element_size()
+            barrier()
+            e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            e0.record()
+            for _ in range(n_e2e):
+                for kname in inp:
+                    inp[kname].copy_(host[kname], non_blocking=True)
+                step()
+                host_out.copy_(out, non_blocking=True)
+            e1.record()
+            barrier()
+            t = torch.tensor([e0.elapsed_time(e1) / n_e2e], device=dev, dtype=torch.float64)
+            if dist is not None:
+                dist.all_reduce(t, op=dist.ReduceOp.MAX)
+            e2e = dict(value=world * L * cfg.batch / (float(t.item()) * 1e-3), unit=UNIT, h2d_bytes_per_step=h2d,
+                       d2h_bytes_per_step=d2h, steps=n_e2e, ms_per_step=float(t.item()))
+            del host, host_out
+        except RuntimeError as ex:      # e.g. not enough pinnable host memory on this machine
+            e2e = dict(value=None, unit=UNIT, h2d_bytes_per_step=0, d2h_bytes_per_step=0, error=str(ex)[:200])
+
+    if rank != 0:
+        if dist is not None:
+            dist.destroy_process_group()
+        return
+    peaks = measured_peaks()
+    flops = attention_flops(cfg)
+    tfl = flops / (t_attn * 1e-3) / 1e12
+    cbytes = condense_bytes(cfg)
+    cgbs = cbytes / (t_cond * 1e-3) / 1e9
+    line = dict(metric=METRIC, value=value, unit=UNIT, n_gpus=world, steps=args.steps, warmup=args.warmup,
+                ms_per_step=ms_per_step, higher_is_better=True, scaling="weak", vs_baseline=None, dtype="bf16",
+                data="synthetic", config=workload_config(cfg, world), clocks=clocks, gpu_launches=int(launches),
+                e2e=e2e,
+                roofline=dict(bound="tensor", achieved=tfl, peak=peaks["tflops_sustained"], unit="TFLOP/s",
+                              frac=tfl / peaks["tflops_sustained"], traffic=None,
+                              kernel="lca_prefill_attention", flops_per_launch=flops, ms_per_launch=t_attn,
+                              peak_kind=f"{peaks['source']} cuBLAS bf16, sustained (kernel timed inside a long step)",
+                              frac_of_burst=tfl / peaks["tflops_burst"], frac_of_nominal_2250=tfl / 2250.0),
+                roofline_condense=dict(bound="hbm", achieved=cgbs, peak=peaks["hbm_gbs"], unit="GB/s",
+                                       frac=cgbs / peaks["hbm_gbs"], traffic=None, kernel="lca_condense (all launches)",
+                                       bytes_per_launch=cbytes, ms_per_launch=t_cond, peak_kind=f"{peaks['source']} copy"),
+                attention_impl=args.attn_impl)
+    if not args.no_cpu_baseline:
+        small = gather_oracle_inputs(cfg, inp, args.ref_rows)
+        v, desc, threads, _ = oracle_sample(cfg, small, args.ref_rows, args.ref_heads)
+        line["cpu_baseline"] = dict(value=v, unit=UNIT, cores=threads, kind="oracle", sample=desc)
+    print(json.dumps(line))
+    if dist is not None:
+        dist.destroy_process_group()
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=5)
+    ap.add_argument("--warmup", type=int, default=3)
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--config", default="mla_128k", choices=[k for k, c in I.CONFIGS.items() if c.variant == "mla" and c.batch == 1])
+    ap.add_argument("--attn-impl", type=int, default=0, help="0 auto, 1 scalar kernel, 2 tensor-core kernel")
+    ap.add_argument("--e2e-steps", type=int, default=2)
+    ap.add_argument("--no-e2e", action="store_true")
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--ref-rows", type=int, default=24, help="query rows in the oracle's bounded sample")
+    ap.add_argument("--ref-heads", type=int, default=16, help="heads per sampled row in the oracle's sample")
+    args = ap.parse_args()
+    rank = int(os.environ.get("RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    local_rank = int(os.environ.get("LOCAL_RANK", "0"))
+    cfg = I.CONFIGS[args.config]
+    if args.impl == "reference":
+        run_reference(args, cfg, rank, world)
+        return
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device: the product path has no CPU fallback")
+    from paper_2604_12452_b200 import build
+    build.build()
+    from paper_2604_12452_b200 import binding as B
+    B.lca_set_attention_impl(args.attn_impl)
+    run_ours(args, cfg, rank, world, local_rank)
+
+
+if __name__ == "__main__":
+    main()

@@ -1,0 +1,154 @@
+/* Latent-Condensed Attention (LCA) for NVIDIA B200 (sm_100a) -- C ABI.
+ *
+ * The library computes the prefill / decode hot path of LCA: condensation of the distant
+ * history in MLA's latent space (query-aware weighted pooling of C^KV, arg-max anchor selection
+ * of K^R) followed by attention of the absorbed-form queries [q_latent | q_rope] over the
+ * condensed representatives plus the uncondensed local window, and the same dual path for
+ * grouped-query attention (pool V, select K).  Section / equation numbers below refer to the
+ * paper "Latent-Condensed Transformer for Efficient Long Context Modeling".
+ *
+ * Conventions that hold for every entry point
+ *   - All tensor pointers are DEVICE pointers owned by the caller, 16-byte aligned, dense
+ *     row-major with the shapes stated; element type bf16 unless stated.  `lca_params*` is a
+ *     HOST pointer.  `stream` is a cudaStream_t passed as void* (NULL = the legacy default stream).
+ *   - Calls are asynchronous on `stream`; nothing is allocated, freed or kept between calls
+ *     unless an entry point says otherwise; the workspace `ws` may be reused by the next call
+ *     on the same stream.
+ *   - Return value: LCA_OK (0) or a negative lca_status.  Arguments are validated on the host
+ *     first; an invalid call launches nothing and writes nothing.
+ *   - Token positions are 0-based in the ABI (the paper's formulas are 1-based).
+ *
+ * Partition of a length-L sequence (Sec. 4.2): m = floor((L-w)/g) groups of g tokens,
+ * G_j = {j*g .. (j+1)*g-1}; the last k = L - m*g = w + (L-w) mod g tokens form the local window.
+ * When L < w+g there is no group: m = 0, k = L and every entry point degenerates to plain
+ * causal attention (Sec. 4.3).  `lca_partition` returns (m, k).
+ *
+ * Condensed-cache layout (Sec. 4.3 "Decoding and Online Cache Update"), per sequence:
+ *   rows 0..m-1   representatives in group order: cache_sem[j] = c_rep_j (Eq. 7, rounded to
+ *                 nearest-even bf16), cache_pos[j] = k^R of the anchor token I_j (Eq. 8, bit copy)
+ *   rows m..m+k-1 the last k tokens in token order (bit copies)
+ * GQA (Sec. 5.4): the same per KV head with cache_sem = pooled V, cache_pos = selected K.
+ */
+#ifndef LCA_H_
+#define LCA_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef enum lca_status {
+  LCA_OK = 0,
+  LCA_ERR_INVALID_ARG = -1,        /* NULL where a pointer is required, non-positive size, ...   */
+  LCA_ERR_UNSUPPORTED_SHAPE = -2,  /* a head dimension / group size no kernel is built for       */
+  LCA_ERR_MISALIGNED = -3,         /* a tensor pointer that is not 16-byte aligned               */
+  LCA_ERR_WORKSPACE_TOO_SMALL = -4,
+  LCA_ERR_CUDA = -5,               /* a CUDA runtime call or a launch failed                     */
+  LCA_ERR_DEVICE_TIMEOUT = -6      /* a bounded device-side wait expired (reported by lca_last_device_status) */
+} lca_status;
+
+enum { LCA_VARIANT_MLA = 0, LCA_VARIANT_GQA = 1 };
+enum { LCA_WS_CONDENSE = 0, LCA_WS_PREFILL = 1, LCA_WS_DECODE = 2 };
+
+/* Problem statement = the REQUIRE line of Alg. 1 (L, C^KV, K^R, Q, w, g) plus the head layout.
+ *   MLA: n_kv_heads = 1, d_sem = d_c (512), d_pos = d_R (64); logits use [sem | pos], values = sem.
+ *   GQA: d_sem = d_pos = head_dim (128); logits use pos (= K) only, values = sem (= V);
+ *        n_q_heads must be a multiple of n_kv_heads.
+ *   n_summary_q: number of trailing queries averaged into the summary query (Alg. 1 line 1;
+ *                Table 8 varies it); 0 means g; clamped to L.
+ *   softmax_scale: 1/sqrt(d_h), used for the importance scores (Sec. 4.2) and the attention (Eq. 10).
+ *   rep_logit_bias: added to the logit of every representative; 0 = Alg. 1 as printed,
+ *                log(g) = the group-size-weighted form analysed in the proof of Theorem 1. */
+typedef struct lca_params {
+  int32_t variant;
+  int32_t batch;
+  int32_t seq_len;
+  int32_t n_q_heads;
+  int32_t n_kv_heads;
+  int32_t d_sem;
+  int32_t d_pos;
+  int32_t group_size;
+  int32_t window;
+  int32_t n_summary_q;
+  float softmax_scale;
+  float rep_logit_bias;
+} lca_params;
+
+/* (m, k) of Sec. 4.2 for one sequence of p->seq_len tokens.  Host only, no device work. */
+int lca_partition(const lca_params* p, int32_t* m, int32_t* k);
+
+/* Bytes of device workspace `which` (LCA_WS_*) needs for these parameters (0 is possible).
+ * Returns 0 for invalid parameters as well; the entry point then reports the error. */
+size_t lca_workspace_bytes(const lca_params* p, int32_t which);
+
+/* Condensation: Alg. 1 lines 1-10 (summary query, Eq. 6 group softmax, Eq. 7 pooling, Eq. 8
+ * anchors, Eq. 9 local window) for `batch` sequences.
+ *   q_tail_sem [B, n, H, d_sem], q_tail_pos [B, n, H, d_pos]: the LAST n = n_summary_q query
+ *       positions of each sequence (MLA: q_latent and q_rope; GQA: q_tail_sem = NULL and
+ *       q_tail_pos = Q).  q_tail_batch_stride = rows (positions) between consecutive sequences
+ *       in these arrays (n for a packed tail, L when pointing into a full [B,L,H,d] tensor).
+ *       Ignored (may be NULL) when qbar_opt is given.
+ *   qbar_opt   [B, n_kv_heads, dk] fp32, dk = d_sem+d_pos (MLA) or d_pos (GQA), or NULL: a
+ *       caller-supplied summary query (e.g. the streaming update of Sec. 4.3).
+ *   kv_sem [B, L, n_kv_heads, d_sem], kv_pos [B, L, n_kv_heads, d_pos]: C^KV, K^R (GQA: V, K).
+ *   cache_sem [B, m+k, n_kv_heads, d_sem], cache_pos [B, m+k, n_kv_heads, d_pos]: out, layout above.
+ *   anchor_idx [B, m, n_kv_heads] int32 out: absolute token index of I_j (lowest index on ties).
+ *   scores_opt [B, n_kv_heads, m*g] fp64 out or NULL: the importance scores s_i the kernel used.
+ *   ws / ws_bytes: >= lca_workspace_bytes(p, LCA_WS_CONDENSE).
+ * Scores, the group softmax and the pooling are evaluated in fp64 (the kernel is HBM-bound),
+ * so anchors follow the fp64 scores and c_rep is rounded once, to bf16. */
+int lca_condense(const lca_params* p, const void* q_tail_sem, const void* q_tail_pos,
+                 int64_t q_tail_batch_stride, const float* qbar_opt, const void* kv_sem,
+                 const void* kv_pos, void* cache_sem, void* cache_pos, int32_t* anchor_idx,
+                 double* scores_opt, void* ws, size_t ws_bytes, void* stream);
+
+/* Prefill attention, Eq. 10 evaluated at every prefix length (causal): the query at position t
+ * attends to the representatives of the m_t = floor((t+1-w)/g) groups that lie wholly outside its
+ * window (0 if t+1 < w+g; read from rows 0..m_t-1 of the cache) and to the tokens m_t*g..t
+ * (read from kv_sem / kv_pos).  window >= seq_len gives dense causal attention (Eq. 5).
+ *   q_sem [B, L, H, d_sem] (MLA; NULL for GQA), q_pos [B, L, H, d_pos]
+ *   kv_sem, kv_pos, cache_sem, cache_pos: as for lca_condense (the cache may be NULL when m = 0)
+ *   out [B, L, H, d_sem] bf16: softmax-weighted sum of the sem vectors (latent space for MLA)
+ *   lse_opt [B, L, H] fp32 or NULL: natural-log sum-exp of the logits of each row
+ * fp32 softmax and accumulation, bf16 tensor-core products. */
+int lca_prefill_attention(const lca_params* p, const void* q_sem, const void* q_pos,
+                          const void* kv_sem, const void* kv_pos, const void* cache_sem,
+                          const void* cache_pos, void* out, float* lse_opt, void* ws,
+                          size_t ws_bytes, void* stream);
+
+/* Decode attention (Sec. 4.3): one new query per sequence attends to every valid row of that
+ * sequence's condensed cache (the caller has appended the new token's own row).
+ *   q_sem [B, H, d_sem] (NULL for GQA), q_pos [B, H, d_pos]
+ *   cache_sem [B, cache_row_capacity, n_kv_heads, d_sem], cache_pos likewise with d_pos
+ *   cache_rows [B] int32 (device): valid rows of each sequence, clamped to [0, cache_row_capacity]
+ *   n_rep: leading rows that are representatives (they receive rep_logit_bias)
+ *   out [B, H, d_sem] bf16, lse_opt [B, H] fp32 or NULL
+ * p->seq_len, group_size and window are not used here. */
+int lca_decode_attention(const lca_params* p, const void* q_sem, const void* q_pos,
+                         const void* cache_sem, const void* cache_pos, const int32_t* cache_rows,
+                         int32_t cache_row_capacity, int32_t n_rep, void* out, float* lse_opt,
+                         void* ws, size_t ws_bytes, void* stream);
+
+/* Which attention implementation lca_prefill_attention / lca_decode_attention use:
+ *   0 = automatic (tensor-core kernels where the shape is supported, else the scalar kernel),
+ *   1 = force the scalar (CUDA-core) kernel, 2 = force the tensor-core kernel (unsupported
+ *   shapes then return LCA_ERR_UNSUPPORTED_SHAPE).  Process-wide; returns the previous value. */
+int lca_set_attention_impl(int impl);
+
+/* Number of kernels the library has launched since it was loaded (all entry points). */
+int64_t lca_launch_count(void);
+
+/* Status word written by bounded device-side waits of the most recent tensor-core launch on the
+ * current device: 0 = none expired.  Synchronises `stream`.  Returns LCA_OK or
+ * LCA_ERR_DEVICE_TIMEOUT / LCA_ERR_CUDA. */
+int lca_last_device_status(void* stream);
+
+const char* lca_status_string(int status);
+int lca_version(void);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* LCA_H_ */

@@ -1,0 +1,180 @@
+// C-ABI entry points of the LCA library: host-side validation and dispatch to the kernels.
+#include <atomic>
+
+#include "lca_common.cuh"
+
+namespace lca {
+static std::atomic<long long> g_launches{0};
+static std::atomic<int> g_attn_impl{0};
+void note_launch(int n) { g_launches.fetch_add(n); }
+
+static bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
+
+static int check_params(const lca_params* p, bool need_partition) {
+  if (!p) return LCA_ERR_INVALID_ARG;
+  if (p->variant != LCA_VARIANT_MLA && p->variant != LCA_VARIANT_GQA) return LCA_ERR_INVALID_ARG;
+  if (p->batch <= 0 || p->n_q_heads <= 0 || p->n_kv_heads <= 0 || p->d_sem <= 0 || p->d_pos <= 0)
+    return LCA_ERR_INVALID_ARG;
+  if (p->n_q_heads % p->n_kv_heads != 0) return LCA_ERR_INVALID_ARG;
+  if (p->variant == LCA_VARIANT_MLA && p->n_kv_heads != 1) return LCA_ERR_INVALID_ARG;
+  if (!(p->softmax_scale > 0.f) || !(p->rep_logit_bias == p->rep_logit_bias)) return LCA_ERR_INVALID_ARG;
+  if (need_partition) {
+    if (p->seq_len <= 0 || p->group_size <= 0 || p->window < 0 || p->n_summary_q < 0)
+      return LCA_ERR_INVALID_ARG;
+  }
+  // feature dimensions must be whole 16-byte rows for the vectorised paths
+  if (p->d_sem % 8 != 0 || p->d_pos % 8 != 0) return LCA_ERR_UNSUPPORTED_SHAPE;
+  return LCA_OK;
+}
+
+static bool simt_shape_ok(const lca_params* p) {
+  if (p->variant == LCA_VARIANT_MLA) return (p->d_sem == 512 || p->d_sem == 128) && p->d_pos == 64;
+  return (p->d_sem == 128 && p->d_pos == 128) || (p->d_sem == 64 && p->d_pos == 64);
+}
+
+static int run_attention(const AttnProblem& a) {
+  const int impl = g_attn_impl.load();
+  if (impl != 1 && attn_tc_supported(a)) {
+    if (a.ws_bytes < attn_tc_workspace_bytes(a)) return LCA_ERR_WORKSPACE_TOO_SMALL;
+    if (attn_tc_workspace_bytes(a) > 0 && (!a.ws || !aligned16(a.ws))) return LCA_ERR_INVALID_ARG;
+    return attn_tc_launch(a);
+  }
+  if (impl == 2) return LCA_ERR_UNSUPPORTED_SHAPE;
+  return attn_simt_launch(a);
+}
+}  // namespace lca
+
+using namespace lca;
+
+extern "C" {
+
+int lca_version(void) { return 100; }
+
+const char* lca_status_string(int s) {
+  switch (s) {
+    case LCA_OK: return "ok";
+    case LCA_ERR_INVALID_ARG: return "invalid argument";
+    case LCA_ERR_UNSUPPORTED_SHAPE: return "unsupported shape";
+    case LCA_ERR_MISALIGNED: return "pointer not 16-byte aligned";
+    case LCA_ERR_WORKSPACE_TOO_SMALL: return "workspace too small";
+    case LCA_ERR_CUDA: return "CUDA error";
+    case LCA_ERR_DEVICE_TIMEOUT: return "device-side wait timed out";
+    default: return "unknown status";
+  }
+}
+
+int64_t lca_launch_count(void) { return (int64_t)g_launches.load(); }
+
+int lca_set_attention_impl(int impl) {
+  if (impl < 0 || impl > 2) return g_attn_impl.load();
+  return g_attn_impl.exchange(impl);
+}
+
+int lca_partition(const lca_params* p, int32_t* m, int32_t* k) {
+  int st = check_params(p, true);
+  if (st != LCA_OK) return st;
+  if (!m || !k) return LCA_ERR_INVALID_ARG;
+  int64_t mm, kk;
+  partition(p->seq_len, p->window, p->group_size, &mm, &kk);
+  *m = (int32_t)mm; *k = (int32_t)kk;
+  return LCA_OK;
+}
+
+size_t lca_workspace_bytes(const lca_params* p, int32_t which) {
+  if (check_params(p, which != LCA_WS_DECODE) != LCA_OK) return 0;
+  if (which == LCA_WS_CONDENSE) return condense_workspace_bytes(p);
+  if (which == LCA_WS_PREFILL || which == LCA_WS_DECODE) {
+    AttnProblem a = {};
+    a.variant = p->variant; a.batch = p->batch; a.q_len = which == LCA_WS_DECODE ? 1 : p->seq_len;
+    a.n_q_heads = p->n_q_heads; a.n_kv_heads = p->n_kv_heads; a.d_sem = p->d_sem; a.d_pos = p->d_pos;
+    a.decode = which == LCA_WS_DECODE; a.seq_len = p->seq_len; a.group_size = p->group_size; a.window = p->window;
+    return attn_tc_supported(a) ? attn_tc_workspace_bytes(a) : 0;
+  }
+  return 0;
+}
+
+int lca_condense(const lca_params* p, const void* q_tail_sem, const void* q_tail_pos,
+                 int64_t q_tail_batch_stride, const float* qbar_opt, const void* kv_sem,
+                 const void* kv_pos, void* cache_sem, void* cache_pos, int32_t* anchor_idx,
+                 double* scores_opt, void* ws, size_t ws_bytes, void* stream) {
+  int st = check_params(p, true);
+  if (st != LCA_OK) return st;
+  int64_t m, k;
+  partition(p->seq_len, p->window, p->group_size, &m, &k);
+  if (!kv_sem || !kv_pos || !cache_sem || !cache_pos) return LCA_ERR_INVALID_ARG;
+  if (m > 0) {
+    if (!anchor_idx) return LCA_ERR_INVALID_ARG;
+    if (!qbar_opt) {
+      if (!q_tail_pos || (p->variant == LCA_VARIANT_MLA && !q_tail_sem)) return LCA_ERR_INVALID_ARG;
+      int n = p->n_summary_q > 0 ? p->n_summary_q : p->group_size;
+      if (n > p->seq_len) n = p->seq_len;
+      if (q_tail_batch_stride < n) return LCA_ERR_INVALID_ARG;
+      if (!aligned16(q_tail_pos) || (q_tail_sem && !aligned16(q_tail_sem))) return LCA_ERR_MISALIGNED;
+    }
+    if (!ws || !aligned16(ws)) return LCA_ERR_INVALID_ARG;
+    if (ws_bytes < condense_workspace_bytes(p)) return LCA_ERR_WORKSPACE_TOO_SMALL;
+    if (condense_smem_bytes(p) > 227u * 1024u) return LCA_ERR_UNSUPPORTED_SHAPE;
+  }
+  if (!aligned16(kv_sem) || !aligned16(kv_pos) || !aligned16(cache_sem) || !aligned16(cache_pos))
+    return LCA_ERR_MISALIGNED;
+  CondenseLaunch c = {p, q_tail_sem, q_tail_pos, q_tail_batch_stride, qbar_opt, kv_sem, kv_pos,
+                      cache_sem, cache_pos, anchor_idx, scores_opt, ws, ws_bytes, (cudaStream_t)stream};
+  return condense_launch(c);
+}
+
+int lca_prefill_attention(const lca_params* p, const void* q_sem, const void* q_pos,
+                          const void* kv_sem, const void* kv_pos, const void* cache_sem,
+                          const void* cache_pos, void* out, float* lse_opt, void* ws,
+                          size_t ws_bytes, void* stream) {
+  int st = check_params(p, true);
+  if (st != LCA_OK) return st;
+  int64_t m, k;
+  partition(p->seq_len, p->window, p->group_size, &m, &k);
+  if (!q_pos || !kv_sem || !kv_pos || !out) return LCA_ERR_INVALID_ARG;
+  if (p->variant == LCA_VARIANT_MLA && !q_sem) return LCA_ERR_INVALID_ARG;
+  if (m > 0 && (!cache_sem || !cache_pos)) return LCA_ERR_INVALID_ARG;
+  if (!aligned16(q_pos) || !aligned16(kv_sem) || !aligned16(kv_pos) || !aligned16(out) ||
+      (q_sem && !aligned16(q_sem)) || (cache_sem && !aligned16(cache_sem)) ||
+      (cache_pos && !aligned16(cache_pos)))
+    return LCA_ERR_MISALIGNED;
+  if (!simt_shape_ok(p)) return LCA_ERR_UNSUPPORTED_SHAPE;
+  AttnProblem a = {};
+  a.variant = p->variant; a.batch = p->batch; a.q_len = p->seq_len; a.n_q_heads = p->n_q_heads;
+  a.n_kv_heads = p->n_kv_heads; a.d_sem = p->d_sem; a.d_pos = p->d_pos; a.decode = 0;
+  a.seq_len = p->seq_len; a.group_size = p->group_size; a.window = p->window;
+  a.cache_rows = nullptr; a.cache_row_capacity = (int)(m + k); a.n_rep_bias = 0;
+  a.softmax_scale = p->softmax_scale; a.rep_logit_bias = p->rep_logit_bias;
+  a.q_sem = q_sem; a.q_pos = q_pos; a.kv_sem = kv_sem; a.kv_pos = kv_pos;
+  a.cache_sem = cache_sem; a.cache_pos = cache_pos; a.out = out; a.lse = lse_opt;
+  a.ws = ws; a.ws_bytes = ws_bytes; a.stream = (cudaStream_t)stream;
+  return run_attention(a);
+}
+
+int lca_decode_attention(const lca_params* p, const void* q_sem, const void* q_pos,
+                         const void* cache_sem, const void* cache_pos, const int32_t* cache_rows,
+                         int32_t cache_row_capacity, int32_t n_rep, void* out, float* lse_opt,
+                         void* ws, size_t ws_bytes, void* stream) {
+  int st = check_params(p, false);
+  if (st != LCA_OK) return st;
+  if (!q_pos || !cache_sem || !cache_pos || !cache_rows || !out) return LCA_ERR_INVALID_ARG;
+  if (p->variant == LCA_VARIANT_MLA && !q_sem) return LCA_ERR_INVALID_ARG;
+  if (cache_row_capacity <= 0 || n_rep < 0) return LCA_ERR_INVALID_ARG;
+  if (!aligned16(q_pos) || !aligned16(cache_sem) || !aligned16(cache_pos) || !aligned16(out) ||
+      (q_sem && !aligned16(q_sem)))
+    return LCA_ERR_MISALIGNED;
+  if (!simt_shape_ok(p)) return LCA_ERR_UNSUPPORTED_SHAPE;
+  AttnProblem a = {};
+  a.variant = p->variant; a.batch = p->batch; a.q_len = 1; a.n_q_heads = p->n_q_heads;
+  a.n_kv_heads = p->n_kv_heads; a.d_sem = p->d_sem; a.d_pos = p->d_pos; a.decode = 1;
+  a.seq_len = 0; a.group_size = 1; a.window = 0;
+  a.cache_rows = cache_rows; a.cache_row_capacity = cache_row_capacity; a.n_rep_bias = n_rep;
+  a.softmax_scale = p->softmax_scale; a.rep_logit_bias = p->rep_logit_bias;
+  a.q_sem = q_sem; a.q_pos = q_pos; a.kv_sem = nullptr; a.kv_pos = nullptr;
+  a.cache_sem = cache_sem; a.cache_pos = cache_pos; a.out = out; a.lse = lse_opt;
+  a.ws = ws; a.ws_bytes = ws_bytes; a.stream = (cudaStream_t)stream;
+  return run_attention(a);
+}
+
+int lca_last_device_status(void* stream) { return attn_tc_device_status((cudaStream_t)stream); }
+
+}  // extern "C"

@@ -1,0 +1,90 @@
+// Shared declarations of the LCA CUDA library (device helpers, launch bookkeeping).
+#pragma once
+
+#include <cuda_bf16.h>
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+#include "../../include/lca.h"
+
+namespace lca {
+
+typedef __nv_bfloat16 bf16;
+typedef __nv_bfloat162 bf162;
+
+// Launch bookkeeping (lca_launch_count).
+void note_launch(int n = 1);
+
+// Partition of Sec. 4.2 on the host.
+inline void partition(int64_t L, int64_t w, int64_t g, int64_t* m, int64_t* k) {
+  if (L < w + g) { *m = 0; *k = L; return; }
+  *m = (L - w) / g;
+  *k = L - (*m) * g;
+}
+
+// Representatives visible to the query at 0-based position p (prefix length p+1).
+__host__ __device__ inline int reps_visible(int p, int w, int g) {
+  int t = p + 1;
+  return (t < w + g) ? 0 : (t - w) / g;
+}
+
+// double -> bf16, round to nearest even with a single rounding: truncate to float, fold the
+// discarded bits into a sticky last bit (round to odd), then let the float->bf16 conversion round.
+__device__ inline bf16 double_to_bf16_rn(double x) {
+  float f = __double2float_rz(x);
+  if ((double)f != x) f = __uint_as_float(__float_as_uint(f) | 1u);
+  return __float2bfloat16_rn(f);
+}
+
+__device__ inline double warp_sum(double v) {
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) v += __shfl_xor_sync(0xffffffffu, v, o);
+  return v;
+}
+__device__ inline float warp_sum(float v) {
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) v += __shfl_xor_sync(0xffffffffu, v, o);
+  return v;
+}
+
+// ---- host-side launchers implemented in the .cu files ---------------------------------------
+struct CondenseLaunch {
+  const lca_params* p;
+  const void* q_tail_sem; const void* q_tail_pos; int64_t q_tail_batch_stride;
+  const float* qbar_opt;
+  const void* kv_sem; const void* kv_pos;
+  void* cache_sem; void* cache_pos; int32_t* anchor_idx; double* scores_opt;
+  void* ws; size_t ws_bytes; cudaStream_t stream;
+};
+size_t condense_workspace_bytes(const lca_params* p);
+int condense_launch(const CondenseLaunch& a);
+size_t condense_smem_bytes(const lca_params* p);
+
+// One description of an attention problem for every implementation.  Each query row (b, t, h)
+// attends to   A) rows [0, n_a) of a "cache" source   and   B) rows [b_first, b_last] of a
+// "token" source, where for prefill n_a = reps_visible(t), B = [n_a*g, t], and for decode
+// n_a = cache_rows[b], B empty.  The first min(n_a, bias_rows) A rows receive rep_logit_bias
+// (prefill: all of them).
+struct AttnProblem {
+  int variant;                 // LCA_VARIANT_*
+  int batch, q_len, n_q_heads, n_kv_heads, d_sem, d_pos;
+  int decode;                  // 0 prefill, 1 decode
+  int seq_len, group_size, window;       // prefill only
+  const int32_t* cache_rows;   // decode only (device)
+  int cache_row_capacity;      // rows per sequence in the cache arrays
+  int n_rep_bias;              // decode: rows that get the bias
+  float softmax_scale, rep_logit_bias;
+  const void* q_sem; const void* q_pos;  // [B, q_len, H, d]
+  const void* kv_sem; const void* kv_pos;        // [B, seq_len, Hkv, d]  (prefill)
+  const void* cache_sem; const void* cache_pos;  // [B, cap, Hkv, d]
+  void* out; float* lse;                  // [B, q_len, H, d_sem], [B, q_len, H]
+  void* ws; size_t ws_bytes;
+  cudaStream_t stream;
+};
+int attn_simt_launch(const AttnProblem& a);     // scalar kernel, every supported head shape
+bool attn_tc_supported(const AttnProblem& a);   // tensor-core (tcgen05) kernels
+size_t attn_tc_workspace_bytes(const AttnProblem& a);
+int attn_tc_launch(const AttnProblem& a);
+int attn_tc_device_status(cudaStream_t stream);
+
+}  // namespace lca

@@ -1,0 +1,227 @@
+"""GPU parity: the CUDA library (through the C ABI) against the CPU oracle on the same seeded bits.
+
+Small cases are compared element by element on every row; they span several KV tiles, a ragged
+tail and the degenerate partitions (no group, window 0, sequence shorter than a group, ...).
+"""
+import math
+
+import numpy as np
+import pytest
+import torch
+
+from oracle import lca_oracle as O
+from paper_2604_12452_b200 import inputs as I
+from tests import helpers as Hh
+
+pytestmark = pytest.mark.gpu
+DEV = "cuda:0"
+
+
+@pytest.fixture(scope="module")
+def B():
+    from paper_2604_12452_b200 import build
+    build.build()
+    from paper_2604_12452_b200 import binding
+    return binding
+
+
+def to_dev(inp):
+    return {k: v.to(DEV) for k, v in inp.items()}
+
+
+def to_cpu(inp):
+    return {k: v.cpu() for k, v in inp.items()}
+
+
+def run_mla(B, cfg, inp_dev, n_summary=0, bias=0.0, impl=0, want_scores=True):
+    p = B.params_from_config(cfg, batch=1, n_summary_q=n_summary, rep_logit_bias=bias)
+    L = cfg.seq_len
+    n = min(L, n_summary if n_summary > 0 else cfg.group_size)
+    qs, qp = inp_dev["q_sem"], inp_dev["q_pos"]
+    cond = B.condense(p, qs[L - n:], qp[L - n:], inp_dev["ckv"], inp_dev["kr"], want_scores=want_scores)
+    prev = B.lca_set_attention_impl(impl)
+    try:
+        out, lse = B.prefill_attention(p, qs, qp, inp_dev["ckv"], inp_dev["kr"], cond["cache_sem"],
+                                       cond["cache_pos"], want_lse=True)
+    finally:
+        B.lca_set_attention_impl(prev)
+    torch.cuda.synchronize()
+    return p, cond, out, lse
+
+
+def one_seq(cond):
+    r = dict(cond)
+    for key in ("cache_sem", "cache_pos", "anchor_idx"):
+        r[key] = cond[key][0]
+    return r
+
+
+MLA_SMALL = [
+    # (L, H, g, w, n_summary)  -- d_c = 512, d_R = 64 throughout
+    (1024, 4, 64, 128, 0),      # config 1 as given
+    (1024, 4, 64, 1024, 0),     # paper-default window: no group, plain MLA
+    (1000, 4, 64, 128, 0),      # ragged: (L - w) mod g = 40 residual tokens
+    (777, 16, 16, 100, 32),     # paper-default group size, odd sizes, 32 summary queries
+    (300, 128, 8, 64, 8),       # many heads (one token per 128-row tile)
+    (130, 4, 64, 0, 0),         # window 0
+    (50, 4, 64, 16, 0),         # shorter than one group
+    (1, 4, 4, 0, 0),            # a single token
+]
+
+
+@pytest.mark.parametrize("L,H,g,w,ns", MLA_SMALL)
+def test_mla_small_cases_match_oracle_on_every_row(B, L, H, g, w, ns):
+    cfg = I.scaled(I.CONFIGS["mla_1k"], seq_len=L, n_q_heads=H, group_size=g, window=w, n_needles=min(8, L))
+    inp = I.make_mla_inputs(cfg, "cpu")
+    p, cond, out, lse = run_mla(B, cfg, to_dev(inp), n_summary=ns)
+    ref = Hh.oracle_mla(inp, g, w, cfg.softmax_scale, rows=np.arange(L), n_summary=ns)
+    Hh.check_condense(one_seq(cond), ref["cond"])
+    if ref["cond"]["m"]:
+        sc = cond["scores"][0, 0].cpu().numpy()
+        np.testing.assert_allclose(sc, ref["cond"]["scores"], rtol=0, atol=1e-12)
+    Hh.check_outputs(out[0], ref["out"], f"mla L={L} H={H} g={g} w={w}")
+    np.testing.assert_allclose(lse[0].cpu().numpy(), ref["lse"], atol=2e-3, rtol=1e-4)
+
+
+def test_mla_stress_peaky_queries_and_exact_ties(B):
+    cfg = I.scaled(I.CONFIGS["mla_1k"], seq_len=1024, n_q_heads=4)
+    inp = I.stress_duplicate_tokens(I.stress_peaky_queries(I.make_mla_inputs(cfg, "cpu"), cfg), cfg)
+    p, cond, out, _ = run_mla(B, cfg, to_dev(inp))
+    ref = Hh.oracle_mla(inp, cfg.group_size, cfg.window, cfg.softmax_scale, rows=np.arange(cfg.seq_len))
+    # the softmax is far from uniform here, and duplicated tokens tie exactly: lowest index wins
+    alpha = ref["cond"]["alpha"].reshape(-1, cfg.group_size)
+    assert alpha.max() > 0.5
+    Hh.check_condense(one_seq(cond), ref["cond"])
+    Hh.check_outputs(out[0], ref["out"], "mla stress")
+
+
+def test_mla_zero_queries_give_mean_pooling(B):
+    cfg = I.scaled(I.CONFIGS["mla_1k"], seq_len=512, n_q_heads=4)
+    inp = I.make_mla_inputs(cfg, "cpu")
+    inp["q_sem"] = torch.zeros_like(inp["q_sem"])
+    inp["q_pos"] = torch.zeros_like(inp["q_pos"])
+    p, cond, out, _ = run_mla(B, cfg, to_dev(inp))
+    ref = Hh.oracle_mla(inp, cfg.group_size, cfg.window, cfg.softmax_scale, rows=np.arange(cfg.seq_len))
+    m = ref["cond"]["m"]
+    assert np.array_equal(ref["cond"]["anchor"], np.arange(m) * cfg.group_size)
+    Hh.check_condense(one_seq(cond), ref["cond"])
+    Hh.check_outputs(out[0], ref["out"], "mla q=0")
+
+
+def test_mla_rep_logit_bias_and_supplied_summary_query(B):
+    cfg = I.scaled(I.CONFIGS["mla_1k"], seq_len=640, n_q_heads=4, group_size=16, window=64)
+    inp = I.make_mla_inputs(cfg, "cpu")
+    d = to_dev(inp)
+    bias = math.log(cfg.group_size)
+    qbar32 = torch.randn(1, 1, 576, generator=torch.Generator().manual_seed(5)).float()
+    p = B.params_from_config(cfg, batch=1, rep_logit_bias=bias)
+    cond = B.condense(p, None, None, d["ckv"], d["kr"], qbar=qbar32.to(DEV), want_scores=True)
+    out, _ = B.prefill_attention(p, d["q_sem"], d["q_pos"], d["ckv"], d["kr"], cond["cache_sem"], cond["cache_pos"])
+    ref = Hh.oracle_mla(inp, cfg.group_size, cfg.window, cfg.softmax_scale, rows=np.arange(cfg.seq_len),
+                        rep_logit_bias=bias, qbar=qbar32[0, 0].double().numpy())
+    Hh.check_condense(one_seq(cond), ref["cond"])
+    Hh.check_outputs(out[0], ref["out"], "mla bias=ln g")
+
+
+def test_mla_batched_sequences_are_independent(B):
+    cfg = I.scaled(I.CONFIGS["mla_1k"], seq_len=384, n_q_heads=4, group_size=32, window=64, batch=3)
+    seqs = [I.make_mla_inputs(cfg, "cpu", batch_index=b) for b in range(3)]
+    stack = {k: torch.stack([s[k] for s in seqs]).to(DEV) for k in seqs[0]}
+    p = B.params_from_config(cfg, batch=3)
+    g = cfg.group_size
+    # summary tail taken straight out of the full [B, L, H, d] query tensors (stride L)
+    L = cfg.seq_len
+    qs_tail = stack["q_sem"][:, L - g:].contiguous()
+    qp_tail = stack["q_pos"][:, L - g:].contiguous()
+    cond = B.condense(p, qs_tail, qp_tail, stack["ckv"], stack["kr"])
+    out, _ = B.prefill_attention(p, stack["q_sem"], stack["q_pos"], stack["ckv"], stack["kr"],
+                                 cond["cache_sem"], cond["cache_pos"])
+    # the same through pointers into the full tensors: tail of sequence b starts L rows after b-1's
+    p2 = B.params_from_config(cfg, batch=3)
+    first_tail_sem = stack["q_sem"].data_ptr() + (L - g) * cfg.n_q_heads * cfg.d_sem * 2
+    first_tail_pos = stack["q_pos"].data_ptr() + (L - g) * cfg.n_q_heads * cfg.d_pos * 2
+    cond2 = B.condense(p2, first_tail_sem, first_tail_pos, stack["ckv"], stack["kr"], q_tail_batch_stride=L)
+    assert torch.equal(cond["cache_sem"], cond2["cache_sem"]) and torch.equal(cond["anchor_idx"], cond2["anchor_idx"])
+    for b in range(3):
+        ref = Hh.oracle_mla(seqs[b], g, cfg.window, cfg.softmax_scale, rows=np.arange(L))
+        r = dict(cond)
+        for key in ("cache_sem", "cache_pos", "anchor_idx"):
+            r[key] = cond[key][b]
+        Hh.check_condense(r, ref["cond"])
+        Hh.check_outputs(out[b], ref["out"], f"batch {b}")
+
+
+GQA_SMALL = [(1024, 32, 8, 64, 128), (515, 8, 2, 16, 40), (96, 4, 4, 64, 64), (260, 32, 8, 64, 0)]
+
+
+@pytest.mark.parametrize("L,Hq,Hkv,g,w", GQA_SMALL)
+def test_gqa_small_cases_match_oracle_on_every_row(B, L, Hq, Hkv, g, w):
+    cfg = I.scaled(I.CONFIGS["gqa_64k"], seq_len=L, n_q_heads=Hq, n_kv_heads=Hkv, group_size=g, window=w,
+                   n_needles=4)
+    inp = I.make_gqa_inputs(cfg, "cpu")
+    d = to_dev(inp)
+    p = B.params_from_config(cfg, batch=1)
+    n = min(L, g)
+    cond = B.condense(p, None, d["q"][L - n:], d["v"], d["k"], want_scores=True)
+    out, lse = B.prefill_attention(p, None, d["q"], d["v"], d["k"], cond["cache_sem"], cond["cache_pos"],
+                                   want_lse=True)
+    ref = Hh.oracle_gqa(inp, g, w, cfg.softmax_scale, rows=np.arange(L))
+    Hh.check_condense(one_seq(cond), ref["cond"], kind="gqa")
+    Hh.check_outputs(out[0], ref["out"], f"gqa L={L}")
+    np.testing.assert_allclose(lse[0].cpu().numpy(), ref["lse"], atol=2e-3, rtol=1e-4)
+
+
+def test_mla_decode_matches_oracle_and_prefill_row(B):
+    # contexts of different lengths share one cache buffer (capacity = longest + 1 appended row)
+    cfg = I.scaled(I.CONFIGS["mla_decode"], batch=3, seq_len=1500, n_q_heads=128, group_size=64, window=256)
+    g, w, H = cfg.group_size, cfg.window, cfg.n_q_heads
+    p = B.params_from_config(cfg, batch=3)
+    m, k = B.lca_partition(p)
+    cap = m + k + 1
+    cache_sem = torch.zeros((3, cap, 1, 512), dtype=torch.bfloat16, device=DEV)
+    cache_pos = torch.zeros((3, cap, 1, 64), dtype=torch.bfloat16, device=DEV)
+    rows = torch.tensor([m + k + 1, m + k + 1, m + k - 5], dtype=torch.int32, device=DEV)
+    q_new_sem = torch.randn((3, H, 512), generator=torch.Generator().manual_seed(1)).bfloat16()
+    q_new_pos = torch.randn((3, H, 64), generator=torch.Generator().manual_seed(2)).bfloat16()
+    refs = []
+    p1 = B.params_from_config(cfg, batch=1)
+    for b in range(3):
+        inp = I.make_mla_inputs(cfg, "cpu", batch_index=b, q_positions=slice(cfg.seq_len - g, cfg.seq_len))
+        d = to_dev(inp)
+        c = B.condense(p1, d["q_sem"], d["q_pos"], d["ckv"], d["kr"])
+        ref = Hh.oracle_mla(inp, g, w, cfg.softmax_scale)
+        Hh.check_condense(one_seq(c), ref["cond"])
+        cache_sem[b, :m + k] = c["cache_sem"][0]
+        cache_pos[b, :m + k] = c["cache_pos"][0]
+        new_sem = torch.randn((1, 512), generator=torch.Generator().manual_seed(10 + b)).bfloat16()
+        new_pos = torch.randn((1, 64), generator=torch.Generator().manual_seed(20 + b)).bfloat16()
+        cache_sem[b, m + k, 0] = new_sem[0].to(DEV)
+        cache_pos[b, m + k, 0] = new_pos[0].to(DEV)
+        nrows = int(rows[b])
+        cs = O.bits_to_f64(Hh.bits(cache_sem[b, :nrows, 0]))
+        cp = O.bits_to_f64(Hh.bits(cache_pos[b, :nrows, 0]))
+        refs.append(O.mla_decode(O.torch_bf16_to_f64(q_new_sem[b]), O.torch_bf16_to_f64(q_new_pos[b]), cs, cp,
+                                 m, Hh.f32(cfg.softmax_scale)))
+    out, lse = B.decode_attention(p, q_new_sem.to(DEV), q_new_pos.to(DEV), cache_sem, cache_pos, rows, m,
+                                  want_lse=True)
+    for b in range(3):
+        Hh.check_outputs(out[b], refs[b][0], f"decode seq {b}")
+        np.testing.assert_allclose(lse[b].cpu().numpy(), refs[b][1], atol=2e-3, rtol=1e-4)
+
+
+def test_dense_window_is_plain_causal_attention(B):
+    # window >= L: the dense-MLA comparison run through the same entry point (Eq. 5), every row.
+    cfg = I.scaled(I.CONFIGS["mla_1k"], seq_len=600, n_q_heads=16, window=600)
+    inp = I.make_mla_inputs(cfg, "cpu")
+    p, cond, out, _ = run_mla(B, cfg, to_dev(inp))
+    assert cond["m"] == 0 and cond["k"] == 600
+    ref = Hh.oracle_mla(inp, cfg.group_size, cfg.window, cfg.softmax_scale, rows=np.arange(600))
+    Hh.check_outputs(out[0], ref["out"], "dense")
+
+
+def test_launches_are_counted(B):
+    cfg = I.scaled(I.CONFIGS["mla_1k"], seq_len=256, n_q_heads=4)
+    inp = to_dev(I.make_mla_inputs(cfg, "cpu"))
+    before = B.lca_launch_count()
+    run_mla(B, cfg, inp)
+    assert B.lca_launch_count() - before >= 5     # 2 summary + condense + 2 copies + attention
