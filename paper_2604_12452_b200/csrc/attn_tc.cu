@@ -1,12 +1,444 @@
-// Tensor-core (tcgen05 / TMEM / TMA) attention kernels.  Placeholder until the kernels land:
-// every shape reports "not supported" so that the dispatcher uses the scalar kernel.
+// Tensor-core attention over the condensed context (Eq. 10 at every prefix length; Sec. 4.3
+// decode) for sm_100a: TMA-staged 128-byte-swizzled tiles, tcgen05.mma with accumulators in
+// tensor memory, online softmax in fp32.
+//
+// One CTA owns a tile of 128 query rows = TB consecutive tokens x HB heads that share one
+// key/value stream.  It walks first the representative rows of the condensed cache that any of
+// its tokens may see, then the local tokens, in tiles of BN keys:
+//     S  = Q K^T        (tcgen05.mma, A = Q and B = K tile from shared memory, D in TMEM)
+//     P  = exp2(S*c - m) with per-row masks only on boundary tiles (4 softmax warps, one row
+//          per thread, S read from TMEM, P written back to TMEM as packed bf16)
+//     O += P V          (tcgen05.mma, A = P from TMEM, B = V tile from shared memory)
+// Roles: warp 0 issues TMA loads, warp 1 owns TMEM and issues every MMA, warps 2..5 do the
+// softmax, the (rare) rescale of O when the running maximum grows by more than 2^8, and the
+// epilogue.  Every wait is bounded; on expiry the CTA records a code in a global status word,
+// drains and returns.
+#include <cstring>
+
 #include "lca_common.cuh"
+#include "tc_common.cuh"
 
 namespace lca {
-bool attn_tc_supported(const AttnProblem&) { return false; }
-size_t attn_tc_workspace_bytes(const AttnProblem&) { return 0; }
-int attn_tc_launch(const AttnProblem&) { return LCA_ERR_UNSUPPORTED_SHAPE; }
-int attn_tc_device_status(cudaStream_t stream) {
-  return cudaStreamSynchronize(stream) == cudaSuccess ? LCA_OK : LCA_ERR_CUDA;
+using namespace tc;
+
+static __device__ int g_tc_status = 0;
+
+static constexpr int ROWS = 128;          // query rows per CTA (TMEM lanes)
+static constexpr int BN = 128;            // keys per tile
+static constexpr int CHUNK_BYTES_Q = ROWS * 128;   // one 64-column chunk of the query tile
+static constexpr int CHUNK_BYTES_KV = BN * 128;    // one 64-column chunk of a key/value tile
+static constexpr float RESCALE_THRESHOLD = 8.0f;   // log2 units
+
+struct TcParams {
+  CUtensorMap q_sem, q_pos, kv_sem, kv_pos, cache_sem, cache_pos;   // 3-D {d, heads, rows}
+  bf16* out; float* lse; const int32_t* cache_rows;
+  int B, q_len, Hq, Hkv, L, g, w, cap, n_rep_bias, decode;
+  int HB, TB, n_tok_tiles, d_out;
+  float scale_log2, bias_log2;
+};
+
+// Shared-memory plan of the 1-CTA kernel.  NK_SEM / NK_POS: 64-column key chunks taken from the
+// sem / pos tensors; NV: value chunks (taken from the sem tensor).  When V_IN_K the value chunks
+// are the first NV key chunks of the same tile (MLA: values are the latents), else they are
+// loaded separately (GQA).
+template <int NK_SEM, int NK_POS, int NV, bool V_IN_K, int STAGES>
+struct Plan1 {
+  static constexpr int NK = NK_SEM + NK_POS;
+  static constexpr int Q_BYTES = NK * CHUNK_BYTES_Q;
+  static constexpr int K_STAGE = NK * CHUNK_BYTES_KV;
+  static constexpr int V_STAGE = V_IN_K ? 0 : NV * CHUNK_BYTES_KV;
+  static constexpr int OFF_Q = 0;
+  static constexpr int OFF_K = OFF_Q + Q_BYTES;
+  static constexpr int OFF_V = OFF_K + STAGES * K_STAGE;
+  static constexpr int OFF_BAR = OFF_V + STAGES * V_STAGE;
+  static constexpr int NBAR = 1 + 4 * STAGES + 2 + 2 + 1;
+  static constexpr int OFF_MISC = OFF_BAR + NBAR * 8;
+  static constexpr int BYTES = OFF_MISC + 16 + 1024;     // + slack to align the base to 1024 B
+  // tensor memory columns
+  static constexpr int TM_S0 = 0, TM_S1 = BN, TM_O = 2 * BN;
+  static constexpr int TM_COLS = 512;
+  static_assert(2 * BN + NV * 64 <= 512, "TMEM budget");
+};
+
+template <int NK_SEM, int NK_POS, int NV, bool V_IN_K, int STAGES>
+__global__ void __launch_bounds__(192, 1)
+attn_tc1_kernel(const __grid_constant__ TcParams p) {
+  using P = Plan1<NK_SEM, NK_POS, NV, V_IN_K, STAGES>;
+  constexpr int NK = P::NK;
+  extern __shared__ unsigned char smem_dyn[];
+  const uint32_t base = (smem_u32(smem_dyn) + 1023u) & ~1023u;
+  unsigned char* base_ptr = smem_dyn + (base - smem_u32(smem_dyn));
+  const uint32_t sQ = base + P::OFF_Q, sK = base + P::OFF_K, sV = base + P::OFF_V;
+  const uint32_t bars = base + P::OFF_BAR;
+  auto BAR_Q = [&]() { return bars; };
+  auto BAR_KFULL = [&](int s) { return bars + 8 * (1 + s); };
+  auto BAR_KEMPTY = [&](int s) { return bars + 8 * (1 + STAGES + s); };
+  auto BAR_VFULL = [&](int s) { return bars + 8 * (1 + 2 * STAGES + s); };
+  auto BAR_VEMPTY = [&](int s) { return bars + 8 * (1 + 3 * STAGES + s); };
+  auto BAR_SFULL = [&](int i) { return bars + 8 * (1 + 4 * STAGES + i); };
+  auto BAR_PFULL = [&](int i) { return bars + 8 * (3 + 4 * STAGES + i); };
+  const uint32_t BAR_ODONE = bars + 8 * (5 + 4 * STAGES);
+  volatile uint32_t* tmem_slot = reinterpret_cast<volatile uint32_t*>(base_ptr + P::OFF_MISC);
+  volatile int* abort_flag = reinterpret_cast<volatile int*>(base_ptr + P::OFF_MISC + 4);
+
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+
+  // ---- which rows, which key tiles
+  const int tile = p.n_tok_tiles - 1 - (int)blockIdx.x;      // heaviest (latest) query tiles first
+  const int hb = blockIdx.y, b = blockIdx.z;
+  const int t0 = tile * p.TB;
+  const int t1 = min(t0 + p.TB, p.q_len) - 1;
+  const int head0 = hb * p.HB;
+  const int hk = (p.Hkv == 1) ? 0 : hb;
+  int nA, nB, first_lo, n_a_lo, n_a_hi;
+  if (p.decode) {
+    n_a_hi = n_a_lo = min(max(p.cache_rows[b], 0), p.cap);
+    first_lo = 0; nB = 0;
+  } else {
+    n_a_lo = reps_visible(t0, p.w, p.g);
+    n_a_hi = reps_visible(t1, p.w, p.g);
+    first_lo = n_a_lo * p.g;
+    nB = (t1 - first_lo + BN) / BN;
+  }
+  nA = (n_a_hi + BN - 1) / BN;
+  const int n_tiles = nA + nB;
+
+  if (threadIdx.x == 0) {
+    mbar_init(BAR_Q(), 1);
+    for (int s = 0; s < STAGES; ++s) {
+      mbar_init(BAR_KFULL(s), 1); mbar_init(BAR_KEMPTY(s), 1);
+      mbar_init(BAR_VFULL(s), 1); mbar_init(BAR_VEMPTY(s), 1);
+    }
+    for (int i = 0; i < 2; ++i) { mbar_init(BAR_SFULL(i), 1); mbar_init(BAR_PFULL(i), 128); }
+    mbar_init(BAR_ODONE, 1);
+    *abort_flag = 0;
+    fence_mbar_init();
+  }
+  if (warp == 1) {                    // TMEM: allocated and freed by the same warp
+    tmem_alloc(smem_u32((const void*)tmem_slot), P::TM_COLS);
+    tmem_relinquish();
+  }
+  tc_fence_before();
+  __syncthreads();
+  tc_fence_after();
+  const uint32_t tmem = *tmem_slot;
+
+  auto fail = [&](int code) {
+    atomicCAS(&g_tc_status, 0, code);
+    *abort_flag = 1;
+  };
+
+  if (warp == 0) {
+    // =============================================================== TMA producer
+    if (lane == 0 && n_tiles > 0) {
+      prefetch_tmap(&p.q_pos); prefetch_tmap(&p.kv_pos); prefetch_tmap(&p.kv_sem);
+      mbar_expect_tx(BAR_Q(), P::Q_BYTES);
+      const int qrow = b * p.q_len + t0;
+      for (int c = 0; c < NK_SEM; ++c) tma_load_3d(sQ + c * CHUNK_BYTES_Q, &p.q_sem, c * 64, head0, qrow, BAR_Q());
+      for (int c = 0; c < NK_POS; ++c) tma_load_3d(sQ + (NK_SEM + c) * CHUNK_BYTES_Q, &p.q_pos, c * 64, head0, qrow, BAR_Q());
+      for (int j = 0; j < n_tiles; ++j) {
+        const int s = j % STAGES, round = j / STAGES;
+        const bool isA = j < nA;
+        const int row = isA ? b * p.cap + j * BN : b * p.L + first_lo + (j - nA) * BN;
+        const CUtensorMap* msem = isA ? &p.cache_sem : &p.kv_sem;
+        const CUtensorMap* mpos = isA ? &p.cache_pos : &p.kv_pos;
+        if (!mbar_wait(BAR_KEMPTY(s), (round & 1) ^ 1, abort_flag)) { fail(ERR_WAIT_KV_EMPTY); break; }
+        mbar_expect_tx(BAR_KFULL(s), P::K_STAGE);
+        for (int c = 0; c < NK_SEM; ++c) tma_load_3d(sK + s * P::K_STAGE + c * CHUNK_BYTES_KV, msem, c * 64, hk, row, BAR_KFULL(s));
+        for (int c = 0; c < NK_POS; ++c) tma_load_3d(sK + s * P::K_STAGE + (NK_SEM + c) * CHUNK_BYTES_KV, mpos, c * 64, hk, row, BAR_KFULL(s));
+        if (!V_IN_K) {
+          if (!mbar_wait(BAR_VEMPTY(s), (round & 1) ^ 1, abort_flag)) { fail(ERR_WAIT_KV_EMPTY); break; }
+          mbar_expect_tx(BAR_VFULL(s), P::V_STAGE);
+          for (int c = 0; c < NV; ++c) tma_load_3d(sV + s * P::V_STAGE + c * CHUNK_BYTES_KV, msem, c * 64, hk, row, BAR_VFULL(s));
+        }
+      }
+    }
+  } else if (warp == 1) {
+    // =============================================================== MMA issuer
+    constexpr uint32_t IDESC_S = umma_idesc_bf16(ROWS, BN, false, false);
+    constexpr uint32_t IDESC_PV = umma_idesc_bf16(ROWS, NV * 64, false, true);
+    bool ok = n_tiles > 0;
+    if (ok && lane == 0) ok = mbar_wait(BAR_Q(), 0, abort_flag);
+    ok = __all_sync(0xffffffffu, ok);
+    if (!ok && n_tiles > 0 && lane == 0) fail(ERR_WAIT_Q);
+    auto issue_pv = [&](int j) -> bool {      // O += P_j V_j   (whole warp enters; lane 0 issues)
+      const int s = j % STAGES, round = j / STAGES;
+      bool good = true;
+      if (lane == 0) {
+        good = mbar_wait(BAR_PFULL(j & 1), (j >> 1) & 1, abort_flag);
+        if (good && !V_IN_K) good = mbar_wait(BAR_VFULL(s), round & 1, abort_flag);
+        if (!good) fail(ERR_WAIT_P_FULL);
+      }
+      good = __all_sync(0xffffffffu, good);
+      if (!good) return false;
+      const uint32_t vbase = V_IN_K ? sK + s * P::K_STAGE : sV + s * P::V_STAGE;
+      // Rows of the cache beyond the valid count (decode, last tile) may hold anything; their
+      // probabilities are exactly 0, so zero the value rows to keep 0 * garbage out of O.
+      if (p.decode && (j + 1) * BN > n_a_hi) {
+        const int first_bad = n_a_hi - j * BN;
+        for (int idx = lane; idx < (BN - first_bad) * 8 * NV; idx += 32) {
+          const int c = idx / ((BN - first_bad) * 8), rem = idx % ((BN - first_bad) * 8);
+          const int r = first_bad + rem / 8, q = rem % 8;
+          const uint32_t a = vbase + c * CHUNK_BYTES_KV + r * 128 + q * 16;
+          asm volatile("st.shared.v4.b32 [%0], {%1, %1, %1, %1};" ::"r"(a), "r"(0) : "memory");
+        }
+        fence_proxy_async_smem();
+        __syncwarp();
+      }
+      if (lane == 0) {
+        tc_fence_after();
+        const uint32_t ptm = tmem + ((j & 1) ? P::TM_S1 : P::TM_S0);
+#pragma unroll
+        for (int k = 0; k < BN / 16; ++k) {
+          const uint64_t bd = umma_desc_sw128(vbase + k * 2048, CHUNK_BYTES_KV, 1024);
+          umma_ts(tmem + P::TM_O, ptm + k * 8, bd, IDESC_PV, (j > 0 || k > 0) ? 1u : 0u);
+        }
+        umma_commit(V_IN_K ? BAR_KEMPTY(s) : BAR_VEMPTY(s));
+        umma_commit(BAR_ODONE);
+      }
+      __syncwarp();
+      return true;
+    };
+    for (int j = 0; ok && j < n_tiles; ++j) {
+      const int s = j % STAGES, round = j / STAGES;
+      if (lane == 0) {
+        ok = mbar_wait(BAR_KFULL(s), round & 1, abort_flag);
+        if (!ok) fail(ERR_WAIT_KV_FULL);
+        if (ok) {
+          tc_fence_after();
+          const uint32_t stm = tmem + ((j & 1) ? P::TM_S1 : P::TM_S0);
+#pragma unroll
+          for (int c = 0; c < NK; ++c) {
+#pragma unroll
+            for (int k = 0; k < 4; ++k) {
+              const uint64_t ad = umma_desc_sw128(sQ + c * CHUNK_BYTES_Q + k * 32, 16, 1024);
+              const uint64_t bd = umma_desc_sw128(sK + s * P::K_STAGE + c * CHUNK_BYTES_KV + k * 32, 16, 1024);
+              umma_ss(stm, ad, bd, IDESC_S, (c > 0 || k > 0) ? 1u : 0u);
+            }
+          }
+          umma_commit(BAR_SFULL(j & 1));
+          if (!V_IN_K) umma_commit(BAR_KEMPTY(s));
+        }
+      }
+      ok = __all_sync(0xffffffffu, ok);
+      if (ok && j >= 1) ok = issue_pv(j - 1);
+    }
+    if (ok && n_tiles > 0) issue_pv(n_tiles - 1);
+  } else {
+    // =============================================================== softmax / epilogue (128 threads)
+    const int quarter = warp & 3;                 // TMEM lanes this warp may touch
+    const int r = quarter * 32 + lane;            // query row of this thread
+    const uint32_t lane_base = (uint32_t)(quarter * 32) << 16;
+    const int tl = r / p.HB, hl = r % p.HB;
+    const int t_row = t0 + tl;
+    const bool row_valid = t_row < p.q_len;
+    int n_a_row, bias_rows, first_row;
+    if (p.decode) { n_a_row = n_a_hi; bias_rows = min(p.n_rep_bias, n_a_row); first_row = 0; }
+    else { n_a_row = reps_visible(min(t_row, p.q_len - 1), p.w, p.g); bias_rows = n_a_row; first_row = n_a_row * p.g; }
+    float m_ref = -INFINITY, l_sum = 0.f;
+    bool ok = true;
+    for (int j = 0; j < n_tiles; ++j) {
+      ok = mbar_wait(BAR_SFULL(j & 1), (j >> 1) & 1, abort_flag);
+      ok = __all_sync(0xffffffffu, ok);
+      if (!ok) { if (lane == 0) fail(ERR_WAIT_S_FULL); break; }
+      tc_fence_after();
+      const uint32_t stm = tmem + lane_base + ((j & 1) ? P::TM_S1 : P::TM_S0);
+      uint32_t sr[4][32];
+#pragma unroll
+      for (int q = 0; q < 4; ++q) tmem_ld32(stm + q * 32, sr[q]);
+      tmem_wait_ld();
+      const bool isA = j < nA;
+      const int key0 = isA ? j * BN : first_lo + (j - nA) * BN;
+      bool need_mask;
+      int lo, hi;                                  // visible columns: lo <= c <= hi
+      if (isA) { lo = 0; hi = n_a_row - key0 - 1; need_mask = key0 + BN > n_a_lo; }
+      else { lo = first_row - key0; hi = t_row - key0; need_mask = (key0 < n_a_hi * p.g) || (key0 + BN - 1 > t0); }
+      const int blim = isA ? bias_rows - key0 : 0;  // columns < blim receive the bias
+      float tmax = -INFINITY;
+#pragma unroll
+      for (int q = 0; q < 4; ++q) {
+#pragma unroll
+        for (int i = 0; i < 32; ++i) {
+          const int c = q * 32 + i;
+          float s = __uint_as_float(sr[q][i]) * p.scale_log2;
+          if (isA && p.bias_log2 != 0.f && c < blim) s += p.bias_log2;
+          if (need_mask && (c < lo || c > hi)) s = -INFINITY;
+          sr[q][i] = __float_as_uint(s);
+          tmax = fmaxf(tmax, s);
+        }
+      }
+      // running maximum: rescale O only when it grows by more than the threshold
+      bool need = false;
+      float factor = 1.f;
+      if (j == 0) m_ref = tmax;
+      else if (tmax > m_ref + RESCALE_THRESHOLD) { need = true; factor = exp2f(m_ref - tmax); }
+      if (__any_sync(0xffffffffu, need)) {
+        ok = mbar_wait(BAR_ODONE, (j - 1) & 1, abort_flag);       // P_{j-1} V_{j-1} has landed in O
+        ok = __all_sync(0xffffffffu, ok);
+        if (!ok) { if (lane == 0) fail(ERR_WAIT_O_DONE); break; }
+        tc_fence_after();
+#pragma unroll
+        for (int q = 0; q < NV * 2; ++q) {
+          uint32_t o[32];
+          tmem_ld32(tmem + lane_base + P::TM_O + q * 32, o);
+          tmem_wait_ld();
+#pragma unroll
+          for (int i = 0; i < 32; ++i) o[i] = __float_as_uint(__uint_as_float(o[i]) * factor);
+          tmem_st32(tmem + lane_base + P::TM_O + q * 32, o);
+        }
+        if (need) { l_sum *= factor; m_ref = tmax; }
+      }
+      const float m_use = (m_ref == -INFINITY) ? 0.f : m_ref;
+      float rs = 0.f;
+#pragma unroll
+      for (int q = 0; q < 4; ++q) {
+        uint32_t pk[16];
+#pragma unroll
+        for (int i = 0; i < 16; ++i) {
+          const float p0 = exp2f(__uint_as_float(sr[q][2 * i]) - m_use);
+          const float p1 = exp2f(__uint_as_float(sr[q][2 * i + 1]) - m_use);
+          rs += p0 + p1;
+          pk[i] = pack_bf16x2(p0, p1);
+        }
+#pragma unroll
+        for (int i = 0; i < 16; ++i) sr[q >> 1][(q & 1) * 16 + i] = pk[i];   // reuse: rows 0,1 of sr now hold P
+      }
+      l_sum += rs;
+      tmem_st32(stm, sr[0]);            // P columns 0..31  (keys 0..63)
+      tmem_st32(stm + 32, sr[1]);       // P columns 32..63 (keys 64..127)
+      tmem_wait_st();
+      tc_fence_before();
+      mbar_arrive(BAR_PFULL(j & 1));
+    }
+    // ---- epilogue: O / l -> bf16 -> global
+    if (ok && n_tiles > 0) {
+      ok = mbar_wait(BAR_ODONE, (n_tiles - 1) & 1, abort_flag);
+      ok = __all_sync(0xffffffffu, ok);
+      if (!ok && lane == 0) fail(ERR_WAIT_O_DONE);
+    }
+    if (ok) {
+      tc_fence_after();
+      const float inv = (n_tiles > 0 && l_sum > 0.f) ? 1.f / l_sum : 0.f;
+      const size_t orow = ((size_t)b * p.q_len + t_row) * p.Hq + head0 + hl;
+      bf16* dst = p.out + orow * p.d_out;
+#pragma unroll
+      for (int q = 0; q < NV * 2; ++q) {
+        uint32_t o[32];
+        if (n_tiles > 0) { tmem_ld32(tmem + lane_base + P::TM_O + q * 32, o); tmem_wait_ld(); }
+        else {
+#pragma unroll
+          for (int i = 0; i < 32; ++i) o[i] = 0;
+        }
+        if (row_valid && hl < p.HB && head0 + hl < p.Hq) {
+          uint4* d4 = reinterpret_cast<uint4*>(dst + q * 32);
+#pragma unroll
+          for (int v = 0; v < 4; ++v) {
+            uint4 w;
+            w.x = pack_bf16x2(__uint_as_float(o[8 * v + 0]) * inv, __uint_as_float(o[8 * v + 1]) * inv);
+            w.y = pack_bf16x2(__uint_as_float(o[8 * v + 2]) * inv, __uint_as_float(o[8 * v + 3]) * inv);
+            w.z = pack_bf16x2(__uint_as_float(o[8 * v + 4]) * inv, __uint_as_float(o[8 * v + 5]) * inv);
+            w.w = pack_bf16x2(__uint_as_float(o[8 * v + 6]) * inv, __uint_as_float(o[8 * v + 7]) * inv);
+            d4[v] = w;
+          }
+        }
+      }
+      if (p.lse && row_valid)
+        p.lse[orow] = (n_tiles > 0 && l_sum > 0.f) ? (m_ref + log2f(l_sum)) * 0.6931471805599453f : -INFINITY;
+    }
+    tc_fence_before();
+  }
+  // ---- teardown: let straggling bulk copies land if the CTA gave up, then free TMEM
+  if (*abort_flag && warp == 0 && lane == 0) {
+    const long long t0c = clock64();
+    while (clock64() - t0c < 2000000ll) { __nanosleep(1000); }
+  }
+  __syncthreads();
+  if (warp == 1) {
+    tc_fence_after();
+    tmem_dealloc(tmem, P::TM_COLS);
+  }
 }
+
+// ----------------------------------------------------------------------------------- host
+typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
+                                  const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
+                                  CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+
+static EncodeTiledFn encode_fn() {
+  static EncodeTiledFn fn = nullptr;
+  if (!fn) {
+    void* ptr = nullptr;
+    cudaDriverEntryPointQueryResult qres;
+    if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &ptr, cudaEnableDefault, &qres) == cudaSuccess &&
+        qres == cudaDriverEntryPointSuccess)
+      fn = reinterpret_cast<EncodeTiledFn>(ptr);
+  }
+  return fn;
+}
+
+// bf16 tensor [rows, heads, d] (d contiguous) viewed as 3-D {d, heads, rows}; box {64, box_heads, box_rows}
+static bool make_map(CUtensorMap* map, const void* ptr, int d, int heads, long long rows, int box_heads, int box_rows) {
+  EncodeTiledFn fn = encode_fn();
+  if (!fn) return false;
+  if (!ptr) { memset(map, 0, sizeof(*map)); return true; }
+  cuuint64_t dims[3] = {(cuuint64_t)d, (cuuint64_t)heads, (cuuint64_t)rows};
+  cuuint64_t strides[2] = {(cuuint64_t)d * 2, (cuuint64_t)d * 2 * heads};
+  cuuint32_t box[3] = {64, (cuuint32_t)box_heads, (cuuint32_t)box_rows};
+  cuuint32_t estr[3] = {1, 1, 1};
+  return fn(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 3, const_cast<void*>(ptr), dims, strides, box, estr,
+            CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+            CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+}
+
+static bool gqa128_shape(const AttnProblem& a) {
+  if (a.variant != LCA_VARIANT_GQA || a.d_sem != 128 || a.d_pos != 128) return false;
+  const int rep = a.n_q_heads / a.n_kv_heads;
+  return rep >= 1 && rep <= 128 && 128 % rep == 0;
+}
+
+bool attn_tc_supported(const AttnProblem& a) { return gqa128_shape(a); }
+size_t attn_tc_workspace_bytes(const AttnProblem&) { return 0; }
+
+int attn_tc_launch(const AttnProblem& a) {
+  if (!gqa128_shape(a)) return LCA_ERR_UNSUPPORTED_SHAPE;
+  TcParams p;
+  memset(&p, 0, sizeof(p));
+  const int rep = a.n_q_heads / a.n_kv_heads;
+  p.HB = rep; p.TB = ROWS / rep;
+  p.B = a.batch; p.q_len = a.q_len; p.Hq = a.n_q_heads; p.Hkv = a.n_kv_heads; p.L = a.seq_len;
+  p.g = a.group_size; p.w = a.window; p.cap = a.cache_row_capacity; p.n_rep_bias = a.n_rep_bias;
+  p.decode = a.decode; p.n_tok_tiles = (a.q_len + p.TB - 1) / p.TB; p.d_out = a.d_sem;
+  p.scale_log2 = a.softmax_scale * 1.4426950408889634f;
+  p.bias_log2 = a.rep_logit_bias * 1.4426950408889634f;
+  p.out = (bf16*)a.out; p.lse = a.lse; p.cache_rows = a.cache_rows;
+  const long long qrows = (long long)a.batch * a.q_len;
+  bool ok = make_map(&p.q_sem, nullptr, 0, 0, 0, 0, 0);
+  ok = ok && make_map(&p.q_pos, a.q_pos, a.d_pos, a.n_q_heads, qrows, p.HB, p.TB);
+  ok = ok && make_map(&p.kv_sem, a.kv_sem, a.d_sem, a.n_kv_heads, (long long)a.batch * a.seq_len, 1, BN);
+  ok = ok && make_map(&p.kv_pos, a.kv_pos, a.d_pos, a.n_kv_heads, (long long)a.batch * a.seq_len, 1, BN);
+  ok = ok && make_map(&p.cache_sem, a.cache_sem, a.d_sem, a.n_kv_heads, (long long)a.batch * a.cache_row_capacity, 1, BN);
+  ok = ok && make_map(&p.cache_pos, a.cache_pos, a.d_pos, a.n_kv_heads, (long long)a.batch * a.cache_row_capacity, 1, BN);
+  if (!ok) return LCA_ERR_CUDA;
+  using PL = Plan1<0, 2, 2, false, 2>;
+  auto kern = attn_tc1_kernel<0, 2, 2, false, 2>;
+  if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, PL::BYTES) != cudaSuccess)
+    return LCA_ERR_CUDA;
+  dim3 grid(p.n_tok_tiles, a.n_kv_heads, a.batch);
+  kern<<<grid, 192, PL::BYTES, a.stream>>>(p);
+  note_launch();
+  return cudaGetLastError() == cudaSuccess ? LCA_OK : LCA_ERR_CUDA;
+}
+
+int attn_tc_device_status(cudaStream_t stream) {
+  if (cudaStreamSynchronize(stream) != cudaSuccess) return LCA_ERR_CUDA;
+  int st = 0;
+  if (cudaMemcpyFromSymbol(&st, g_tc_status, sizeof(int)) != cudaSuccess) return LCA_ERR_CUDA;
+  if (st != 0) {
+    int zero = 0;
+    cudaMemcpyToSymbol(g_tc_status, &zero, sizeof(int));
+    return LCA_ERR_DEVICE_TIMEOUT;
+  }
+  return LCA_OK;
+}
+
 }  // namespace lca

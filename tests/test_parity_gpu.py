@@ -165,6 +165,7 @@ def test_gqa_small_cases_match_oracle_on_every_row(B, L, Hq, Hkv, g, w):
     cond = B.condense(p, None, d["q"][L - n:], d["v"], d["k"], want_scores=True)
     out, lse = B.prefill_attention(p, None, d["q"], d["v"], d["k"], cond["cache_sem"], cond["cache_pos"],
                                    want_lse=True)
+    assert B.lca_last_device_status() == 0
     ref = Hh.oracle_gqa(inp, g, w, cfg.softmax_scale, rows=np.arange(L))
     Hh.check_condense(one_seq(cond), ref["cond"], kind="gqa")
     Hh.check_outputs(out[0], ref["out"], f"gqa L={L}")
