@@ -8,7 +8,7 @@ import sys
 PKG = os.path.dirname(os.path.abspath(__file__))
 CSRC = os.path.join(PKG, "csrc")
 LIB = os.path.join(PKG, "liblca.so")
-SOURCES = ["lca_api.cu", "condense.cu", "attn_simt.cu", "attn_tc.cu"]
+SOURCES = ["lca_api.cu", "condense.cu", "attn_simt.cu", "attn_tc.cu", "attn_tc2.cu"]
 NVCC_FLAGS = ["-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo", "-O3", "-std=c++17",
               "--use_fast_math", "-Xcompiler", "-fPIC", "-shared"]
 

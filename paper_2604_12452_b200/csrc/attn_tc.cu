@@ -13,6 +13,7 @@
 // softmax, the (rare) rescale of O when the running maximum grows by more than 2^8, and the
 // epilogue.  Every wait is bounded; on expiry the CTA records a code in a global status word,
 // drains and returns.
+#include <cstdio>
 #include <cstring>
 
 #include "lca_common.cuh"
@@ -377,7 +378,7 @@ static EncodeTiledFn encode_fn() {
 }
 
 // bf16 tensor [rows, heads, d] (d contiguous) viewed as 3-D {d, heads, rows}; box {64, box_heads, box_rows}
-static bool make_map(CUtensorMap* map, const void* ptr, int d, int heads, long long rows, int box_heads, int box_rows) {
+bool make_tensor_map_3d(CUtensorMap* map, const void* ptr, int d, int heads, long long rows, int box_heads, int box_rows) {
   EncodeTiledFn fn = encode_fn();
   if (!fn) return false;
   if (!ptr) { memset(map, 0, sizeof(*map)); return true; }
@@ -396,10 +397,15 @@ static bool gqa128_shape(const AttnProblem& a) {
   return rep >= 1 && rep <= 128 && 128 % rep == 0;
 }
 
-bool attn_tc_supported(const AttnProblem& a) { return gqa128_shape(a); }
+bool attn_tc2_supported(const AttnProblem& a);
+int attn_tc2_launch(const AttnProblem& a);
+int attn_tc2_take_status();
+
+bool attn_tc_supported(const AttnProblem& a) { return gqa128_shape(a) || attn_tc2_supported(a); }
 size_t attn_tc_workspace_bytes(const AttnProblem&) { return 0; }
 
 int attn_tc_launch(const AttnProblem& a) {
+  if (attn_tc2_supported(a)) return attn_tc2_launch(a);
   if (!gqa128_shape(a)) return LCA_ERR_UNSUPPORTED_SHAPE;
   TcParams p;
   memset(&p, 0, sizeof(p));
@@ -412,12 +418,12 @@ int attn_tc_launch(const AttnProblem& a) {
   p.bias_log2 = a.rep_logit_bias * 1.4426950408889634f;
   p.out = (bf16*)a.out; p.lse = a.lse; p.cache_rows = a.cache_rows;
   const long long qrows = (long long)a.batch * a.q_len;
-  bool ok = make_map(&p.q_sem, nullptr, 0, 0, 0, 0, 0);
-  ok = ok && make_map(&p.q_pos, a.q_pos, a.d_pos, a.n_q_heads, qrows, p.HB, p.TB);
-  ok = ok && make_map(&p.kv_sem, a.kv_sem, a.d_sem, a.n_kv_heads, (long long)a.batch * a.seq_len, 1, BN);
-  ok = ok && make_map(&p.kv_pos, a.kv_pos, a.d_pos, a.n_kv_heads, (long long)a.batch * a.seq_len, 1, BN);
-  ok = ok && make_map(&p.cache_sem, a.cache_sem, a.d_sem, a.n_kv_heads, (long long)a.batch * a.cache_row_capacity, 1, BN);
-  ok = ok && make_map(&p.cache_pos, a.cache_pos, a.d_pos, a.n_kv_heads, (long long)a.batch * a.cache_row_capacity, 1, BN);
+  bool ok = make_tensor_map_3d(&p.q_sem, nullptr, 0, 0, 0, 0, 0);
+  ok = ok && make_tensor_map_3d(&p.q_pos, a.q_pos, a.d_pos, a.n_q_heads, qrows, p.HB, p.TB);
+  ok = ok && make_tensor_map_3d(&p.kv_sem, a.kv_sem, a.d_sem, a.n_kv_heads, (long long)a.batch * a.seq_len, 1, BN);
+  ok = ok && make_tensor_map_3d(&p.kv_pos, a.kv_pos, a.d_pos, a.n_kv_heads, (long long)a.batch * a.seq_len, 1, BN);
+  ok = ok && make_tensor_map_3d(&p.cache_sem, a.cache_sem, a.d_sem, a.n_kv_heads, (long long)a.batch * a.cache_row_capacity, 1, BN);
+  ok = ok && make_tensor_map_3d(&p.cache_pos, a.cache_pos, a.d_pos, a.n_kv_heads, (long long)a.batch * a.cache_row_capacity, 1, BN);
   if (!ok) return LCA_ERR_CUDA;
   using PL = Plan1<0, 2, 2, false, 2>;
   auto kern = attn_tc1_kernel<0, 2, 2, false, 2>;
@@ -433,6 +439,11 @@ int attn_tc_device_status(cudaStream_t stream) {
   if (cudaStreamSynchronize(stream) != cudaSuccess) return LCA_ERR_CUDA;
   int st = 0;
   if (cudaMemcpyFromSymbol(&st, g_tc_status, sizeof(int)) != cudaSuccess) return LCA_ERR_CUDA;
+  const int st2 = attn_tc2_take_status();
+  if (st2 < 0) return LCA_ERR_CUDA;
+  if (st2 != 0) { fprintf(stderr, "lca: CTA-pair attention kernel gave up waiting (code %d)\n", st2); }
+  if (st != 0) { fprintf(stderr, "lca: attention kernel gave up waiting (code %d)\n", st); }
+  if (st == 0 && st2 != 0) return LCA_ERR_DEVICE_TIMEOUT;
   if (st != 0) {
     int zero = 0;
     cudaMemcpyToSymbol(g_tc_status, &zero, sizeof(int));

@@ -1,0 +1,420 @@
+// MLA-shaped (d_c = 512, d_R = 64) attention over the condensed context on CTA pairs.
+//
+// The absorbed MLA shape does not fit one SM: 128 query rows x 512 fp32 output columns is the
+// whole of tensor memory, and a 128 x 576 bf16 query tile is 144 KB of shared memory.  So two
+// CTAs of a cluster share one tile of 128 query rows (TB tokens x HB heads) and issue
+// tcgen05.mma with cta_group::2:
+//   * each CTA holds 64 of the query rows (72 KB) and, per tile of 128 keys, 64 of the keys with
+//     all 576 columns (B operand of S = Q K^T is split by keys) and all 128 keys of 256 of the
+//     512 value columns (B operand of O += P V is split by output columns);
+//   * S lands as 128 lanes x 64 columns per CTA (lanes 0-63: keys 0-63, lanes 64-127: keys
+//     64-127 of the CTA's 64 rows), O as 128 lanes x 256 columns;
+//   * softmax threads (one per lane) exchange the row maximum of the two key halves through
+//     shared memory, write P as bf16 into a 128-byte-swizzled shared tile (A operand of PV)
+//     and signal the even CTA, whose MMA warp issues every tcgen05.mma for the pair.
+// Everything else (tile walk over representatives then local tokens, boundary-only masks, lazy
+// rescale of O, bounded waits with a status word) follows the single-CTA kernel.
+#include <cstring>
+
+#include "lca_common.cuh"
+#include "tc_common.cuh"
+
+namespace lca {
+using namespace tc;
+
+static __device__ int g_tc2_status = 0;
+
+namespace pair {
+constexpr int BN = 128;                 // keys per tile (64 per CTA for S)
+constexpr int NKC = 9;                  // 64-column key chunks: 8 latent + 1 rope
+constexpr int QCH = 64 * 128;           // bytes of one query chunk  (64 rows)
+constexpr int KCH = 64 * 128;           // bytes of one key chunk    (64 keys)
+constexpr int VCH = 128 * 128;          // bytes of one value chunk  (128 keys x 64 columns)
+constexpr int PCH = 64 * 128;           // bytes of one P chunk      (64 rows x 64 keys)
+constexpr int Q_BYTES = NKC * QCH, K_BYTES = NKC * KCH, V_BYTES = 4 * VCH, P_BYTES = 2 * PCH;
+constexpr int OFF_Q = 0, OFF_K = OFF_Q + Q_BYTES, OFF_V = OFF_K + K_BYTES, OFF_P = OFF_V + V_BYTES;
+constexpr int OFF_BAR = OFF_P + P_BYTES;
+constexpr int OFF_MISC = OFF_BAR + 128, OFF_RED = OFF_BAR + 256;
+constexpr int SMEM_BYTES = OFF_BAR + 256 + 2 * 128 * 4;     // 230656
+constexpr int TM_S0 = 0, TM_S1 = 64, TM_O = 128, TM_COLS = 512;
+constexpr int THREADS = 224;            // warps: 0 K/Q loads, 1 MMA + TMEM, 2-5 softmax, 6 V loads
+constexpr float RESCALE_THRESHOLD = 8.0f;
+static_assert(SMEM_BYTES <= 232448, "shared memory budget of one SM");
+}  // namespace pair
+
+struct Tc2Params {
+  CUtensorMap q_sem, q_pos;       // queries, box of 64 rows
+  CUtensorMap k_sem, k_pos;       // per-token latents / rope keys, box of 64 rows
+  CUtensorMap c_sem, c_pos;       // condensed cache, box of 64 rows
+  CUtensorMap v_sem, cv_sem;      // values (latents) from tokens / cache, box of 128 rows
+  bf16* out; float* lse; const int32_t* cache_rows;
+  int B, q_len, H, L, g, w, cap, n_rep_bias, decode;
+  int HB, TB, n_tok_tiles;
+  float scale_log2, bias_log2;
+};
+
+__global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(pair::THREADS, 1)
+attn_tc2_kernel(const __grid_constant__ Tc2Params p) {
+  using namespace pair;
+  extern __shared__ __align__(1024) unsigned char smem[];
+  const uint32_t base = smem_u32(smem);
+  const uint32_t sQ = base + OFF_Q, sK = base + OFF_K, sV = base + OFF_V, sP = base + OFF_P;
+  const uint32_t bars = base + OFF_BAR;
+  const uint32_t BAR_Q = bars, BAR_KFULL = bars + 8, BAR_KEMPTY = bars + 16, BAR_VFULL = bars + 24,
+                 BAR_VEMPTY = bars + 32, BAR_SFULL0 = bars + 40, BAR_SFULL1 = bars + 48,
+                 BAR_PFULL = bars + 56, BAR_ODONE = bars + 64;
+  volatile uint32_t* tmem_slot = reinterpret_cast<volatile uint32_t*>(smem + OFF_MISC);
+  volatile int* abort_flag = reinterpret_cast<volatile int*>(smem + OFF_MISC + 4);
+  volatile float* red = reinterpret_cast<volatile float*>(smem + OFF_RED);    // [2][128]
+
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const uint32_t rank = cluster_ctarank();       // 0 = even CTA: issues the MMAs, owns the "full" barriers
+
+  // ---- which rows, which key tiles (identical in both CTAs of the pair)
+  const int tile = p.n_tok_tiles - 1 - (int)(blockIdx.x >> 1);       // heaviest query tiles first
+  const int hb = blockIdx.y, b = blockIdx.z;
+  const int t0 = tile * p.TB;
+  const int t1 = min(t0 + p.TB, p.q_len) - 1;
+  const int head0 = hb * p.HB;
+  int nA, nB, first_lo, n_a_lo, n_a_hi;
+  if (p.decode) {
+    n_a_hi = n_a_lo = min(max(p.cache_rows[b], 0), p.cap);
+    first_lo = 0; nB = 0;
+  } else {
+    n_a_lo = reps_visible(t0, p.w, p.g);
+    n_a_hi = reps_visible(t1, p.w, p.g);
+    first_lo = n_a_lo * p.g;
+    nB = (t1 - first_lo + BN) / BN;
+  }
+  nA = (n_a_hi + BN - 1) / BN;
+  const int n_tiles = nA + nB;
+
+  if (threadIdx.x == 0) {
+    mbar_init(BAR_Q, 1); mbar_init(BAR_KFULL, 1); mbar_init(BAR_KEMPTY, 1);
+    mbar_init(BAR_VFULL, 1); mbar_init(BAR_VEMPTY, 1);
+    mbar_init(BAR_SFULL0, 1); mbar_init(BAR_SFULL1, 1);
+    mbar_init(BAR_PFULL, 256); mbar_init(BAR_ODONE, 1);
+    *abort_flag = (base & 1023u) ? 1 : 0;
+    fence_mbar_init();
+  }
+  if (warp == 1) {
+    tmem_alloc_pair(smem_u32((const void*)tmem_slot), TM_COLS);
+    tmem_relinquish_pair();
+  }
+  tc_fence_before();
+  __syncthreads();
+  cluster_sync_all();                              // both CTAs' barriers are initialised
+  tc_fence_after();
+  const uint32_t tmem = *tmem_slot;
+
+  auto fail = [&](int code) {
+    atomicCAS(&g_tc2_status, 0, code);
+    *abort_flag = 1;
+  };
+  if (threadIdx.x == 0 && (base & 1023u)) atomicCAS(&g_tc2_status, 0, 100);
+
+  // rows of this CTA inside the pair tile: global row rg = 64*rank + rl = tl*HB + hl
+  const int row0 = 64 * (int)rank;
+
+  if (warp == 0) {
+    // =============================================== producer: Q once, then the key part of each tile
+    if (lane == 0 && n_tiles > 0 && !*abort_flag) {
+      const uint32_t q_bar = mapa_u32(BAR_Q, 0), k_bar = mapa_u32(BAR_KFULL, 0);
+      if (rank == 0) mbar_expect_tx(BAR_Q, 2 * Q_BYTES);
+      const int qtok = b * p.q_len + t0 + row0 / p.HB, qhead = head0 + row0 % p.HB;
+      for (int c = 0; c < 8; ++c) tma_load_3d_pair(sQ + c * QCH, &p.q_sem, c * 64, qhead, qtok, q_bar);
+      tma_load_3d_pair(sQ + 8 * QCH, &p.q_pos, 0, qhead, qtok, q_bar);
+      for (int j = 0; j < n_tiles; ++j) {
+        const bool isA = j < nA;
+        const int row = (isA ? b * p.cap + j * BN : b * p.L + first_lo + (j - nA) * BN) + 64 * (int)rank;
+        if (!mbar_wait(BAR_KEMPTY, (j & 1) ^ 1, abort_flag)) { fail(ERR_WAIT_KV_EMPTY); break; }
+        if (rank == 0) mbar_expect_tx(BAR_KFULL, 2 * K_BYTES);
+        const CUtensorMap* ms = isA ? &p.c_sem : &p.k_sem;
+        const CUtensorMap* mp = isA ? &p.c_pos : &p.k_pos;
+        for (int c = 0; c < 8; ++c) tma_load_3d_pair(sK + c * KCH, ms, c * 64, 0, row, k_bar);
+        tma_load_3d_pair(sK + 8 * KCH, mp, 0, 0, row, k_bar);
+      }
+    }
+  } else if (warp == 6) {
+    // =============================================== producer: the value part of each tile
+    if (lane == 0 && n_tiles > 0 && !*abort_flag) {
+      const uint32_t v_bar = mapa_u32(BAR_VFULL, 0);
+      for (int j = 0; j < n_tiles; ++j) {
+        const bool isA = j < nA;
+        const int row = isA ? b * p.cap + j * BN : b * p.L + first_lo + (j - nA) * BN;
+        if (!mbar_wait(BAR_VEMPTY, (j & 1) ^ 1, abort_flag)) { fail(ERR_WAIT_KV_EMPTY); break; }
+        if (rank == 0) mbar_expect_tx(BAR_VFULL, 2 * V_BYTES);
+        const CUtensorMap* mv = isA ? &p.cv_sem : &p.v_sem;
+        // output columns of this CTA: [128*rank, +128) of the first 256, then of the second 256
+        for (int i = 0; i < 4; ++i) {
+          const int col = (i >> 1) * 256 + 128 * (int)rank + (i & 1) * 64;
+          tma_load_3d_pair(sV + i * VCH, mv, col, 0, row, v_bar);
+        }
+      }
+    }
+  } else if (warp == 1) {
+    // =============================================== MMA issuer (even CTA only)
+    if (rank == 0 && lane == 0 && n_tiles > 0) {
+      constexpr uint32_t IDESC_S = umma_idesc_bf16(128, BN, false, false);
+      constexpr uint32_t IDESC_PV = umma_idesc_bf16(128, 256, false, true);
+      bool ok = mbar_wait(BAR_Q, 0, abort_flag);
+      if (!ok) fail(ERR_WAIT_Q);
+      auto issue_pv = [&](int j) -> bool {
+        if (!mbar_wait(BAR_PFULL, j & 1, abort_flag)) { fail(ERR_WAIT_P_FULL); return false; }
+        if (!mbar_wait(BAR_VFULL, j & 1, abort_flag)) { fail(ERR_WAIT_KV_FULL); return false; }
+        tc_fence_after();
+#pragma unroll
+        for (int n2 = 0; n2 < 2; ++n2) {
+#pragma unroll
+          for (int k = 0; k < BN / 16; ++k) {
+            const uint64_t ad = umma_desc_sw128(sP + (k >> 2) * PCH + (k & 3) * 32, 16, 1024);
+            const uint64_t bd = umma_desc_sw128(sV + n2 * 2 * VCH + k * 2048, VCH, 1024);
+            umma_ss_pair(tmem + TM_O + n2 * 128, ad, bd, IDESC_PV, (j > 0 || k > 0) ? 1u : 0u);
+          }
+        }
+        umma_commit_pair(BAR_VEMPTY, 3);
+        umma_commit_pair(BAR_ODONE, 3);
+        return true;
+      };
+      for (int j = 0; ok && j < n_tiles; ++j) {
+        ok = mbar_wait(BAR_KFULL, j & 1, abort_flag);
+        if (!ok) { fail(ERR_WAIT_KV_FULL); break; }
+        tc_fence_after();
+        const uint32_t stm = tmem + ((j & 1) ? TM_S1 : TM_S0);
+#pragma unroll
+        for (int c = 0; c < NKC; ++c) {
+#pragma unroll
+          for (int k = 0; k < 4; ++k) {
+            const uint64_t ad = umma_desc_sw128(sQ + c * QCH + k * 32, 16, 1024);
+            const uint64_t bd = umma_desc_sw128(sK + c * KCH + k * 32, 16, 1024);
+            umma_ss_pair(stm, ad, bd, IDESC_S, (c > 0 || k > 0) ? 1u : 0u);
+          }
+        }
+        umma_commit_pair((j & 1) ? BAR_SFULL1 : BAR_SFULL0, 3);
+        umma_commit_pair(BAR_KEMPTY, 3);
+        if (j >= 1) ok = issue_pv(j - 1);
+      }
+      if (ok) issue_pv(n_tiles - 1);
+    }
+  } else {
+    // =============================================== softmax / epilogue: 128 threads, one per TMEM lane
+    const int quarter = warp & 3;
+    const int ln = quarter * 32 + lane;           // TMEM lane
+    const int rl = ln & 63, half = ln >> 6;       // row inside this CTA, key half of the tile
+    const uint32_t lane_base = (uint32_t)(quarter * 32) << 16;
+    const int rg = row0 + rl;
+    const int tl = rg / p.HB, hl = rg % p.HB;
+    const int t_row = t0 + tl;
+    const bool row_valid = t_row < p.q_len;
+    int n_a_row, bias_rows, first_row;
+    if (p.decode) { n_a_row = n_a_hi; bias_rows = min(p.n_rep_bias, n_a_row); first_row = 0; }
+    else { n_a_row = reps_visible(min(t_row, p.q_len - 1), p.w, p.g); bias_rows = n_a_row; first_row = n_a_row * p.g; }
+    const uint32_t pfull_addr = mapa_u32(BAR_PFULL, 0);
+    float m_ref = -INFINITY, l_sum = 0.f;
+    volatile int* fail_word = reinterpret_cast<volatile int*>(smem + OFF_MISC + 16);   // [2], softmax threads only
+    if (ln < 2) fail_word[ln] = 0;
+    asm volatile("bar.sync 1, 128;" ::: "memory");
+    // All 128 threads execute exactly one named barrier per tile, whatever happens: a thread whose
+    // wait expired marks the tile's fail word before the barrier and everybody leaves after it.
+    bool ok = !*abort_flag;
+    for (int j = 0; j < n_tiles; ++j) {
+      if (ok) {
+        ok = mbar_wait((j & 1) ? BAR_SFULL1 : BAR_SFULL0, (j >> 1) & 1, abort_flag);
+        if (!ok && lane == 0) fail(ERR_WAIT_S_FULL);
+      }
+      ok = __all_sync(0xffffffffu, ok);
+      const uint32_t stm = tmem + lane_base + ((j & 1) ? TM_S1 : TM_S0);
+      uint32_t sr[2][32];
+      float tmax = -INFINITY;
+      const bool isA = j < nA;
+      const int tile_key0 = isA ? j * BN : first_lo + (j - nA) * BN;
+      const int key0 = tile_key0 + 64 * half;     // first key of this thread's 64 columns
+      if (ok) {
+        tc_fence_after();
+        tmem_ld32(stm, sr[0]);
+        tmem_ld32(stm + 32, sr[1]);
+        tmem_wait_ld();
+        bool need_mask;
+        int lo, hi;
+        if (isA) { lo = 0; hi = n_a_row - key0 - 1; need_mask = tile_key0 + BN > n_a_lo; }
+        else { lo = first_row - key0; hi = t_row - key0; need_mask = (tile_key0 < n_a_hi * p.g) || (tile_key0 + BN - 1 > t0); }
+        const int blim = isA ? bias_rows - key0 : 0;
+#pragma unroll
+        for (int q = 0; q < 2; ++q) {
+#pragma unroll
+          for (int i = 0; i < 32; ++i) {
+            const int c = q * 32 + i;
+            float s = __uint_as_float(sr[q][i]) * p.scale_log2;
+            if (isA && p.bias_log2 != 0.f && c < blim) s += p.bias_log2;
+            if (need_mask && (c < lo || c > hi)) s = -INFINITY;
+            sr[q][i] = __float_as_uint(s);
+            tmax = fmaxf(tmax, s);
+          }
+        }
+      } else {
+        fail_word[j & 1] = 1;
+      }
+      // the two key halves of a row live in different warps: combine their maxima
+      red[(j & 1) * 128 + ln] = tmax;
+      asm volatile("bar.sync 1, 128;" ::: "memory");
+      if (fail_word[j & 1]) { ok = false; break; }          // uniform over the 128 threads
+      tmax = fmaxf(tmax, red[(j & 1) * 128 + (ln ^ 64)]);
+      bool need = false;
+      float factor = 1.f;
+      if (j == 0) m_ref = tmax;
+      else if (tmax > m_ref + RESCALE_THRESHOLD) { need = true; factor = exp2f(m_ref - tmax); }
+      if (j >= 1) {
+        // P (one buffer) and O are free once P_{j-1} V_{j-1} has completed
+        ok = mbar_wait(BAR_ODONE, (j - 1) & 1, abort_flag);
+        if (!ok && lane == 0) fail(ERR_WAIT_O_DONE);
+        ok = __all_sync(0xffffffffu, ok);
+        if (!ok) continue;                                   // reported at the next tile's barrier
+        tc_fence_after();
+      }
+      if (__any_sync(0xffffffffu, need)) {
+#pragma unroll
+        for (int q = 0; q < 8; ++q) {
+          uint32_t o[32];
+          tmem_ld32(tmem + lane_base + TM_O + q * 32, o);
+          tmem_wait_ld();
+#pragma unroll
+          for (int i = 0; i < 32; ++i) o[i] = __float_as_uint(__uint_as_float(o[i]) * factor);
+          tmem_st32(tmem + lane_base + TM_O + q * 32, o);
+        }
+        tmem_wait_st();
+      }
+      if (need) { l_sum *= factor; m_ref = tmax; }
+      const float m_use = (m_ref == -INFINITY) ? 0.f : m_ref;
+      float rs = 0.f;
+      const uint32_t prow = sP + half * PCH + rl * 128;
+#pragma unroll
+      for (int s8 = 0; s8 < 8; ++s8) {             // 16-byte slot s8 holds keys 8*s8 .. 8*s8+7
+        uint32_t pk[4];
+#pragma unroll
+        for (int i = 0; i < 4; ++i) {
+          const int c = s8 * 8 + 2 * i;
+          const float p0 = exp2f(__uint_as_float(sr[c >> 5][c & 31]) - m_use);
+          const float p1 = exp2f(__uint_as_float(sr[(c + 1) >> 5][(c + 1) & 31]) - m_use);
+          rs += p0 + p1;
+          pk[i] = pack_bf16x2(p0, p1);
+        }
+        const uint32_t a = prow + ((s8 ^ (rl & 7)) << 4);
+        asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(a), "r"(pk[0]), "r"(pk[1]), "r"(pk[2]), "r"(pk[3]) : "memory");
+      }
+      l_sum += rs;
+      fence_proxy_async_smem();                   // P is read by the tensor core (async proxy)
+      tc_fence_before();
+      if (rank == 0) mbar_arrive(BAR_PFULL); else mbar_arrive_cluster(pfull_addr);
+    }
+    // ---- epilogue
+    if (ok && n_tiles > 0) {
+      ok = mbar_wait(BAR_ODONE, (n_tiles - 1) & 1, abort_flag);
+      ok = __all_sync(0xffffffffu, ok);
+      if (!ok && lane == 0) fail(ERR_WAIT_O_DONE);
+    }
+    // total row sum = sum over both key halves
+    red[ln] = l_sum;
+    asm volatile("bar.sync 1, 128;" ::: "memory");
+    const float l_tot = l_sum + red[ln ^ 64];
+    if (ok) {
+      tc_fence_after();
+      const float inv = (n_tiles > 0 && l_tot > 0.f) ? 1.f / l_tot : 0.f;
+      const size_t orow = ((size_t)b * p.q_len + t_row) * p.H + head0 + hl;
+      bf16* dst = p.out + orow * 512;
+#pragma unroll
+      for (int q = 0; q < 8; ++q) {
+        uint32_t o[32];
+        if (n_tiles > 0) { tmem_ld32(tmem + lane_base + TM_O + q * 32, o); tmem_wait_ld(); }
+        else {
+#pragma unroll
+          for (int i = 0; i < 32; ++i) o[i] = 0;
+        }
+        if (row_valid) {
+          // TMEM columns [0,128): output columns 128*half + c ; [128,256): 256 + 128*half + (c-128)
+          const int col = (q >> 2) * 256 + 128 * half + (q & 3) * 32;
+          uint4* d4 = reinterpret_cast<uint4*>(dst + col);
+#pragma unroll
+          for (int v = 0; v < 4; ++v) {
+            uint4 w;
+            w.x = pack_bf16x2(__uint_as_float(o[8 * v + 0]) * inv, __uint_as_float(o[8 * v + 1]) * inv);
+            w.y = pack_bf16x2(__uint_as_float(o[8 * v + 2]) * inv, __uint_as_float(o[8 * v + 3]) * inv);
+            w.z = pack_bf16x2(__uint_as_float(o[8 * v + 4]) * inv, __uint_as_float(o[8 * v + 5]) * inv);
+            w.w = pack_bf16x2(__uint_as_float(o[8 * v + 6]) * inv, __uint_as_float(o[8 * v + 7]) * inv);
+            d4[v] = w;
+          }
+        }
+      }
+      if (p.lse && row_valid && half == 0)
+        p.lse[orow] = (n_tiles > 0 && l_tot > 0.f) ? (m_ref + log2f(l_tot)) * 0.6931471805599453f : -INFINITY;
+    }
+    tc_fence_before();
+  }
+  // ---- teardown
+  if (*abort_flag && (warp == 0 || warp == 6) && lane == 0) {
+    const long long t0c = clock64();
+    while (clock64() - t0c < 2000000ll) { __nanosleep(1000); }
+  }
+  __syncthreads();
+  cluster_sync_all();                              // the peer is done with this CTA's memory and TMEM
+  if (warp == 1) {
+    tc_fence_after();
+    tmem_dealloc_pair(tmem, TM_COLS);
+  }
+}
+
+// ----------------------------------------------------------------------------------- host
+bool make_tensor_map_3d(CUtensorMap* map, const void* ptr, int d, int heads, long long rows, int box_heads, int box_rows);
+
+bool attn_tc2_supported(const AttnProblem& a) {
+  if (a.variant != LCA_VARIANT_MLA || a.d_sem != 512 || a.d_pos != 64 || a.n_kv_heads != 1) return false;
+  if (a.decode) return false;
+  const int H = a.n_q_heads;
+  if (H >= 128) return H % 128 == 0;
+  return H >= 1 && (128 % H) == 0;      // each CTA of the pair takes whole tokens
+}
+
+int attn_tc2_launch(const AttnProblem& a) {
+  using namespace pair;
+  if (!attn_tc2_supported(a)) return LCA_ERR_UNSUPPORTED_SHAPE;
+  Tc2Params p;
+  memset(&p, 0, sizeof(p));
+  const int H = a.n_q_heads;
+  p.HB = H >= 128 ? 128 : H;
+  p.TB = 128 / p.HB;
+  p.B = a.batch; p.q_len = a.q_len; p.H = H; p.L = a.seq_len; p.g = a.group_size; p.w = a.window;
+  p.cap = a.cache_row_capacity; p.n_rep_bias = a.n_rep_bias; p.decode = a.decode;
+  p.n_tok_tiles = (a.q_len + p.TB - 1) / p.TB;
+  p.scale_log2 = a.softmax_scale * 1.4426950408889634f;
+  p.bias_log2 = a.rep_logit_bias * 1.4426950408889634f;
+  p.out = (bf16*)a.out; p.lse = a.lse; p.cache_rows = a.cache_rows;
+  const int hbc = p.HB >= 64 ? 64 : p.HB, tbc = 64 / hbc;
+  const long long qrows = (long long)a.batch * a.q_len, krows = (long long)a.batch * a.seq_len,
+                  crows = (long long)a.batch * a.cache_row_capacity;
+  bool ok = make_tensor_map_3d(&p.q_sem, a.q_sem, 512, H, qrows, hbc, tbc);
+  ok = ok && make_tensor_map_3d(&p.q_pos, a.q_pos, 64, H, qrows, hbc, tbc);
+  ok = ok && make_tensor_map_3d(&p.k_sem, a.kv_sem, 512, 1, krows, 1, 64);
+  ok = ok && make_tensor_map_3d(&p.k_pos, a.kv_pos, 64, 1, krows, 1, 64);
+  ok = ok && make_tensor_map_3d(&p.v_sem, a.kv_sem, 512, 1, krows, 1, 128);
+  ok = ok && make_tensor_map_3d(&p.c_sem, a.cache_sem, 512, 1, crows, 1, 64);
+  ok = ok && make_tensor_map_3d(&p.c_pos, a.cache_pos, 64, 1, crows, 1, 64);
+  ok = ok && make_tensor_map_3d(&p.cv_sem, a.cache_sem, 512, 1, crows, 1, 128);
+  if (!ok) return LCA_ERR_CUDA;
+  if (cudaFuncSetAttribute(attn_tc2_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM_BYTES) != cudaSuccess)
+    return LCA_ERR_CUDA;
+  dim3 grid(2 * p.n_tok_tiles, H >= 128 ? H / 128 : 1, a.batch);
+  attn_tc2_kernel<<<grid, THREADS, SMEM_BYTES, a.stream>>>(p);
+  note_launch();
+  return cudaGetLastError() == cudaSuccess ? LCA_OK : LCA_ERR_CUDA;
+}
+
+int attn_tc2_take_status() {
+  int st = 0;
+  if (cudaMemcpyFromSymbol(&st, g_tc2_status, sizeof(int)) != cudaSuccess) return -1;
+  if (st != 0) {
+    int zero = 0;
+    cudaMemcpyToSymbol(g_tc2_status, &zero, sizeof(int));
+  }
+  return st;
+}
+
+}  // namespace lca

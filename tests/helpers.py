@@ -10,7 +10,8 @@ from oracle import lca_oracle as O
 
 ATOL = 2e-2          # max-abs bound on outputs of unit scale (bf16 inputs, fp32 accumulation)
 RTOL = 2.0 ** -7     # one bf16 ulp of the reference, for outputs larger than unit scale
-MEAN_ATOL = 2e-3
+MEAN_ATOL = 2e-3     # mean-abs bound on outputs of unit scale
+MEAN_RTOL = 2.0 ** -9  # half a bf16 ulp of the mean output magnitude (the output format's own rounding)
 
 
 def f32(x: float) -> float:
@@ -93,7 +94,9 @@ def bf16_ulp_distance(a_bits: np.ndarray, b_bits: np.ndarray) -> np.ndarray:
 
 
 def check_outputs(got: torch.Tensor, ref: np.ndarray, what: str = ""):
-    """max-abs <= ATOL + RTOL*|ref| element-wise and mean-abs <= MEAN_ATOL; returns the stats."""
+    """max-abs <= ATOL + RTOL*|ref| element-wise and mean-abs <= MEAN_ATOL + MEAN_RTOL*mean|ref|;
+    returns the stats.  The relative terms only matter where outputs exceed unit scale (rows that
+    lock onto a x4 "needle" token reach |out| ~ 16, where one bf16 ulp is already 0.06)."""
     g = got.detach().float().cpu().numpy().astype(np.float64)
     err = np.abs(g - ref)
     bound = ATOL + RTOL * np.abs(ref)
@@ -102,7 +105,7 @@ def check_outputs(got: torch.Tensor, ref: np.ndarray, what: str = ""):
                  worst_ratio=worst, max_ref=float(np.abs(ref).max()) if err.size else 0.0)
     assert np.isfinite(g).all(), f"{what}: non-finite output"
     assert worst <= 1.0, f"{what}: {stats}"
-    assert stats["mean_abs"] <= MEAN_ATOL, f"{what}: {stats}"
+    assert stats["mean_abs"] <= MEAN_ATOL + MEAN_RTOL * float(np.abs(ref).mean()), f"{what}: {stats}"
     return stats
 
 
