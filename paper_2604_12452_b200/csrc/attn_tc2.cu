@@ -24,18 +24,32 @@ using namespace tc;
 
 static __device__ int g_tc2_status = 0;
 
+#ifdef LCA_TC2_TRACE
+// Debug build only: per-phase clock64 stamps of one CTA pair (block 0), read back by a test script.
+static __device__ long long g_trace[8192];
+#define TRACE(slot, j) do { if (blockIdx.x < 2 && blockIdx.y == 0 && blockIdx.z == 0 && (j) < 60) g_trace[(int)rank * 4096 + (j) * 16 + (slot)] = clock64(); } while (0)
+#else
+#define TRACE(slot, j) do { } while (0)
+#endif
+
 namespace pair {
 constexpr int BN = 128;                 // keys per tile (64 per CTA for S)
 constexpr int NKC = 9;                  // 64-column key chunks: 8 latent + 1 rope
+#ifndef LCA_TC2_KG
+#define LCA_TC2_KG 3
+#endif
+constexpr int KG = LCA_TC2_KG;          // key chunks per ring slot (one full/empty barrier pair each)
+constexpr int NKG = NKC / KG;
+static_assert(NKC % KG == 0, "key chunks per slot must divide 9");
 constexpr int QCH = 64 * 128;           // bytes of one query chunk  (64 rows)
 constexpr int KCH = 64 * 128;           // bytes of one key chunk    (64 keys)
-constexpr int VCH = 128 * 128;          // bytes of one value chunk  (128 keys x 64 columns)
+constexpr int VCH = 64 * 128;           // bytes of one value chunk  (64 keys x 64 columns)
 constexpr int PCH = 64 * 128;           // bytes of one P chunk      (64 rows x 64 keys)
-constexpr int Q_BYTES = NKC * QCH, K_BYTES = NKC * KCH, V_BYTES = 4 * VCH, P_BYTES = 2 * PCH;
+constexpr int Q_BYTES = NKC * QCH, K_BYTES = NKC * KCH, V_BYTES = 8 * VCH, P_BYTES = 2 * PCH;
 constexpr int OFF_Q = 0, OFF_K = OFF_Q + Q_BYTES, OFF_V = OFF_K + K_BYTES, OFF_P = OFF_V + V_BYTES;
 constexpr int OFF_BAR = OFF_P + P_BYTES;
-constexpr int OFF_MISC = OFF_BAR + 128, OFF_RED = OFF_BAR + 256;
-constexpr int SMEM_BYTES = OFF_BAR + 256 + 2 * 128 * 4;     // 230656
+constexpr int OFF_MISC = OFF_BAR + 256, OFF_RED = OFF_BAR + 512;
+constexpr int SMEM_BYTES = OFF_BAR + 512 + 2 * 128 * 4;     // 230912
 constexpr int TM_S0 = 0, TM_S1 = 64, TM_O = 128, TM_COLS = 512;
 constexpr int THREADS = 224;            // warps: 0 K/Q loads, 1 MMA + TMEM, 2-5 softmax, 6 V loads
 constexpr float RESCALE_THRESHOLD = 8.0f;
@@ -46,7 +60,6 @@ struct Tc2Params {
   CUtensorMap q_sem, q_pos;       // queries, box of 64 rows
   CUtensorMap k_sem, k_pos;       // per-token latents / rope keys, box of 64 rows
   CUtensorMap c_sem, c_pos;       // condensed cache, box of 64 rows
-  CUtensorMap v_sem, cv_sem;      // values (latents) from tokens / cache, box of 128 rows
   bf16* out; float* lse; const int32_t* cache_rows;
   int B, q_len, H, L, g, w, cap, n_rep_bias, decode;
   int HB, TB, n_tok_tiles;
@@ -60,9 +73,15 @@ attn_tc2_kernel(const __grid_constant__ Tc2Params p) {
   const uint32_t base = smem_u32(smem);
   const uint32_t sQ = base + OFF_Q, sK = base + OFF_K, sV = base + OFF_V, sP = base + OFF_P;
   const uint32_t bars = base + OFF_BAR;
-  const uint32_t BAR_Q = bars, BAR_KFULL = bars + 8, BAR_KEMPTY = bars + 16, BAR_VFULL = bars + 24,
-                 BAR_VEMPTY = bars + 32, BAR_SFULL0 = bars + 40, BAR_SFULL1 = bars + 48,
-                 BAR_PFULL = bars + 56, BAR_ODONE = bars + 64;
+  // The key part of a tile is a ring of its nine 64-column chunks and the value part a ring of its
+  // two 64-key halves: a slot is refilled with the next tile's data as soon as the MMAs that read
+  // it have completed, so the loads of tile j+1 run underneath the MMAs of tile j.
+  const uint32_t BAR_Q = bars, BAR_SFULL0 = bars + 8, BAR_SFULL1 = bars + 16, BAR_PFULL = bars + 24,
+                 BAR_ODONE = bars + 32;
+  auto BAR_KFULL = [&](int c) { return bars + 40 + 8 * c; };            // 9
+  auto BAR_KEMPTY = [&](int c) { return bars + 40 + 72 + 8 * c; };      // 9
+  auto BAR_VFULL = [&](int h) { return bars + 40 + 144 + 8 * h; };      // 2
+  auto BAR_VEMPTY = [&](int h) { return bars + 40 + 160 + 8 * h; };     // 2
   volatile uint32_t* tmem_slot = reinterpret_cast<volatile uint32_t*>(smem + OFF_MISC);
   volatile int* abort_flag = reinterpret_cast<volatile int*>(smem + OFF_MISC + 4);
   volatile float* red = reinterpret_cast<volatile float*>(smem + OFF_RED);    // [2][128]
@@ -90,8 +109,9 @@ attn_tc2_kernel(const __grid_constant__ Tc2Params p) {
   const int n_tiles = nA + nB;
 
   if (threadIdx.x == 0) {
-    mbar_init(BAR_Q, 1); mbar_init(BAR_KFULL, 1); mbar_init(BAR_KEMPTY, 1);
-    mbar_init(BAR_VFULL, 1); mbar_init(BAR_VEMPTY, 1);
+    mbar_init(BAR_Q, 1);
+    for (int c = 0; c < NKG; ++c) { mbar_init(BAR_KFULL(c), 1); mbar_init(BAR_KEMPTY(c), 1); }
+    for (int h = 0; h < 2; ++h) { mbar_init(BAR_VFULL(h), 1); mbar_init(BAR_VEMPTY(h), 1); }
     mbar_init(BAR_SFULL0, 1); mbar_init(BAR_SFULL1, 1);
     mbar_init(BAR_PFULL, 256); mbar_init(BAR_ODONE, 1);
     *abort_flag = (base & 1023u) ? 1 : 0;
@@ -119,7 +139,7 @@ attn_tc2_kernel(const __grid_constant__ Tc2Params p) {
   if (warp == 0) {
     // =============================================== producer: Q once, then the key part of each tile
     if (lane == 0 && n_tiles > 0 && !*abort_flag) {
-      const uint32_t q_bar = mapa_u32(BAR_Q, 0), k_bar = mapa_u32(BAR_KFULL, 0);
+      const uint32_t q_bar = mapa_u32(BAR_Q, 0);
       if (rank == 0) mbar_expect_tx(BAR_Q, 2 * Q_BYTES);
       const int qtok = b * p.q_len + t0 + row0 / p.HB, qhead = head0 + row0 % p.HB;
       for (int c = 0; c < 8; ++c) tma_load_3d_pair(sQ + c * QCH, &p.q_sem, c * 64, qhead, qtok, q_bar);
@@ -127,29 +147,38 @@ attn_tc2_kernel(const __grid_constant__ Tc2Params p) {
       for (int j = 0; j < n_tiles; ++j) {
         const bool isA = j < nA;
         const int row = (isA ? b * p.cap + j * BN : b * p.L + first_lo + (j - nA) * BN) + 64 * (int)rank;
-        if (!mbar_wait(BAR_KEMPTY, (j & 1) ^ 1, abort_flag)) { fail(ERR_WAIT_KV_EMPTY); break; }
-        if (rank == 0) mbar_expect_tx(BAR_KFULL, 2 * K_BYTES);
         const CUtensorMap* ms = isA ? &p.c_sem : &p.k_sem;
         const CUtensorMap* mp = isA ? &p.c_pos : &p.k_pos;
-        for (int c = 0; c < 8; ++c) tma_load_3d_pair(sK + c * KCH, ms, c * 64, 0, row, k_bar);
-        tma_load_3d_pair(sK + 8 * KCH, mp, 0, 0, row, k_bar);
+        bool good = true;
+        for (int gk = 0; gk < NKG; ++gk) {
+          if (!mbar_wait(BAR_KEMPTY(gk), (j & 1) ^ 1, abort_flag)) { fail(ERR_WAIT_KV_EMPTY); good = false; break; }
+          if (rank == 0) mbar_expect_tx(BAR_KFULL(gk), 2 * KG * KCH);
+          const uint32_t k_bar = mapa_u32(BAR_KFULL(gk), 0);
+          for (int c = gk * KG; c < (gk + 1) * KG; ++c)
+            tma_load_3d_pair(sK + c * KCH, c < 8 ? ms : mp, c < 8 ? c * 64 : 0, 0, row, k_bar);
+        }
+        if (!good) break;
       }
     }
   } else if (warp == 6) {
     // =============================================== producer: the value part of each tile
     if (lane == 0 && n_tiles > 0 && !*abort_flag) {
-      const uint32_t v_bar = mapa_u32(BAR_VFULL, 0);
       for (int j = 0; j < n_tiles; ++j) {
         const bool isA = j < nA;
         const int row = isA ? b * p.cap + j * BN : b * p.L + first_lo + (j - nA) * BN;
-        if (!mbar_wait(BAR_VEMPTY, (j & 1) ^ 1, abort_flag)) { fail(ERR_WAIT_KV_EMPTY); break; }
-        if (rank == 0) mbar_expect_tx(BAR_VFULL, 2 * V_BYTES);
-        const CUtensorMap* mv = isA ? &p.cv_sem : &p.v_sem;
-        // output columns of this CTA: [128*rank, +128) of the first 256, then of the second 256
-        for (int i = 0; i < 4; ++i) {
-          const int col = (i >> 1) * 256 + 128 * (int)rank + (i & 1) * 64;
-          tma_load_3d_pair(sV + i * VCH, mv, col, 0, row, v_bar);
+        const CUtensorMap* mv = isA ? &p.c_sem : &p.k_sem;
+        bool good = true;
+        for (int kh = 0; kh < 2; ++kh) {            // keys [64*kh, 64*kh+64) of the tile
+          if (!mbar_wait(BAR_VEMPTY(kh), (j & 1) ^ 1, abort_flag)) { fail(ERR_WAIT_KV_EMPTY); good = false; break; }
+          if (rank == 0) mbar_expect_tx(BAR_VFULL(kh), 2 * 4 * VCH);
+          const uint32_t v_bar = mapa_u32(BAR_VFULL(kh), 0);
+          // output columns of this CTA: [128*rank, +128) of the first 256, then of the second 256
+          for (int i = 0; i < 4; ++i) {
+            const int col = (i >> 1) * 256 + 128 * (int)rank + (i & 1) * 64;
+            tma_load_3d_pair(sV + (kh * 4 + i) * VCH, mv, col, 0, row + 64 * kh, v_bar);
+          }
         }
+        if (!good) break;
       }
     }
   } else if (warp == 1) {
@@ -160,38 +189,52 @@ attn_tc2_kernel(const __grid_constant__ Tc2Params p) {
       bool ok = mbar_wait(BAR_Q, 0, abort_flag);
       if (!ok) fail(ERR_WAIT_Q);
       auto issue_pv = [&](int j) -> bool {
+        TRACE(3, j);
         if (!mbar_wait(BAR_PFULL, j & 1, abort_flag)) { fail(ERR_WAIT_P_FULL); return false; }
-        if (!mbar_wait(BAR_VFULL, j & 1, abort_flag)) { fail(ERR_WAIT_KV_FULL); return false; }
-        tc_fence_after();
+        TRACE(4, j);
 #pragma unroll
-        for (int n2 = 0; n2 < 2; ++n2) {
+        for (int kh = 0; kh < 2; ++kh) {
+          if (!mbar_wait(BAR_VFULL(kh), j & 1, abort_flag)) { fail(ERR_WAIT_KV_FULL); return false; }
+          tc_fence_after();
 #pragma unroll
-          for (int k = 0; k < BN / 16; ++k) {
-            const uint64_t ad = umma_desc_sw128(sP + (k >> 2) * PCH + (k & 3) * 32, 16, 1024);
-            const uint64_t bd = umma_desc_sw128(sV + n2 * 2 * VCH + k * 2048, VCH, 1024);
-            umma_ss_pair(tmem + TM_O + n2 * 128, ad, bd, IDESC_PV, (j > 0 || k > 0) ? 1u : 0u);
+          for (int n2 = 0; n2 < 2; ++n2) {
+#pragma unroll
+            for (int k = 0; k < 4; ++k) {
+              const uint64_t ad = umma_desc_sw128(sP + kh * PCH + k * 32, 16, 1024);
+              const uint64_t bd = umma_desc_sw128(sV + (kh * 4 + n2 * 2) * VCH + k * 2048, VCH, 1024);
+              umma_ss_pair(tmem + TM_O + n2 * 128, ad, bd, IDESC_PV, (j > 0 || kh > 0 || k > 0) ? 1u : 0u);
+            }
           }
+          umma_commit_pair(BAR_VEMPTY(kh), 3);
         }
-        umma_commit_pair(BAR_VEMPTY, 3);
         umma_commit_pair(BAR_ODONE, 3);
+        TRACE(5, j);
         return true;
       };
       for (int j = 0; ok && j < n_tiles; ++j) {
-        ok = mbar_wait(BAR_KFULL, j & 1, abort_flag);
-        if (!ok) { fail(ERR_WAIT_KV_FULL); break; }
-        tc_fence_after();
         const uint32_t stm = tmem + ((j & 1) ? TM_S1 : TM_S0);
+        TRACE(0, j);
 #pragma unroll
-        for (int c = 0; c < NKC; ++c) {
+        for (int gk = 0; gk < NKG; ++gk) {
+          ok = mbar_wait(BAR_KFULL(gk), j & 1, abort_flag);
+          if (gk == 0) TRACE(1, j);
+          if (!ok) { fail(ERR_WAIT_KV_FULL); break; }
+          tc_fence_after();
 #pragma unroll
-          for (int k = 0; k < 4; ++k) {
-            const uint64_t ad = umma_desc_sw128(sQ + c * QCH + k * 32, 16, 1024);
-            const uint64_t bd = umma_desc_sw128(sK + c * KCH + k * 32, 16, 1024);
-            umma_ss_pair(stm, ad, bd, IDESC_S, (c > 0 || k > 0) ? 1u : 0u);
+          for (int cc = 0; cc < KG; ++cc) {
+            const int c = gk * KG + cc;
+#pragma unroll
+            for (int k = 0; k < 4; ++k) {
+              const uint64_t ad = umma_desc_sw128(sQ + c * QCH + k * 32, 16, 1024);
+              const uint64_t bd = umma_desc_sw128(sK + c * KCH + k * 32, 16, 1024);
+              umma_ss_pair(stm, ad, bd, IDESC_S, (c > 0 || k > 0) ? 1u : 0u);
+            }
           }
+          umma_commit_pair(BAR_KEMPTY(gk), 3);
         }
+        if (!ok) break;
         umma_commit_pair((j & 1) ? BAR_SFULL1 : BAR_SFULL0, 3);
-        umma_commit_pair(BAR_KEMPTY, 3);
+        TRACE(2, j);
         if (j >= 1) ok = issue_pv(j - 1);
       }
       if (ok) issue_pv(n_tiles - 1);
@@ -218,10 +261,12 @@ attn_tc2_kernel(const __grid_constant__ Tc2Params p) {
     // wait expired marks the tile's fail word before the barrier and everybody leaves after it.
     bool ok = !*abort_flag;
     for (int j = 0; j < n_tiles; ++j) {
+      if (ln == 0) TRACE(8, j);
       if (ok) {
         ok = mbar_wait((j & 1) ? BAR_SFULL1 : BAR_SFULL0, (j >> 1) & 1, abort_flag);
         if (!ok && lane == 0) fail(ERR_WAIT_S_FULL);
       }
+      if (ln == 0) TRACE(9, j);
       ok = __all_sync(0xffffffffu, ok);
       const uint32_t stm = tmem + lane_base + ((j & 1) ? TM_S1 : TM_S0);
       uint32_t sr[2][32];
@@ -263,6 +308,7 @@ attn_tc2_kernel(const __grid_constant__ Tc2Params p) {
       float factor = 1.f;
       if (j == 0) m_ref = tmax;
       else if (tmax > m_ref + RESCALE_THRESHOLD) { need = true; factor = exp2f(m_ref - tmax); }
+      if (ln == 0) TRACE(10, j);
       if (j >= 1) {
         // P (one buffer) and O are free once P_{j-1} V_{j-1} has completed
         ok = mbar_wait(BAR_ODONE, (j - 1) & 1, abort_flag);
@@ -271,6 +317,7 @@ attn_tc2_kernel(const __grid_constant__ Tc2Params p) {
         if (!ok) continue;                                   // reported at the next tile's barrier
         tc_fence_after();
       }
+      if (ln == 0) TRACE(11, j);
       if (__any_sync(0xffffffffu, need)) {
 #pragma unroll
         for (int q = 0; q < 8; ++q) {
@@ -305,6 +352,7 @@ attn_tc2_kernel(const __grid_constant__ Tc2Params p) {
       fence_proxy_async_smem();                   // P is read by the tensor core (async proxy)
       tc_fence_before();
       if (rank == 0) mbar_arrive(BAR_PFULL); else mbar_arrive_cluster(pfull_addr);
+      if (ln == 0) TRACE(12, j);
     }
     // ---- epilogue
     if (ok && n_tiles > 0) {
@@ -394,10 +442,8 @@ int attn_tc2_launch(const AttnProblem& a) {
   ok = ok && make_tensor_map_3d(&p.q_pos, a.q_pos, 64, H, qrows, hbc, tbc);
   ok = ok && make_tensor_map_3d(&p.k_sem, a.kv_sem, 512, 1, krows, 1, 64);
   ok = ok && make_tensor_map_3d(&p.k_pos, a.kv_pos, 64, 1, krows, 1, 64);
-  ok = ok && make_tensor_map_3d(&p.v_sem, a.kv_sem, 512, 1, krows, 1, 128);
   ok = ok && make_tensor_map_3d(&p.c_sem, a.cache_sem, 512, 1, crows, 1, 64);
   ok = ok && make_tensor_map_3d(&p.c_pos, a.cache_pos, 64, 1, crows, 1, 64);
-  ok = ok && make_tensor_map_3d(&p.cv_sem, a.cache_sem, 512, 1, crows, 1, 128);
   if (!ok) return LCA_ERR_CUDA;
   if (cudaFuncSetAttribute(attn_tc2_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM_BYTES) != cudaSuccess)
     return LCA_ERR_CUDA;
@@ -406,6 +452,12 @@ int attn_tc2_launch(const AttnProblem& a) {
   note_launch();
   return cudaGetLastError() == cudaSuccess ? LCA_OK : LCA_ERR_CUDA;
 }
+
+#ifdef LCA_TC2_TRACE
+extern "C" int lca_debug_read_trace(long long* dst) {
+  return cudaMemcpyFromSymbol(dst, g_trace, sizeof(long long) * 8192) == cudaSuccess ? 0 : -1;
+}
+#endif
 
 int attn_tc2_take_status() {
   int st = 0;
