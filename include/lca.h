@@ -46,7 +46,8 @@ typedef enum lca_status {
   LCA_ERR_MISALIGNED = -3,         /* a tensor pointer that is not 16-byte aligned               */
   LCA_ERR_WORKSPACE_TOO_SMALL = -4,
   LCA_ERR_CUDA = -5,               /* a CUDA runtime call or a launch failed                     */
-  LCA_ERR_DEVICE_TIMEOUT = -6      /* a bounded device-side wait expired (reported by lca_last_device_status) */
+  LCA_ERR_DEVICE_TIMEOUT = -6,     /* a bounded device-side wait expired (reported by lca_last_device_status) */
+  LCA_ERR_STATIC_SCRATCH_EXCEEDED = -7  /* lca_condense_static_scratch: the problem needs more than LCA_STATIC_SCRATCH_BYTES */
 } lca_status;
 
 enum { LCA_VARIANT_MLA = 0, LCA_VARIANT_GQA = 1 };
@@ -103,6 +104,36 @@ int lca_condense(const lca_params* p, const void* q_tail_sem, const void* q_tail
                  int64_t q_tail_batch_stride, const float* qbar_opt, const void* kv_sem,
                  const void* kv_pos, void* cache_sem, void* cache_pos, int32_t* anchor_idx,
                  double* scores_opt, void* ws, size_t ws_bytes, void* stream);
+
+/* The same condensation for callers that cannot allocate device memory.  (The paper has no
+ * counterpart: this entry point exists only for the way the library is called.)
+ *
+ * Who needs it: code that runs where cudaMalloc is off limits -- a plug-in inside a serving
+ * process whose memory is handed out once at start-up by its own pool, a real-time loop that
+ * may not take the allocator's lock, a host thread that is not allowed to synchronise the
+ * device (cudaMalloc and cudaFree may do that).  lca_condense needs a few hundred KB of scratch
+ * for the summary query; here that scratch is a fixed array of LCA_STATIC_SCRATCH_BYTES that is
+ * part of the library image on every GPU that loads it, from load until the process exits.
+ *
+ * Arguments, results and arithmetic are those of lca_condense without `ws` / `ws_bytes`; the
+ * output is bit-identical.  The call allocates nothing and frees nothing.
+ *   - Limit: lca_workspace_bytes(p, LCA_WS_CONDENSE) must not exceed LCA_STATIC_SCRATCH_BYTES
+ *     (1 MiB: one MLA sequence with up to 128 heads and 64 summary positions uses 0.6 MB; a
+ *     batch of 64 such sequences does not fit).  Larger problems return
+ *     LCA_ERR_STATIC_SCRATCH_EXCEEDED and launch nothing: use lca_condense with your own buffer.
+ *   - The first call on each device looks up the array's device address (the device that is
+ *     current at the call).  Make that first call outside any stream capture; later calls on the
+ *     same device do no set-up work.
+ *   - All calls on one device share the one array, and it keeps whatever the previous call left
+ *     there.  Nothing in it has to start at zero: every element a call reads was written earlier
+ *     in that same call.  Two calls that may overlap on the GPU (different streams, no
+ *     dependency between them) race on the array and give wrong results; order them. */
+#define LCA_STATIC_SCRATCH_BYTES (1u << 20)
+int lca_condense_static_scratch(const lca_params* p, const void* q_tail_sem, const void* q_tail_pos,
+                                int64_t q_tail_batch_stride, const float* qbar_opt,
+                                const void* kv_sem, const void* kv_pos, void* cache_sem,
+                                void* cache_pos, int32_t* anchor_idx, double* scores_opt,
+                                void* stream);
 
 /* Prefill attention, Eq. 10 evaluated at every prefix length (causal): the query at position t
  * attends to the representatives of the m_t = floor((t+1-w)/g) groups that lie wholly outside its

@@ -21,6 +21,8 @@ from . import build as _build
 LCA_OK = 0
 LCA_VARIANT_MLA, LCA_VARIANT_GQA = 0, 1
 LCA_WS_CONDENSE, LCA_WS_PREFILL, LCA_WS_DECODE = 0, 1, 2
+LCA_STATIC_SCRATCH_BYTES = 1 << 20
+LCA_ERR_STATIC_SCRATCH_EXCEEDED = -7
 ATTN_AUTO, ATTN_SCALAR, ATTN_TENSOR = 0, 1, 2
 
 
@@ -59,6 +61,8 @@ def _load() -> C.CDLL:
     lib.lca_workspace_bytes.argtypes = [P, i32]
     lib.lca_condense.restype = C.c_int
     lib.lca_condense.argtypes = [P, vp, vp, i64, vp, vp, vp, vp, vp, vp, vp, vp, sz, vp]
+    lib.lca_condense_static_scratch.restype = C.c_int
+    lib.lca_condense_static_scratch.argtypes = [P, vp, vp, i64, vp, vp, vp, vp, vp, vp, vp, vp]
     lib.lca_prefill_attention.restype = C.c_int
     lib.lca_prefill_attention.argtypes = [P, vp, vp, vp, vp, vp, vp, vp, vp, vp, sz, vp]
     lib.lca_decode_attention.restype = C.c_int
@@ -129,6 +133,16 @@ def lca_condense(params, q_tail_sem, q_tail_pos, q_tail_batch_stride, qbar_opt, 
                                  int(q_tail_batch_stride), _ptr(qbar_opt), _ptr(kv_sem), _ptr(kv_pos),
                                  _ptr(cache_sem), _ptr(cache_pos), _ptr(anchor_idx), _ptr(scores_opt),
                                  _ptr(ws), wsb, _stream(stream)))
+
+
+def lca_condense_static_scratch(params, q_tail_sem, q_tail_pos, q_tail_batch_stride, qbar_opt, kv_sem,
+                                kv_pos, cache_sem, cache_pos, anchor_idx, scores_opt, stream=None) -> int:
+    """lca_condense without a workspace argument: the scratch is a fixed array inside the library
+    (for callers that must not allocate device memory).  Same outputs, bit for bit."""
+    return int(_lib.lca_condense_static_scratch(C.byref(params), _ptr(q_tail_sem), _ptr(q_tail_pos),
+                                                int(q_tail_batch_stride), _ptr(qbar_opt), _ptr(kv_sem),
+                                                _ptr(kv_pos), _ptr(cache_sem), _ptr(cache_pos),
+                                                _ptr(anchor_idx), _ptr(scores_opt), _stream(stream)))
 
 
 def lca_prefill_attention(params, q_sem, q_pos, kv_sem, kv_pos, cache_sem, cache_pos, out, lse_opt,

@@ -7,6 +7,8 @@
 // are written straight into the condensed cache.  All arithmetic is fp64: it costs a few percent
 // of the fp64 pipe at HBM speed and makes the arg-max and the bf16 rounding of c_rep follow the
 // exact scores rather than an fp32 accumulation order.
+#include <mutex>
+
 #include "lca_common.cuh"
 
 namespace lca {
@@ -287,6 +289,27 @@ int condense_launch(const CondenseLaunch& c) {
     note_launch(2);
   }
   return cudaGetLastError() == cudaSuccess ? LCA_OK : LCA_ERR_CUDA;
+}
+
+// ------------------------------------------------------------------ fixed scratch (no allocation)
+// Scratch of lca_condense_static_scratch: part of the library image on every device.  In host
+// code the name below is only a handle; the device address comes from cudaGetSymbolAddress, asked
+// once per device with that device current, and that address is what the kernels receive.
+static __device__ __align__(256) unsigned char g_condense_static_scratch[LCA_STATIC_SCRATCH_BYTES];
+
+int condense_static_scratch_address(void** out) {
+  static std::mutex mu;
+  static void* addr[64] = {};
+  int dev = 0;
+  if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return LCA_ERR_CUDA;
+  std::lock_guard<std::mutex> lock(mu);
+  if (!addr[dev]) {
+    void* p = nullptr;
+    if (cudaGetSymbolAddress(&p, g_condense_static_scratch) != cudaSuccess || !p) return LCA_ERR_CUDA;
+    addr[dev] = p;
+  }
+  *out = addr[dev];
+  return LCA_OK;
 }
 
 }  // namespace lca

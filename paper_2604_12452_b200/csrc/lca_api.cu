@@ -59,6 +59,7 @@ const char* lca_status_string(int s) {
     case LCA_ERR_WORKSPACE_TOO_SMALL: return "workspace too small";
     case LCA_ERR_CUDA: return "CUDA error";
     case LCA_ERR_DEVICE_TIMEOUT: return "device-side wait timed out";
+    case LCA_ERR_STATIC_SCRATCH_EXCEEDED: return "problem needs more scratch than the fixed LCA_STATIC_SCRATCH_BYTES array; use lca_condense with a caller buffer";
     default: return "unknown status";
   }
 }
@@ -120,6 +121,21 @@ int lca_condense(const lca_params* p, const void* q_tail_sem, const void* q_tail
   CondenseLaunch c = {p, q_tail_sem, q_tail_pos, q_tail_batch_stride, qbar_opt, kv_sem, kv_pos,
                       cache_sem, cache_pos, anchor_idx, scores_opt, ws, ws_bytes, (cudaStream_t)stream};
   return condense_launch(c);
+}
+
+int lca_condense_static_scratch(const lca_params* p, const void* q_tail_sem, const void* q_tail_pos,
+                                int64_t q_tail_batch_stride, const float* qbar_opt,
+                                const void* kv_sem, const void* kv_pos, void* cache_sem,
+                                void* cache_pos, int32_t* anchor_idx, double* scores_opt,
+                                void* stream) {
+  int st = check_params(p, true);
+  if (st != LCA_OK) return st;
+  if (condense_workspace_bytes(p) > (size_t)LCA_STATIC_SCRATCH_BYTES) return LCA_ERR_STATIC_SCRATCH_EXCEEDED;
+  void* scratch = nullptr;
+  st = condense_static_scratch_address(&scratch);     // first call on a device: one address look-up
+  if (st != LCA_OK) return st;
+  return lca_condense(p, q_tail_sem, q_tail_pos, q_tail_batch_stride, qbar_opt, kv_sem, kv_pos,
+                      cache_sem, cache_pos, anchor_idx, scores_opt, scratch, LCA_STATIC_SCRATCH_BYTES, stream);
 }
 
 int lca_prefill_attention(const lca_params* p, const void* q_sem, const void* q_pos,
