@@ -398,12 +398,11 @@ static bool gqa128_shape(const AttnProblem& a) {
 }
 
 bool attn_tc2_supported(const AttnProblem& a);
-size_t attn_tc2_workspace_bytes(const AttnProblem& a);
 int attn_tc2_launch(const AttnProblem& a);
 int attn_tc2_take_status();
 
 bool attn_tc_supported(const AttnProblem& a) { return gqa128_shape(a) || attn_tc2_supported(a); }
-size_t attn_tc_workspace_bytes(const AttnProblem& a) { return attn_tc2_supported(a) ? attn_tc2_workspace_bytes(a) : 0; }
+size_t attn_tc_workspace_bytes(const AttnProblem&) { return 0; }
 
 int attn_tc_launch(const AttnProblem& a) {
   if (attn_tc2_supported(a)) return attn_tc2_launch(a);
