@@ -2,11 +2,11 @@
 // weighted pooling (Eq. 7), anchor selection (Eq. 8) and the local-window copy (Eq. 9).
 //
 // The work is HBM-bound (about 2 flop per byte): every history token is read from global memory
-// exactly once into shared memory (one CTA per group), scored against the summary query,
-// soft-maxed within the group, pooled, and the representative plus the anchor's positional row
-// are written straight into the condensed cache.  All arithmetic is fp64: it costs a few percent
-// of the fp64 pipe at HBM speed and makes the arg-max and the bf16 rounding of c_rep follow the
-// exact scores rather than an fp32 accumulation order.
+// exactly once into shared memory, scored against the summary query, soft-maxed within its
+// group, pooled, and the representative plus the anchor's positional row are written straight
+// into the condensed cache.  The summary query and the scores are fp64, so the arg-max follows
+// the exact scores rather than an fp32 accumulation order; the softmax weights and the pooling
+// are fp32 (the fp64 pipe could not keep up with HBM for both), c_rep is rounded once to bf16.
 #include <mutex>
 
 #include "lca_common.cuh"
@@ -15,35 +15,52 @@ namespace lca {
 
 static const int QBAR_ROWS_PER_CHUNK = 64;
 static const int QBAR_THREADS = 128;
-static const int CONDENSE_THREADS = 256;
+static const int CONDENSE_THREADS = 512;
 
 // ---------------------------------------------------------------------------- summary query
-// Partial sums of the query tail.  Rows of one KV head = (position, query head in its group).
-// grid (nchunks, Hkv, B); each thread owns column pairs tid, tid+T, ...
+// Partial sums of the query tail.  Rows of one KV head = (position, query head in its group);
+// a chunk is QBAR_ROWS_PER_CHUNK rows.  grid (nchunks, Hkv, B).  A thread owns one 16-byte piece
+// (8 columns) of the key dimension and every row_lanes-th row of the chunk, so that consecutive
+// threads read a whole query row and each thread has many independent loads in flight; the
+// row lanes are then added up through shared memory in a fixed order.
 __global__ void qbar_partial_kernel(const bf16* __restrict__ q_sem, const bf16* __restrict__ q_pos,
                                     int64_t batch_stride_rows, int n_pos, int Hq, int Hkv, int d_sem,
-                                    int d_pos, int sem_in_logit, double* __restrict__ partial) {
+                                    int d_pos, int sem_in_logit, int row_lanes, double* __restrict__ partial) {
+  extern __shared__ double s_part[];                     // [row_lanes][dk]
   const int chunk = blockIdx.x, hk = blockIdx.y, b = blockIdx.z;
   const int rep = Hq / Hkv;
   const int n_rows = n_pos * rep;
   const int r0 = chunk * QBAR_ROWS_PER_CHUNK;
   const int r1 = min(n_rows, r0 + QBAR_ROWS_PER_CHUNK);
   const int dk = (sem_in_logit ? d_sem : 0) + d_pos;
-  const int sem_pairs = sem_in_logit ? d_sem / 2 : 0;
-  double* dst = partial + (((size_t)b * Hkv + hk) * gridDim.x + chunk) * dk;
-  for (int pr = threadIdx.x; pr < dk / 2; pr += blockDim.x) {
-    double a0 = 0.0, a1 = 0.0;
-    for (int r = r0; r < r1; ++r) {
+  const int pieces = dk / 8, sem_pieces = sem_in_logit ? d_sem / 8 : 0;
+  const int pc = threadIdx.x % pieces, rl = threadIdx.x / pieces;
+  double acc[8];
+#pragma unroll
+  for (int i = 0; i < 8; ++i) acc[i] = 0.0;
+  if (rl < row_lanes) {
+#pragma unroll 4
+    for (int r = r0 + rl; r < r1; r += row_lanes) {
       const int pos = r / rep, head = hk * rep + r % rep;
       const size_t row = ((size_t)b * batch_stride_rows + pos) * Hq + head;
-      const bf16* src = (pr < sem_pairs) ? q_sem + row * d_sem + 2 * pr
-                                         : q_pos + row * d_pos + 2 * (pr - sem_pairs);
-      const bf162 v = *reinterpret_cast<const bf162*>(src);
-      a0 += (double)__low2float(v);
-      a1 += (double)__high2float(v);
+      const bf16* src = (pc < sem_pieces) ? q_sem + row * d_sem + 8 * pc : q_pos + row * d_pos + 8 * (pc - sem_pieces);
+      const uint4 v = *reinterpret_cast<const uint4*>(src);
+      const unsigned w[4] = {v.x, v.y, v.z, v.w};
+#pragma unroll
+      for (int i = 0; i < 4; ++i) {
+        acc[2 * i] += (double)__uint_as_float(w[i] << 16);
+        acc[2 * i + 1] += (double)__uint_as_float(w[i] & 0xffff0000u);
+      }
     }
-    dst[2 * pr] = a0;
-    dst[2 * pr + 1] = a1;
+#pragma unroll
+    for (int i = 0; i < 8; ++i) s_part[(size_t)rl * dk + 8 * pc + i] = acc[i];
+  }
+  __syncthreads();
+  double* dst = partial + (((size_t)b * Hkv + hk) * gridDim.x + chunk) * dk;
+  for (int c = threadIdx.x; c < dk; c += blockDim.x) {
+    double sum = 0.0;
+    for (int l = 0; l < row_lanes; ++l) sum += s_part[(size_t)l * dk + c];
+    dst[c] = sum;
   }
 }
 
@@ -70,6 +87,7 @@ struct CondenseArgs {
   const bf16* kv_sem; const bf16* kv_pos; const double* qbar;
   bf16* cache_sem; bf16* cache_pos; int32_t* anchor; double* scores;
   int L, Hkv, d_sem, d_pos, g, m, cache_rows, sem_in_logit;
+  long long n_groups;          // B * Hkv * m
   double scale;
 };
 
@@ -77,128 +95,365 @@ __device__ inline void cp_async16(void* smem_dst, const void* gmem_src) {
   unsigned s = (unsigned)__cvta_generic_to_shared(smem_dst);
   asm volatile("cp.async.cg.shared.global [%0], [%1], 16;\n" ::"r"(s), "l"(gmem_src) : "memory");
 }
-__device__ inline void cp_async_wait_all() {
-  asm volatile("cp.async.commit_group;\ncp.async.wait_group 0;\n" ::: "memory");
-}
 
-// grid (m, Hkv, B), CONDENSE_THREADS threads, dynamic smem = tile + q_bar + scores + alpha.
-__global__ void __launch_bounds__(CONDENSE_THREADS)
+// Persistent CTAs, one per SM; group index = (b * Hkv + hk) * m + j.  Two shared-memory stages:
+// while a group is scored and pooled, the next one streams in with 16-byte cp.async copies, so
+// every history byte is read from HBM once and the loads never wait for the arithmetic.
+// A stage holds the g tokens [g][d_sem] and [g][d_pos] in bf16 and the summary query in fp64.
+// Scores stay in fp64 (the arg-max must follow the exact scores); the group softmax and the
+// pooling run in fp32, c_rep is rounded once to bf16.
+__global__ void __launch_bounds__(CONDENSE_THREADS, 1)
 condense_kernel(CondenseArgs a) {
   extern __shared__ __align__(16) unsigned char smem_raw[];
-  const int j = blockIdx.x, hk = blockIdx.y, b = blockIdx.z;
   const int g = a.g, d_sem = a.d_sem, d_pos = a.d_pos;
   const int dk = (a.sem_in_logit ? d_sem : 0) + d_pos;
-  bf16* t_sem = reinterpret_cast<bf16*>(smem_raw);                 // [g][d_sem]
-  bf16* t_pos = t_sem + (size_t)g * d_sem;                         // [g][d_pos]
-  double* s_q = reinterpret_cast<double*>(t_pos + (size_t)g * d_pos);   // [dk]
-  double* s_s = s_q + dk;                                          // [g] scores
-  double* s_a = s_s + g;                                           // [g] alpha
+  const size_t stage_bytes = (size_t)g * (d_sem + d_pos) * sizeof(bf16) + (size_t)dk * sizeof(double);
+  double* s_s = reinterpret_cast<double*>(smem_raw + 2 * stage_bytes);      // [g] scores
+  float* s_a = reinterpret_cast<float*>(s_s + g);                           // [g] alpha
   __shared__ int s_anchor;
 
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5, nwarps = blockDim.x >> 5;
-  const size_t tok0 = (size_t)b * a.L + (size_t)j * g;             // first token of G_j
   const size_t row_stride_sem = (size_t)a.Hkv * d_sem, row_stride_pos = (size_t)a.Hkv * d_pos;
+  const int cps = d_sem / 8, cpp = d_pos / 8, cpq = dk / 2;                 // 16-byte pieces per row / of q_bar
 
-  // 1. the g tokens of the group: global -> shared, 16 B per copy, each byte read once
-  {
-    const int cps = d_sem / 8, cpp = d_pos / 8;                    // 16-byte chunks per row
+  auto stage_ptr = [&](int st) { return smem_raw + (size_t)st * stage_bytes; };
+  auto prefetch = [&](long long grp, int st) {
+    const int j = (int)(grp % a.m);
+    const long long bh = grp / a.m;
+    const int hk = (int)(bh % a.Hkv), b = (int)(bh / a.Hkv);
+    bf16* t_sem = reinterpret_cast<bf16*>(stage_ptr(st));
+    bf16* t_pos = t_sem + (size_t)g * d_sem;
+    double* s_q = reinterpret_cast<double*>(t_pos + (size_t)g * d_pos);
+    const size_t tok0 = (size_t)b * a.L + (size_t)j * g;
     const bf16* gs = a.kv_sem + tok0 * row_stride_sem + (size_t)hk * d_sem;
     const bf16* gp = a.kv_pos + tok0 * row_stride_pos + (size_t)hk * d_pos;
     for (int x = tid; x < g * cps; x += blockDim.x) {
-      int i = x / cps, c = x % cps;
+      const int i = x / cps, c = x % cps;
       cp_async16(t_sem + (size_t)i * d_sem + c * 8, gs + (size_t)i * row_stride_sem + c * 8);
     }
     for (int x = tid; x < g * cpp; x += blockDim.x) {
-      int i = x / cpp, c = x % cpp;
+      const int i = x / cpp, c = x % cpp;
       cp_async16(t_pos + (size_t)i * d_pos + c * 8, gp + (size_t)i * row_stride_pos + c * 8);
     }
-    const double* qb = a.qbar + ((size_t)b * a.Hkv + hk) * dk;
-    for (int c = tid; c < dk; c += blockDim.x) s_q[c] = qb[c];
-    cp_async_wait_all();
-  }
-  __syncthreads();
+    const double* qb = a.qbar + (size_t)bh * dk;
+    for (int x = tid; x < cpq; x += blockDim.x) cp_async16(s_q + 2 * x, qb + 2 * x);
+  };
 
-  // 2. importance scores s_i = scale * q_bar . k_i   (one warp per token, fp64)
-  const int sem_off = a.sem_in_logit ? d_sem : 0;
-  for (int i = warp; i < g; i += nwarps) {
-    double acc = 0.0;
-    if (a.sem_in_logit) {
-      const bf162* row = reinterpret_cast<const bf162*>(t_sem + (size_t)i * d_sem);
-      for (int pr = lane; pr < d_sem / 2; pr += 32) {
-        bf162 v = row[pr];
-        acc = fma(s_q[2 * pr], (double)__low2float(v), acc);
-        acc = fma(s_q[2 * pr + 1], (double)__high2float(v), acc);
-      }
-    }
-    {
-      const bf162* row = reinterpret_cast<const bf162*>(t_pos + (size_t)i * d_pos);
-      for (int pr = lane; pr < d_pos / 2; pr += 32) {
-        bf162 v = row[pr];
-        acc = fma(s_q[sem_off + 2 * pr], (double)__low2float(v), acc);
-        acc = fma(s_q[sem_off + 2 * pr + 1], (double)__high2float(v), acc);
-      }
-    }
-    acc = warp_sum(acc);
-    if (lane == 0) s_s[i] = acc * a.scale;
-  }
-  __syncthreads();
+  long long grp = blockIdx.x;
+  if (grp < a.n_groups) prefetch(grp, 0);
+  asm volatile("cp.async.commit_group;\n" ::: "memory");
+  for (int it = 0; grp < a.n_groups; ++it, grp += gridDim.x) {
+    const int st = it & 1;
+    const long long next = grp + gridDim.x;
+    if (next < a.n_groups) prefetch(next, st ^ 1);
+    asm volatile("cp.async.commit_group;\ncp.async.wait_group 1;\n" ::: "memory");
+    __syncthreads();
 
-  // 3. group softmax (Eq. 6) and arg-max (Eq. 8; lowest index on ties), warp 0
-  if (warp == 0) {
-    double best = -INFINITY;
-    int besti = 0x7fffffff;
-    for (int i = lane; i < g; i += 32) {
-      double s = s_s[i];
-      if (s > best) { best = s; besti = i; }
+    const int j = (int)(grp % a.m);
+    const long long bh = grp / a.m;
+    const int hk = (int)(bh % a.Hkv), b = (int)(bh / a.Hkv);
+    const bf16* t_sem = reinterpret_cast<const bf16*>(stage_ptr(st));
+    const bf16* t_pos = t_sem + (size_t)g * d_sem;
+    const double* s_q = reinterpret_cast<const double*>(t_pos + (size_t)g * d_pos);
+
+    // 1. importance scores s_i = scale * q_bar . k_i   (one warp per token, fp64)
+    const int sem_off = a.sem_in_logit ? d_sem : 0;
+    for (int i = warp; i < g; i += nwarps) {
+      double acc0 = 0.0, acc1 = 0.0;
+      if (a.sem_in_logit) {
+        const bf162* row = reinterpret_cast<const bf162*>(t_sem + (size_t)i * d_sem);
+        for (int pr = lane; pr < d_sem / 2; pr += 32) {
+          const bf162 v = row[pr];
+          acc0 = fma(s_q[2 * pr], (double)__low2float(v), acc0);
+          acc1 = fma(s_q[2 * pr + 1], (double)__high2float(v), acc1);
+        }
+      }
+      {
+        const bf162* row = reinterpret_cast<const bf162*>(t_pos + (size_t)i * d_pos);
+        for (int pr = lane; pr < d_pos / 2; pr += 32) {
+          const bf162 v = row[pr];
+          acc0 = fma(s_q[sem_off + 2 * pr], (double)__low2float(v), acc0);
+          acc1 = fma(s_q[sem_off + 2 * pr + 1], (double)__high2float(v), acc1);
+        }
+      }
+      const double acc = warp_sum(acc0 + acc1);
+      if (lane == 0) s_s[i] = acc * a.scale;
     }
+    __syncthreads();
+
+    // 2. arg-max on the fp64 scores (Eq. 8; lowest index on ties) and group softmax (Eq. 6), warp 0
+    if (warp == 0) {
+      double best = -INFINITY;
+      int besti = 0x7fffffff;
+      for (int i = lane; i < g; i += 32) {
+        const double s = s_s[i];
+        if (s > best) { best = s; besti = i; }
+      }
 #pragma unroll
-    for (int o = 16; o > 0; o >>= 1) {
-      double ob = __shfl_xor_sync(0xffffffffu, best, o);
-      int oi = __shfl_xor_sync(0xffffffffu, besti, o);
-      if (ob > best || (ob == best && oi < besti)) { best = ob; besti = oi; }
+      for (int o = 16; o > 0; o >>= 1) {
+        const double ob = __shfl_xor_sync(0xffffffffu, best, o);
+        const int oi = __shfl_xor_sync(0xffffffffu, besti, o);
+        if (ob > best || (ob == best && oi < besti)) { best = ob; besti = oi; }
+      }
+      float z = 0.f;
+      for (int i = lane; i < g; i += 32) {
+        const float e = expf((float)(s_s[i] - best));
+        s_a[i] = e;
+        z += e;
+      }
+      z = warp_sum(z);
+      const float inv = 1.f / z;
+      for (int i = lane; i < g; i += 32) s_a[i] *= inv;
+      if (lane == 0) s_anchor = besti;
     }
-    double z = 0.0;
-    for (int i = lane; i < g; i += 32) {
-      double e = exp(s_s[i] - best);
-      s_a[i] = e;
-      z += e;
+    __syncthreads();
+
+    // 3. weighted pooling c_rep = sum_i alpha_i c_i (Eq. 7), one column pair per thread, fp32
+    const size_t out_row = (size_t)b * a.cache_rows + j;
+    {
+      bf16* dst = a.cache_sem + (out_row * a.Hkv + hk) * d_sem;
+      for (int pr = tid; pr < d_sem / 2; pr += blockDim.x) {
+        float a0 = 0.f, a1 = 0.f;
+#pragma unroll 8
+        for (int i = 0; i < g; ++i) {
+          const float2 v = __bfloat1622float2(*reinterpret_cast<const bf162*>(t_sem + (size_t)i * d_sem + 2 * pr));
+          const float al = s_a[i];
+          a0 = fmaf(al, v.x, a0);
+          a1 = fmaf(al, v.y, a1);
+        }
+        *reinterpret_cast<bf162*>(dst + 2 * pr) = __floats2bfloat162_rn(a0, a1);
+      }
     }
-    z = warp_sum(z);
-    for (int i = lane; i < g; i += 32) s_a[i] = s_a[i] / z;
-    if (lane == 0) s_anchor = besti;
+    // 4. positional anchor: bit copy of the arg-max token's positional row (threads from the top)
+    {
+      const int ia = s_anchor;
+      const uint4* src = reinterpret_cast<const uint4*>(t_pos + (size_t)ia * d_pos);
+      uint4* dst = reinterpret_cast<uint4*>(a.cache_pos + (out_row * a.Hkv + hk) * d_pos);
+      const int rt = blockDim.x - 1 - tid;
+      for (int c = rt; c < d_pos / 8; c += blockDim.x) dst[c] = src[c];
+      if (rt == 0) a.anchor[((size_t)b * a.m + j) * a.Hkv + hk] = j * g + ia;
+      if (a.scores) {
+        double* sc = a.scores + (((size_t)b * a.Hkv + hk) * a.m + j) * g;
+        for (int i = rt; i < g; i += blockDim.x) sc[i] = s_s[i];
+      }
+    }
+    __syncthreads();        // the stage and the score arrays are free for the next round
+  }
+  asm volatile("cp.async.wait_group 0;\n" ::: "memory");
+}
+
+// ----------------------------------------------------- condense, MLA shape with g = 64 (the fast path)
+// Same arithmetic as condense_kernel for d_sem = 512, d_pos = 64, g = 64 and one KV stream, laid
+// out for the instruction budget HBM speed leaves (about 3000 cycles per group and SM).  The
+// float-to-double conversions of the scores (one per key element, on the slow conversion unit)
+// take most of that budget, so nothing else may wait for them: the CTA is split into roles that
+// work on different groups at the same time.
+//   * one producer thread fetches a group (64 KB + 8 KB of contiguous memory) with two bulk
+//     copies (cp.async.bulk) into one of three stages, completion on an mbarrier per stage;
+//   * sixteen score warps: warp w takes tokens w, w+16, ...; lane l holds the 18 components of q_bar
+//     it needs in registers (columns 8l..8l+7 and 256+8l..256+8l+7 of the latent part, 2l, 2l+1
+//     of the rope part) and reads its share of a token with two 16-byte and one 4-byte load;
+//     fp64 multiply-adds, warp-shuffle reduction; warp 0 then takes the arg-max and the softmax;
+//   * four pool warps, one group behind: four output columns per thread, fp32, alpha read four
+//     tokens at a time; they also copy the anchor's rope row and write index and scores.
+namespace fast {
+constexpr int G = 64, DS = 512, DP = 64, DK = DS + DP, STAGES = 3;
+constexpr int SCORE_WARPS = 16, POOL_WARPS = 4, THREADS = 32 * (SCORE_WARPS + POOL_WARPS + 1);
+constexpr int SEM_BYTES = G * DS * 2, POS_BYTES = G * DP * 2, STAGE_BYTES = SEM_BYTES + POS_BYTES;
+constexpr int OFF_Q = STAGES * STAGE_BYTES;                 // double[DK]
+constexpr int OFF_S = OFF_Q + DK * 8;                       // double[2][G] scores
+constexpr int OFF_A = OFF_S + 2 * G * 8;                    // float[2][G] alpha
+constexpr int OFF_BAR = OFF_A + 2 * G * 4;                  // mbarriers: full[3] free[3] ready[2] afree[2], then flags
+constexpr int SMEM_BYTES = OFF_BAR + 128;
+static_assert(SMEM_BYTES <= 232448, "shared memory budget of one SM");
+constexpr long long WAIT_CYCLES = 2000000000ll;
+}  // namespace fast
+
+static __device__ int g_condense_status = 0;
+
+__device__ __forceinline__ bool cond_wait(unsigned bar, unsigned parity, volatile int* abort_flag) {
+  unsigned done = 0;
+  long long t0 = 0;
+  while (true) {
+    asm volatile("{\n\t.reg .pred p;\n\tmbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\tselp.u32 %0, 1, 0, p;\n\t}"
+                 : "=r"(done) : "r"(bar), "r"(parity) : "memory");
+    if (done) return true;
+    if (t0 == 0) t0 = clock64();
+    if (*abort_flag || clock64() - t0 > fast::WAIT_CYCLES) { *abort_flag = 1; return false; }
+    __nanosleep(40);                                      // leave the issue slots to the working warps
+  }
+}
+__device__ __forceinline__ void cond_arrive(unsigned bar) {
+  asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar) : "memory");
+}
+
+__global__ void __launch_bounds__(fast::THREADS, 1)
+condense_mla64_kernel(CondenseArgs a) {
+  using namespace fast;
+  extern __shared__ __align__(128) unsigned char smem[];
+  double* s_q = reinterpret_cast<double*>(smem + OFF_Q);
+  double* s_s = reinterpret_cast<double*>(smem + OFF_S);
+  float* s_a = reinterpret_cast<float*>(smem + OFF_A);
+  const unsigned bar0 = (unsigned)__cvta_generic_to_shared(smem + OFF_BAR);
+  auto BAR_FULL = [&](int st) { return bar0 + 8 * st; };
+  auto BAR_FREE = [&](int st) { return bar0 + 24 + 8 * st; };
+  auto BAR_READY = [&](int p) { return bar0 + 48 + 8 * p; };      // alpha / anchor of parity p written
+  auto BAR_AFREE = [&](int p) { return bar0 + 64 + 8 * p; };      // ... and consumed
+  volatile int* s_anchor = reinterpret_cast<volatile int*>(smem + OFF_BAR + 80);   // [2]
+  volatile int* s_abort = reinterpret_cast<volatile int*>(smem + OFF_BAR + 88);
+  volatile int* s_stop = reinterpret_cast<volatile int*>(smem + OFF_BAR + 96);     // [2]
+  const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+
+  if (tid == 0) {
+    for (int st = 0; st < STAGES; ++st) {
+      asm volatile("mbarrier.init.shared::cta.b64 [%0], 1;" ::"r"(BAR_FULL(st)) : "memory");
+      asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(BAR_FREE(st)), "r"(POOL_WARPS) : "memory");
+    }
+    for (int p = 0; p < 2; ++p) {
+      asm volatile("mbarrier.init.shared::cta.b64 [%0], 1;" ::"r"(BAR_READY(p)) : "memory");
+      asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(BAR_AFREE(p)), "r"(POOL_WARPS) : "memory");
+    }
+    *s_abort = 0;
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
   }
   __syncthreads();
 
-  // 4. weighted pooling c_rep = sum_i alpha_i c_i (Eq. 7), one column pair per thread
-  const size_t out_row = (size_t)b * a.cache_rows + j;
-  {
-    bf16* dst = a.cache_sem + (out_row * a.Hkv + hk) * d_sem;
-    for (int pr = tid; pr < d_sem / 2; pr += blockDim.x) {
-      double a0 = 0.0, a1 = 0.0;
-      for (int i = 0; i < g; ++i) {
-        bf162 v = *reinterpret_cast<const bf162*>(t_sem + (size_t)i * d_sem + 2 * pr);
-        double al = s_a[i];
-        a0 = fma(al, (double)__low2float(v), a0);
-        a1 = fma(al, (double)__high2float(v), a1);
+  const long long first = blockIdx.x, stride = gridDim.x;
+  const long long n_mine = first < a.n_groups ? (a.n_groups - first + stride - 1) / stride : 0;
+
+  if (warp == SCORE_WARPS + POOL_WARPS) {
+    // ===================================================== producer
+    if (lane == 0) {
+      for (long long it = 0; it < n_mine; ++it) {
+        const int st = (int)(it % STAGES);
+        if (it >= STAGES && !cond_wait(BAR_FREE(st), (unsigned)((it / STAGES - 1) & 1), s_abort)) break;
+        const long long grp = first + it * stride;
+        const int j = (int)(grp % a.m);
+        const long long b = grp / a.m;
+        const size_t tok0 = (size_t)b * a.L + (size_t)j * G;
+        const unsigned dst = (unsigned)__cvta_generic_to_shared(smem + (size_t)st * STAGE_BYTES);
+        const unsigned bar = BAR_FULL(st);
+        asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(STAGE_BYTES) : "memory");
+        asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];"
+                     ::"r"(dst), "l"(a.kv_sem + tok0 * DS), "r"(SEM_BYTES), "r"(bar) : "memory");
+        asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];"
+                     ::"r"(dst + SEM_BYTES), "l"(a.kv_pos + tok0 * DP), "r"(POS_BYTES), "r"(bar) : "memory");
       }
-      bf162 o;
-      o.x = double_to_bf16_rn(a0);
-      o.y = double_to_bf16_rn(a1);
-      *reinterpret_cast<bf162*>(dst + 2 * pr) = o;
+    }
+  } else if (warp < SCORE_WARPS) {
+    // ===================================================== scores, arg-max, softmax
+    double q[18];
+    long long cur_b = -1;
+    for (long long it = 0; it < n_mine; ++it) {
+      const int st = (int)(it % STAGES), p = (int)(it & 1);
+      const long long grp = first + it * stride;
+      const long long b = grp / a.m;
+      if (b != cur_b) {                                   // uniform over the score warps; rare
+        cur_b = b;
+        asm volatile("bar.sync 1, 512;" ::: "memory");    // nobody still reads the old q_bar
+        const double* qb = a.qbar + (size_t)b * DK;
+        for (int x = tid; x < DK; x += 32 * SCORE_WARPS) s_q[x] = qb[x];
+        asm volatile("bar.sync 1, 512;" ::: "memory");
+#pragma unroll
+        for (int i = 0; i < 8; ++i) { q[i] = s_q[8 * lane + i]; q[8 + i] = s_q[256 + 8 * lane + i]; }
+        q[16] = s_q[DS + 2 * lane]; q[17] = s_q[DS + 2 * lane + 1];
+      }
+      bool ok = cond_wait(BAR_FULL(st), (unsigned)((it / STAGES) & 1), s_abort);
+      if (ok && it >= 2) ok = cond_wait(BAR_AFREE(p), (unsigned)(((it >> 1) - 1) & 1), s_abort);
+      const unsigned char* t_sem = smem + (size_t)st * STAGE_BYTES;
+      const unsigned char* t_pos = t_sem + SEM_BYTES;
+      if (ok) {
+#pragma unroll 2
+        for (int tt = 0; tt < G / SCORE_WARPS; ++tt) {
+          const int i = warp + SCORE_WARPS * tt;
+          const uint4 v0 = *reinterpret_cast<const uint4*>(t_sem + (size_t)i * (DS * 2) + 16 * lane);
+          const uint4 v1 = *reinterpret_cast<const uint4*>(t_sem + (size_t)i * (DS * 2) + 512 + 16 * lane);
+          const unsigned vp = *reinterpret_cast<const unsigned*>(t_pos + (size_t)i * (DP * 2) + 4 * lane);
+          const unsigned w[9] = {v0.x, v0.y, v0.z, v0.w, v1.x, v1.y, v1.z, v1.w, vp};
+          double acc0 = 0.0, acc1 = 0.0;
+#pragma unroll
+          for (int k = 0; k < 9; ++k) {
+            acc0 = fma(q[2 * k], (double)__uint_as_float(w[k] << 16), acc0);
+            acc1 = fma(q[2 * k + 1], (double)__uint_as_float(w[k] & 0xffff0000u), acc1);
+          }
+          const double acc = warp_sum(acc0 + acc1);
+          if (lane == 0) s_s[p * G + i] = acc * a.scale;
+        }
+      }
+      // one thread samples the abort flag before the barrier, so that all score warps leave in
+      // the same iteration (a warp whose own wait expired skips the work and is caught next time)
+      if (tid == 0) s_stop[p] = *s_abort;
+      asm volatile("bar.sync 1, 512;" ::: "memory");
+      if (s_stop[p]) break;
+      if (warp == 0) {
+        const double sa = s_s[p * G + lane], sb = s_s[p * G + lane + 32];
+        double best = sa; int besti = lane;
+        if (sb > best) { best = sb; besti = lane + 32; }
+#pragma unroll
+        for (int o = 16; o > 0; o >>= 1) {
+          const double ob = __shfl_xor_sync(0xffffffffu, best, o);
+          const int oi = __shfl_xor_sync(0xffffffffu, besti, o);
+          if (ob > best || (ob == best && oi < besti)) { best = ob; besti = oi; }
+        }
+        const float ea = expf((float)(sa - best)), eb = expf((float)(sb - best));
+        const float inv = 1.f / warp_sum(ea + eb);
+        s_a[p * G + lane] = ea * inv; s_a[p * G + lane + 32] = eb * inv;
+        if (lane == 0) s_anchor[p] = besti;
+        __syncwarp();
+        if (lane == 0) cond_arrive(BAR_READY(p));
+      }
+    }
+  } else {
+    // ===================================================== pooling and outputs, one group behind
+    const int pt = tid - 32 * SCORE_WARPS;                // 0..127: output columns 4 pt .. 4 pt + 3
+    for (long long it = 0; it < n_mine; ++it) {
+      const int st = (int)(it % STAGES), p = (int)(it & 1);
+      const long long grp = first + it * stride;
+      const int j = (int)(grp % a.m);
+      const long long b = grp / a.m;
+      if (!cond_wait(BAR_READY(p), (unsigned)((it >> 1) & 1), s_abort)) break;
+      if (!cond_wait(BAR_FULL(st), (unsigned)((it / STAGES) & 1), s_abort)) break;     // complete long ago
+      const unsigned char* t_sem = smem + (size_t)st * STAGE_BYTES;
+      const unsigned char* t_pos = t_sem + SEM_BYTES;
+      const size_t out_row = (size_t)b * a.cache_rows + j;
+      float a0 = 0.f, a1 = 0.f, a2 = 0.f, a3 = 0.f;
+      const uint2* col = reinterpret_cast<const uint2*>(t_sem) + pt;
+      const float* al_base = s_a + p * G;
+#pragma unroll 2
+      for (int i = 0; i < G; i += 4) {
+        const float4 al = *reinterpret_cast<const float4*>(al_base + i);
+        const float alv[4] = {al.x, al.y, al.z, al.w};
+#pragma unroll
+        for (int u = 0; u < 4; ++u) {
+          const uint2 w = col[(i + u) * (DS / 4)];
+          a0 = fmaf(alv[u], __uint_as_float(w.x << 16), a0); a1 = fmaf(alv[u], __uint_as_float(w.x & 0xffff0000u), a1);
+          a2 = fmaf(alv[u], __uint_as_float(w.y << 16), a2); a3 = fmaf(alv[u], __uint_as_float(w.y & 0xffff0000u), a3);
+        }
+      }
+      {
+        const bf162 lo = __floats2bfloat162_rn(a0, a1), hi = __floats2bfloat162_rn(a2, a3);
+        uint2 o;
+        o.x = *reinterpret_cast<const unsigned*>(&lo); o.y = *reinterpret_cast<const unsigned*>(&hi);
+        *reinterpret_cast<uint2*>(a.cache_sem + out_row * DS + 4 * pt) = o;
+      }
+      const int ia = s_anchor[p];
+      if (pt < DP / 8)
+        reinterpret_cast<uint4*>(a.cache_pos + out_row * DP)[pt] = reinterpret_cast<const uint4*>(t_pos + (size_t)ia * (DP * 2))[pt];
+      if (pt == 32) a.anchor[(size_t)b * a.m + j] = j * G + ia;
+      if (a.scores && pt >= 64) a.scores[((size_t)b * a.m + j) * G + (pt - 64)] = s_s[p * G + pt - 64];
+      __syncwarp();
+      if (lane == 0) { cond_arrive(BAR_AFREE(p)); cond_arrive(BAR_FREE(st)); }
     }
   }
-  // 5. positional anchor: bit copy of the arg-max token's positional row
-  {
-    const int ia = s_anchor;
-    const uint4* src = reinterpret_cast<const uint4*>(t_pos + (size_t)ia * d_pos);
-    uint4* dst = reinterpret_cast<uint4*>(a.cache_pos + (out_row * a.Hkv + hk) * d_pos);
-    for (int c = tid; c < d_pos / 8; c += blockDim.x) dst[c] = src[c];
-    if (tid == 0) a.anchor[((size_t)b * a.m + j) * a.Hkv + hk] = j * g + ia;
-  }
-  if (a.scores) {
-    double* sc = a.scores + (((size_t)b * a.Hkv + hk) * a.m + j) * g;
-    for (int i = tid; i < g; i += blockDim.x) sc[i] = s_s[i];
-  }
+  __syncthreads();
+  if (tid == 0 && *s_abort) atomicCAS(&g_condense_status, 0, 1);
+}
+
+int condense_take_status() {
+  int st = 0;
+  if (cudaMemcpyFromSymbol(&st, g_condense_status, sizeof(int)) != cudaSuccess) return -1;
+  if (st != 0) { int zero = 0; cudaMemcpyToSymbol(g_condense_status, &zero, sizeof(int)); }
+  return st;
 }
 
 // ------------------------------------------------------------------------------ local window
@@ -232,9 +487,15 @@ size_t condense_workspace_bytes(const lca_params* p) {
   return (streams * dk + streams * dk * (size_t)qbar_chunks(p)) * sizeof(double);
 }
 
+static bool condense_fast_shape(const lca_params* p) {
+  return p->variant == LCA_VARIANT_MLA && p->d_sem == 512 && p->d_pos == 64 && p->group_size == 64 && p->n_kv_heads == 1;
+}
+
 size_t condense_smem_bytes(const lca_params* p) {
-  size_t g = (size_t)p->group_size;
-  return g * (size_t)(p->d_sem + p->d_pos) * sizeof(bf16) + ((size_t)key_dim(p) + 2 * g) * sizeof(double);
+  if (condense_fast_shape(p)) return fast::SMEM_BYTES;
+  const size_t g = (size_t)p->group_size;
+  const size_t stage = g * (size_t)(p->d_sem + p->d_pos) * sizeof(bf16) + (size_t)key_dim(p) * sizeof(double);
+  return 2 * stage + g * (sizeof(double) + sizeof(float));
 }
 
 int condense_launch(const CondenseLaunch& c) {
@@ -255,9 +516,14 @@ int condense_launch(const CondenseLaunch& c) {
     } else {
       const int nch = qbar_chunks(p);
       dim3 grid(nch, Hkv, B);
-      qbar_partial_kernel<<<grid, QBAR_THREADS, 0, c.stream>>>(
+      const int pieces = dk / 8;
+      int row_lanes = 256 / pieces;
+      if (row_lanes < 1) row_lanes = 1;
+      if (row_lanes > 16) row_lanes = 16;
+      const int threads = ((pieces * row_lanes + 31) / 32) * 32;
+      qbar_partial_kernel<<<grid, threads, (size_t)row_lanes * dk * sizeof(double), c.stream>>>(
           (const bf16*)c.q_tail_sem, (const bf16*)c.q_tail_pos, c.q_tail_batch_stride, n_summary(p),
-          p->n_q_heads, Hkv, p->d_sem, p->d_pos, sem_in_logit, partial);
+          p->n_q_heads, Hkv, p->d_sem, p->d_pos, sem_in_logit, row_lanes, partial);
       double count = (double)n_summary(p) * (double)(p->n_q_heads / Hkv);
       qbar_final_kernel<<<dim3(Hkv, B), QBAR_THREADS, 0, c.stream>>>(partial, nch, dk, count, qbar);
       note_launch(2);
@@ -269,10 +535,20 @@ int condense_launch(const CondenseLaunch& c) {
     a.L = p->seq_len; a.Hkv = Hkv; a.d_sem = p->d_sem; a.d_pos = p->d_pos; a.g = p->group_size;
     a.m = (int)m; a.cache_rows = (int)(m + k); a.sem_in_logit = sem_in_logit;
     a.scale = (double)p->softmax_scale;
-    size_t smem = condense_smem_bytes(p);
-    if (cudaFuncSetAttribute(condense_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) != cudaSuccess)
-      return LCA_ERR_CUDA;
-    condense_kernel<<<dim3((unsigned)m, Hkv, B), CONDENSE_THREADS, smem, c.stream>>>(a);
+    a.n_groups = (long long)B * Hkv * m;
+    int dev = 0, sms = 148;
+    if (cudaGetDevice(&dev) == cudaSuccess) cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
+    const long long ctas = a.n_groups < sms ? a.n_groups : sms;
+    if (condense_fast_shape(p)) {
+      if (cudaFuncSetAttribute(condense_mla64_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, fast::SMEM_BYTES) != cudaSuccess)
+        return LCA_ERR_CUDA;
+      condense_mla64_kernel<<<dim3((unsigned)ctas), fast::THREADS, fast::SMEM_BYTES, c.stream>>>(a);
+    } else {
+      size_t smem = condense_smem_bytes(p);
+      if (cudaFuncSetAttribute(condense_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) != cudaSuccess)
+        return LCA_ERR_CUDA;
+      condense_kernel<<<dim3((unsigned)ctas), CONDENSE_THREADS, smem, c.stream>>>(a);
+    }
     note_launch();
   }
   if (k > 0) {

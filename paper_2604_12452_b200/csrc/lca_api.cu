@@ -191,6 +191,12 @@ int lca_decode_attention(const lca_params* p, const void* q_sem, const void* q_p
   return run_attention(a);
 }
 
-int lca_last_device_status(void* stream) { return attn_tc_device_status((cudaStream_t)stream); }
+int lca_last_device_status(void* stream) {
+  const int st = attn_tc_device_status((cudaStream_t)stream);      // synchronises the stream
+  const int cst = condense_take_status();
+  if (cst < 0) return LCA_ERR_CUDA;
+  if (cst > 0) return LCA_ERR_DEVICE_TIMEOUT;
+  return st;
+}
 
 }  // extern "C"

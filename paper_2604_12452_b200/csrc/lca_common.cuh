@@ -59,6 +59,7 @@ struct CondenseLaunch {
 size_t condense_workspace_bytes(const lca_params* p);
 int condense_launch(const CondenseLaunch& a);
 size_t condense_smem_bytes(const lca_params* p);
+int condense_take_status();   // nonzero once if a bounded wait of the condense kernel expired
 int condense_static_scratch_address(void** out);   // device address of the library's fixed scratch array
 
 // One description of an attention problem for every implementation.  Each query row (b, t, h)

@@ -111,7 +111,7 @@ def check_outputs(got: torch.Tensor, ref: np.ndarray, what: str = ""):
 
 def check_condense(res: dict, cond: dict, kind: str = "mla"):
     """Compare the device cache with the oracle's: anchors, copied rows and layout bit-exact;
-    c_rep bit-exact up to counted 1-ulp differences.  `res` holds one sequence (batch index
+    c_rep within one bf16 ulp (fp32 pooling against fp64), differences counted.  `res` holds one sequence (batch index
     already taken)."""
     m, k = cond["m"], cond["k"]
     assert res["m"] == m and res["k"] == k
@@ -128,6 +128,15 @@ def check_condense(res: dict, cond: dict, kind: str = "mla"):
     assert np.array_equal(got_sem[m:], ref_sem[m:]), "local-window rows differ"
     ulp = bf16_ulp_distance(got_sem[:m], ref_sem[:m])
     n_off = int((ulp > 0).sum())
-    assert (ulp <= 1).all(), f"c_rep off by more than one bf16 ulp: max {ulp.max()}"
-    assert n_off <= max(1, ulp.size // 100000), f"too many 1-ulp c_rep differences: {n_off}/{ulp.size}"
+    # The kernel pools in fp32 and the oracle in fp64.  A sum of g terms carries an absolute error
+    # of at most g * 2^-24 * sum_i alpha_i |c_i| <= g * 2^-24 * max|c|; where the pooled value is
+    # not tiny that is far below one bf16 ulp, so c_rep is within one ulp; where the terms cancel
+    # (|c_rep| << |c_i|) an ulp is smaller than that error and the absolute bound applies.
+    g_max = 64
+    abs_err = np.abs(O.bits_to_f64(got_sem[:m]) - O.bits_to_f64(ref_sem[:m]))
+    abs_bound = g_max * 2.0 ** -24 * float(np.abs(O.bits_to_f64(ref_sem)).max()) if ref_sem.size else 0.0
+    bad = (ulp > 1) & (abs_err > abs_bound)
+    assert not bad.any(), f"c_rep off by more than one bf16 ulp and more than {abs_bound:.2e}: max ulp {ulp.max()}"
+    # a bf16 rounding boundary (spacing 2^-8 relative) is crossed by about one element in 2500
+    assert n_off <= max(2, ulp.size // 250), f"too many c_rep differences: {n_off}/{ulp.size}"
     return dict(crep_one_ulp=n_off, crep_elems=int(ulp.size))
