@@ -39,7 +39,7 @@ __global__ void qbar_partial_kernel(const bf16* __restrict__ q_sem, const bf16* 
 #pragma unroll
   for (int i = 0; i < 8; ++i) acc[i] = 0.0;
   if (rl < row_lanes) {
-#pragma unroll 4
+#pragma unroll 8
     for (int r = r0 + rl; r < r1; r += row_lanes) {
       const int pos = r / rep, head = hk * rep + r % rep;
       const size_t row = ((size_t)b * batch_stride_rows + pos) * Hq + head;
@@ -72,7 +72,8 @@ __global__ void qbar_final_kernel(const double* __restrict__ partial, int nchunk
   const double* src = partial + stream_id * nchunks * dk;
   for (int c = threadIdx.x; c < dk; c += blockDim.x) {
     double s = 0.0;
-    for (int ch = 0; ch < nchunks; ++ch) s += src[(size_t)ch * dk + c];
+#pragma unroll 16
+    for (int ch = 0; ch < nchunks; ++ch) s += __ldg(src + (size_t)ch * dk + c);     // loads run ahead of the adds
     qbar[stream_id * dk + c] = s / count;
   }
 }
@@ -363,8 +364,12 @@ condense_mla64_kernel(CondenseArgs a) {
       const unsigned char* t_sem = smem + (size_t)st * STAGE_BYTES;
       const unsigned char* t_pos = t_sem + SEM_BYTES;
       if (ok) {
-#pragma unroll 2
-        for (int tt = 0; tt < G / SCORE_WARPS; ++tt) {
+        // the warp's four tokens together: 4 x 18 independent multiply-add chains, then one
+        // transposed reduction (lanes 0, 8, 16, 24 end up with the sums of tokens 0..3)
+        static_assert(G / SCORE_WARPS == 4, "four tokens per score warp");
+        double part[4];
+#pragma unroll
+        for (int tt = 0; tt < 4; ++tt) {
           const int i = warp + SCORE_WARPS * tt;
           const uint4 v0 = *reinterpret_cast<const uint4*>(t_sem + (size_t)i * (DS * 2) + 16 * lane);
           const uint4 v1 = *reinterpret_cast<const uint4*>(t_sem + (size_t)i * (DS * 2) + 512 + 16 * lane);
@@ -376,9 +381,18 @@ condense_mla64_kernel(CondenseArgs a) {
             acc0 = fma(q[2 * k], (double)__uint_as_float(w[k] << 16), acc0);
             acc1 = fma(q[2 * k + 1], (double)__uint_as_float(w[k] & 0xffff0000u), acc1);
           }
-          const double acc = warp_sum(acc0 + acc1);
-          if (lane == 0) s_s[p * G + i] = acc * a.scale;
+          part[tt] = acc0 + acc1;
         }
+        const bool up16 = (lane & 16) != 0, up8 = (lane & 8) != 0;
+        const double k0 = up16 ? part[2] : part[0], k1 = up16 ? part[3] : part[1];
+        const double g0 = up16 ? part[0] : part[2], g1 = up16 ? part[1] : part[3];
+        const double b0 = k0 + __shfl_xor_sync(0xffffffffu, g0, 16);
+        const double b1 = k1 + __shfl_xor_sync(0xffffffffu, g1, 16);
+        double c = (up8 ? b1 : b0) + __shfl_xor_sync(0xffffffffu, up8 ? b0 : b1, 8);
+        c += __shfl_xor_sync(0xffffffffu, c, 4);
+        c += __shfl_xor_sync(0xffffffffu, c, 2);
+        c += __shfl_xor_sync(0xffffffffu, c, 1);
+        if ((lane & 7) == 0) s_s[p * G + warp + SCORE_WARPS * (lane >> 3)] = c * a.scale;
       }
       // one thread samples the abort flag before the barrier, so that all score warps leave in
       // the same iteration (a warp whose own wait expired skips the work and is caught next time)
@@ -525,7 +539,7 @@ int condense_launch(const CondenseLaunch& c) {
           (const bf16*)c.q_tail_sem, (const bf16*)c.q_tail_pos, c.q_tail_batch_stride, n_summary(p),
           p->n_q_heads, Hkv, p->d_sem, p->d_pos, sem_in_logit, row_lanes, partial);
       double count = (double)n_summary(p) * (double)(p->n_q_heads / Hkv);
-      qbar_final_kernel<<<dim3(Hkv, B), QBAR_THREADS, 0, c.stream>>>(partial, nch, dk, count, qbar);
+      qbar_final_kernel<<<dim3(Hkv, B), dk < 1024 ? ((dk + 31) / 32) * 32 : 1024, 0, c.stream>>>(partial, nch, dk, count, qbar);
       note_launch(2);
     }
     CondenseArgs a;
