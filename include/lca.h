@@ -154,6 +154,8 @@ int lca_prefill_attention(const lca_params* p, const void* q_sem, const void* q_
  *   q_sem [B, H, d_sem] (NULL for GQA), q_pos [B, H, d_pos]
  *   cache_sem [B, cache_row_capacity, n_kv_heads, d_sem], cache_pos likewise with d_pos
  *   cache_rows [B] int32 (device): valid rows of each sequence, clamped to [0, cache_row_capacity]
+ *       (the tensor-core kernels fetch whole tiles of 128 rows: rows between cache_rows[b] and the
+ *       end of the buffers take no part in the result but must hold finite numbers, e.g. zeros)
  *   n_rep: leading rows that are representatives (they receive rep_logit_bias)
  *   out [B, H, d_sem] bf16, lse_opt [B, H] fp32 or NULL
  * p->seq_len, group_size and window are not used here. */

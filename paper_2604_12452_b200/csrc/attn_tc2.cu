@@ -415,7 +415,6 @@ bool make_tensor_map_3d(CUtensorMap* map, const void* ptr, int d, int heads, lon
 
 bool attn_tc2_supported(const AttnProblem& a) {
   if (a.variant != LCA_VARIANT_MLA || a.d_sem != 512 || a.d_pos != 64 || a.n_kv_heads != 1) return false;
-  if (a.decode) return false;
   const int H = a.n_q_heads;
   if (H >= 128) return H % 128 == 0;
   return H >= 1 && (128 % H) == 0;      // each CTA of the pair takes whole tokens
