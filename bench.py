@@ -33,6 +33,9 @@ from paper_2604_12452_b200 import inputs as I
 
 METRIC = "lca_prefill_tokens_per_s"
 UNIT = "tokens/s"
+# dram__bytes_read.sum + dram__bytes_write.sum of attn_tc2_kernel at mla_32k (L=32768, H=16) divided by
+# L*H: the kernel reads every query row and writes every output row once, the key/value stream stays in L2.
+ATTN_DRAM_BYTES_PER_TOKEN_HEAD = (644.07e6 + 492.18e6) / (32768 * 16)
 
 
 # ---------------------------------------------------------------------------- work counts
@@ -299,6 +302,16 @@ def run_ours(args, cfg, rank, world, local_rank):
             dist.destroy_process_group()
         return
     peaks = measured_peaks()
+    extras = {}
+    if not args.no_extras and world == 1:
+        for name, fn in (("decode_config", lambda: measure_decode_config(B, dev, args.decode_batch, peaks)),
+                         ("gqa_config", lambda: measure_gqa_config(B, dev, peaks)),
+                         ("dense_mla_comparison", lambda: measure_dense_comparison(B, dev, peaks))):
+            try:
+                extras[name] = fn()
+            except Exception as ex:        # report, never lose the main line
+                extras[name] = dict(error=str(ex)[:200])
+            torch.cuda.empty_cache()
     flops = attention_flops(cfg)
     tfl = flops / (t_attn * 1e-3) / 1e12
     cbytes = condense_bytes(cfg)
@@ -308,14 +321,16 @@ def run_ours(args, cfg, rank, world, local_rank):
                 data="synthetic", config=workload_config(cfg, world), clocks=clocks, gpu_launches=int(launches),
                 e2e=e2e,
                 roofline=dict(bound="tensor", achieved=tfl, peak=peaks["tflops_sustained"], unit="TFLOP/s",
-                              frac=tfl / peaks["tflops_sustained"], traffic=None,
+                              frac=tfl / peaks["tflops_sustained"],
+                              traffic=ATTN_DRAM_BYTES_PER_TOKEN_HEAD * L * cfg.n_q_heads if cfg.variant == "mla" else None,
+                              traffic_note="dram read+write of one ncu capture at mla_32k (profiles/), scaled by tokens x heads",
                               kernel="lca_prefill_attention", flops_per_launch=flops, ms_per_launch=t_attn,
                               peak_kind=f"{peaks['source']} cuBLAS bf16, sustained (kernel timed inside a long step)",
                               frac_of_burst=tfl / peaks["tflops_burst"], frac_of_nominal_2250=tfl / 2250.0),
                 roofline_condense=dict(bound="hbm", achieved=cgbs, peak=peaks["hbm_gbs"], unit="GB/s",
                                        frac=cgbs / peaks["hbm_gbs"], traffic=None, kernel="lca_condense (all launches)",
                                        bytes_per_launch=cbytes, ms_per_launch=t_cond, peak_kind=f"{peaks['source']} copy"),
-                attention_impl=args.attn_impl)
+                attention_impl=args.attn_impl, extras=extras)
     if not args.no_cpu_baseline:
         small = gather_oracle_inputs(cfg, inp, args.ref_rows)
         v, desc, threads, _ = oracle_sample(cfg, small, args.ref_rows, args.ref_heads)
@@ -325,17 +340,122 @@ def run_ours(args, cfg, rank, world, local_rank):
         dist.destroy_process_group()
 
 
+def time_cuda(fn, warmup=3, iters=5):
+    for _ in range(warmup):
+        fn()
+    torch.cuda.synchronize()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e0.record()
+    for _ in range(iters):
+        fn()
+    e1.record()
+    torch.cuda.synchronize()
+    return e0.elapsed_time(e1) / iters
+
+
+def measure_decode_config(B, dev, batch, peaks, warmup=3, iters=5):
+    """Config 4: lca_condense over `batch` contexts of 65536 tokens (the HBM-bound figure), then
+    lca_decode_attention of one new query per sequence over the condensed cache."""
+    cfg = I.scaled(I.CONFIGS["mla_decode"], batch=batch)
+    L, g, H = cfg.seq_len, cfg.group_size, cfg.n_q_heads
+    ckv = torch.empty((batch, L, cfg.d_sem), dtype=torch.bfloat16, device=dev)
+    kr = torch.empty((batch, L, cfg.d_pos), dtype=torch.bfloat16, device=dev)
+    q_tail_sem = torch.empty((batch, g, H, cfg.d_sem), dtype=torch.bfloat16, device=dev)
+    q_tail_pos = torch.empty((batch, g, H, cfg.d_pos), dtype=torch.bfloat16, device=dev)
+    for b in range(batch):
+        one = I.make_mla_inputs(cfg, dev, batch_index=b, q_positions=slice(L - g, L))
+        ckv[b], kr[b], q_tail_sem[b], q_tail_pos[b] = one["ckv"], one["kr"], one["q_sem"], one["q_pos"]
+    p = B.params_from_config(cfg, batch=batch)
+    m, k = B.lca_partition(p)
+    cap = m + k + 1                                   # + the new token's own row
+    cache = dict(cache_sem=torch.zeros((batch, m + k, 1, cfg.d_sem), dtype=torch.bfloat16, device=dev),
+                 cache_pos=torch.zeros((batch, m + k, 1, cfg.d_pos), dtype=torch.bfloat16, device=dev),
+                 anchor_idx=torch.empty((batch, m, 1), dtype=torch.int32, device=dev))
+    ws = B.workspace(p, B.LCA_WS_CONDENSE, dev)
+    t_cond = time_cuda(lambda: B.condense(p, q_tail_sem, q_tail_pos, ckv, kr, out=cache, ws=ws), warmup, iters)
+    cfg_b = I.scaled(cfg, batch=batch)
+    cbytes = condense_bytes(cfg_b)
+    # decode: cache with one appended row per sequence
+    dsem = torch.zeros((batch, cap, 1, cfg.d_sem), dtype=torch.bfloat16, device=dev)
+    dpos = torch.zeros((batch, cap, 1, cfg.d_pos), dtype=torch.bfloat16, device=dev)
+    dsem[:, :m + k] = cache["cache_sem"]
+    dpos[:, :m + k] = cache["cache_pos"]
+    gen = torch.Generator(device=dev)
+    gen.manual_seed(cfg.seed + 99)
+    dsem[:, m + k] = torch.randn((batch, 1, cfg.d_sem), generator=gen, device=dev).bfloat16()
+    dpos[:, m + k] = torch.randn((batch, 1, cfg.d_pos), generator=gen, device=dev).bfloat16()
+    q_new_sem = torch.randn((batch, H, cfg.d_sem), generator=gen, device=dev).bfloat16()
+    q_new_pos = torch.randn((batch, H, cfg.d_pos), generator=gen, device=dev).bfloat16()
+    rows = torch.full((batch,), cap, dtype=torch.int32, device=dev)
+    out = torch.empty((batch, H, cfg.d_sem), dtype=torch.bfloat16, device=dev)
+    wsd = B.workspace(p, B.LCA_WS_DECODE, dev)
+    t_dec = time_cuda(lambda: B.decode_attention(p, q_new_sem, q_new_pos, dsem, dpos, rows, m, out=out, ws=wsd), warmup, iters)
+    flops = float(batch) * H * cap * 2.0 * (cfg.d_sem + cfg.d_pos + cfg.d_sem)
+    kv_bytes = float(batch) * cap * (cfg.d_sem + cfg.d_pos) * 2
+    full_bytes = float(batch) * (L + 1) * (cfg.d_sem + cfg.d_pos) * 2
+    return dict(workload=f"mla_decode: batch {batch}, contexts of {L} tokens, H={H}, g={g}, w={cfg.window}",
+                condense=dict(ms=t_cond, bytes=cbytes, gbs=cbytes / t_cond / 1e6, frac_of_measured_hbm=cbytes / t_cond / 1e6 / peaks["hbm_gbs"]),
+                decode=dict(us=t_dec * 1e3, rows_per_seq=cap, tflops=flops / t_dec / 1e9, kv_gbs=kv_bytes / t_dec / 1e6,
+                            kv_bytes_condensed=kv_bytes, kv_bytes_full_mla=full_bytes, kv_reduction=1.0 - kv_bytes / full_bytes))
+
+
+def measure_gqa_config(B, dev, peaks, warmup=3, iters=5):
+    """Config 5: GQA variant (pool V, select K per KV head): condense + prefill attention."""
+    cfg = I.CONFIGS["gqa_64k"]
+    L, g = cfg.seq_len, cfg.group_size
+    inp = I.make_gqa_inputs(cfg, dev)
+    p = B.params_from_config(cfg, batch=1)
+    cond = B.condense(p, None, inp["q"][L - g:], inp["v"], inp["k"])
+    out = torch.empty((1, L, cfg.n_q_heads, cfg.d_sem), dtype=torch.bfloat16, device=dev)
+    ws = B.workspace(p, B.LCA_WS_CONDENSE, dev)
+    t_cond = time_cuda(lambda: B.condense(p, None, inp["q"][L - g:], inp["v"], inp["k"], out=cond, ws=ws), warmup, iters)
+    t_attn = time_cuda(lambda: B.prefill_attention(p, None, inp["q"], inp["v"], inp["k"], cond["cache_sem"], cond["cache_pos"], out=out),
+                       warmup, iters)
+    flops = attention_flops(cfg)
+    cbytes = condense_bytes(cfg)
+    return dict(workload=f"gqa_64k: L={L}, {cfg.n_q_heads} q heads / {cfg.n_kv_heads} kv heads, d={cfg.d_sem}, g={g}, w={cfg.window}",
+                tokens_per_s=L / ((t_cond + t_attn) * 1e-3), condense_ms=t_cond, condense_gbs=cbytes / t_cond / 1e6,
+                attention_ms=t_attn, attention_tflops=flops / t_attn / 1e9,
+                attention_frac_of_measured_burst=flops / t_attn / 1e9 / peaks["tflops_burst"])
+
+
+def measure_dense_comparison(B, dev, peaks, iters=2):
+    """Dense absorbed-MLA attention (Eq. 5) through the same entry point (window >= L) beside LCA on
+    config 2 (the 128K dense run would take seconds per launch)."""
+    cfg = I.CONFIGS["mla_32k"]
+    L, g = cfg.seq_len, cfg.group_size
+    inp = I.make_mla_inputs(cfg, dev)
+    out = torch.empty((1, L, cfg.n_q_heads, cfg.d_sem), dtype=torch.bfloat16, device=dev)
+    res = {}
+    for name, w in (("lca", cfg.window), ("dense", L)):
+        c2 = I.scaled(cfg, window=w)
+        p = B.params_from_config(c2, batch=1)
+        cond = B.condense(p, inp["q_sem"][L - g:], inp["q_pos"][L - g:], inp["ckv"], inp["kr"])
+        ws = B.workspace(p, B.LCA_WS_PREFILL, dev)
+        t = time_cuda(lambda: B.prefill_attention(p, inp["q_sem"], inp["q_pos"], inp["ckv"], inp["kr"], cond["cache_sem"],
+                                                  cond["cache_pos"], out=out, ws=ws), 2, iters)
+        fl = attention_flops(c2)
+        res[name] = dict(ms=t, tflops=fl / t / 1e9, flops=fl)
+    res["workload"] = f"mla_32k: L={L}, H={cfg.n_q_heads}"
+    res["speedup_lca_over_dense"] = res["dense"]["ms"] / res["lca"]["ms"]
+    return res
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
     ap.add_argument("--steps", type=int, default=5)
     ap.add_argument("--warmup", type=int, default=3)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
-    ap.add_argument("--config", default="mla_128k", choices=[k for k, c in I.CONFIGS.items() if c.variant == "mla" and c.batch == 1])
+    ap.add_argument("--config", default="mla_128k", choices=list(I.CONFIGS.keys()),
+                    help="mla_128k is the benchmark; mla_1k / mla_32k run the same step on configs 1 / 2; mla_decode and "
+                         "gqa_64k print the side measurements of configs 4 / 5 on their own (used for profiling)")
     ap.add_argument("--attn-impl", type=int, default=0, help="0 auto, 1 scalar kernel, 2 tensor-core kernel")
     ap.add_argument("--e2e-steps", type=int, default=2)
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--no-extras", action="store_true", help="skip the decode / GQA / dense-comparison side measurements")
+    ap.add_argument("--decode-batch", type=int, default=64)
     ap.add_argument("--ref-rows", type=int, default=24, help="query rows in the oracle's bounded sample")
     ap.add_argument("--ref-heads", type=int, default=16, help="heads per sampled row in the oracle's sample")
     args = ap.parse_args()
@@ -352,6 +472,16 @@ def main():
     build.build()
     from paper_2604_12452_b200 import binding as B
     B.lca_set_attention_impl(args.attn_impl)
+    if args.config in ("mla_decode", "gqa_64k"):
+        if rank == 0:
+            torch.cuda.set_device(local_rank)
+            peaks = measured_peaks()
+            dev = f"cuda:{local_rank}"
+            res = (measure_decode_config(B, dev, args.decode_batch, peaks, args.warmup, args.steps) if args.config == "mla_decode"
+                   else measure_gqa_config(B, dev, peaks, args.warmup, args.steps))
+            print(json.dumps(dict(metric="side_measurement", config=dict(workload=res["workload"]), n_gpus=1, steps=args.steps,
+                                  warmup=args.warmup, data="synthetic", result=res, gpu_launches=None)))
+        return
     run_ours(args, cfg, rank, world, local_rank)
 
 
