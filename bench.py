@@ -63,6 +63,19 @@ def condense_bytes(cfg) -> float:
     return float(cfg.batch) * (m * g * row + min(g, L) * qrow + m * row + 4 * m * cfg.n_kv_heads + 2 * k * row)
 
 
+def max_over_ranks(ms: float, dist, device) -> float:
+    """The time of a multi-rank step is the slowest rank's (replicas run independently)."""
+    t = torch.tensor([ms], device=device, dtype=torch.float64)
+    if dist is not None:
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    return float(t.item())
+
+
+def whole_job_value(tokens_per_rank: int, world: int, ms_per_step: float) -> float:
+    """tokens/s over all ranks: every rank processes its own sequence in the same wall time."""
+    return world * tokens_per_rank / (ms_per_step * 1e-3)
+
+
 def measured_peaks():
     path = os.path.join(ROOT, "MEASURED_PEAKS.json")
     if os.path.exists(path):
@@ -262,12 +275,9 @@ def run_ours(args, cfg, rank, world, local_rank):
     status = B.lca_last_device_status()
     if status != 0:
         raise RuntimeError(f"device status {status}: {B.lca_status_string(status)}")
-    tmax = torch.tensor([total_ms], device=dev, dtype=torch.float64)
-    if dist is not None:
-        dist.all_reduce(tmax, op=dist.ReduceOp.MAX)
-    total_ms = float(tmax.item())
+    total_ms = max_over_ranks(total_ms, dist, dev)
     ms_per_step = total_ms / args.steps
-    value = world * L * cfg.batch / (ms_per_step * 1e-3)
+    value = whole_job_value(L * cfg.batch, world, ms_per_step)
 
     # ---- end to end: pinned host buffers, H2D of the step's inputs and D2H of its output inside the timing
     e2e = None
@@ -288,11 +298,9 @@ def run_ours(args, cfg, rank, world, local_rank):
                 host_out.copy_(out, non_blocking=True)
             e1.record()
             barrier()
-            t = torch.tensor([e0.elapsed_time(e1) / n_e2e], device=dev, dtype=torch.float64)
-            if dist is not None:
-                dist.all_reduce(t, op=dist.ReduceOp.MAX)
-            e2e = dict(value=world * L * cfg.batch / (float(t.item()) * 1e-3), unit=UNIT, h2d_bytes_per_step=h2d,
-                       d2h_bytes_per_step=d2h, steps=n_e2e, ms_per_step=float(t.item()))
+            t_e2e = max_over_ranks(e0.elapsed_time(e1) / n_e2e, dist, dev)
+            e2e = dict(value=whole_job_value(L * cfg.batch, world, t_e2e), unit=UNIT, h2d_bytes_per_step=h2d,
+                       d2h_bytes_per_step=d2h, steps=n_e2e, ms_per_step=t_e2e)
             del host, host_out
         except RuntimeError as ex:      # e.g. not enough pinnable host memory on this machine
             e2e = dict(value=None, unit=UNIT, h2d_bytes_per_step=0, d2h_bytes_per_step=0, error=str(ex)[:200])

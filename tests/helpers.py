@@ -140,3 +140,20 @@ def check_condense(res: dict, cond: dict, kind: str = "mla"):
     # a bf16 rounding boundary (spacing 2^-8 relative) is crossed by about one element in 2500
     assert n_off <= max(2, ulp.size // 250), f"too many c_rep differences: {n_off}/{ulp.size}"
     return dict(crep_one_ulp=n_off, crep_elems=int(ulp.size))
+
+
+def oracle_mla_sampled(ckv, kr, q_tail_sem, q_tail_pos, q_rows_sem, q_rows_pos, rows, g, w, scale, heads=None):
+    """Oracle for one full-size MLA sequence when only some query rows are on the host: the
+    condensation of the whole sequence plus the listed prefill rows (torch bf16 CPU tensors in)."""
+    ckv64, kr64 = O.torch_bf16_to_f64(ckv), O.torch_bf16_to_f64(kr)
+    qbar = O.mla_summary_query(O.torch_bf16_to_f64(q_tail_sem), O.torch_bf16_to_f64(q_tail_pos))
+    cond = O.mla_condense(qbar, ckv64, kr64, g, w, f32(scale))
+    m = cond["m"]
+    rep_sem = O.bits_to_f64(cond["cache_sem_bits"][:m]) if m else None
+    rep_pos = O.bits_to_f64(cond["cache_pos_bits"][:m]) if m else None
+    qs, qp = q_rows_sem, q_rows_pos
+    if heads is not None:
+        qs, qp = qs[:, heads], qp[:, heads]
+    out, lse = O.mla_prefill_rows(O.torch_bf16_to_f64(qs), O.torch_bf16_to_f64(qp), np.asarray(rows, dtype=np.int64),
+                                  ckv64, kr64, rep_sem, rep_pos, g, w, f32(scale))
+    return dict(cond=cond, out=out, lse=lse)

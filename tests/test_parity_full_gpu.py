@@ -1,0 +1,120 @@
+"""GPU parity at the full benchmark sizes, in the launch configuration bench.py times.
+
+The oracle cannot compute 131072 x 128 output rows, so the condensed cache is compared in full
+(anchors, copied rows, representatives) and the attention output on a stratified sample of query
+positions (window / group boundaries, both ends, seeded uniform positions) with all heads.
+"""
+import numpy as np
+import pytest
+import torch
+
+from oracle import lca_oracle as O
+from paper_2604_12452_b200 import inputs as I
+from tests import helpers as Hh
+
+pytestmark = pytest.mark.gpu
+DEV = "cuda:0"
+
+
+@pytest.fixture(scope="module")
+def B():
+    from paper_2604_12452_b200 import build
+    build.build()
+    from paper_2604_12452_b200 import binding
+    return binding
+
+
+def one_seq(cond, b=0):
+    r = dict(cond)
+    for key in ("cache_sem", "cache_pos", "anchor_idx"):
+        r[key] = cond[key][b]
+    return r
+
+
+def check_mla_full(B, name, n_uniform):
+    cfg = I.CONFIGS[name]
+    L, g, w = cfg.seq_len, cfg.group_size, cfg.window
+    inp = I.make_mla_inputs(cfg, DEV)
+    p = B.params_from_config(cfg, batch=1)
+    cond = B.condense(p, inp["q_sem"][L - g:], inp["q_pos"][L - g:], inp["ckv"], inp["kr"])
+    out, lse = B.prefill_attention(p, inp["q_sem"], inp["q_pos"], inp["ckv"], inp["kr"], cond["cache_sem"],
+                                   cond["cache_pos"], want_lse=True)
+    torch.cuda.synchronize()
+    assert B.lca_last_device_status() == 0
+    needles = [int(x) for x in I.needle_positions(cfg)]
+    extra = [n + d for n in needles[:4] for d in (-1, 0, 1)] + [8191, 8192, 8193]
+    rows = Hh.sample_positions(L, g, w, extra=extra, n_uniform=n_uniform, seed=3)
+    idx = torch.from_numpy(rows).to(DEV)
+    ref = Hh.oracle_mla_sampled(inp["ckv"].cpu(), inp["kr"].cpu(), inp["q_sem"][L - g:].cpu(), inp["q_pos"][L - g:].cpu(),
+                                inp["q_sem"][idx].cpu(), inp["q_pos"][idx].cpu(), rows, g, w, cfg.softmax_scale)
+    Hh.check_condense(one_seq(cond), ref["cond"])
+    st = Hh.check_outputs(out[0][idx], ref["out"], f"{name} sampled rows")
+    np.testing.assert_allclose(lse[0][idx].cpu().numpy(), ref["lse"], atol=2e-3, rtol=1e-4)
+    return st
+
+
+def test_config2_mla_32k_full_size(B):
+    check_mla_full(B, "mla_32k", n_uniform=40)
+
+
+def test_config3_mla_128k_full_size(B):
+    check_mla_full(B, "mla_128k", n_uniform=24)
+
+
+def test_config5_gqa_64k_full_size(B):
+    cfg = I.CONFIGS["gqa_64k"]
+    L, g, w = cfg.seq_len, cfg.group_size, cfg.window
+    inp = I.make_gqa_inputs(cfg, DEV)
+    p = B.params_from_config(cfg, batch=1)
+    cond = B.condense(p, None, inp["q"][L - g:], inp["v"], inp["k"])
+    out, _ = B.prefill_attention(p, None, inp["q"], inp["v"], inp["k"], cond["cache_sem"], cond["cache_pos"])
+    torch.cuda.synchronize()
+    assert B.lca_last_device_status() == 0
+    rows = Hh.sample_positions(L, g, w, n_uniform=24, seed=5)
+    idx = torch.from_numpy(rows).to(DEV)
+    k64, v64 = O.torch_bf16_to_f64(inp["k"].cpu()), O.torch_bf16_to_f64(inp["v"].cpu())
+    qbar = O.gqa_summary_query(O.torch_bf16_to_f64(inp["q"][L - g:].cpu()), cfg.n_kv_heads)
+    rc = O.gqa_condense(qbar, k64, v64, g, w, Hh.f32(cfg.softmax_scale))
+    Hh.check_condense(one_seq(cond), rc, kind="gqa")
+    m = rc["m"]
+    ro, _ = O.gqa_prefill_rows(O.torch_bf16_to_f64(inp["q"][idx].cpu()), rows, k64, v64, O.bits_to_f64(rc["cache_k_bits"][:m]),
+                               O.bits_to_f64(rc["cache_v_bits"][:m]), g, w, Hh.f32(cfg.softmax_scale))
+    Hh.check_outputs(out[0][idx], ro, "gqa_64k sampled rows")
+
+
+def test_config4_batched_condense_and_decode_full_size(B):
+    cfg = I.CONFIGS["mla_decode"]
+    Bsz, L, g, w, H = cfg.batch, cfg.seq_len, cfg.group_size, cfg.window, cfg.n_q_heads
+    ckv = torch.empty((Bsz, L, 512), dtype=torch.bfloat16, device=DEV)
+    kr = torch.empty((Bsz, L, 64), dtype=torch.bfloat16, device=DEV)
+    qts = torch.empty((Bsz, g, H, 512), dtype=torch.bfloat16, device=DEV)
+    qtp = torch.empty((Bsz, g, H, 64), dtype=torch.bfloat16, device=DEV)
+    for b in range(Bsz):
+        one = I.make_mla_inputs(cfg, DEV, batch_index=b, q_positions=slice(L - g, L))
+        ckv[b], kr[b], qts[b], qtp[b] = one["ckv"], one["kr"], one["q_sem"], one["q_pos"]
+    p = B.params_from_config(cfg, batch=Bsz)
+    m, k = B.lca_partition(p)
+    cond = B.condense(p, qts, qtp, ckv, kr)
+    cap = m + k + 1
+    dsem = torch.zeros((Bsz, cap, 1, 512), dtype=torch.bfloat16, device=DEV)
+    dpos = torch.zeros((Bsz, cap, 1, 64), dtype=torch.bfloat16, device=DEV)
+    dsem[:, :m + k] = cond["cache_sem"]
+    dpos[:, :m + k] = cond["cache_pos"]
+    gen = torch.Generator(device=DEV)
+    gen.manual_seed(77)
+    dsem[:, m + k] = torch.randn((Bsz, 1, 512), generator=gen, device=DEV).bfloat16()
+    dpos[:, m + k] = torch.randn((Bsz, 1, 64), generator=gen, device=DEV).bfloat16()
+    qs = torch.randn((Bsz, H, 512), generator=gen, device=DEV).bfloat16()
+    qp = torch.randn((Bsz, H, 64), generator=gen, device=DEV).bfloat16()
+    rows = torch.full((Bsz,), cap, dtype=torch.int32, device=DEV)
+    out, lse = B.decode_attention(p, qs, qp, dsem, dpos, rows, m, want_lse=True)
+    torch.cuda.synchronize()
+    assert B.lca_last_device_status() == 0
+    for b in (0, 1, 31, 63):
+        qbar = O.mla_summary_query(O.torch_bf16_to_f64(qts[b].cpu()), O.torch_bf16_to_f64(qtp[b].cpu()))
+        rc = O.mla_condense(qbar, O.torch_bf16_to_f64(ckv[b].cpu()), O.torch_bf16_to_f64(kr[b].cpu()), g, w, Hh.f32(cfg.softmax_scale))
+        Hh.check_condense(one_seq(cond, b), rc)
+        ro, rl = O.mla_decode(O.torch_bf16_to_f64(qs[b].cpu()), O.torch_bf16_to_f64(qp[b].cpu()), O.bits_to_f64(Hh.bits(dsem[b, :, 0])),
+                              O.bits_to_f64(Hh.bits(dpos[b, :, 0])), m, Hh.f32(cfg.softmax_scale))
+        Hh.check_outputs(out[b], ro, f"decode seq {b}")
+        np.testing.assert_allclose(lse[b].cpu().numpy(), rl, atol=2e-3, rtol=1e-4)
