@@ -398,13 +398,37 @@ def measure_decode_config(B, dev, batch, peaks, warmup=3, iters=5):
     out = torch.empty((batch, H, cfg.d_sem), dtype=torch.bfloat16, device=dev)
     wsd = B.workspace(p, B.LCA_WS_DECODE, dev)
     t_dec = time_cuda(lambda: B.decode_attention(p, q_new_sem, q_new_pos, dsem, dpos, rows, m, out=out, ws=wsd), warmup, iters)
+    # online cache update (Sec. 4.3) at the moment every sequence has w + g buffered tokens
+    upd = None
+    try:
+        cap_u = m + cfg.window + g
+        usem = torch.randn((batch, cap_u, 1, cfg.d_sem), generator=gen, device=dev).bfloat16()
+        upos = torch.randn((batch, cap_u, 1, cfg.d_pos), generator=gen, device=dev).bfloat16()
+        wsu = B.workspace(p, B.LCA_WS_UPDATE, dev)
+        times = []
+        for _ in range(3):
+            n_rep_t = torch.full((batch,), m, dtype=torch.int32, device=dev)
+            rows_t = torch.full((batch,), cap_u, dtype=torch.int32, device=dev)
+            torch.cuda.synchronize()
+            e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            e0.record()
+            B.decode_update(p, q_tail_sem, q_tail_pos, usem, upos, n_rep_t, rows_t, ws=wsu)
+            e1.record()
+            torch.cuda.synchronize()
+            times.append(e0.elapsed_time(e1))
+        upd = dict(us_per_update_all_sequences=min(times) * 1e3, amortised_us_per_token=min(times) * 1e3 / g,
+                   note="every g-th decode step: summary query, condense the earliest g buffered tokens, move the window up")
+        del usem, upos
+    except Exception as ex:
+        upd = dict(error=str(ex)[:200])
     flops = float(batch) * H * cap * 2.0 * (cfg.d_sem + cfg.d_pos + cfg.d_sem)
     kv_bytes = float(batch) * cap * (cfg.d_sem + cfg.d_pos) * 2
     full_bytes = float(batch) * (L + 1) * (cfg.d_sem + cfg.d_pos) * 2
     return dict(workload=f"mla_decode: batch {batch}, contexts of {L} tokens, H={H}, g={g}, w={cfg.window}",
                 condense=dict(ms=t_cond, bytes=cbytes, gbs=cbytes / t_cond / 1e6, frac_of_measured_hbm=cbytes / t_cond / 1e6 / peaks["hbm_gbs"]),
                 decode=dict(us=t_dec * 1e3, rows_per_seq=cap, tflops=flops / t_dec / 1e9, kv_gbs=kv_bytes / t_dec / 1e6,
-                            kv_bytes_condensed=kv_bytes, kv_bytes_full_mla=full_bytes, kv_reduction=1.0 - kv_bytes / full_bytes))
+                            kv_bytes_condensed=kv_bytes, kv_bytes_full_mla=full_bytes, kv_reduction=1.0 - kv_bytes / full_bytes),
+                online_update=upd)
 
 
 def measure_gqa_config(B, dev, peaks, warmup=3, iters=5):

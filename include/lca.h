@@ -51,7 +51,7 @@ typedef enum lca_status {
 } lca_status;
 
 enum { LCA_VARIANT_MLA = 0, LCA_VARIANT_GQA = 1 };
-enum { LCA_WS_CONDENSE = 0, LCA_WS_PREFILL = 1, LCA_WS_DECODE = 2 };
+enum { LCA_WS_CONDENSE = 0, LCA_WS_PREFILL = 1, LCA_WS_DECODE = 2, LCA_WS_UPDATE = 3 };
 
 /* Problem statement = the REQUIRE line of Alg. 1 (L, C^KV, K^R, Q, w, g) plus the head layout.
  *   MLA: n_kv_heads = 1, d_sem = d_c (512), d_pos = d_R (64); logits use [sem | pos], values = sem.
@@ -163,6 +163,28 @@ int lca_decode_attention(const lca_params* p, const void* q_sem, const void* q_p
                          const void* cache_sem, const void* cache_pos, const int32_t* cache_rows,
                          int32_t cache_row_capacity, int32_t n_rep, void* out, float* lse_opt,
                          void* ws, size_t ws_bytes, void* stream);
+
+/* Online cache update while decoding (Sec. 4.3 "Decoding and Online Cache Update").  The caller
+ * appends the row of every newly generated token after the valid rows of its sequence and counts
+ * it in cache_rows[b].  This call then looks at every sequence: when its uncondensed tokens
+ * (cache_rows[b] - n_rep[b]) have reached window + group_size, the EARLIEST group_size of them are
+ * condensed into one representative with the summary query of the last queries (importance
+ * scores as in Sec. 4.2, Eq. 6 softmax, Eq. 7 pooling, Eq. 8 anchor), the representative is
+ * written to row n_rep[b], the remaining tokens move up by group_size - 1 rows, n_rep[b] grows by
+ * one and cache_rows[b] shrinks by group_size - 1: the cache stays at m + w .. m + w + g - 1 rows
+ * in the layout [representatives ; tokens in order].  Sequences below the threshold are untouched.
+ *   q_tail_sem / q_tail_pos / q_tail_batch_stride / qbar_opt: the last n_summary_q (0 = g) queries
+ *       of each sequence or a ready summary query, exactly as for lca_condense
+ *   cache_sem [B, cache_row_capacity, n_kv_heads, d_sem], cache_pos likewise: in / out
+ *   n_rep [B], cache_rows [B] int32 (device): in / out
+ *   anchor_out [B, n_kv_heads] int32 (device): offset 0..g-1 of the anchor token inside the
+ *       condensed group, or -1 where nothing was condensed
+ *   ws / ws_bytes: >= lca_workspace_bytes(p, LCA_WS_UPDATE); p->seq_len is not used. */
+int lca_decode_update(const lca_params* p, const void* q_tail_sem, const void* q_tail_pos,
+                      int64_t q_tail_batch_stride, const float* qbar_opt, void* cache_sem,
+                      void* cache_pos, int32_t cache_row_capacity, int32_t* n_rep,
+                      int32_t* cache_rows, int32_t* anchor_out, void* ws, size_t ws_bytes,
+                      void* stream);
 
 /* Which attention implementation lca_prefill_attention / lca_decode_attention use:
  *   0 = automatic (tensor-core kernels where the shape is supported, else the scalar kernel),

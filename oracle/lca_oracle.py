@@ -275,3 +275,28 @@ def gqa_decode(q, cache_k, cache_v, n_rep, scale, rep_logit_bias=0.0):
         out[h * rep:(h + 1) * rep] = o
         lse[h * rep:(h + 1) * rep] = l
     return out, lse
+
+
+# ------------------------------------------------------------------- online cache update
+def mla_decode_update(cache_sem_bits: np.ndarray, cache_pos_bits: np.ndarray, n_rep: int, n_rows: int,
+                      qbar: np.ndarray, g: int, w: int, scale: float):
+    """Sec. 4.3 "Decoding and Online Cache Update" for one sequence.
+
+    cache_*_bits [rows, d] are bf16 bit patterns: rows 0..n_rep-1 the representatives, rows
+    n_rep..n_rows-1 the buffered tokens in order.  When the buffer holds w + g tokens, its earliest g
+    tokens are condensed with the summary query q_bar (scores of Sec. 4.2, Eq. 6 softmax, Eq. 7
+    pooling, Eq. 8 anchor) into one representative that is appended to the representatives; the
+    other tokens keep their order.  Returns (cache_sem_bits, cache_pos_bits, n_rep, n_rows, anchor)
+    with anchor = offset of the anchor token in the condensed group, or -1 when nothing happened.
+    """
+    if n_rows - n_rep < w + g:
+        return cache_sem_bits, cache_pos_bits, n_rep, n_rows, -1
+    grp_sem = bits_to_f64(cache_sem_bits[n_rep:n_rep + g])
+    grp_pos = bits_to_f64(cache_pos_bits[n_rep:n_rep + g])
+    r = condense_stream(np.concatenate([grp_sem, grp_pos], axis=1), grp_sem, qbar, g, 0, scale)   # one group
+    assert r["m"] == 1
+    ia = int(r["anchor"][0])
+    new_sem = np.concatenate([cache_sem_bits[:n_rep], round_bf16_bits(r["pooled"]), cache_sem_bits[n_rep + g:n_rows]], axis=0)
+    new_pos = np.concatenate([cache_pos_bits[:n_rep], cache_pos_bits[n_rep + ia:n_rep + ia + 1],
+                              cache_pos_bits[n_rep + g:n_rows]], axis=0)
+    return new_sem, new_pos, n_rep + 1, n_rows - (g - 1), ia

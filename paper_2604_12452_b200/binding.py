@@ -20,7 +20,7 @@ from . import build as _build
 
 LCA_OK = 0
 LCA_VARIANT_MLA, LCA_VARIANT_GQA = 0, 1
-LCA_WS_CONDENSE, LCA_WS_PREFILL, LCA_WS_DECODE = 0, 1, 2
+LCA_WS_CONDENSE, LCA_WS_PREFILL, LCA_WS_DECODE, LCA_WS_UPDATE = 0, 1, 2, 3
 LCA_STATIC_SCRATCH_BYTES = 1 << 20
 LCA_ERR_STATIC_SCRATCH_EXCEEDED = -7
 ATTN_AUTO, ATTN_SCALAR, ATTN_TENSOR = 0, 1, 2
@@ -67,6 +67,8 @@ def _load() -> C.CDLL:
     lib.lca_prefill_attention.argtypes = [P, vp, vp, vp, vp, vp, vp, vp, vp, vp, sz, vp]
     lib.lca_decode_attention.restype = C.c_int
     lib.lca_decode_attention.argtypes = [P, vp, vp, vp, vp, vp, i32, i32, vp, vp, vp, sz, vp]
+    lib.lca_decode_update.restype = C.c_int
+    lib.lca_decode_update.argtypes = [P, vp, vp, i64, vp, vp, vp, i32, vp, vp, vp, vp, sz, vp]
     lib.lca_last_device_status.restype = C.c_int
     lib.lca_last_device_status.argtypes = [vp]
     return lib
@@ -162,6 +164,14 @@ def lca_decode_attention(params, q_sem, q_pos, cache_sem, cache_pos, cache_rows,
                                          _stream(stream)))
 
 
+def lca_decode_update(params, q_tail_sem, q_tail_pos, q_tail_batch_stride, qbar_opt, cache_sem, cache_pos,
+                      cache_row_capacity, n_rep, cache_rows, anchor_out, ws, ws_bytes=None, stream=None) -> int:
+    wsb = _nbytes(ws) if ws_bytes is None else int(ws_bytes)
+    return int(_lib.lca_decode_update(C.byref(params), _ptr(q_tail_sem), _ptr(q_tail_pos), int(q_tail_batch_stride),
+                                      _ptr(qbar_opt), _ptr(cache_sem), _ptr(cache_pos), int(cache_row_capacity),
+                                      _ptr(n_rep), _ptr(cache_rows), _ptr(anchor_out), _ptr(ws), wsb, _stream(stream)))
+
+
 def lca_last_device_status(stream=None) -> int:
     return int(_lib.lca_last_device_status(_stream(stream)))
 
@@ -249,3 +259,17 @@ def decode_attention(params: LcaParams, q_sem, q_pos, cache_sem, cache_pos, cach
                               ws, stream=stream)
     _check(st, "lca_decode_attention")
     return out, lse
+
+
+def decode_update(params: LcaParams, q_tail_sem, q_tail_pos, cache_sem, cache_pos, n_rep, cache_rows,
+                  qbar: Optional[torch.Tensor] = None, ws=None, stream=None):
+    """Run lca_decode_update in place on the cache buffers and counters; returns anchor offsets [B, Hkv]."""
+    dev = cache_sem.device
+    anchor = torch.empty((params.batch, params.n_kv_heads), dtype=torch.int32, device=dev)
+    if ws is None:
+        ws = workspace(params, LCA_WS_UPDATE, dev)
+    n = params.n_summary_q if params.n_summary_q > 0 else params.group_size
+    st = lca_decode_update(params, q_tail_sem, q_tail_pos, n, qbar, cache_sem, cache_pos, cache_sem.shape[1], n_rep,
+                           cache_rows, anchor, ws, stream=stream)
+    _check(st, "lca_decode_update")
+    return anchor

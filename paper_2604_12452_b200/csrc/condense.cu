@@ -581,6 +581,172 @@ int condense_launch(const CondenseLaunch& c) {
   return cudaGetLastError() == cudaSuccess ? LCA_OK : LCA_ERR_CUDA;
 }
 
+// ------------------------------------------------------------------ online cache update (decode)
+// Sec. 4.3 "Decoding and Online Cache Update": when the buffer of uncondensed tokens of a sequence
+// has grown to window + g rows, its earliest g tokens become one representative (Eq. 6-8 with the
+// summary query of the last g queries), stored right after the existing representatives, and the
+// remaining tokens move up by g - 1 rows, so the cache keeps the layout [representatives ; tokens].
+struct UpdateArgs {
+  bf16* cache_sem; bf16* cache_pos; const double* qbar;
+  int32_t* n_rep; int32_t* n_rows; int32_t* anchor_out;
+  int cap, Hkv, d_sem, d_pos, g, w, sem_in_logit;
+  double scale;
+};
+
+// grid (Hkv, B), 256 threads: condense rows n_rep .. n_rep + g - 1 of one KV stream.  Same
+// arithmetic as the condense kernels: fp64 scores, arg-max on them, fp32 softmax and pooling.
+__global__ void __launch_bounds__(256) update_condense_kernel(UpdateArgs a) {
+  extern __shared__ __align__(16) unsigned char smem_raw[];
+  const int hk = blockIdx.x, b = blockIdx.y;
+  const int nr = a.n_rep[b], rows = a.n_rows[b];
+  const int g = a.g, d_sem = a.d_sem, d_pos = a.d_pos;
+  if (rows - nr < a.w + g || nr + g > a.cap) {           // nothing to condense yet
+    if (threadIdx.x == 0) a.anchor_out[b * a.Hkv + hk] = -1;
+    return;
+  }
+  const int dk = (a.sem_in_logit ? d_sem : 0) + d_pos;
+  bf16* t_sem = reinterpret_cast<bf16*>(smem_raw);
+  bf16* t_pos = t_sem + (size_t)g * d_sem;
+  double* s_q = reinterpret_cast<double*>(t_pos + (size_t)g * d_pos);
+  double* s_s = s_q + dk;
+  float* s_a = reinterpret_cast<float*>(s_s + g);
+  __shared__ int s_anchor;
+  const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5, nwarps = blockDim.x >> 5;
+  const size_t row0 = (size_t)b * a.cap + nr;
+  const size_t rs_sem = (size_t)a.Hkv * d_sem, rs_pos = (size_t)a.Hkv * d_pos;
+  bf16* gs = a.cache_sem + row0 * rs_sem + (size_t)hk * d_sem;
+  bf16* gp = a.cache_pos + row0 * rs_pos + (size_t)hk * d_pos;
+  const int cps = d_sem / 8, cpp = d_pos / 8;
+  for (int x = tid; x < g * cps; x += blockDim.x) {
+    const int i = x / cps, c = x % cps;
+    reinterpret_cast<uint4*>(t_sem + (size_t)i * d_sem)[c] = reinterpret_cast<const uint4*>(gs + (size_t)i * rs_sem)[c];
+  }
+  for (int x = tid; x < g * cpp; x += blockDim.x) {
+    const int i = x / cpp, c = x % cpp;
+    reinterpret_cast<uint4*>(t_pos + (size_t)i * d_pos)[c] = reinterpret_cast<const uint4*>(gp + (size_t)i * rs_pos)[c];
+  }
+  const double* qb = a.qbar + ((size_t)b * a.Hkv + hk) * dk;
+  for (int c = tid; c < dk; c += blockDim.x) s_q[c] = qb[c];
+  __syncthreads();
+  const int sem_off = a.sem_in_logit ? d_sem : 0;
+  for (int i = warp; i < g; i += nwarps) {
+    double acc = 0.0;
+    if (a.sem_in_logit)
+      for (int c = lane; c < d_sem; c += 32) acc = fma(s_q[c], (double)__bfloat162float(t_sem[(size_t)i * d_sem + c]), acc);
+    for (int c = lane; c < d_pos; c += 32) acc = fma(s_q[sem_off + c], (double)__bfloat162float(t_pos[(size_t)i * d_pos + c]), acc);
+    acc = warp_sum(acc);
+    if (lane == 0) s_s[i] = acc * a.scale;
+  }
+  __syncthreads();
+  if (warp == 0) {
+    double best = -INFINITY;
+    int besti = 0x7fffffff;
+    for (int i = lane; i < g; i += 32) { const double v = s_s[i]; if (v > best) { best = v; besti = i; } }
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) {
+      const double ob = __shfl_xor_sync(0xffffffffu, best, o);
+      const int oi = __shfl_xor_sync(0xffffffffu, besti, o);
+      if (ob > best || (ob == best && oi < besti)) { best = ob; besti = oi; }
+    }
+    float z = 0.f;
+    for (int i = lane; i < g; i += 32) { const float e = expf((float)(s_s[i] - best)); s_a[i] = e; z += e; }
+    z = warp_sum(z);
+    const float inv = 1.f / z;
+    for (int i = lane; i < g; i += 32) s_a[i] *= inv;
+    if (lane == 0) s_anchor = besti;
+  }
+  __syncthreads();
+  for (int c = tid; c < d_sem; c += blockDim.x) {
+    float acc = 0.f;
+    for (int i = 0; i < g; ++i) acc = fmaf(s_a[i], __bfloat162float(t_sem[(size_t)i * d_sem + c]), acc);
+    gs[c] = __float2bfloat16_rn(acc);                    // row n_rep of this stream: the new representative
+  }
+  const int ia = s_anchor;
+  for (int c = tid; c < d_pos; c += blockDim.x) gp[c] = t_pos[(size_t)ia * d_pos + c];
+  if (tid == 0) a.anchor_out[b * a.Hkv + hk] = ia;
+}
+
+// grid (B), 1024 threads: move rows [n_rep + g, n_rows) up to [n_rep + 1, ...) and update the
+// counters.  Source and destination overlap (destination below source), so the rows are moved in
+// ascending chunks that are loaded completely before any of their bytes is stored.
+__global__ void __launch_bounds__(1024) update_shift_kernel(UpdateArgs a) {
+  const int b = blockIdx.x;
+  const int nr = a.n_rep[b], rows = a.n_rows[b];
+  if (rows - nr < a.w + a.g || nr + a.g > a.cap) return;
+  const int n_move = rows - (nr + a.g);
+  for (int pass = 0; pass < 2; ++pass) {
+    const size_t row16 = (size_t)a.Hkv * (pass ? a.d_pos : a.d_sem) * sizeof(bf16) / 16;
+    uint4* base = reinterpret_cast<uint4*>(pass ? a.cache_pos : a.cache_sem) + (size_t)b * a.cap * row16;
+    const uint4* src = base + (size_t)(nr + a.g) * row16;
+    uint4* dst = base + (size_t)(nr + 1) * row16;
+    const size_t n16 = (size_t)n_move * row16;
+    if (a.g > 1)
+      for (size_t c0 = 0; c0 < n16; c0 += 4 * 1024) {
+        uint4 v[4];
+#pragma unroll
+        for (int u = 0; u < 4; ++u) { const size_t i = c0 + u * 1024 + threadIdx.x; if (i < n16) v[u] = src[i]; }
+        __syncthreads();
+#pragma unroll
+        for (int u = 0; u < 4; ++u) { const size_t i = c0 + u * 1024 + threadIdx.x; if (i < n16) dst[i] = v[u]; }
+        __syncthreads();
+      }
+  }
+  if (threadIdx.x == 0) { a.n_rep[b] = nr + 1; a.n_rows[b] = rows - (a.g - 1); }
+}
+
+size_t update_workspace_bytes(const lca_params* p) {
+  const int n = p->n_summary_q > 0 ? p->n_summary_q : p->group_size;
+  const int rows = n * (p->n_q_heads / p->n_kv_heads);
+  const size_t chunks = (size_t)(rows + QBAR_ROWS_PER_CHUNK - 1) / QBAR_ROWS_PER_CHUNK;
+  return (size_t)p->batch * p->n_kv_heads * key_dim(p) * (1 + chunks) * sizeof(double);
+}
+
+size_t update_smem_bytes(const lca_params* p) {
+  const size_t g = (size_t)p->group_size;
+  return g * (size_t)(p->d_sem + p->d_pos) * sizeof(bf16) + (size_t)key_dim(p) * sizeof(double) + g * (sizeof(double) + sizeof(float));
+}
+
+int update_launch(const lca_params* p, const void* q_tail_sem, const void* q_tail_pos, int64_t q_tail_batch_stride,
+                  const float* qbar_opt, void* cache_sem, void* cache_pos, int cap, int32_t* n_rep, int32_t* n_rows,
+                  int32_t* anchor_out, void* ws, cudaStream_t stream) {
+  const int dk = key_dim(p), B = p->batch, Hkv = p->n_kv_heads;
+  const int sem_in_logit = p->variant == LCA_VARIANT_MLA;
+  double* qbar = reinterpret_cast<double*>(ws);
+  double* partial = qbar + (size_t)B * Hkv * dk;
+  if (qbar_opt) {
+    const int n = B * Hkv * dk;
+    qbar_widen_kernel<<<(n + 255) / 256, 256, 0, stream>>>(qbar_opt, qbar, n);
+    note_launch();
+  } else {
+    const int n = p->n_summary_q > 0 ? p->n_summary_q : p->group_size;
+    const int rows = n * (p->n_q_heads / Hkv);
+    const int nch = (rows + QBAR_ROWS_PER_CHUNK - 1) / QBAR_ROWS_PER_CHUNK;
+    const int pieces = dk / 8;
+    int row_lanes = 256 / pieces;
+    if (row_lanes < 1) row_lanes = 1;
+    if (row_lanes > 16) row_lanes = 16;
+    const int threads = ((pieces * row_lanes + 31) / 32) * 32;
+    qbar_partial_kernel<<<dim3(nch, Hkv, B), threads, (size_t)row_lanes * dk * sizeof(double), stream>>>(
+        (const bf16*)q_tail_sem, (const bf16*)q_tail_pos, q_tail_batch_stride, n, p->n_q_heads, Hkv, p->d_sem, p->d_pos,
+        sem_in_logit, row_lanes, partial);
+    qbar_final_kernel<<<dim3(Hkv, B), dk < 1024 ? ((dk + 31) / 32) * 32 : 1024, 0, stream>>>(
+        partial, nch, dk, (double)n * (double)(p->n_q_heads / Hkv), qbar);
+    note_launch(2);
+  }
+  UpdateArgs a;
+  a.cache_sem = (bf16*)cache_sem; a.cache_pos = (bf16*)cache_pos; a.qbar = qbar;
+  a.n_rep = n_rep; a.n_rows = n_rows; a.anchor_out = anchor_out;
+  a.cap = cap; a.Hkv = Hkv; a.d_sem = p->d_sem; a.d_pos = p->d_pos; a.g = p->group_size; a.w = p->window;
+  a.sem_in_logit = sem_in_logit; a.scale = (double)p->softmax_scale;
+  const size_t smem = update_smem_bytes(p);
+  if (cudaFuncSetAttribute(update_condense_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) != cudaSuccess)
+    return LCA_ERR_CUDA;
+  update_condense_kernel<<<dim3(Hkv, B), 256, smem, stream>>>(a);
+  update_shift_kernel<<<dim3(B), 1024, 0, stream>>>(a);
+  note_launch(2);
+  return cudaGetLastError() == cudaSuccess ? LCA_OK : LCA_ERR_CUDA;
+}
+
 // ------------------------------------------------------------------ fixed scratch (no allocation)
 // Scratch of lca_condense_static_scratch: part of the library image on every device.  In host
 // code the name below is only a handle; the device address comes from cudaGetSymbolAddress, asked

@@ -82,8 +82,9 @@ int lca_partition(const lca_params* p, int32_t* m, int32_t* k) {
 }
 
 size_t lca_workspace_bytes(const lca_params* p, int32_t which) {
-  if (check_params(p, which != LCA_WS_DECODE) != LCA_OK) return 0;
+  if (check_params(p, which != LCA_WS_DECODE && which != LCA_WS_UPDATE) != LCA_OK) return 0;
   if (which == LCA_WS_CONDENSE) return condense_workspace_bytes(p);
+  if (which == LCA_WS_UPDATE) return update_workspace_bytes(p);
   if (which == LCA_WS_PREFILL || which == LCA_WS_DECODE) {
     AttnProblem a = {};
     a.variant = p->variant; a.batch = p->batch; a.q_len = which == LCA_WS_DECODE ? 1 : p->seq_len;
@@ -189,6 +190,30 @@ int lca_decode_attention(const lca_params* p, const void* q_sem, const void* q_p
   a.cache_sem = cache_sem; a.cache_pos = cache_pos; a.out = out; a.lse = lse_opt;
   a.ws = ws; a.ws_bytes = ws_bytes; a.stream = (cudaStream_t)stream;
   return run_attention(a);
+}
+
+int lca_decode_update(const lca_params* p, const void* q_tail_sem, const void* q_tail_pos,
+                      int64_t q_tail_batch_stride, const float* qbar_opt, void* cache_sem,
+                      void* cache_pos, int32_t cache_row_capacity, int32_t* n_rep,
+                      int32_t* cache_rows, int32_t* anchor_out, void* ws, size_t ws_bytes,
+                      void* stream) {
+  int st = check_params(p, false);
+  if (st != LCA_OK) return st;
+  if (p->group_size <= 0 || p->window < 0 || p->n_summary_q < 0) return LCA_ERR_INVALID_ARG;
+  if (!cache_sem || !cache_pos || !n_rep || !cache_rows || !anchor_out || cache_row_capacity <= 0)
+    return LCA_ERR_INVALID_ARG;
+  if (!qbar_opt) {
+    if (!q_tail_pos || (p->variant == LCA_VARIANT_MLA && !q_tail_sem)) return LCA_ERR_INVALID_ARG;
+    const int n = p->n_summary_q > 0 ? p->n_summary_q : p->group_size;
+    if (q_tail_batch_stride < n) return LCA_ERR_INVALID_ARG;
+    if (!aligned16(q_tail_pos) || (q_tail_sem && !aligned16(q_tail_sem))) return LCA_ERR_MISALIGNED;
+  }
+  if (!aligned16(cache_sem) || !aligned16(cache_pos)) return LCA_ERR_MISALIGNED;
+  if (!ws || !aligned16(ws)) return LCA_ERR_INVALID_ARG;
+  if (ws_bytes < update_workspace_bytes(p)) return LCA_ERR_WORKSPACE_TOO_SMALL;
+  if (update_smem_bytes(p) > 227u * 1024u) return LCA_ERR_UNSUPPORTED_SHAPE;
+  return update_launch(p, q_tail_sem, q_tail_pos, q_tail_batch_stride, qbar_opt, cache_sem, cache_pos,
+                       cache_row_capacity, n_rep, cache_rows, anchor_out, ws, (cudaStream_t)stream);
 }
 
 int lca_last_device_status(void* stream) {

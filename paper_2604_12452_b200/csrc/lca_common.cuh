@@ -59,6 +59,11 @@ struct CondenseLaunch {
 size_t condense_workspace_bytes(const lca_params* p);
 int condense_launch(const CondenseLaunch& a);
 size_t condense_smem_bytes(const lca_params* p);
+size_t update_workspace_bytes(const lca_params* p);
+size_t update_smem_bytes(const lca_params* p);
+int update_launch(const lca_params* p, const void* q_tail_sem, const void* q_tail_pos, int64_t q_tail_batch_stride,
+                  const float* qbar_opt, void* cache_sem, void* cache_pos, int cap, int32_t* n_rep, int32_t* n_rows,
+                  int32_t* anchor_out, void* ws, cudaStream_t stream);
 int condense_take_status();   // nonzero once if a bounded wait of the condense kernel expired
 int condense_static_scratch_address(void** out);   // device address of the library's fixed scratch array
 

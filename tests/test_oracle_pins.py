@@ -448,3 +448,52 @@ def test_mla_cache_layout_and_bit_exact_copies():
     assert np.array_equal(r["cache_pos_bits"][m:], KRb[L - k:])
     assert np.array_equal(r["cache_pos_bits"][:m], KRb[r["anchor"]])    # anchors copied bit-exactly
     assert np.array_equal(r["cache_sem_bits"][:m], O.round_bf16_bits(r["c_rep"]))
+
+
+def test_online_cache_update_reproduces_alg1_on_the_longer_sequence():
+    """Streaming (Sec. 4.3) against Alg. 1: feed tokens one at a time and condense whenever the buffer
+    reaches w + g tokens.  With one fixed summary query for every update the cache after T more tokens
+    must equal the cache Alg. 1 builds from scratch on the longer sequence with that summary query:
+    same representatives, same anchors, same tokens in the window, nothing lost or duplicated."""
+    rng = RNG(21)
+    g, w, dc, dr = 4, 6, 8, 4
+    L0, T = w + 2 * g + 3, 3 * g + 2
+    import torch
+    C = torch.from_numpy(rng.standard_normal((L0 + T, dc))).bfloat16()
+    KR = torch.from_numpy(rng.standard_normal((L0 + T, dr))).bfloat16()
+    Cb, KRb = O.torch_bf16_to_bits(C), O.torch_bf16_to_bits(KR)
+    qbar = rng.standard_normal(dc + dr)
+    scale = 0.3
+    start = O.mla_condense(qbar, O.bits_to_f64(Cb[:L0]), O.bits_to_f64(KRb[:L0]), g, w, scale)
+    sem, pos = start["cache_sem_bits"], start["cache_pos_bits"]
+    n_rep, n_rows = start["m"], start["m"] + start["k"]
+    sizes = []
+    for t in range(L0, L0 + T):
+        sem = np.concatenate([sem[:n_rows], Cb[t:t + 1]], axis=0)          # the new token's row
+        pos = np.concatenate([pos[:n_rows], KRb[t:t + 1]], axis=0)
+        n_rows += 1
+        sem, pos, n_rep, n_rows, _ = O.mla_decode_update(sem, pos, n_rep, n_rows, qbar, g, w, scale)
+        sizes.append(n_rows - n_rep)
+        whole = O.mla_condense(qbar, O.bits_to_f64(Cb[:t + 1]), O.bits_to_f64(KRb[:t + 1]), g, w, scale)
+        assert n_rep == whole["m"] and n_rows == whole["m"] + whole["k"]
+        assert np.array_equal(sem[:n_rows], whole["cache_sem_bits"])
+        assert np.array_equal(pos[:n_rows], whole["cache_pos_bits"])
+    assert min(sizes) == w and max(sizes) == w + g - 1                       # the buffer breathes between w and w+g-1
+
+
+def test_online_cache_update_waits_for_a_full_group_and_zero_query_gives_the_mean():
+    rng = RNG(22)
+    g, w, dc, dr = 4, 3, 6, 2
+    import torch
+    rows = w + g
+    sem = O.torch_bf16_to_bits(torch.from_numpy(rng.standard_normal((rows, dc))).bfloat16())
+    pos = O.torch_bf16_to_bits(torch.from_numpy(rng.standard_normal((rows, dr))).bfloat16())
+    # one token short: untouched
+    s2, p2, nr, nrows, ia = O.mla_decode_update(sem[:-1], pos[:-1], 0, rows - 1, np.zeros(dc + dr), g, w, 1.0)
+    assert ia == -1 and nr == 0 and nrows == rows - 1 and s2 is sem[:-1].base or np.array_equal(s2, sem[:-1])
+    # threshold reached, q_bar = 0: uniform weights -> mean of the earliest g tokens, anchor = first of them
+    s3, p3, nr, nrows, ia = O.mla_decode_update(sem, pos, 0, rows, np.zeros(dc + dr), g, w, 1.0)
+    assert (nr, nrows, ia) == (1, w + 1, 0)
+    mean = O.bits_to_f64(sem[:g]).mean(axis=0)
+    assert np.array_equal(s3[0], O.round_bf16_bits(mean))
+    assert np.array_equal(p3[0], pos[0]) and np.array_equal(s3[1:], sem[g:]) and np.array_equal(p3[1:], pos[g:])

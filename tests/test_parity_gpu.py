@@ -226,3 +226,61 @@ def test_launches_are_counted(B):
     before = B.lca_launch_count()
     run_mla(B, cfg, inp)
     assert B.lca_launch_count() - before >= 5     # 2 summary + condense + 2 copies + attention
+
+
+def test_online_cache_update_matches_oracle_over_many_decode_steps(B):
+    # three sequences in different phases of the buffer; 2 g + 5 generated tokens each, so every
+    # sequence condenses two or three times; a fresh summary query (last g queries) at every step
+    cfg = I.scaled(I.CONFIGS["mla_decode"], batch=3, seq_len=0, n_q_heads=16, group_size=16, window=40)
+    g, w, H, Bsz = cfg.group_size, cfg.window, cfg.n_q_heads, 3
+    cap = 8 + w + g + 4
+    gen = torch.Generator().manual_seed(11)
+    p = B.params_from_config(cfg, batch=Bsz)
+    n_rep0 = [3, 5, 0]
+    n_loc0 = [w + g - 1, w + 3, w]
+    sem = torch.zeros((Bsz, cap, 1, 512), dtype=torch.bfloat16)
+    pos = torch.zeros((Bsz, cap, 1, 64), dtype=torch.bfloat16)
+    for b in range(Bsz):
+        n = n_rep0[b] + n_loc0[b]
+        sem[b, :n, 0] = torch.randn((n, 512), generator=gen).bfloat16()
+        pos[b, :n, 0] = torch.randn((n, 64), generator=gen).bfloat16()
+    d_sem, d_pos = sem.to(DEV), pos.to(DEV)
+    d_nrep = torch.tensor(n_rep0, dtype=torch.int32, device=DEV)
+    d_rows = torch.tensor([a + c for a, c in zip(n_rep0, n_loc0)], dtype=torch.int32, device=DEV)
+    o_sem = [Hh.bits(sem[b, :, 0]) for b in range(Bsz)]
+    o_pos = [Hh.bits(pos[b, :, 0]) for b in range(Bsz)]
+    o_nrep, o_rows = list(n_rep0), [a + c for a, c in zip(n_rep0, n_loc0)]
+    n_updates = 0
+    for step in range(2 * g + 5):
+        new_sem = torch.randn((Bsz, 512), generator=gen).bfloat16()
+        new_pos = torch.randn((Bsz, 64), generator=gen).bfloat16()
+        q_tail_sem = torch.randn((Bsz, g, H, 512), generator=gen).bfloat16()
+        q_tail_pos = torch.randn((Bsz, g, H, 64), generator=gen).bfloat16()
+        rows_now = d_rows.cpu().tolist()
+        for b in range(Bsz):                       # the caller appends the new token's row
+            d_sem[b, rows_now[b], 0] = new_sem[b].to(DEV)
+            d_pos[b, rows_now[b], 0] = new_pos[b].to(DEV)
+        d_rows += 1
+        anchor = B.decode_update(p, q_tail_sem.to(DEV), q_tail_pos.to(DEV), d_sem, d_pos, d_nrep, d_rows)
+        torch.cuda.synchronize()
+        for b in range(Bsz):
+            o_sem[b][o_rows[b]] = Hh.bits(new_sem[b])
+            o_pos[b][o_rows[b]] = Hh.bits(new_pos[b])
+            o_rows[b] += 1
+            qbar = O.mla_summary_query(O.torch_bf16_to_f64(q_tail_sem[b]), O.torch_bf16_to_f64(q_tail_pos[b]))
+            s2, p2, o_nrep[b], o_rows[b], ia = O.mla_decode_update(o_sem[b][:o_rows[b]], o_pos[b][:o_rows[b]], o_nrep[b],
+                                                                 o_rows[b], qbar, g, w, Hh.f32(cfg.softmax_scale))
+            o_sem[b] = np.concatenate([s2, np.zeros((cap - len(s2), 512), np.uint16)])
+            o_pos[b] = np.concatenate([p2, np.zeros((cap - len(p2), 64), np.uint16)])
+            n_updates += ia >= 0
+            assert int(anchor[b, 0]) == ia
+        assert d_nrep.cpu().tolist() == o_nrep and d_rows.cpu().tolist() == o_rows
+        for b in range(Bsz):
+            n, r = o_rows[b], o_nrep[b]
+            got_sem, got_pos = Hh.bits(d_sem[b, :n, 0]), Hh.bits(d_pos[b, :n, 0])
+            assert np.array_equal(got_pos, o_pos[b][:n])                       # anchors and tokens: bit copies
+            assert np.array_equal(got_sem[r:], o_sem[b][r:n])                  # buffered tokens in order
+            ulp = Hh.bf16_ulp_distance(got_sem[:r], o_sem[b][:r])
+            assert (ulp <= 1).all()                                            # representatives: fp32 pooling
+            o_sem[b][:r] = got_sem[:r]                                         # carry the device's rounding forward
+    assert n_updates >= 6
