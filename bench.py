@@ -473,13 +473,45 @@ def measure_dense_comparison(B, dev, peaks, iters=2):
     return res
 
 
+def measure_scaling(B, dev, peaks, lengths=(65536, 131072, 262144, 524288, 1048576), dense_up_to=131072):
+    """Context-length scaling with the paper's own hyper-parameters (g = 16, w = 1024) on a
+    DeepSeek-V2-Lite-shaped layer (16 heads): prefill time of LCA and, while affordable, of dense
+    absorbed MLA through the same kernel; KV-cache rows kept."""
+    rows = []
+    for L in lengths:
+        cfg = I.scaled(I.CONFIGS["mla_32k"], name=f"v2lite_{L}", seq_len=L, group_size=16, window=1024, needle_every=4096)
+        g = cfg.group_size
+        inp = I.make_mla_inputs(cfg, dev)
+        out = torch.empty((1, L, cfg.n_q_heads, cfg.d_sem), dtype=torch.bfloat16, device=dev)
+        p = B.params_from_config(cfg, batch=1)
+        m, k = B.lca_partition(p)
+        cond = B.condense(p, inp["q_sem"][L - g:], inp["q_pos"][L - g:], inp["ckv"], inp["kr"])
+        wsc = B.workspace(p, B.LCA_WS_CONDENSE, dev)
+        t_c = time_cuda(lambda: B.condense(p, inp["q_sem"][L - g:], inp["q_pos"][L - g:], inp["ckv"], inp["kr"], out=cond, ws=wsc), 1, 2)
+        t_a = time_cuda(lambda: B.prefill_attention(p, inp["q_sem"], inp["q_pos"], inp["ckv"], inp["kr"], cond["cache_sem"],
+                                                    cond["cache_pos"], out=out), 1, 2)
+        row = dict(seq_len=L, cache_rows=m + k, kv_reduction=1.0 - (m + k) / L, condense_ms=t_c, attention_ms=t_a,
+                   attention_tflops=attention_flops(cfg) / t_a / 1e9, tokens_per_s=L / ((t_c + t_a) * 1e-3))
+        if L <= dense_up_to:
+            cd = I.scaled(cfg, window=L)
+            pd = B.params_from_config(cd, batch=1)
+            cdn = B.condense(pd, inp["q_sem"][L - g:], inp["q_pos"][L - g:], inp["ckv"], inp["kr"])
+            t_d = time_cuda(lambda: B.prefill_attention(pd, inp["q_sem"], inp["q_pos"], inp["ckv"], inp["kr"], cdn["cache_sem"],
+                                                        cdn["cache_pos"], out=out), 1, 1)
+            row.update(dense_attention_ms=t_d, dense_tflops=attention_flops(cd) / t_d / 1e9, speedup_over_dense=t_d / (t_c + t_a))
+        rows.append(row)
+        del inp, out, cond
+        torch.cuda.empty_cache()
+    return dict(workload="V2-Lite-shaped layer, H=16, paper defaults g=16, w=1024", rows=rows)
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
     ap.add_argument("--steps", type=int, default=5)
     ap.add_argument("--warmup", type=int, default=3)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
-    ap.add_argument("--config", default="mla_128k", choices=list(I.CONFIGS.keys()),
+    ap.add_argument("--config", default="mla_128k", choices=list(I.CONFIGS.keys()) + ["scaling"],
                     help="mla_128k is the benchmark; mla_1k / mla_32k run the same step on configs 1 / 2; mla_decode and "
                          "gqa_64k print the side measurements of configs 4 / 5 on their own (used for profiling)")
     ap.add_argument("--attn-impl", type=int, default=0, help="0 auto, 1 scalar kernel, 2 tensor-core kernel")
@@ -494,7 +526,7 @@ def main():
     rank = int(os.environ.get("RANK", "0"))
     world = int(os.environ.get("WORLD_SIZE", "1"))
     local_rank = int(os.environ.get("LOCAL_RANK", "0"))
-    cfg = I.CONFIGS[args.config]
+    cfg = I.CONFIGS.get(args.config, I.CONFIGS["mla_128k"])
     if args.impl == "reference":
         run_reference(args, cfg, rank, world)
         return
@@ -504,6 +536,13 @@ def main():
     build.build()
     from paper_2604_12452_b200 import binding as B
     B.lca_set_attention_impl(args.attn_impl)
+    if args.config == "scaling":
+        if rank == 0:
+            torch.cuda.set_device(local_rank)
+            res = measure_scaling(B, f"cuda:{local_rank}", measured_peaks())
+            print(json.dumps(dict(metric="side_measurement", config=dict(workload=res["workload"]), n_gpus=1, data="synthetic",
+                                  result=res, gpu_launches=None)))
+        return
     if args.config in ("mla_decode", "gqa_64k"):
         if rank == 0:
             torch.cuda.set_device(local_rank)
