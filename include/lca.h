@@ -51,6 +51,11 @@ typedef enum lca_status {
 } lca_status;
 
 enum { LCA_VARIANT_MLA = 0, LCA_VARIANT_GQA = 1 };
+/* How a group is reduced to one vector (Table 5 ablates these for c_rep and for k^R_rep):
+ *   MAXPOOL  element-wise maximum over the g tokens      MEANPOOL  plain mean
+ *   WEIGHTED sum_i alpha_i x_i with the Eq. 6 weights    MAXSEL    the vector of the arg-max token (Eq. 8)
+ * DEFAULT is the method itself: WEIGHTED for the semantic part (Eq. 7), MAXSEL for the positional part. */
+enum { LCA_REDUCE_DEFAULT = 0, LCA_REDUCE_MAXPOOL = 1, LCA_REDUCE_MEANPOOL = 2, LCA_REDUCE_WEIGHTED = 3, LCA_REDUCE_MAXSEL = 4 };
 enum { LCA_WS_CONDENSE = 0, LCA_WS_PREFILL = 1, LCA_WS_DECODE = 2, LCA_WS_UPDATE = 3 };
 
 /* Problem statement = the REQUIRE line of Alg. 1 (L, C^KV, K^R, Q, w, g) plus the head layout.
@@ -61,7 +66,9 @@ enum { LCA_WS_CONDENSE = 0, LCA_WS_PREFILL = 1, LCA_WS_DECODE = 2, LCA_WS_UPDATE
  *                Table 8 varies it); 0 means g; clamped to L.
  *   softmax_scale: 1/sqrt(d_h), used for the importance scores (Sec. 4.2) and the attention (Eq. 10).
  *   rep_logit_bias: added to the logit of every representative; 0 = Alg. 1 as printed,
- *                log(g) = the group-size-weighted form analysed in the proof of Theorem 1. */
+ *                log(g) = the group-size-weighted form analysed in the proof of Theorem 1.
+ *   sem_reducer / pos_reducer: 0 = the method (Eq. 7 / Eq. 8); other values reproduce the operators
+ *                ablated in Table 5 (lca_condense only; lca_decode_update always uses the method's). */
 typedef struct lca_params {
   int32_t variant;
   int32_t batch;
@@ -75,6 +82,8 @@ typedef struct lca_params {
   int32_t n_summary_q;
   float softmax_scale;
   float rep_logit_bias;
+  int32_t sem_reducer;   /* LCA_REDUCE_*: how lca_condense forms cache_sem[j] (c_rep; GQA: v_rep) */
+  int32_t pos_reducer;   /* LCA_REDUCE_*: how it forms cache_pos[j] (k^R_rep; GQA: k_rep).  anchor_idx is always the arg-max token */
 } lca_params;
 
 /* (m, k) of Sec. 4.2 for one sequence of p->seq_len tokens.  Host only, no device work. */

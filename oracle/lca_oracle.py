@@ -162,13 +162,36 @@ def decode_rows(q: np.ndarray, ckey: np.ndarray, cval: np.ndarray, n_rep: int, s
     return out, lse
 
 
+# --------------------------------------------------------------------- ablation reducers
+def reduce_groups(x: np.ndarray, alpha: np.ndarray, anchor: np.ndarray, g: int, m: int, mode: str) -> np.ndarray:
+    """One vector per group from the g vectors x[j*g:(j+1)*g] (Table 5 operators):
+    "weighted" = sum_i alpha_i x_i (Eq. 7), "maxsel" = x of the arg-max token (Eq. 8),
+    "meanpool" = plain mean, "maxpool" = element-wise maximum."""
+    x = _f64(x)
+    out = np.zeros((m, x.shape[1]))
+    for j in range(m):
+        grp = x[j * g:(j + 1) * g]
+        if mode == "weighted":
+            out[j] = (alpha[j * g:(j + 1) * g, None] * grp).sum(axis=0)
+        elif mode == "maxsel":
+            out[j] = x[anchor[j]]
+        elif mode == "meanpool":
+            out[j] = grp.sum(axis=0) / g
+        elif mode == "maxpool":
+            out[j] = grp.max(axis=0)
+        else:
+            raise ValueError(mode)
+    return out
+
+
 # ------------------------------------------------------------------------------ MLA flavour
 def mla_summary_query(q_sem_tail: np.ndarray, q_pos_tail: np.ndarray) -> np.ndarray:
     """q_bar over [q_latent | q_rope] of the last n positions and all heads -> [d_c + d_R]."""
     return summary_query(np.concatenate([_f64(q_sem_tail), _f64(q_pos_tail)], axis=-1))
 
 
-def mla_condense(qbar: np.ndarray, ckv: np.ndarray, kr: np.ndarray, g: int, w: int, scale: float):
+def mla_condense(qbar: np.ndarray, ckv: np.ndarray, kr: np.ndarray, g: int, w: int, scale: float,
+                 sem_reducer: str = "weighted", pos_reducer: str = "maxsel"):
     """Condensed MLA cache of one sequence (Alg. 1 lines 2-10).
 
     Returns dict with
@@ -184,9 +207,11 @@ def mla_condense(qbar: np.ndarray, ckv: np.ndarray, kr: np.ndarray, g: int, w: i
     r = condense_stream(key, ckv, qbar, g, w, scale)
     m, k = r["m"], r["k"]
     L = ckv.shape[0]
-    cache_sem = np.concatenate([r["pooled"], ckv[L - k:]], axis=0)
-    cache_pos = np.concatenate([kr[r["anchor"]] if m else np.zeros((0, kr.shape[1])), kr[L - k:]], axis=0)
-    return dict(scores=r["scores"], alpha=r["alpha"], c_rep=r["pooled"], anchor=r["anchor"],
+    c_rep = r["pooled"] if sem_reducer == "weighted" else reduce_groups(ckv, r["alpha"], r["anchor"], g, m, sem_reducer)
+    k_rep = reduce_groups(kr, r["alpha"], r["anchor"], g, m, pos_reducer)
+    cache_sem = np.concatenate([c_rep, ckv[L - k:]], axis=0)
+    cache_pos = np.concatenate([k_rep, kr[L - k:]], axis=0)
+    return dict(scores=r["scores"], alpha=r["alpha"], c_rep=c_rep, anchor=r["anchor"],
                 cache_sem_bits=round_bf16_bits(cache_sem), cache_pos_bits=round_bf16_bits(cache_pos),
                 m=m, k=k)
 

@@ -24,6 +24,7 @@ LCA_WS_CONDENSE, LCA_WS_PREFILL, LCA_WS_DECODE, LCA_WS_UPDATE = 0, 1, 2, 3
 LCA_STATIC_SCRATCH_BYTES = 1 << 20
 LCA_ERR_STATIC_SCRATCH_EXCEEDED = -7
 ATTN_AUTO, ATTN_SCALAR, ATTN_TENSOR = 0, 1, 2
+REDUCE_DEFAULT, REDUCE_MAXPOOL, REDUCE_MEANPOOL, REDUCE_WEIGHTED, REDUCE_MAXSEL = 0, 1, 2, 3, 4
 
 
 class LcaParams(C.Structure):
@@ -32,7 +33,7 @@ class LcaParams(C.Structure):
                 ("n_q_heads", C.c_int32), ("n_kv_heads", C.c_int32), ("d_sem", C.c_int32),
                 ("d_pos", C.c_int32), ("group_size", C.c_int32), ("window", C.c_int32),
                 ("n_summary_q", C.c_int32), ("softmax_scale", C.c_float),
-                ("rep_logit_bias", C.c_float)]
+                ("rep_logit_bias", C.c_float), ("sem_reducer", C.c_int32), ("pos_reducer", C.c_int32)]
 
 
 class LcaError(RuntimeError):
@@ -182,7 +183,7 @@ def make_params(variant: str, batch: int, seq_len: int, n_q_heads: int, n_kv_hea
                 n_summary_q: int = 0, rep_logit_bias: float = 0.0) -> LcaParams:
     v = LCA_VARIANT_MLA if variant == "mla" else LCA_VARIANT_GQA
     return LcaParams(v, batch, seq_len, n_q_heads, n_kv_heads, d_sem, d_pos, group_size, window,
-                     n_summary_q, softmax_scale, rep_logit_bias)
+                     n_summary_q, softmax_scale, rep_logit_bias, 0, 0)
 
 
 def params_from_config(cfg, batch: Optional[int] = None, **kw) -> LcaParams:

@@ -88,6 +88,7 @@ struct CondenseArgs {
   const bf16* kv_sem; const bf16* kv_pos; const double* qbar;
   bf16* cache_sem; bf16* cache_pos; int32_t* anchor; double* scores;
   int L, Hkv, d_sem, d_pos, g, m, cache_rows, sem_in_logit;
+  int sem_reducer, pos_reducer;   // LCA_REDUCE_* with DEFAULT already resolved
   long long n_groups;          // B * Hkv * m
   double scale;
 };
@@ -209,29 +210,32 @@ condense_kernel(CondenseArgs a) {
     }
     __syncthreads();
 
-    // 3. weighted pooling c_rep = sum_i alpha_i c_i (Eq. 7), one column pair per thread, fp32
+    // 3. the representative: semantic part (Eq. 7 by default) and positional part (Eq. 8 by
+    //    default), each reduced over the g tokens by the chosen operator, one column pair per thread
     const size_t out_row = (size_t)b * a.cache_rows + j;
-    {
-      bf16* dst = a.cache_sem + (out_row * a.Hkv + hk) * d_sem;
-      for (int pr = tid; pr < d_sem / 2; pr += blockDim.x) {
-        float a0 = 0.f, a1 = 0.f;
+    const int ia = s_anchor;
+    auto reduce = [&](const bf16* tile, int d, int mode, bf16* dst, int tid0) {
+      for (int pr = tid0; pr < d / 2; pr += blockDim.x) {
+        if (mode == LCA_REDUCE_MAXSEL) {
+          *reinterpret_cast<bf162*>(dst + 2 * pr) = *reinterpret_cast<const bf162*>(tile + (size_t)ia * d + 2 * pr);
+          continue;
+        }
+        float a0 = mode == LCA_REDUCE_MAXPOOL ? -INFINITY : 0.f, a1 = a0;
 #pragma unroll 8
         for (int i = 0; i < g; ++i) {
-          const float2 v = __bfloat1622float2(*reinterpret_cast<const bf162*>(t_sem + (size_t)i * d_sem + 2 * pr));
-          const float al = s_a[i];
-          a0 = fmaf(al, v.x, a0);
-          a1 = fmaf(al, v.y, a1);
+          const float2 v = __bfloat1622float2(*reinterpret_cast<const bf162*>(tile + (size_t)i * d + 2 * pr));
+          if (mode == LCA_REDUCE_MAXPOOL) { a0 = fmaxf(a0, v.x); a1 = fmaxf(a1, v.y); }
+          else if (mode == LCA_REDUCE_MEANPOOL) { a0 += v.x; a1 += v.y; }
+          else { const float al = s_a[i]; a0 = fmaf(al, v.x, a0); a1 = fmaf(al, v.y, a1); }
         }
+        if (mode == LCA_REDUCE_MEANPOOL) { a0 /= (float)g; a1 /= (float)g; }
         *reinterpret_cast<bf162*>(dst + 2 * pr) = __floats2bfloat162_rn(a0, a1);
       }
-    }
-    // 4. positional anchor: bit copy of the arg-max token's positional row (threads from the top)
+    };
+    reduce(t_sem, d_sem, a.sem_reducer, a.cache_sem + (out_row * a.Hkv + hk) * d_sem, tid);
+    reduce(t_pos, d_pos, a.pos_reducer, a.cache_pos + (out_row * a.Hkv + hk) * d_pos, blockDim.x - 1 - tid);
     {
-      const int ia = s_anchor;
-      const uint4* src = reinterpret_cast<const uint4*>(t_pos + (size_t)ia * d_pos);
-      uint4* dst = reinterpret_cast<uint4*>(a.cache_pos + (out_row * a.Hkv + hk) * d_pos);
       const int rt = blockDim.x - 1 - tid;
-      for (int c = rt; c < d_pos / 8; c += blockDim.x) dst[c] = src[c];
       if (rt == 0) a.anchor[((size_t)b * a.m + j) * a.Hkv + hk] = j * g + ia;
       if (a.scores) {
         double* sc = a.scores + (((size_t)b * a.Hkv + hk) * a.m + j) * g;
@@ -502,7 +506,9 @@ size_t condense_workspace_bytes(const lca_params* p) {
 }
 
 static bool condense_fast_shape(const lca_params* p) {
-  return p->variant == LCA_VARIANT_MLA && p->d_sem == 512 && p->d_pos == 64 && p->group_size == 64 && p->n_kv_heads == 1;
+  const bool method = (p->sem_reducer == LCA_REDUCE_DEFAULT || p->sem_reducer == LCA_REDUCE_WEIGHTED) &&
+                      (p->pos_reducer == LCA_REDUCE_DEFAULT || p->pos_reducer == LCA_REDUCE_MAXSEL);
+  return method && p->variant == LCA_VARIANT_MLA && p->d_sem == 512 && p->d_pos == 64 && p->group_size == 64 && p->n_kv_heads == 1;
 }
 
 size_t condense_smem_bytes(const lca_params* p) {
@@ -550,6 +556,8 @@ int condense_launch(const CondenseLaunch& c) {
     a.m = (int)m; a.cache_rows = (int)(m + k); a.sem_in_logit = sem_in_logit;
     a.scale = (double)p->softmax_scale;
     a.n_groups = (long long)B * Hkv * m;
+    a.sem_reducer = p->sem_reducer == LCA_REDUCE_DEFAULT ? LCA_REDUCE_WEIGHTED : p->sem_reducer;
+    a.pos_reducer = p->pos_reducer == LCA_REDUCE_DEFAULT ? LCA_REDUCE_MAXSEL : p->pos_reducer;
     int dev = 0, sms = 148;
     if (cudaGetDevice(&dev) == cudaSuccess) cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
     const long long ctas = a.n_groups < sms ? a.n_groups : sms;

@@ -18,6 +18,7 @@ static int check_params(const lca_params* p, bool need_partition) {
   if (p->n_q_heads % p->n_kv_heads != 0) return LCA_ERR_INVALID_ARG;
   if (p->variant == LCA_VARIANT_MLA && p->n_kv_heads != 1) return LCA_ERR_INVALID_ARG;
   if (!(p->softmax_scale > 0.f) || !(p->rep_logit_bias == p->rep_logit_bias)) return LCA_ERR_INVALID_ARG;
+  if (p->sem_reducer < 0 || p->sem_reducer > 4 || p->pos_reducer < 0 || p->pos_reducer > 4) return LCA_ERR_INVALID_ARG;
   if (need_partition) {
     if (p->seq_len <= 0 || p->group_size <= 0 || p->window < 0 || p->n_summary_q < 0)
       return LCA_ERR_INVALID_ARG;

@@ -497,3 +497,31 @@ def test_online_cache_update_waits_for_a_full_group_and_zero_query_gives_the_mea
     mean = O.bits_to_f64(sem[:g]).mean(axis=0)
     assert np.array_equal(s3[0], O.round_bf16_bits(mean))
     assert np.array_equal(p3[0], pos[0]) and np.array_equal(s3[1:], sem[g:]) and np.array_equal(p3[1:], pos[g:])
+
+
+def test_ablation_reducers_have_their_defining_properties():
+    """Table 5 operators: the method's pair is the default; mean pooling is weighted pooling at a zero
+    summary query; max selection returns a member of the group bit for bit; max pooling dominates every
+    member coordinate-wise and is attained; weighted pooling of the rope keys stays in their hull."""
+    rng = RNG(31)
+    L, g, w, dc, dr = 70, 8, 6, 5, 4
+    C, KR = rng.standard_normal((L, dc)), rng.standard_normal((L, dr))
+    qbar = rng.standard_normal(dc + dr)
+    base = O.mla_condense(qbar, C, KR, g, w, 0.4)
+    m = base["m"]
+    same = O.mla_condense(qbar, C, KR, g, w, 0.4, "weighted", "maxsel")
+    assert np.array_equal(base["cache_sem_bits"], same["cache_sem_bits"]) and np.array_equal(base["cache_pos_bits"], same["cache_pos_bits"])
+    mean = O.mla_condense(qbar, C, KR, g, w, 0.4, "meanpool", "meanpool")
+    zero = O.mla_condense(np.zeros(dc + dr), C, KR, g, w, 0.4, "weighted", "weighted")
+    np.testing.assert_allclose(mean["c_rep"], zero["c_rep"], rtol=1e-13, atol=1e-15)
+    sel = O.mla_condense(qbar, C, KR, g, w, 0.4, "maxsel", "maxsel")
+    mx = O.mla_condense(qbar, C, KR, g, w, 0.4, "maxpool", "maxpool")
+    wk = O.mla_condense(qbar, C, KR, g, w, 0.4, "weighted", "weighted")
+    for j in range(m):
+        grp, grk = C[j * g:(j + 1) * g], KR[j * g:(j + 1) * g]
+        assert np.array_equal(sel["c_rep"][j], C[base["anchor"][j]])
+        assert (mx["c_rep"][j] >= grp).all() and all(mx["c_rep"][j][c] in grp[:, c] for c in range(dc))
+        kw = O.bits_to_f64(wk["cache_pos_bits"][j])
+        assert (kw >= grk.min(axis=0) - 0.02).all() and (kw <= grk.max(axis=0) + 0.02).all()
+    # anchors do not depend on the reducers
+    assert np.array_equal(mx["anchor"], base["anchor"]) and np.array_equal(mean["anchor"], base["anchor"])

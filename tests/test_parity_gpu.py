@@ -284,3 +284,32 @@ def test_online_cache_update_matches_oracle_over_many_decode_steps(B):
             assert (ulp <= 1).all()                                            # representatives: fp32 pooling
             o_sem[b][:r] = got_sem[:r]                                         # carry the device's rounding forward
     assert n_updates >= 6
+
+
+REDUCERS = {"maxpool": 1, "meanpool": 2, "weighted": 3, "maxsel": 4}
+
+
+@pytest.mark.parametrize("sem", list(REDUCERS))
+@pytest.mark.parametrize("pos", list(REDUCERS))
+def test_ablation_reducers_match_oracle(B, sem, pos):
+    cfg = I.scaled(I.CONFIGS["mla_1k"], seq_len=400, n_q_heads=4, group_size=32, window=48)
+    inp = I.stress_peaky_queries(I.make_mla_inputs(cfg, "cpu"), cfg)
+    d = to_dev(inp)
+    L, g = cfg.seq_len, cfg.group_size
+    p = B.params_from_config(cfg, batch=1, sem_reducer=REDUCERS[sem], pos_reducer=REDUCERS[pos])
+    cond = B.condense(p, d["q_sem"][L - g:], d["q_pos"][L - g:], d["ckv"], d["kr"])
+    torch.cuda.synchronize()
+    qbar = O.mla_summary_query(O.torch_bf16_to_f64(inp["q_sem"][L - g:]), O.torch_bf16_to_f64(inp["q_pos"][L - g:]))
+    ref = O.mla_condense(qbar, O.torch_bf16_to_f64(inp["ckv"]), O.torch_bf16_to_f64(inp["kr"]), g, cfg.window,
+                         Hh.f32(cfg.softmax_scale), sem, pos)
+    m, k = ref["m"], ref["k"]
+    got_sem, got_pos = Hh.bits(cond["cache_sem"][0, :, 0]), Hh.bits(cond["cache_pos"][0, :, 0])
+    assert np.array_equal(cond["anchor_idx"][0, :, 0].cpu().numpy(), ref["anchor"])
+    assert np.array_equal(got_sem[m:], ref["cache_sem_bits"][m:]) and np.array_equal(got_pos[m:], ref["cache_pos_bits"][m:])
+    for got, want, mode in ((got_sem[:m], ref["cache_sem_bits"][:m], sem), (got_pos[:m], ref["cache_pos_bits"][:m], pos)):
+        if mode in ("maxsel", "maxpool"):
+            assert np.array_equal(got, want)                       # selections and maxima are exact
+        else:
+            ulp = Hh.bf16_ulp_distance(got, want)
+            tiny = np.abs(O.bits_to_f64(got) - O.bits_to_f64(want)) <= 32 * 2.0 ** -24 * 20.0
+            assert ((ulp <= 1) | tiny).all()                       # fp32 sums of g terms against fp64
