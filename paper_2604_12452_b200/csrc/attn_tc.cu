@@ -9,8 +9,8 @@
 //     P  = exp2(S*c - m) with per-row masks only on boundary tiles (4 softmax warps, one row
 //          per thread, S read from TMEM, P written back to TMEM as packed bf16)
 //     O += P V          (tcgen05.mma, A = P from TMEM, B = V tile from shared memory)
-// Roles: warp 0 issues TMA loads, warp 1 owns TMEM and issues every MMA, warps 2..5 do the
-// softmax, the (rare) rescale of O when the running maximum grows by more than 2^8, and the
+// Roles: warp 0 issues TMA loads, warp 1 owns TMEM and issues every MMA, warps 2..9 do the
+// softmax (two threads per row), the (rare) rescale of O when the running maximum grows by more than 2^8, and the
 // epilogue.  Every wait is bounded; on expiry the CTA records a code in a global status word,
 // drains and returns.
 #include <cstdio>
@@ -54,7 +54,8 @@ struct Plan1 {
   static constexpr int OFF_BAR = OFF_V + STAGES * V_STAGE;
   static constexpr int NBAR = 1 + 4 * STAGES + 2 + 2 + 1;
   static constexpr int OFF_MISC = OFF_BAR + NBAR * 8;
-  static constexpr int BYTES = OFF_MISC + 16 + 1024;     // + slack to align the base to 1024 B
+  static constexpr int OFF_RED = OFF_MISC + 16;          // float [3][2][128]: row maxima (two tiles in flight) and row sums
+  static constexpr int BYTES = OFF_RED + 6 * 128 * 4 + 1024;     // + slack to align the base to 1024 B
   // tensor memory columns
   static constexpr int TM_S0 = 0, TM_S1 = BN, TM_O = 2 * BN;
   static constexpr int TM_COLS = 512;
@@ -62,7 +63,7 @@ struct Plan1 {
 };
 
 template <int NK_SEM, int NK_POS, int NV, bool V_IN_K, int STAGES>
-__global__ void __launch_bounds__(192, 1)
+__global__ void __launch_bounds__(320, 1)
 attn_tc1_kernel(const __grid_constant__ TcParams p) {
   using P = Plan1<NK_SEM, NK_POS, NV, V_IN_K, STAGES>;
   constexpr int NK = P::NK;
@@ -110,7 +111,7 @@ attn_tc1_kernel(const __grid_constant__ TcParams p) {
       mbar_init(BAR_KFULL(s), 1); mbar_init(BAR_KEMPTY(s), 1);
       mbar_init(BAR_VFULL(s), 1); mbar_init(BAR_VEMPTY(s), 1);
     }
-    for (int i = 0; i < 2; ++i) { mbar_init(BAR_SFULL(i), 1); mbar_init(BAR_PFULL(i), 128); }
+    for (int i = 0; i < 2; ++i) { mbar_init(BAR_SFULL(i), 1); mbar_init(BAR_PFULL(i), 256); }
     mbar_init(BAR_ODONE, 1);
     *abort_flag = 0;
     fence_mbar_init();
@@ -226,8 +227,13 @@ attn_tc1_kernel(const __grid_constant__ TcParams p) {
     }
     if (ok && n_tiles > 0) issue_pv(n_tiles - 1);
   } else {
-    // =============================================================== softmax / epilogue (128 threads)
-    const int quarter = warp & 3;                 // TMEM lanes this warp may touch
+    // =============================================================== softmax / epilogue (256 threads)
+    // Two threads per query row: warps 2-5 take keys 0..63 of a tile, warps 6-9 keys 64..127 (a
+    // warp may only touch the 32 TMEM lanes of its quarter, warp & 3).  One thread per row was
+    // twice as slow as the tensor core at this head size.  The halves combine their row maxima
+    // through shared memory; that barrier also orders every read of S before any write of P,
+    // which reuses the S columns.
+    const int quarter = warp & 3, half = warp >= 6 ? 1 : 0;
     const int r = quarter * 32 + lane;            // query row of this thread
     const uint32_t lane_base = (uint32_t)(quarter * 32) << 16;
     const int tl = r / p.HB, hl = r % p.HB;
@@ -236,38 +242,55 @@ attn_tc1_kernel(const __grid_constant__ TcParams p) {
     int n_a_row, bias_rows, first_row;
     if (p.decode) { n_a_row = n_a_hi; bias_rows = min(p.n_rep_bias, n_a_row); first_row = 0; }
     else { n_a_row = reps_visible(min(t_row, p.q_len - 1), p.w, p.g); bias_rows = n_a_row; first_row = n_a_row * p.g; }
+    volatile float* red = reinterpret_cast<volatile float*>(base_ptr + P::OFF_RED);          // [3][2][128]
+    volatile int* fail_word = reinterpret_cast<volatile int*>(base_ptr + P::OFF_MISC + 8);   // [2]
+    if (half == 0 && r < 2) fail_word[r] = 0;
+    asm volatile("bar.sync 1, 256;" ::: "memory");
+    // All 256 threads execute exactly one named barrier per tile, whatever happens: a thread whose
+    // wait expired marks the tile's fail word before the barrier and everybody leaves after it.
     float m_ref = -INFINITY, l_sum = 0.f;
     bool ok = true;
     for (int j = 0; j < n_tiles; ++j) {
-      ok = mbar_wait(BAR_SFULL(j & 1), (j >> 1) & 1, abort_flag);
-      ok = __all_sync(0xffffffffu, ok);
-      if (!ok) { if (lane == 0) fail(ERR_WAIT_S_FULL); break; }
-      tc_fence_after();
-      const uint32_t stm = tmem + lane_base + ((j & 1) ? P::TM_S1 : P::TM_S0);
-      uint32_t sr[4][32];
-#pragma unroll
-      for (int q = 0; q < 4; ++q) tmem_ld32(stm + q * 32, sr[q]);
-      tmem_wait_ld();
-      const bool isA = j < nA;
-      const int key0 = isA ? j * BN : first_lo + (j - nA) * BN;
-      bool need_mask;
-      int lo, hi;                                  // visible columns: lo <= c <= hi
-      if (isA) { lo = 0; hi = n_a_row - key0 - 1; need_mask = key0 + BN > n_a_lo; }
-      else { lo = first_row - key0; hi = t_row - key0; need_mask = (key0 < n_a_hi * p.g) || (key0 + BN - 1 > t0); }
-      const int blim = isA ? bias_rows - key0 : 0;  // columns < blim receive the bias
-      float tmax = -INFINITY;
-#pragma unroll
-      for (int q = 0; q < 4; ++q) {
-#pragma unroll
-        for (int i = 0; i < 32; ++i) {
-          const int c = q * 32 + i;
-          float s = __uint_as_float(sr[q][i]) * p.scale_log2;
-          if (isA && p.bias_log2 != 0.f && c < blim) s += p.bias_log2;
-          if (need_mask && (c < lo || c > hi)) s = -INFINITY;
-          sr[q][i] = __float_as_uint(s);
-          tmax = fmaxf(tmax, s);
-        }
+      if (ok) {
+        ok = mbar_wait(BAR_SFULL(j & 1), (j >> 1) & 1, abort_flag);
+        if (!ok && lane == 0) fail(ERR_WAIT_S_FULL);
       }
+      ok = __all_sync(0xffffffffu, ok);
+      const uint32_t stm = tmem + lane_base + ((j & 1) ? P::TM_S1 : P::TM_S0);
+      uint32_t sr[2][32];
+      float tmax = -INFINITY;
+      const bool isA = j < nA;
+      const int key0 = (isA ? j * BN : first_lo + (j - nA) * BN) + 64 * half;   // first key of this thread's columns
+      if (ok) {
+        tc_fence_after();
+        tmem_ld32(stm + 64 * half, sr[0]);
+        tmem_ld32(stm + 64 * half + 32, sr[1]);
+        tmem_wait_ld();
+        const int tile_key0 = key0 - 64 * half;
+        bool need_mask;
+        int lo, hi;                                  // visible columns of this thread: lo <= c <= hi
+        if (isA) { lo = 0; hi = n_a_row - key0 - 1; need_mask = tile_key0 + BN > n_a_lo; }
+        else { lo = first_row - key0; hi = t_row - key0; need_mask = (tile_key0 < n_a_hi * p.g) || (tile_key0 + BN - 1 > t0); }
+        const int blim = isA ? bias_rows - key0 : 0;  // columns < blim receive the bias
+#pragma unroll
+        for (int q = 0; q < 2; ++q) {
+#pragma unroll
+          for (int i = 0; i < 32; ++i) {
+            const int c = q * 32 + i;
+            float s = __uint_as_float(sr[q][i]) * p.scale_log2;
+            if (isA && p.bias_log2 != 0.f && c < blim) s += p.bias_log2;
+            if (need_mask && (c < lo || c > hi)) s = -INFINITY;
+            sr[q][i] = __float_as_uint(s);
+            tmax = fmaxf(tmax, s);
+          }
+        }
+      } else {
+        fail_word[j & 1] = 1;
+      }
+      red[((j & 1) * 2 + half) * 128 + r] = tmax;
+      asm volatile("bar.sync 1, 256;" ::: "memory");
+      if (fail_word[j & 1]) { ok = false; continue; }          // uniform over the 256 threads
+      tmax = fmaxf(tmax, red[((j & 1) * 2 + (half ^ 1)) * 128 + r]);
       // running maximum: rescale O only when it grows by more than the threshold
       bool need = false;
       float factor = 1.f;
@@ -275,11 +298,12 @@ attn_tc1_kernel(const __grid_constant__ TcParams p) {
       else if (tmax > m_ref + RESCALE_THRESHOLD) { need = true; factor = exp2f(m_ref - tmax); }
       if (__any_sync(0xffffffffu, need)) {
         ok = mbar_wait(BAR_ODONE, (j - 1) & 1, abort_flag);       // P_{j-1} V_{j-1} has landed in O
+        if (!ok && lane == 0) fail(ERR_WAIT_O_DONE);
         ok = __all_sync(0xffffffffu, ok);
-        if (!ok) { if (lane == 0) fail(ERR_WAIT_O_DONE); break; }
+        if (!ok) continue;                                        // reported at the next tile's barrier
         tc_fence_after();
 #pragma unroll
-        for (int q = 0; q < NV * 2; ++q) {
+        for (int q = NV * half; q < NV * half + NV; ++q) {         // this half's share of the O columns
           uint32_t o[32];
           tmem_ld32(tmem + lane_base + P::TM_O + q * 32, o);
           tmem_wait_ld();
@@ -291,22 +315,16 @@ attn_tc1_kernel(const __grid_constant__ TcParams p) {
       }
       const float m_use = (m_ref == -INFINITY) ? 0.f : m_ref;
       float rs = 0.f;
+      uint32_t pk[32];
 #pragma unroll
-      for (int q = 0; q < 4; ++q) {
-        uint32_t pk[16];
-#pragma unroll
-        for (int i = 0; i < 16; ++i) {
-          const float p0 = exp2f(__uint_as_float(sr[q][2 * i]) - m_use);
-          const float p1 = exp2f(__uint_as_float(sr[q][2 * i + 1]) - m_use);
-          rs += p0 + p1;
-          pk[i] = pack_bf16x2(p0, p1);
-        }
-#pragma unroll
-        for (int i = 0; i < 16; ++i) sr[q >> 1][(q & 1) * 16 + i] = pk[i];   // reuse: rows 0,1 of sr now hold P
+      for (int i = 0; i < 32; ++i) {
+        const float p0 = exp2f(__uint_as_float(sr[i >> 4][(2 * i) & 31]) - m_use);
+        const float p1 = exp2f(__uint_as_float(sr[i >> 4][(2 * i + 1) & 31]) - m_use);
+        rs += p0 + p1;
+        pk[i] = pack_bf16x2(p0, p1);
       }
       l_sum += rs;
-      tmem_st32(stm, sr[0]);            // P columns 0..31  (keys 0..63)
-      tmem_st32(stm + 32, sr[1]);       // P columns 32..63 (keys 64..127)
+      tmem_st32(stm + 32 * half, pk);     // P columns 32*half .. 32*half+31 = keys 64*half .. 64*half+63
       tmem_wait_st();
       tc_fence_before();
       mbar_arrive(BAR_PFULL(j & 1));
@@ -314,16 +332,20 @@ attn_tc1_kernel(const __grid_constant__ TcParams p) {
     // ---- epilogue: O / l -> bf16 -> global
     if (ok && n_tiles > 0) {
       ok = mbar_wait(BAR_ODONE, (n_tiles - 1) & 1, abort_flag);
-      ok = __all_sync(0xffffffffu, ok);
       if (!ok && lane == 0) fail(ERR_WAIT_O_DONE);
     }
-    if (ok) {
+    ok = __all_sync(0xffffffffu, ok);
+    if (!ok) fail_word[0] = fail_word[1] = 1;
+    red[(4 + half) * 128 + r] = l_sum;
+    asm volatile("bar.sync 1, 256;" ::: "memory");
+    if (!fail_word[0]) {
+      const float l_tot = l_sum + red[(4 + (half ^ 1)) * 128 + r];
       tc_fence_after();
-      const float inv = (n_tiles > 0 && l_sum > 0.f) ? 1.f / l_sum : 0.f;
+      const float inv = (n_tiles > 0 && l_tot > 0.f) ? 1.f / l_tot : 0.f;
       const size_t orow = ((size_t)b * p.q_len + t_row) * p.Hq + head0 + hl;
       bf16* dst = p.out + orow * p.d_out;
 #pragma unroll
-      for (int q = 0; q < NV * 2; ++q) {
+      for (int q = NV * half; q < NV * half + NV; ++q) {
         uint32_t o[32];
         if (n_tiles > 0) { tmem_ld32(tmem + lane_base + P::TM_O + q * 32, o); tmem_wait_ld(); }
         else {
@@ -343,8 +365,8 @@ attn_tc1_kernel(const __grid_constant__ TcParams p) {
           }
         }
       }
-      if (p.lse && row_valid)
-        p.lse[orow] = (n_tiles > 0 && l_sum > 0.f) ? (m_ref + log2f(l_sum)) * 0.6931471805599453f : -INFINITY;
+      if (p.lse && row_valid && half == 0)
+        p.lse[orow] = (n_tiles > 0 && l_tot > 0.f) ? (m_ref + log2f(l_tot)) * 0.6931471805599453f : -INFINITY;
     }
     tc_fence_before();
   }
@@ -430,7 +452,7 @@ int attn_tc_launch(const AttnProblem& a) {
   if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, PL::BYTES) != cudaSuccess)
     return LCA_ERR_CUDA;
   dim3 grid(p.n_tok_tiles, a.n_kv_heads, a.batch);
-  kern<<<grid, 192, PL::BYTES, a.stream>>>(p);
+  kern<<<grid, 320, PL::BYTES, a.stream>>>(p);
   note_launch();
   return cudaGetLastError() == cudaSuccess ? LCA_OK : LCA_ERR_CUDA;
 }
