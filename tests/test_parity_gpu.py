@@ -313,3 +313,44 @@ def test_ablation_reducers_match_oracle(B, sem, pos):
             ulp = Hh.bf16_ulp_distance(got, want)
             tiny = np.abs(O.bits_to_f64(got) - O.bits_to_f64(want)) <= 32 * 2.0 ** -24 * 20.0
             assert ((ulp <= 1) | tiny).all()                       # fp32 sums of g terms against fp64
+
+
+def test_gqa_decode_matches_oracle(B):
+    # GQA cache: K anchors / pooled V per KV head; sequences of different valid lengths share one buffer,
+    # rows past the valid count are left as zeros (they take no part in the result)
+    cfg = I.scaled(I.CONFIGS["gqa_64k"], batch=3, seq_len=900, n_q_heads=32, n_kv_heads=8, group_size=64, window=128)
+    g, w, Hq, Hkv, d = cfg.group_size, cfg.window, cfg.n_q_heads, cfg.n_kv_heads, cfg.d_sem
+    p1 = B.params_from_config(cfg, batch=1)
+    m, k = B.lca_partition(p1)
+    cap = m + k + 1
+    cache_v = torch.zeros((3, cap, Hkv, d), dtype=torch.bfloat16, device=DEV)
+    cache_k = torch.zeros((3, cap, Hkv, d), dtype=torch.bfloat16, device=DEV)
+    valid = [m + k + 1, m + k - 37, m + 1]
+    gen = torch.Generator().manual_seed(3)
+    q_new = torch.randn((3, Hq, d), generator=gen).bfloat16()
+    refs = []
+    for b in range(3):
+        inp = I.make_gqa_inputs(cfg, "cpu", batch_index=b)
+        dv = to_dev(inp)
+        c = B.condense(p1, None, dv["q"][cfg.seq_len - g:], dv["v"], dv["k"])
+        ref = Hh.oracle_gqa(inp, g, w, cfg.softmax_scale)
+        Hh.check_condense(one_seq(c), ref["cond"], kind="gqa")
+        cache_v[b, :m + k] = c["cache_sem"][0]
+        cache_k[b, :m + k] = c["cache_pos"][0]
+        cache_v[b, m + k] = torch.randn((Hkv, d), generator=gen).bfloat16().to(DEV)
+        cache_k[b, m + k] = torch.randn((Hkv, d), generator=gen).bfloat16().to(DEV)
+        n = valid[b]
+        refs.append(O.gqa_decode(O.torch_bf16_to_f64(q_new[b]), O.bits_to_f64(Hh.bits(cache_k[b, :n])),
+                                 O.bits_to_f64(Hh.bits(cache_v[b, :n])), m, Hh.f32(cfg.softmax_scale), 0.25))
+    p = B.params_from_config(cfg, batch=3, rep_logit_bias=0.25)
+    rows = torch.tensor(valid, dtype=torch.int32, device=DEV)
+    for impl in (0, 1):                                  # tensor-core kernel, then the scalar kernel
+        prev = B.lca_set_attention_impl(impl)
+        try:
+            out, lse = B.decode_attention(p, None, q_new.to(DEV), cache_v, cache_k, rows, m, want_lse=True)
+        finally:
+            B.lca_set_attention_impl(prev)
+        assert B.lca_last_device_status() == 0
+        for b in range(3):
+            Hh.check_outputs(out[b], refs[b][0], f"gqa decode seq {b} impl {impl}")
+            np.testing.assert_allclose(lse[b].cpu().numpy(), refs[b][1], atol=2e-3, rtol=1e-4)
