@@ -14,7 +14,6 @@
 namespace lca {
 
 static const int QBAR_ROWS_PER_CHUNK = 64;
-static const int QBAR_THREADS = 128;
 static const int CONDENSE_THREADS = 512;
 
 // ---------------------------------------------------------------------------- summary query

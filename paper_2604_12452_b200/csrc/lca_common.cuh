@@ -28,14 +28,6 @@ __host__ __device__ inline int reps_visible(int p, int w, int g) {
   return (t < w + g) ? 0 : (t - w) / g;
 }
 
-// double -> bf16, round to nearest even with a single rounding: truncate to float, fold the
-// discarded bits into a sticky last bit (round to odd), then let the float->bf16 conversion round.
-__device__ inline bf16 double_to_bf16_rn(double x) {
-  float f = __double2float_rz(x);
-  if ((double)f != x) f = __uint_as_float(__float_as_uint(f) | 1u);
-  return __float2bfloat16_rn(f);
-}
-
 __device__ inline double warp_sum(double v) {
 #pragma unroll
   for (int o = 16; o > 0; o >>= 1) v += __shfl_xor_sync(0xffffffffu, v, o);
