@@ -186,6 +186,11 @@ attn_tc2_kernel(const __grid_constant__ Tc2Params p) {
     if (rank == 0 && lane == 0 && n_tiles > 0) {
       constexpr uint32_t IDESC_S = umma_idesc_bf16(128, BN, false, false);
       constexpr uint32_t IDESC_PV = umma_idesc_bf16(128, 256, false, true);
+      // The issuing thread's own instructions between two tcgen05.mma are not hidden behind the
+      // tensor core, so the shared-memory descriptors are built once and only their start-address
+      // field (low word) is advanced per instruction.
+      const uint64_t qd0 = umma_desc_sw128(sQ, 16, 1024), kd0 = umma_desc_sw128(sK, 16, 1024);
+      const uint64_t pd0 = umma_desc_sw128(sP, 16, 1024), vd0 = umma_desc_sw128(sV, VCH, 1024);
       bool ok = mbar_wait(BAR_Q, 0, abort_flag);
       if (!ok) fail(ERR_WAIT_Q);
       auto issue_pv = [&](int j) -> bool {
@@ -196,12 +201,13 @@ attn_tc2_kernel(const __grid_constant__ Tc2Params p) {
         for (int kh = 0; kh < 2; ++kh) {
           if (!mbar_wait(BAR_VFULL(kh), j & 1, abort_flag)) { fail(ERR_WAIT_KV_FULL); return false; }
           tc_fence_after();
+          // descriptors differ from the precomputed bases only in the 16-byte-unit start address
 #pragma unroll
           for (int n2 = 0; n2 < 2; ++n2) {
 #pragma unroll
             for (int k = 0; k < 4; ++k) {
-              const uint64_t ad = umma_desc_sw128(sP + kh * PCH + k * 32, 16, 1024);
-              const uint64_t bd = umma_desc_sw128(sV + (kh * 4 + n2 * 2) * VCH + k * 2048, VCH, 1024);
+              const uint64_t ad = desc_add(pd0, (kh * PCH + k * 32) >> 4);
+              const uint64_t bd = desc_add(vd0, ((kh * 4 + n2 * 2) * VCH + k * 2048) >> 4);
               umma_ss_pair(tmem + TM_O + n2 * 128, ad, bd, IDESC_PV, (j > 0 || kh > 0 || k > 0) ? 1u : 0u);
             }
           }
@@ -225,8 +231,8 @@ attn_tc2_kernel(const __grid_constant__ Tc2Params p) {
             const int c = gk * KG + cc;
 #pragma unroll
             for (int k = 0; k < 4; ++k) {
-              const uint64_t ad = umma_desc_sw128(sQ + c * QCH + k * 32, 16, 1024);
-              const uint64_t bd = umma_desc_sw128(sK + c * KCH + k * 32, 16, 1024);
+              const uint64_t ad = desc_add(qd0, (c * QCH + k * 32) >> 4);
+              const uint64_t bd = desc_add(kd0, (c * KCH + k * 32) >> 4);
               umma_ss_pair(stm, ad, bd, IDESC_S, (c > 0 || k > 0) ? 1u : 0u);
             }
           }

@@ -128,6 +128,16 @@ __device__ __forceinline__ uint64_t umma_desc_sw128(uint32_t smem_addr, uint32_t
   return d;
 }
 
+// The same descriptor with its start address advanced by `units16` 16-byte units (the address
+// field occupies the low 14 bits of the low word; shared-memory addresses stay below 256 KB, so
+// the sum never carries out of the field).
+__device__ __forceinline__ uint64_t desc_add(uint64_t desc, uint32_t units16) {
+  uint32_t lo = (uint32_t)desc + units16, hi = (uint32_t)(desc >> 32);
+  uint64_t r;
+  asm("mov.b64 %0, {%1, %2};" : "=l"(r) : "r"(lo), "r"(hi));
+  return r;
+}
+
 // Instruction descriptor for kind::f16 with bf16 operands and an fp32 accumulator.
 __host__ __device__ constexpr uint32_t umma_idesc_bf16(int M, int N, bool a_mn_major, bool b_mn_major) {
   return (1u << 4)                      // accumulator format: f32
