@@ -191,10 +191,10 @@ attn_tc1_kernel(const __grid_constant__ TcParams p) {
         tc_fence_after();
         const uint32_t ptm = tmem + ((j & 1) ? P::TM_S1 : P::TM_S0);
 #pragma unroll
-        for (int k = 0; k < BN / 16; ++k) {
-          const uint64_t bd = umma_desc_sw128(vbase + k * 2048, CHUNK_BYTES_KV, 1024);
-          umma_ts(tmem + P::TM_O, ptm + k * 8, bd, IDESC_PV, (j > 0 || k > 0) ? 1u : 0u);
-        }
+        const uint64_t vd0 = umma_desc_sw128(vbase, CHUNK_BYTES_KV, 1024);
+#pragma unroll
+        for (int k = 0; k < BN / 16; ++k)
+          umma_ts(tmem + P::TM_O, ptm + k * 8, desc_add(vd0, (k * 2048) >> 4), IDESC_PV, (j > 0 || k > 0) ? 1u : 0u);
         umma_commit(V_IN_K ? BAR_KEMPTY(s) : BAR_VEMPTY(s));
         umma_commit(BAR_ODONE);
       }
@@ -210,13 +210,14 @@ attn_tc1_kernel(const __grid_constant__ TcParams p) {
           tc_fence_after();
           const uint32_t stm = tmem + ((j & 1) ? P::TM_S1 : P::TM_S0);
 #pragma unroll
+          // descriptors are built once per tile; per instruction only the start address moves
+          const uint64_t qd0 = umma_desc_sw128(sQ, 16, 1024), kd0 = umma_desc_sw128(sK + s * P::K_STAGE, 16, 1024);
+#pragma unroll
           for (int c = 0; c < NK; ++c) {
 #pragma unroll
-            for (int k = 0; k < 4; ++k) {
-              const uint64_t ad = umma_desc_sw128(sQ + c * CHUNK_BYTES_Q + k * 32, 16, 1024);
-              const uint64_t bd = umma_desc_sw128(sK + s * P::K_STAGE + c * CHUNK_BYTES_KV + k * 32, 16, 1024);
-              umma_ss(stm, ad, bd, IDESC_S, (c > 0 || k > 0) ? 1u : 0u);
-            }
+            for (int k = 0; k < 4; ++k)
+              umma_ss(stm, desc_add(qd0, (c * CHUNK_BYTES_Q + k * 32) >> 4), desc_add(kd0, (c * CHUNK_BYTES_KV + k * 32) >> 4),
+                      IDESC_S, (c > 0 || k > 0) ? 1u : 0u);
           }
           umma_commit(BAR_SFULL(j & 1));
           if (!V_IN_K) umma_commit(BAR_KEMPTY(s));
