@@ -277,6 +277,7 @@ attn_tc2_kernel(const __grid_constant__ Tc2Params p) {
       const uint32_t stm = tmem + lane_base + ((j & 1) ? TM_S1 : TM_S0);
       uint32_t sr[2][32];
       float tmax = -INFINITY;
+      bool plain = false;
       const bool isA = j < nA;
       const int tile_key0 = isA ? j * BN : first_lo + (j - nA) * BN;
       const int key0 = tile_key0 + 64 * half;     // first key of this thread's 64 columns
@@ -290,16 +291,27 @@ attn_tc2_kernel(const __grid_constant__ Tc2Params p) {
         if (isA) { lo = 0; hi = n_a_row - key0 - 1; need_mask = tile_key0 + BN > n_a_lo; }
         else { lo = first_row - key0; hi = t_row - key0; need_mask = (tile_key0 < n_a_hi * p.g) || (tile_key0 + BN - 1 > t0); }
         const int blim = isA ? bias_rows - key0 : 0;
+        plain = !need_mask && !(isA && p.bias_log2 != 0.f);
+        if (plain) {
+          // interior tile: the raw products stay in sr, the (positive) scale is applied to the maximum
+          // here and folded into the exponent's multiply-add below
 #pragma unroll
-        for (int q = 0; q < 2; ++q) {
+          for (int q = 0; q < 2; ++q)
 #pragma unroll
-          for (int i = 0; i < 32; ++i) {
-            const int c = q * 32 + i;
-            float s = __uint_as_float(sr[q][i]) * p.scale_log2;
-            if (isA && p.bias_log2 != 0.f && c < blim) s += p.bias_log2;
-            if (need_mask && (c < lo || c > hi)) s = -INFINITY;
-            sr[q][i] = __float_as_uint(s);
-            tmax = fmaxf(tmax, s);
+            for (int i = 0; i < 32; ++i) tmax = fmaxf(tmax, __uint_as_float(sr[q][i]));
+          tmax *= p.scale_log2;
+        } else {
+#pragma unroll
+          for (int q = 0; q < 2; ++q) {
+#pragma unroll
+            for (int i = 0; i < 32; ++i) {
+              const int c = q * 32 + i;
+              float s = __uint_as_float(sr[q][i]) * p.scale_log2;
+              if (isA && p.bias_log2 != 0.f && c < blim) s += p.bias_log2;
+              if (need_mask && (c < lo || c > hi)) s = -INFINITY;
+              sr[q][i] = __float_as_uint(s);
+              tmax = fmaxf(tmax, s);
+            }
           }
         }
       } else {
@@ -338,6 +350,7 @@ attn_tc2_kernel(const __grid_constant__ Tc2Params p) {
       }
       if (need) { l_sum *= factor; m_ref = tmax; }
       const float m_use = (m_ref == -INFINITY) ? 0.f : m_ref;
+      const float e_mul = plain ? p.scale_log2 : 1.f;       // sr holds raw products (plain) or scaled logits
       float rs = 0.f;
       const uint32_t prow = sP + half * PCH + rl * 128;
 #pragma unroll
@@ -346,8 +359,8 @@ attn_tc2_kernel(const __grid_constant__ Tc2Params p) {
 #pragma unroll
         for (int i = 0; i < 4; ++i) {
           const int c = s8 * 8 + 2 * i;
-          const float p0 = exp2f(__uint_as_float(sr[c >> 5][c & 31]) - m_use);
-          const float p1 = exp2f(__uint_as_float(sr[(c + 1) >> 5][(c + 1) & 31]) - m_use);
+          const float p0 = exp2f(fmaf(__uint_as_float(sr[c >> 5][c & 31]), e_mul, -m_use));
+          const float p1 = exp2f(fmaf(__uint_as_float(sr[(c + 1) >> 5][(c + 1) & 31]), e_mul, -m_use));
           rs += p0 + p1;
           pk[i] = pack_bf16x2(p0, p1);
         }
