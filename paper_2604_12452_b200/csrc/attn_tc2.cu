@@ -295,11 +295,13 @@ attn_tc2_kernel(const __grid_constant__ Tc2Params p) {
         if (plain) {
           // interior tile: the raw products stay in sr, the (positive) scale is applied to the maximum
           // here and folded into the exponent's multiply-add below
+          float t0m = -INFINITY, t1m = -INFINITY, t2m = -INFINITY, t3m = -INFINITY;    // four short chains
 #pragma unroll
-          for (int q = 0; q < 2; ++q)
-#pragma unroll
-            for (int i = 0; i < 32; ++i) tmax = fmaxf(tmax, __uint_as_float(sr[q][i]));
-          tmax *= p.scale_log2;
+          for (int i = 0; i < 32; i += 2) {
+            t0m = fmaxf(t0m, __uint_as_float(sr[0][i])); t1m = fmaxf(t1m, __uint_as_float(sr[0][i + 1]));
+            t2m = fmaxf(t2m, __uint_as_float(sr[1][i])); t3m = fmaxf(t3m, __uint_as_float(sr[1][i + 1]));
+          }
+          tmax = fmaxf(fmaxf(t0m, t1m), fmaxf(t2m, t3m)) * p.scale_log2;
         } else {
 #pragma unroll
           for (int q = 0; q < 2; ++q) {
@@ -327,6 +329,21 @@ attn_tc2_kernel(const __grid_constant__ Tc2Params p) {
       if (j == 0) m_ref = tmax;
       else if (tmax > m_ref + RESCALE_THRESHOLD) { need = true; factor = exp2f(m_ref - tmax); }
       if (ln == 0) TRACE(10, j);
+      // The probabilities depend only on S and the (new) reference maximum: compute and pack them
+      // while P V of the previous tile is still running, then wait, rescale O if needed, and store.
+      const float m_new = need ? tmax : m_ref;
+      const float m_use = (m_new == -INFINITY) ? 0.f : m_new;
+      const float e_mul = plain ? p.scale_log2 : 1.f;       // sr holds raw products (plain) or scaled logits
+      float rs0 = 0.f, rs1 = 0.f;
+      uint32_t pk[32];
+#pragma unroll
+      for (int i = 0; i < 32; ++i) {
+        const int c = 2 * i;
+        const float p0 = exp2f(fmaf(__uint_as_float(sr[c >> 5][c & 31]), e_mul, -m_use));
+        const float p1 = exp2f(fmaf(__uint_as_float(sr[(c + 1) >> 5][(c + 1) & 31]), e_mul, -m_use));
+        rs0 += p0; rs1 += p1;
+        pk[i] = pack_bf16x2(p0, p1);
+      }
       if (j >= 1) {
         // P (one buffer) and O are free once P_{j-1} V_{j-1} has completed
         ok = mbar_wait(BAR_ODONE, (j - 1) & 1, abort_flag);
@@ -349,24 +366,13 @@ attn_tc2_kernel(const __grid_constant__ Tc2Params p) {
         tmem_wait_st();
       }
       if (need) { l_sum *= factor; m_ref = tmax; }
-      const float m_use = (m_ref == -INFINITY) ? 0.f : m_ref;
-      const float e_mul = plain ? p.scale_log2 : 1.f;       // sr holds raw products (plain) or scaled logits
-      float rs = 0.f;
       const uint32_t prow = sP + half * PCH + rl * 128;
 #pragma unroll
       for (int s8 = 0; s8 < 8; ++s8) {             // 16-byte slot s8 holds keys 8*s8 .. 8*s8+7
-        uint32_t pk[4];
-#pragma unroll
-        for (int i = 0; i < 4; ++i) {
-          const int c = s8 * 8 + 2 * i;
-          const float p0 = exp2f(fmaf(__uint_as_float(sr[c >> 5][c & 31]), e_mul, -m_use));
-          const float p1 = exp2f(fmaf(__uint_as_float(sr[(c + 1) >> 5][(c + 1) & 31]), e_mul, -m_use));
-          rs += p0 + p1;
-          pk[i] = pack_bf16x2(p0, p1);
-        }
         const uint32_t a = prow + ((s8 ^ (rl & 7)) << 4);
-        asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(a), "r"(pk[0]), "r"(pk[1]), "r"(pk[2]), "r"(pk[3]) : "memory");
+        asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(a), "r"(pk[4 * s8]), "r"(pk[4 * s8 + 1]), "r"(pk[4 * s8 + 2]), "r"(pk[4 * s8 + 3]) : "memory");
       }
+      const float rs = rs0 + rs1;
       l_sum += rs;
       fence_proxy_async_smem();                   // P is read by the tensor core (async proxy)
       tc_fence_before();
