@@ -278,11 +278,13 @@ attn_tc1_kernel(const __grid_constant__ TcParams p) {
         if (plain) {
           // interior tile: the raw products stay in sr, the (positive) scale is applied to the maximum
           // here and folded into the exponent's multiply-add below
+          float t0m = -INFINITY, t1m = -INFINITY, t2m = -INFINITY, t3m = -INFINITY;    // four short chains
 #pragma unroll
-          for (int q = 0; q < 2; ++q)
-#pragma unroll
-            for (int i = 0; i < 32; ++i) tmax = fmaxf(tmax, __uint_as_float(sr[q][i]));
-          tmax *= p.scale_log2;
+          for (int i = 0; i < 32; i += 2) {
+            t0m = fmaxf(t0m, __uint_as_float(sr[0][i])); t1m = fmaxf(t1m, __uint_as_float(sr[0][i + 1]));
+            t2m = fmaxf(t2m, __uint_as_float(sr[1][i])); t3m = fmaxf(t3m, __uint_as_float(sr[1][i + 1]));
+          }
+          tmax = fmaxf(fmaxf(t0m, t1m), fmaxf(t2m, t3m)) * p.scale_log2;
         } else {
 #pragma unroll
           for (int q = 0; q < 2; ++q) {
@@ -327,17 +329,17 @@ attn_tc1_kernel(const __grid_constant__ TcParams p) {
         if (need) { l_sum *= factor; m_ref = tmax; }
       }
       const float m_use = (m_ref == -INFINITY) ? 0.f : m_ref;
-      float rs = 0.f;
+      float rs0 = 0.f, rs1 = 0.f;
       uint32_t pk[32];
       const float e_mul = plain ? p.scale_log2 : 1.f;       // sr holds raw products (plain) or scaled logits
 #pragma unroll
       for (int i = 0; i < 32; ++i) {
         const float p0 = exp2f(fmaf(__uint_as_float(sr[i >> 4][(2 * i) & 31]), e_mul, -m_use));
         const float p1 = exp2f(fmaf(__uint_as_float(sr[i >> 4][(2 * i + 1) & 31]), e_mul, -m_use));
-        rs += p0 + p1;
+        rs0 += p0; rs1 += p1;
         pk[i] = pack_bf16x2(p0, p1);
       }
-      l_sum += rs;
+      l_sum += rs0 + rs1;
       tmem_st32(stm + 32 * half, pk);     // P columns 32*half .. 32*half+31 = keys 64*half .. 64*half+63
       tmem_wait_st();
       tc_fence_before();
