@@ -36,7 +36,7 @@ namespace pair {
 constexpr int BN = 128;                 // keys per tile (64 per CTA for S)
 constexpr int NKC = 9;                  // 64-column key chunks: 8 latent + 1 rope
 #ifndef LCA_TC2_KG
-#define LCA_TC2_KG 3
+#define LCA_TC2_KG 9
 #endif
 constexpr int KG = LCA_TC2_KG;          // key chunks per ring slot (one full/empty barrier pair each)
 constexpr int NKG = NKC / KG;
