@@ -190,7 +190,6 @@ attn_tc1_kernel(const __grid_constant__ TcParams p) {
       if (lane == 0) {
         tc_fence_after();
         const uint32_t ptm = tmem + ((j & 1) ? P::TM_S1 : P::TM_S0);
-#pragma unroll
         const uint64_t vd0 = umma_desc_sw128(vbase, CHUNK_BYTES_KV, 1024);
 #pragma unroll
         for (int k = 0; k < BN / 16; ++k)
@@ -209,7 +208,6 @@ attn_tc1_kernel(const __grid_constant__ TcParams p) {
         if (ok) {
           tc_fence_after();
           const uint32_t stm = tmem + ((j & 1) ? P::TM_S1 : P::TM_S0);
-#pragma unroll
           // descriptors are built once per tile; per instruction only the start address moves
           const uint64_t qd0 = umma_desc_sw128(sQ, 16, 1024), kd0 = umma_desc_sw128(sK + s * P::K_STAGE, 16, 1024);
 #pragma unroll
@@ -423,6 +421,22 @@ bool make_tensor_map_3d(CUtensorMap* map, const void* ptr, int d, int heads, lon
   cuuint64_t dims[3] = {(cuuint64_t)d, (cuuint64_t)heads, (cuuint64_t)rows};
   cuuint64_t strides[2] = {(cuuint64_t)d * 2, (cuuint64_t)d * 2 * heads};
   cuuint32_t box[3] = {64, (cuuint32_t)box_heads, (cuuint32_t)box_rows};
+  cuuint32_t estr[3] = {1, 1, 1};
+  return fn(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 3, const_cast<void*>(ptr), dims, strides, box, estr,
+            CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+            CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+}
+
+// A [rows][64 * chunks] bf16 matrix seen as (64 columns, rows, 64-column chunks): one box then brings
+// several column chunks of the same rows, each landing as its own 128-byte-swizzled [rows][64] block
+// (chunk after chunk), in a single request instead of one request per chunk.
+bool make_tensor_map_chunks(CUtensorMap* map, const void* ptr, int chunks, long long rows, int box_rows, int box_chunks) {
+  EncodeTiledFn fn = encode_fn();
+  if (!fn) return false;
+  if (!ptr) { memset(map, 0, sizeof(*map)); return true; }
+  cuuint64_t dims[3] = {64, (cuuint64_t)rows, (cuuint64_t)chunks};
+  cuuint64_t strides[2] = {(cuuint64_t)chunks * 128, 128};
+  cuuint32_t box[3] = {64, (cuuint32_t)box_rows, (cuuint32_t)box_chunks};
   cuuint32_t estr[3] = {1, 1, 1};
   return fn(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 3, const_cast<void*>(ptr), dims, strides, box, estr,
             CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,

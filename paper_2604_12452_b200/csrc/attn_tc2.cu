@@ -35,12 +35,13 @@ static __device__ long long g_trace[8192];
 namespace pair {
 constexpr int BN = 128;                 // keys per tile (64 per CTA for S)
 constexpr int NKC = 9;                  // 64-column key chunks: 8 latent + 1 rope
-#ifndef LCA_TC2_KG
-#define LCA_TC2_KG 9
-#endif
-constexpr int KG = LCA_TC2_KG;          // key chunks per ring slot (one full/empty barrier pair each)
-constexpr int NKG = NKC / KG;
-static_assert(NKC % KG == 0, "key chunks per slot must divide 9");
+// The key part of a tile is one buffer, filled and released in NKG pieces (2: rope chunk + latent
+// chunks 0-3, then latent chunks 4-7, so that a refill starts while S = Q K^T still reads the other
+// piece).  One piece measured faster: every extra wait / commit pair in the issuing thread costs
+// more than the earlier refill gains.
+constexpr int NKG = 1;
+constexpr int KBOX = 8 / NKG;           // latent column chunks brought by one TMA request of the key part
+constexpr int VBOX = 2;                 // column chunks brought by one request of the value part
 constexpr int QCH = 64 * 128;           // bytes of one query chunk  (64 rows)
 constexpr int KCH = 64 * 128;           // bytes of one key chunk    (64 keys)
 constexpr int VCH = 64 * 128;           // bytes of one value chunk  (64 keys x 64 columns)
@@ -58,8 +59,9 @@ static_assert(SMEM_BYTES <= 232448, "shared memory budget of one SM");
 
 struct Tc2Params {
   CUtensorMap q_sem, q_pos;       // queries, box of 64 rows
-  CUtensorMap k_sem, k_pos;       // per-token latents / rope keys, box of 64 rows
-  CUtensorMap c_sem, c_pos;       // condensed cache, box of 64 rows
+  CUtensorMap k_pos, c_pos;       // rope keys of the tokens / of the condensed cache, box of 64 rows
+  CUtensorMap k_sem, c_sem;       // latents seen as (64 columns, rows, chunks): box of 64 rows x KBOX chunks
+  CUtensorMap k_val, c_val;       // the same memory, box of 64 rows x VBOX chunks
   bf16* out; float* lse; const int32_t* cache_rows;
   int B, q_len, H, L, g, w, cap, n_rep_bias, decode;
   int HB, TB, n_tok_tiles;
@@ -73,13 +75,13 @@ attn_tc2_kernel(const __grid_constant__ Tc2Params p) {
   const uint32_t base = smem_u32(smem);
   const uint32_t sQ = base + OFF_Q, sK = base + OFF_K, sV = base + OFF_V, sP = base + OFF_P;
   const uint32_t bars = base + OFF_BAR;
-  // The key part of a tile is a ring of its nine 64-column chunks and the value part a ring of its
-  // two 64-key halves: a slot is refilled with the next tile's data as soon as the MMAs that read
-  // it have completed, so the loads of tile j+1 run underneath the MMAs of tile j.
+  // One buffer for the key part of a tile (nine 64-column chunks) and one for each 64-key half of
+  // its value part: a buffer is refilled with the next tile's data as soon as the MMAs that read it
+  // have completed, so the loads of tile j+1 run underneath the remaining MMAs of tile j.
   const uint32_t BAR_Q = bars, BAR_SFULL0 = bars + 8, BAR_SFULL1 = bars + 16, BAR_PFULL = bars + 24,
                  BAR_ODONE = bars + 32;
-  auto BAR_KFULL = [&](int c) { return bars + 40 + 8 * c; };            // 9
-  auto BAR_KEMPTY = [&](int c) { return bars + 40 + 72 + 8 * c; };      // 9
+  auto BAR_KFULL = [&](int c) { return bars + 40 + 8 * c; };            // NKG (room for 9)
+  auto BAR_KEMPTY = [&](int c) { return bars + 40 + 72 + 8 * c; };      // NKG (room for 9)
   auto BAR_VFULL = [&](int h) { return bars + 40 + 144 + 8 * h; };      // 2
   auto BAR_VEMPTY = [&](int h) { return bars + 40 + 160 + 8 * h; };     // 2
   volatile uint32_t* tmem_slot = reinterpret_cast<volatile uint32_t*>(smem + OFF_MISC);
@@ -152,10 +154,11 @@ attn_tc2_kernel(const __grid_constant__ Tc2Params p) {
         bool good = true;
         for (int gk = 0; gk < NKG; ++gk) {
           if (!mbar_wait(BAR_KEMPTY(gk), (j & 1) ^ 1, abort_flag)) { fail(ERR_WAIT_KV_EMPTY); good = false; break; }
-          if (rank == 0) mbar_expect_tx(BAR_KFULL(gk), 2 * KG * KCH);
+          const int n_sem = 8 / NKG, n_all = n_sem + (gk == 0 ? 1 : 0);
+          if (rank == 0) mbar_expect_tx(BAR_KFULL(gk), 2 * n_all * KCH);
           const uint32_t k_bar = mapa_u32(BAR_KFULL(gk), 0);
-          for (int c = gk * KG; c < (gk + 1) * KG; ++c)
-            tma_load_3d_pair(sK + c * KCH, c < 8 ? ms : mp, c < 8 ? c * 64 : 0, 0, row, k_bar);
+          if (gk == 0) tma_load_3d_pair(sK + 8 * KCH, mp, 0, 0, row, k_bar);
+          for (int c = gk * n_sem; c < (gk + 1) * n_sem; c += KBOX) tma_load_3d_pair(sK + c * KCH, ms, 0, row, c, k_bar);
         }
         if (!good) break;
       }
@@ -166,16 +169,16 @@ attn_tc2_kernel(const __grid_constant__ Tc2Params p) {
       for (int j = 0; j < n_tiles; ++j) {
         const bool isA = j < nA;
         const int row = isA ? b * p.cap + j * BN : b * p.L + first_lo + (j - nA) * BN;
-        const CUtensorMap* mv = isA ? &p.c_sem : &p.k_sem;
+        const CUtensorMap* mv = isA ? &p.c_val : &p.k_val;
         bool good = true;
         for (int kh = 0; kh < 2; ++kh) {            // keys [64*kh, 64*kh+64) of the tile
           if (!mbar_wait(BAR_VEMPTY(kh), (j & 1) ^ 1, abort_flag)) { fail(ERR_WAIT_KV_EMPTY); good = false; break; }
           if (rank == 0) mbar_expect_tx(BAR_VFULL(kh), 2 * 4 * VCH);
           const uint32_t v_bar = mapa_u32(BAR_VFULL(kh), 0);
           // output columns of this CTA: [128*rank, +128) of the first 256, then of the second 256
-          for (int i = 0; i < 4; ++i) {
-            const int col = (i >> 1) * 256 + 128 * (int)rank + (i & 1) * 64;
-            tma_load_3d_pair(sV + (kh * 4 + i) * VCH, mv, col, 0, row + 64 * kh, v_bar);
+          for (int i = 0; i < 4; i += VBOX) {
+            const int chunk = (i >> 1) * 4 + 2 * (int)rank + (i & 1);
+            tma_load_3d_pair(sV + (kh * 4 + i) * VCH, mv, 0, row + 64 * kh, chunk, v_bar);
           }
         }
         if (!good) break;
@@ -226,14 +229,15 @@ attn_tc2_kernel(const __grid_constant__ Tc2Params p) {
           if (gk == 0) TRACE(1, j);
           if (!ok) { fail(ERR_WAIT_KV_FULL); break; }
           tc_fence_after();
+          constexpr int n_sem = 8 / NKG;
 #pragma unroll
-          for (int cc = 0; cc < KG; ++cc) {
-            const int c = gk * KG + cc;
+          for (int cc = (gk == 0 ? -1 : 0); cc < n_sem; ++cc) {
+            const int c = cc < 0 ? 8 : gk * n_sem + cc;         // the rope chunk goes first
 #pragma unroll
             for (int k = 0; k < 4; ++k) {
               const uint64_t ad = desc_add(qd0, (c * QCH + k * 32) >> 4);
               const uint64_t bd = desc_add(kd0, (c * KCH + k * 32) >> 4);
-              umma_ss_pair(stm, ad, bd, IDESC_S, (c > 0 || k > 0) ? 1u : 0u);
+              umma_ss_pair(stm, ad, bd, IDESC_S, (c != 8 || k > 0) ? 1u : 0u);
             }
           }
           umma_commit_pair(BAR_KEMPTY(gk), 3);
@@ -437,6 +441,7 @@ attn_tc2_kernel(const __grid_constant__ Tc2Params p) {
 
 // ----------------------------------------------------------------------------------- host
 bool make_tensor_map_3d(CUtensorMap* map, const void* ptr, int d, int heads, long long rows, int box_heads, int box_rows);
+bool make_tensor_map_chunks(CUtensorMap* map, const void* ptr, int chunks, long long rows, int box_rows, int box_chunks);
 
 bool attn_tc2_supported(const AttnProblem& a) {
   if (a.variant != LCA_VARIANT_MLA || a.d_sem != 512 || a.d_pos != 64 || a.n_kv_heads != 1) return false;
@@ -464,10 +469,12 @@ int attn_tc2_launch(const AttnProblem& a) {
                   crows = (long long)a.batch * a.cache_row_capacity;
   bool ok = make_tensor_map_3d(&p.q_sem, a.q_sem, 512, H, qrows, hbc, tbc);
   ok = ok && make_tensor_map_3d(&p.q_pos, a.q_pos, 64, H, qrows, hbc, tbc);
-  ok = ok && make_tensor_map_3d(&p.k_sem, a.kv_sem, 512, 1, krows, 1, 64);
   ok = ok && make_tensor_map_3d(&p.k_pos, a.kv_pos, 64, 1, krows, 1, 64);
-  ok = ok && make_tensor_map_3d(&p.c_sem, a.cache_sem, 512, 1, crows, 1, 64);
   ok = ok && make_tensor_map_3d(&p.c_pos, a.cache_pos, 64, 1, crows, 1, 64);
+  ok = ok && make_tensor_map_chunks(&p.k_sem, a.kv_sem, 8, krows, 64, KBOX);
+  ok = ok && make_tensor_map_chunks(&p.c_sem, a.cache_sem, 8, crows, 64, KBOX);
+  ok = ok && make_tensor_map_chunks(&p.k_val, a.kv_sem, 8, krows, 64, VBOX);
+  ok = ok && make_tensor_map_chunks(&p.c_val, a.cache_sem, 8, crows, 64, VBOX);
   if (!ok) return LCA_ERR_CUDA;
   if (cudaFuncSetAttribute(attn_tc2_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM_BYTES) != cudaSuccess)
     return LCA_ERR_CUDA;
