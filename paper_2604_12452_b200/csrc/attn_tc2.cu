@@ -88,7 +88,8 @@ attn_tc2_kernel(const __grid_constant__ Tc2Params p) {
   volatile int* abort_flag = reinterpret_cast<volatile int*>(smem + OFF_MISC + 4);
   volatile float* red = reinterpret_cast<volatile float*>(smem + OFF_RED);    // [2][128]
 
-  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  // the warp index through a shuffle: provably warp-uniform, so the role branches below are uniform branches
+  const int warp = __shfl_sync(0xffffffffu, (int)(threadIdx.x >> 5), 0), lane = threadIdx.x & 31;
   const uint32_t rank = cluster_ctarank();       // 0 = even CTA: issues the MMAs, owns the "full" barriers
 
   // ---- which rows, which key tiles (identical in both CTAs of the pair)
@@ -186,7 +187,9 @@ attn_tc2_kernel(const __grid_constant__ Tc2Params p) {
     }
   } else if (warp == 1) {
     // =============================================== MMA issuer (even CTA only)
-    if (rank == 0 && lane == 0 && n_tiles > 0) {
+    // The whole warp walks the loop (every lane polls the barriers); one elected lane issues.
+    if (rank == 0 && n_tiles > 0) {
+      const uint32_t leader = elect_one();
       constexpr uint32_t IDESC_S = umma_idesc_bf16(128, BN, false, false);
       constexpr uint32_t IDESC_PV = umma_idesc_bf16(128, 256, false, true);
       // The issuing thread's own instructions between two tcgen05.mma are not hidden behind the
@@ -195,14 +198,14 @@ attn_tc2_kernel(const __grid_constant__ Tc2Params p) {
       const uint64_t qd0 = umma_desc_sw128(sQ, 16, 1024), kd0 = umma_desc_sw128(sK, 16, 1024);
       const uint64_t pd0 = umma_desc_sw128(sP, 16, 1024), vd0 = umma_desc_sw128(sV, VCH, 1024);
       bool ok = mbar_wait(BAR_Q, 0, abort_flag);
-      if (!ok) fail(ERR_WAIT_Q);
+      if (!ok) if (leader) fail(ERR_WAIT_Q);
       auto issue_pv = [&](int j) -> bool {
         TRACE(3, j);
-        if (!mbar_wait(BAR_PFULL, j & 1, abort_flag)) { fail(ERR_WAIT_P_FULL); return false; }
+        if (!mbar_wait(BAR_PFULL, j & 1, abort_flag)) { if (leader) fail(ERR_WAIT_P_FULL); return false; }
         TRACE(4, j);
 #pragma unroll
         for (int kh = 0; kh < 2; ++kh) {
-          if (!mbar_wait(BAR_VFULL(kh), j & 1, abort_flag)) { fail(ERR_WAIT_KV_FULL); return false; }
+          if (!mbar_wait(BAR_VFULL(kh), j & 1, abort_flag)) { if (leader) fail(ERR_WAIT_KV_FULL); return false; }
           tc_fence_after();
           // descriptors differ from the precomputed bases only in the 16-byte-unit start address
 #pragma unroll
@@ -211,12 +214,12 @@ attn_tc2_kernel(const __grid_constant__ Tc2Params p) {
             for (int k = 0; k < 4; ++k) {
               const uint64_t ad = desc_add(pd0, (kh * PCH + k * 32) >> 4);
               const uint64_t bd = desc_add(vd0, ((kh * 4 + n2 * 2) * VCH + k * 2048) >> 4);
-              umma_ss_pair(tmem + TM_O + n2 * 128, ad, bd, IDESC_PV, (j > 0 || kh > 0 || k > 0) ? 1u : 0u);
+              umma_ss_pair_elected(leader, tmem + TM_O + n2 * 128, ad, bd, IDESC_PV, (j > 0 || kh > 0 || k > 0) ? 1u : 0u);
             }
           }
-          umma_commit_pair(BAR_VEMPTY(kh), 3);
+          umma_commit_pair_elected(leader, BAR_VEMPTY(kh), 3);
         }
-        umma_commit_pair(BAR_ODONE, 3);
+        umma_commit_pair_elected(leader, BAR_ODONE, 3);
         TRACE(5, j);
         return true;
       };
@@ -227,7 +230,7 @@ attn_tc2_kernel(const __grid_constant__ Tc2Params p) {
         for (int gk = 0; gk < NKG; ++gk) {
           ok = mbar_wait(BAR_KFULL(gk), j & 1, abort_flag);
           if (gk == 0) TRACE(1, j);
-          if (!ok) { fail(ERR_WAIT_KV_FULL); break; }
+          if (!ok) { if (leader) fail(ERR_WAIT_KV_FULL); break; }
           tc_fence_after();
           constexpr int n_sem = 8 / NKG;
 #pragma unroll
@@ -237,13 +240,13 @@ attn_tc2_kernel(const __grid_constant__ Tc2Params p) {
             for (int k = 0; k < 4; ++k) {
               const uint64_t ad = desc_add(qd0, (c * QCH + k * 32) >> 4);
               const uint64_t bd = desc_add(kd0, (c * KCH + k * 32) >> 4);
-              umma_ss_pair(stm, ad, bd, IDESC_S, (c != 8 || k > 0) ? 1u : 0u);
+              umma_ss_pair_elected(leader, stm, ad, bd, IDESC_S, (c != 8 || k > 0) ? 1u : 0u);
             }
           }
-          umma_commit_pair(BAR_KEMPTY(gk), 3);
+          umma_commit_pair_elected(leader, BAR_KEMPTY(gk), 3);
         }
         if (!ok) break;
-        umma_commit_pair((j & 1) ? BAR_SFULL1 : BAR_SFULL0, 3);
+        umma_commit_pair_elected(leader, (j & 1) ? BAR_SFULL1 : BAR_SFULL0, 3);
         TRACE(2, j);
         if (j >= 1) ok = issue_pv(j - 1);
       }
