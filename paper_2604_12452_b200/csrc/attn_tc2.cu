@@ -84,6 +84,7 @@ attn_tc2_kernel(const __grid_constant__ Tc2Params p) {
   auto BAR_KEMPTY = [&](int c) { return bars + 40 + 72 + 8 * c; };      // NKG (room for 9)
   auto BAR_VFULL = [&](int h) { return bars + 40 + 144 + 8 * h; };      // 2
   auto BAR_VEMPTY = [&](int h) { return bars + 40 + 160 + 8 * h; };     // 2
+  const uint32_t BAR_PLOCAL = bars + 224;        // odd CTA: its 128 softmax threads -> its relay thread
   volatile uint32_t* tmem_slot = reinterpret_cast<volatile uint32_t*>(smem + OFF_MISC);
   volatile int* abort_flag = reinterpret_cast<volatile int*>(smem + OFF_MISC + 4);
   volatile float* red = reinterpret_cast<volatile float*>(smem + OFF_RED);    // [2][128]
@@ -116,7 +117,8 @@ attn_tc2_kernel(const __grid_constant__ Tc2Params p) {
     for (int c = 0; c < NKG; ++c) { mbar_init(BAR_KFULL(c), 1); mbar_init(BAR_KEMPTY(c), 1); }
     for (int h = 0; h < 2; ++h) { mbar_init(BAR_VFULL(h), 1); mbar_init(BAR_VEMPTY(h), 1); }
     mbar_init(BAR_SFULL0, 1); mbar_init(BAR_SFULL1, 1);
-    mbar_init(BAR_PFULL, 256); mbar_init(BAR_ODONE, 1);
+    mbar_init(BAR_PFULL, 129); mbar_init(BAR_ODONE, 1);     // 128 threads of the even CTA + the odd CTA's relay
+    mbar_init(BAR_PLOCAL, 128);
     *abort_flag = (base & 1023u) ? 1 : 0;
     fence_mbar_init();
   }
@@ -252,6 +254,17 @@ attn_tc2_kernel(const __grid_constant__ Tc2Params p) {
       }
       if (ok) issue_pv(n_tiles - 1);
     }
+    // =============================================== relay (odd CTA): "P of this CTA is complete" -> even CTA
+    // A release-arrive on a barrier of the other CTA stalls its thread for 1000-2000 cycles.  The odd CTA's
+    // softmax threads therefore arrive on a barrier of their own CTA and this otherwise idle thread forwards
+    // one arrival per tile (its acquire on the local barrier and release on the remote one chain the ordering).
+    if (rank == 1 && lane == 0 && n_tiles > 0) {
+      const uint32_t pfull_addr = mapa_u32(BAR_PFULL, 0);
+      for (int j = 0; j < n_tiles; ++j) {
+        if (!mbar_wait(BAR_PLOCAL, j & 1, abort_flag)) { fail(ERR_WAIT_P_FULL); break; }
+        mbar_arrive_cluster_relaxed(pfull_addr);
+      }
+    }
   } else {
     // =============================================== softmax / epilogue: 128 threads, one per TMEM lane
     const int quarter = warp & 3;
@@ -265,7 +278,6 @@ attn_tc2_kernel(const __grid_constant__ Tc2Params p) {
     int n_a_row, bias_rows, first_row;
     if (p.decode) { n_a_row = n_a_hi; bias_rows = min(p.n_rep_bias, n_a_row); first_row = 0; }
     else { n_a_row = reps_visible(min(t_row, p.q_len - 1), p.w, p.g); bias_rows = n_a_row; first_row = n_a_row * p.g; }
-    const uint32_t pfull_addr = mapa_u32(BAR_PFULL, 0);
     float m_ref = -INFINITY, l_sum = 0.f;
     volatile int* fail_word = reinterpret_cast<volatile int*>(smem + OFF_MISC + 16);   // [2], softmax threads only
     if (ln < 2) fail_word[ln] = 0;
@@ -383,7 +395,7 @@ attn_tc2_kernel(const __grid_constant__ Tc2Params p) {
       l_sum += rs;
       fence_proxy_async_smem();                   // P is read by the tensor core (async proxy)
       tc_fence_before();
-      if (rank == 0) mbar_arrive(BAR_PFULL); else mbar_arrive_cluster(pfull_addr);
+      mbar_arrive(rank == 0 ? BAR_PFULL : BAR_PLOCAL);
       if (ln == 0) TRACE(12, j);
     }
     // ---- epilogue
