@@ -35,12 +35,16 @@ static __device__ long long g_trace[8192];
 namespace pair {
 constexpr int BN = 128;                 // keys per tile (64 per CTA for S)
 constexpr int NKC = 9;                  // 64-column key chunks: 8 latent + 1 rope
-// The key part of a tile is one buffer, filled and released in NKG pieces (2: rope chunk + latent
-// chunks 0-3, then latent chunks 4-7, so that a refill starts while S = Q K^T still reads the other
-// piece).  One piece measured faster: every extra wait / commit pair in the issuing thread costs
-// more than the earlier refill gains.
-constexpr int NKG = 1;
-constexpr int KBOX = 8 / NKG;           // latent column chunks brought by one TMA request of the key part
+// The key part of a tile is one buffer, filled and released in NKG pieces, so that the refill of a piece
+// starts while S = Q K^T still reads the others.  S takes the chunks in the order rope, latent 0..7; piece p
+// covers positions [piece_begin(p), piece_begin(p + 1)) of that order.
+#ifndef LCA_TC2_NKG
+#define LCA_TC2_NKG 2
+#endif
+constexpr int NKG = LCA_TC2_NKG;
+static_assert(NKG >= 1 && NKG <= 3, "pieces of the key buffer");
+__host__ __device__ constexpr int piece_begin(int p) { return NKG == 1 ? 9 * p : NKG == 2 ? (p == 0 ? 0 : p == 1 ? 5 : 9) : 3 * p; }
+constexpr int KBOX = NKG == 1 ? 8 : NKG == 2 ? 4 : 1;   // latent column chunks brought by one TMA request of the key part
 constexpr int VBOX = 2;                 // column chunks brought by one request of the value part
 constexpr int QCH = 64 * 128;           // bytes of one query chunk  (64 rows)
 constexpr int KCH = 64 * 128;           // bytes of one key chunk    (64 keys)
@@ -157,11 +161,11 @@ attn_tc2_kernel(const __grid_constant__ Tc2Params p) {
         bool good = true;
         for (int gk = 0; gk < NKG; ++gk) {
           if (!mbar_wait(BAR_KEMPTY(gk), (j & 1) ^ 1, abort_flag)) { fail(ERR_WAIT_KV_EMPTY); good = false; break; }
-          const int n_sem = 8 / NKG, n_all = n_sem + (gk == 0 ? 1 : 0);
-          if (rank == 0) mbar_expect_tx(BAR_KFULL(gk), 2 * n_all * KCH);
+          const int pos0 = piece_begin(gk), pos1 = piece_begin(gk + 1);
+          if (rank == 0) mbar_expect_tx(BAR_KFULL(gk), 2 * (pos1 - pos0) * KCH);
           const uint32_t k_bar = mapa_u32(BAR_KFULL(gk), 0);
-          if (gk == 0) tma_load_3d_pair(sK + 8 * KCH, mp, 0, 0, row, k_bar);
-          for (int c = gk * n_sem; c < (gk + 1) * n_sem; c += KBOX) tma_load_3d_pair(sK + c * KCH, ms, 0, row, c, k_bar);
+          if (pos0 == 0) tma_load_3d_pair(sK + 8 * KCH, mp, 0, 0, row, k_bar);
+          for (int c = max(pos0 - 1, 0); c < pos1 - 1; c += KBOX) tma_load_3d_pair(sK + c * KCH, ms, 0, row, c, k_bar);
         }
         if (!good) break;
       }
@@ -234,10 +238,9 @@ attn_tc2_kernel(const __grid_constant__ Tc2Params p) {
           if (gk == 0) TRACE(1, j);
           if (!ok) { if (leader) fail(ERR_WAIT_KV_FULL); break; }
           tc_fence_after();
-          constexpr int n_sem = 8 / NKG;
 #pragma unroll
-          for (int cc = (gk == 0 ? -1 : 0); cc < n_sem; ++cc) {
-            const int c = cc < 0 ? 8 : gk * n_sem + cc;         // the rope chunk goes first
+          for (int pos = piece_begin(gk); pos < piece_begin(gk + 1); ++pos) {
+            const int c = pos == 0 ? 8 : pos - 1;               // the rope chunk goes first
 #pragma unroll
             for (int k = 0; k < 4; ++k) {
               const uint64_t ad = desc_add(qd0, (c * QCH + k * 32) >> 4);
