@@ -83,7 +83,8 @@ attn_tc1_kernel(const __grid_constant__ TcParams p) {
   volatile uint32_t* tmem_slot = reinterpret_cast<volatile uint32_t*>(base_ptr + P::OFF_MISC);
   volatile int* abort_flag = reinterpret_cast<volatile int*>(base_ptr + P::OFF_MISC + 4);
 
-  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  // the warp index through a shuffle: provably warp-uniform, so the role branches below are uniform branches
+  const int warp = __shfl_sync(0xffffffffu, (int)(threadIdx.x >> 5), 0), lane = threadIdx.x & 31;
 
   // ---- which rows, which key tiles
   const int tile = p.n_tok_tiles - 1 - (int)blockIdx.x;      // heaviest (latest) query tiles first
@@ -157,22 +158,21 @@ attn_tc1_kernel(const __grid_constant__ TcParams p) {
     }
   } else if (warp == 1) {
     // =============================================================== MMA issuer
+    // The whole warp walks the loop converged (every lane polls the barriers); one elected lane issues.
     constexpr uint32_t IDESC_S = umma_idesc_bf16(ROWS, BN, false, false);
     constexpr uint32_t IDESC_PV = umma_idesc_bf16(ROWS, NV * 64, false, true);
+    const uint32_t leader = elect_one();
     bool ok = n_tiles > 0;
-    if (ok && lane == 0) ok = mbar_wait(BAR_Q(), 0, abort_flag);
-    ok = __all_sync(0xffffffffu, ok);
-    if (!ok && n_tiles > 0 && lane == 0) fail(ERR_WAIT_Q);
-    auto issue_pv = [&](int j) -> bool {      // O += P_j V_j   (whole warp enters; lane 0 issues)
+    if (ok) {
+      ok = mbar_wait(BAR_Q(), 0, abort_flag);
+      if (!ok && leader) fail(ERR_WAIT_Q);
+    }
+    const uint64_t qd0 = umma_desc_sw128(sQ, 16, 1024);
+    auto issue_pv = [&](int j) -> bool {      // O += P_j V_j
       const int s = j % STAGES, round = j / STAGES;
-      bool good = true;
-      if (lane == 0) {
-        good = mbar_wait(BAR_PFULL(j & 1), (j >> 1) & 1, abort_flag);
-        if (good && !V_IN_K) good = mbar_wait(BAR_VFULL(s), round & 1, abort_flag);
-        if (!good) fail(ERR_WAIT_P_FULL);
-      }
-      good = __all_sync(0xffffffffu, good);
-      if (!good) return false;
+      bool good = mbar_wait(BAR_PFULL(j & 1), (j >> 1) & 1, abort_flag);
+      if (good && !V_IN_K) good = mbar_wait(BAR_VFULL(s), round & 1, abort_flag);
+      if (!good) { if (leader) fail(ERR_WAIT_P_FULL); return false; }
       const uint32_t vbase = V_IN_K ? sK + s * P::K_STAGE : sV + s * P::V_STAGE;
       // Rows of the cache beyond the valid count (decode, last tile) may hold anything; their
       // probabilities are exactly 0, so zero the value rows to keep 0 * garbage out of O.
@@ -187,42 +187,34 @@ attn_tc1_kernel(const __grid_constant__ TcParams p) {
         fence_proxy_async_smem();
         __syncwarp();
       }
-      if (lane == 0) {
-        tc_fence_after();
-        const uint32_t ptm = tmem + ((j & 1) ? P::TM_S1 : P::TM_S0);
-        const uint64_t vd0 = umma_desc_sw128(vbase, CHUNK_BYTES_KV, 1024);
+      tc_fence_after();
+      const uint32_t ptm = tmem + ((j & 1) ? P::TM_S1 : P::TM_S0);
+      const uint64_t vd0 = umma_desc_sw128(vbase, CHUNK_BYTES_KV, 1024);
 #pragma unroll
-        for (int k = 0; k < BN / 16; ++k)
-          umma_ts(tmem + P::TM_O, ptm + k * 8, desc_add(vd0, (k * 2048) >> 4), IDESC_PV, (j > 0 || k > 0) ? 1u : 0u);
-        umma_commit(V_IN_K ? BAR_KEMPTY(s) : BAR_VEMPTY(s));
-        umma_commit(BAR_ODONE);
-      }
-      __syncwarp();
+      for (int k = 0; k < BN / 16; ++k)
+        umma_ts_elected(leader, tmem + P::TM_O, ptm + k * 8, desc_add(vd0, (k * 2048) >> 4), IDESC_PV, (j > 0 || k > 0) ? 1u : 0u);
+      umma_commit_elected(leader, V_IN_K ? BAR_KEMPTY(s) : BAR_VEMPTY(s));
+      umma_commit_elected(leader, BAR_ODONE);
       return true;
     };
     for (int j = 0; ok && j < n_tiles; ++j) {
       const int s = j % STAGES, round = j / STAGES;
-      if (lane == 0) {
-        ok = mbar_wait(BAR_KFULL(s), round & 1, abort_flag);
-        if (!ok) fail(ERR_WAIT_KV_FULL);
-        if (ok) {
-          tc_fence_after();
-          const uint32_t stm = tmem + ((j & 1) ? P::TM_S1 : P::TM_S0);
-          // descriptors are built once per tile; per instruction only the start address moves
-          const uint64_t qd0 = umma_desc_sw128(sQ, 16, 1024), kd0 = umma_desc_sw128(sK + s * P::K_STAGE, 16, 1024);
+      ok = mbar_wait(BAR_KFULL(s), round & 1, abort_flag);
+      if (!ok) { if (leader) fail(ERR_WAIT_KV_FULL); break; }
+      tc_fence_after();
+      const uint32_t stm = tmem + ((j & 1) ? P::TM_S1 : P::TM_S0);
+      // descriptors are built once; per instruction only the start address moves
+      const uint64_t kd0 = umma_desc_sw128(sK + s * P::K_STAGE, 16, 1024);
 #pragma unroll
-          for (int c = 0; c < NK; ++c) {
+      for (int c = 0; c < NK; ++c) {
 #pragma unroll
-            for (int k = 0; k < 4; ++k)
-              umma_ss(stm, desc_add(qd0, (c * CHUNK_BYTES_Q + k * 32) >> 4), desc_add(kd0, (c * CHUNK_BYTES_KV + k * 32) >> 4),
-                      IDESC_S, (c > 0 || k > 0) ? 1u : 0u);
-          }
-          umma_commit(BAR_SFULL(j & 1));
-          if (!V_IN_K) umma_commit(BAR_KEMPTY(s));
-        }
+        for (int k = 0; k < 4; ++k)
+          umma_ss_elected(leader, stm, desc_add(qd0, (c * CHUNK_BYTES_Q + k * 32) >> 4),
+                          desc_add(kd0, (c * CHUNK_BYTES_KV + k * 32) >> 4), IDESC_S, (c > 0 || k > 0) ? 1u : 0u);
       }
-      ok = __all_sync(0xffffffffu, ok);
-      if (ok && j >= 1) ok = issue_pv(j - 1);
+      umma_commit_elected(leader, BAR_SFULL(j & 1));
+      if (!V_IN_K) umma_commit_elected(leader, BAR_KEMPTY(s));
+      if (j >= 1) ok = issue_pv(j - 1);
     }
     if (ok && n_tiles > 0) issue_pv(n_tiles - 1);
   } else {
