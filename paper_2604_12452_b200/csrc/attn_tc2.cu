@@ -14,6 +14,11 @@
 //     and signal the even CTA, whose MMA warp issues every tcgen05.mma for the pair.
 // Everything else (tile walk over representatives then local tokens, boundary-only masks, lazy
 // rescale of O, bounded waits with a status word) follows the single-CTA kernel.
+//
+// A CTA pair is persistent: it takes work items (tiles of 128 query rows) from the heaviest (latest
+// tokens) down in a fixed stride.  Barriers and tensor memory are set up once; the query tile of the
+// next item is fetched as soon as the last S product of the current one has completed, and its first
+// products run while the softmax threads still normalise and store the current output.
 #include <cstring>
 
 #include "lca_common.cuh"
@@ -54,7 +59,7 @@ constexpr int Q_BYTES = NKC * QCH, K_BYTES = NKC * KCH, V_BYTES = 8 * VCH, P_BYT
 constexpr int OFF_Q = 0, OFF_K = OFF_Q + Q_BYTES, OFF_V = OFF_K + K_BYTES, OFF_P = OFF_V + V_BYTES;
 constexpr int OFF_BAR = OFF_P + P_BYTES;
 constexpr int OFF_MISC = OFF_BAR + 256, OFF_RED = OFF_BAR + 512;
-constexpr int SMEM_BYTES = OFF_BAR + 512 + 2 * 128 * 4;     // 230912
+constexpr int SMEM_BYTES = OFF_BAR + 512 + 3 * 128 * 4;     // 231424
 constexpr int TM_S0 = 0, TM_S1 = 64, TM_O = 128, TM_COLS = 512;
 constexpr int THREADS = 224;            // warps: 0 K/Q loads, 1 MMA + TMEM, 2-5 softmax, 6 V loads
 constexpr float RESCALE_THRESHOLD = 8.0f;
@@ -68,9 +73,40 @@ struct Tc2Params {
   CUtensorMap k_val, c_val;       // the same memory, box of 64 rows x VBOX chunks
   bf16* out; float* lse; const int32_t* cache_rows;
   int B, q_len, H, L, g, w, cap, n_rep_bias, decode;
-  int HB, TB, n_tok_tiles;
+  int HB, TB, n_tok_tiles, n_head_blocks;
+  long long n_items;              // query tiles x head blocks x batch
   float scale_log2, bias_log2;
 };
+
+// One work item = one tile of 128 query rows; the same arithmetic in every role of both CTAs.
+struct Item {
+  int b, head0, t0, t1;
+  int n_a_lo, n_a_hi, first_lo, nA, n_tiles;
+};
+__device__ __forceinline__ Item make_item(const Tc2Params& p, long long idx) {
+  Item it;
+  // heaviest query tiles (latest tokens) first; batch and head block vary fastest
+  const long long per_tile = (long long)p.n_head_blocks * p.B;
+  const int tile = p.n_tok_tiles - 1 - (int)(idx / per_tile);
+  const int rem = (int)(idx % per_tile);
+  it.b = rem / p.n_head_blocks;
+  it.head0 = (rem % p.n_head_blocks) * p.HB;
+  it.t0 = tile * p.TB;
+  it.t1 = min(it.t0 + p.TB, p.q_len) - 1;
+  int nB;
+  if (p.decode) {
+    it.n_a_hi = it.n_a_lo = min(max(p.cache_rows[it.b], 0), p.cap);
+    it.first_lo = 0; nB = 0;
+  } else {
+    it.n_a_lo = reps_visible(it.t0, p.w, p.g);
+    it.n_a_hi = reps_visible(it.t1, p.w, p.g);
+    it.first_lo = it.n_a_lo * p.g;
+    nB = (it.t1 - it.first_lo + pair::BN) / pair::BN;
+  }
+  it.nA = (it.n_a_hi + pair::BN - 1) / pair::BN;
+  it.n_tiles = it.nA + nB;
+  return it;
+}
 
 __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(pair::THREADS, 1)
 attn_tc2_kernel(const __grid_constant__ Tc2Params p) {
@@ -81,7 +117,9 @@ attn_tc2_kernel(const __grid_constant__ Tc2Params p) {
   const uint32_t bars = base + OFF_BAR;
   // One buffer for the key part of a tile (nine 64-column chunks) and one for each 64-key half of
   // its value part: a buffer is refilled with the next tile's data as soon as the MMAs that read it
-  // have completed, so the loads of tile j+1 run underneath the remaining MMAs of tile j.
+  // have completed, so the loads of tile j+1 run underneath the remaining MMAs of tile j.  Tiles are
+  // counted through all items of the pair (jt), which is what every per-tile barrier phase follows;
+  // the per-item barriers (Q, QFREE, OLAST, OFREE, OLOCAL) follow the count of non-empty items.
   const uint32_t BAR_Q = bars, BAR_SFULL0 = bars + 8, BAR_SFULL1 = bars + 16, BAR_PFULL = bars + 24,
                  BAR_ODONE = bars + 32;
   auto BAR_KFULL = [&](int c) { return bars + 40 + 8 * c; };            // NKG (room for 9)
@@ -89,32 +127,19 @@ attn_tc2_kernel(const __grid_constant__ Tc2Params p) {
   auto BAR_VFULL = [&](int h) { return bars + 40 + 144 + 8 * h; };      // 2
   auto BAR_VEMPTY = [&](int h) { return bars + 40 + 160 + 8 * h; };     // 2
   const uint32_t BAR_PLOCAL = bars + 224;        // odd CTA: its 128 softmax threads -> its relay thread
+  const uint32_t BAR_QFREE = bars + 216;         // last S of an item done: the query tile may be replaced
+  const uint32_t BAR_OLAST = bars + 232;         // last P V of an item done: O is complete
+  const uint32_t BAR_OFREE = bars + 240;         // O has been read out by both CTAs: the next item may overwrite it
+  const uint32_t BAR_OLOCAL = bars + 248;        // odd CTA: O read out by its 128 threads -> its relay thread
   volatile uint32_t* tmem_slot = reinterpret_cast<volatile uint32_t*>(smem + OFF_MISC);
   volatile int* abort_flag = reinterpret_cast<volatile int*>(smem + OFF_MISC + 4);
-  volatile float* red = reinterpret_cast<volatile float*>(smem + OFF_RED);    // [2][128]
+  volatile float* red = reinterpret_cast<volatile float*>(smem + OFF_RED);    // [3][128]
 
   // the warp index through a shuffle: provably warp-uniform, so the role branches below are uniform branches
   const int warp = __shfl_sync(0xffffffffu, (int)(threadIdx.x >> 5), 0), lane = threadIdx.x & 31;
   const uint32_t rank = cluster_ctarank();       // 0 = even CTA: issues the MMAs, owns the "full" barriers
 
-  // ---- which rows, which key tiles (identical in both CTAs of the pair)
-  const int tile = p.n_tok_tiles - 1 - (int)(blockIdx.x >> 1);       // heaviest query tiles first
-  const int hb = blockIdx.y, b = blockIdx.z;
-  const int t0 = tile * p.TB;
-  const int t1 = min(t0 + p.TB, p.q_len) - 1;
-  const int head0 = hb * p.HB;
-  int nA, nB, first_lo, n_a_lo, n_a_hi;
-  if (p.decode) {
-    n_a_hi = n_a_lo = min(max(p.cache_rows[b], 0), p.cap);
-    first_lo = 0; nB = 0;
-  } else {
-    n_a_lo = reps_visible(t0, p.w, p.g);
-    n_a_hi = reps_visible(t1, p.w, p.g);
-    first_lo = n_a_lo * p.g;
-    nB = (t1 - first_lo + BN) / BN;
-  }
-  nA = (n_a_hi + BN - 1) / BN;
-  const int n_tiles = nA + nB;
+  const long long pair_id = blockIdx.x >> 1, n_pairs = gridDim.x >> 1;
 
   if (threadIdx.x == 0) {
     mbar_init(BAR_Q, 1);
@@ -123,6 +148,7 @@ attn_tc2_kernel(const __grid_constant__ Tc2Params p) {
     mbar_init(BAR_SFULL0, 1); mbar_init(BAR_SFULL1, 1);
     mbar_init(BAR_PFULL, 129); mbar_init(BAR_ODONE, 1);     // 128 threads of the even CTA + the odd CTA's relay
     mbar_init(BAR_PLOCAL, 128);
+    mbar_init(BAR_QFREE, 1); mbar_init(BAR_OLAST, 1); mbar_init(BAR_OFREE, 129); mbar_init(BAR_OLOCAL, 128);
     *abort_flag = (base & 1023u) ? 1 : 0;
     fence_mbar_init();
   }
@@ -146,72 +172,91 @@ attn_tc2_kernel(const __grid_constant__ Tc2Params p) {
   const int row0 = 64 * (int)rank;
 
   if (warp == 0) {
-    // =============================================== producer: Q once, then the key part of each tile
-    if (lane == 0 && n_tiles > 0 && !*abort_flag) {
+    // =============================================== producer: Q of each item, then the key part of each tile
+    if (lane == 0 && !*abort_flag) {
       const uint32_t q_bar = mapa_u32(BAR_Q, 0);
-      if (rank == 0) mbar_expect_tx(BAR_Q, 2 * Q_BYTES);
-      const int qtok = b * p.q_len + t0 + row0 / p.HB, qhead = head0 + row0 % p.HB;
-      for (int c = 0; c < 8; ++c) tma_load_3d_pair(sQ + c * QCH, &p.q_sem, c * 64, qhead, qtok, q_bar);
-      tma_load_3d_pair(sQ + 8 * QCH, &p.q_pos, 0, qhead, qtok, q_bar);
-      for (int j = 0; j < n_tiles; ++j) {
-        const bool isA = j < nA;
-        const int row = (isA ? b * p.cap + j * BN : b * p.L + first_lo + (j - nA) * BN) + 64 * (int)rank;
-        const CUtensorMap* ms = isA ? &p.c_sem : &p.k_sem;
-        const CUtensorMap* mp = isA ? &p.c_pos : &p.k_pos;
-        bool good = true;
-        for (int gk = 0; gk < NKG; ++gk) {
-          if (!mbar_wait(BAR_KEMPTY(gk), (j & 1) ^ 1, abort_flag)) { fail(ERR_WAIT_KV_EMPTY); good = false; break; }
-          const int pos0 = piece_begin(gk), pos1 = piece_begin(gk + 1);
-          if (rank == 0) mbar_expect_tx(BAR_KFULL(gk), 2 * (pos1 - pos0) * KCH);
-          const uint32_t k_bar = mapa_u32(BAR_KFULL(gk), 0);
-          if (pos0 == 0) tma_load_3d_pair(sK + 8 * KCH, mp, 0, 0, row, k_bar);
-          for (int c = max(pos0 - 1, 0); c < pos1 - 1; c += KBOX) tma_load_3d_pair(sK + c * KCH, ms, 0, row, c, k_bar);
+      uint32_t jt = 0, n_item = 0;
+      bool good = true;
+      for (long long idx = pair_id; good && idx < p.n_items; idx += n_pairs) {
+        const Item it = make_item(p, idx);
+        if (it.n_tiles == 0) continue;             // nothing to attend to (decode with an empty cache): no loads, no phases
+        // the query tile may be replaced once the last S of the previous item has completed
+        if (!mbar_wait(BAR_QFREE, (n_item & 1) ^ 1, abort_flag)) { fail(ERR_WAIT_Q); break; }
+        if (rank == 0) mbar_expect_tx(BAR_Q, 2 * Q_BYTES);
+        const int qtok = it.b * p.q_len + it.t0 + row0 / p.HB, qhead = it.head0 + row0 % p.HB;
+        for (int c = 0; c < 8; ++c) tma_load_3d_pair(sQ + c * QCH, &p.q_sem, c * 64, qhead, qtok, q_bar);
+        tma_load_3d_pair(sQ + 8 * QCH, &p.q_pos, 0, qhead, qtok, q_bar);
+        ++n_item;
+        for (int j = 0; good && j < it.n_tiles; ++j, ++jt) {
+          const bool isA = j < it.nA;
+          const int row = (isA ? it.b * p.cap + j * BN : it.b * p.L + it.first_lo + (j - it.nA) * BN) + 64 * (int)rank;
+          const CUtensorMap* ms = isA ? &p.c_sem : &p.k_sem;
+          const CUtensorMap* mp = isA ? &p.c_pos : &p.k_pos;
+          for (int gk = 0; gk < NKG; ++gk) {
+            if (!mbar_wait(BAR_KEMPTY(gk), (jt & 1) ^ 1, abort_flag)) { fail(ERR_WAIT_KV_EMPTY); good = false; break; }
+            const int pos0 = piece_begin(gk), pos1 = piece_begin(gk + 1);
+            if (rank == 0) mbar_expect_tx(BAR_KFULL(gk), 2 * (pos1 - pos0) * KCH);
+            const uint32_t k_bar = mapa_u32(BAR_KFULL(gk), 0);
+            if (pos0 == 0) tma_load_3d_pair(sK + 8 * KCH, mp, 0, 0, row, k_bar);
+            for (int c = max(pos0 - 1, 0); c < pos1 - 1; c += KBOX) tma_load_3d_pair(sK + c * KCH, ms, 0, row, c, k_bar);
+          }
         }
-        if (!good) break;
       }
     }
   } else if (warp == 6) {
     // =============================================== producer: the value part of each tile
-    if (lane == 0 && n_tiles > 0 && !*abort_flag) {
-      for (int j = 0; j < n_tiles; ++j) {
-        const bool isA = j < nA;
-        const int row = isA ? b * p.cap + j * BN : b * p.L + first_lo + (j - nA) * BN;
-        const CUtensorMap* mv = isA ? &p.c_val : &p.k_val;
-        bool good = true;
-        for (int kh = 0; kh < 2; ++kh) {            // keys [64*kh, 64*kh+64) of the tile
-          if (!mbar_wait(BAR_VEMPTY(kh), (j & 1) ^ 1, abort_flag)) { fail(ERR_WAIT_KV_EMPTY); good = false; break; }
-          if (rank == 0) mbar_expect_tx(BAR_VFULL(kh), 2 * 4 * VCH);
-          const uint32_t v_bar = mapa_u32(BAR_VFULL(kh), 0);
-          // output columns of this CTA: [128*rank, +128) of the first 256, then of the second 256
-          for (int i = 0; i < 4; i += VBOX) {
-            const int chunk = (i >> 1) * 4 + 2 * (int)rank + (i & 1);
-            tma_load_3d_pair(sV + (kh * 4 + i) * VCH, mv, 0, row + 64 * kh, chunk, v_bar);
+    if (lane == 0 && !*abort_flag) {
+      uint32_t jt = 0;
+      bool good = true;
+      for (long long idx = pair_id; good && idx < p.n_items; idx += n_pairs) {
+        const Item it = make_item(p, idx);
+        for (int j = 0; good && j < it.n_tiles; ++j, ++jt) {
+          const bool isA = j < it.nA;
+          const int row = isA ? it.b * p.cap + j * BN : it.b * p.L + it.first_lo + (j - it.nA) * BN;
+          const CUtensorMap* mv = isA ? &p.c_val : &p.k_val;
+          for (int kh = 0; kh < 2; ++kh) {            // keys [64*kh, 64*kh+64) of the tile
+            if (!mbar_wait(BAR_VEMPTY(kh), (jt & 1) ^ 1, abort_flag)) { fail(ERR_WAIT_KV_EMPTY); good = false; break; }
+            if (rank == 0) mbar_expect_tx(BAR_VFULL(kh), 2 * 4 * VCH);
+            const uint32_t v_bar = mapa_u32(BAR_VFULL(kh), 0);
+            // output columns of this CTA: [128*rank, +128) of the first 256, then of the second 256
+            for (int i = 0; i < 4; i += VBOX) {
+              const int chunk = (i >> 1) * 4 + 2 * (int)rank + (i & 1);
+              tma_load_3d_pair(sV + (kh * 4 + i) * VCH, mv, 0, row + 64 * kh, chunk, v_bar);
+            }
           }
         }
-        if (!good) break;
       }
     }
   } else if (warp == 1) {
     // =============================================== MMA issuer (even CTA only)
     // The whole warp walks the loop (every lane polls the barriers); one elected lane issues.
-    if (rank == 0 && n_tiles > 0) {
+    if (rank == 0 && !*abort_flag) {
       const uint32_t leader = elect_one();
       constexpr uint32_t IDESC_S = umma_idesc_bf16(128, BN, false, false);
       constexpr uint32_t IDESC_PV = umma_idesc_bf16(128, 256, false, true);
-      // The issuing thread's own instructions between two tcgen05.mma are not hidden behind the
-      // tensor core, so the shared-memory descriptors are built once and only their start-address
-      // field (low word) is advanced per instruction.
+      // The shared-memory descriptors are built once and only their start-address field (low word)
+      // is advanced per instruction.
       const uint64_t qd0 = umma_desc_sw128(sQ, 16, 1024), kd0 = umma_desc_sw128(sK, 16, 1024);
       const uint64_t pd0 = umma_desc_sw128(sP, 16, 1024), vd0 = umma_desc_sw128(sV, VCH, 1024);
-      bool ok = mbar_wait(BAR_Q, 0, abort_flag);
-      if (!ok) if (leader) fail(ERR_WAIT_Q);
-      auto issue_pv = [&](int j) -> bool {
-        TRACE(3, j);
-        if (!mbar_wait(BAR_PFULL, j & 1, abort_flag)) { if (leader) fail(ERR_WAIT_P_FULL); return false; }
-        TRACE(4, j);
+      uint32_t jt = 0, n_item = 0;                  // tiles issued so far (all items), non-empty items started
+      bool ok = true;
+      // P V of a tile is issued after S of the next one (so that S runs while the softmax threads work);
+      // the tile whose P V is still to be issued:
+      bool pending = false, pend_first = false, pend_last = false;
+      uint32_t pend_t = 0, pend_item = 0;
+      auto issue_pending_pv = [&]() -> bool {
+        const uint32_t t = pend_t;
+        pending = false;
+        TRACE(3, t);
+        if (pend_first && pend_item > 0) {
+          // O of the previous item has been read out by the epilogue threads of both CTAs
+          if (!mbar_wait(BAR_OFREE, (pend_item - 1) & 1, abort_flag)) { if (leader) fail(ERR_WAIT_O_DONE); return false; }
+        }
+        if (!mbar_wait(BAR_PFULL, t & 1, abort_flag)) { if (leader) fail(ERR_WAIT_P_FULL); return false; }
+        TRACE(4, t);
 #pragma unroll
         for (int kh = 0; kh < 2; ++kh) {
-          if (!mbar_wait(BAR_VFULL(kh), j & 1, abort_flag)) { if (leader) fail(ERR_WAIT_KV_FULL); return false; }
+          if (!mbar_wait(BAR_VFULL(kh), t & 1, abort_flag)) { if (leader) fail(ERR_WAIT_KV_FULL); return false; }
           tc_fence_after();
           // descriptors differ from the precomputed bases only in the 16-byte-unit start address
 #pragma unroll
@@ -220,52 +265,83 @@ attn_tc2_kernel(const __grid_constant__ Tc2Params p) {
             for (int k = 0; k < 4; ++k) {
               const uint64_t ad = desc_add(pd0, (kh * PCH + k * 32) >> 4);
               const uint64_t bd = desc_add(vd0, ((kh * 4 + n2 * 2) * VCH + k * 2048) >> 4);
-              umma_ss_pair_elected(leader, tmem + TM_O + n2 * 128, ad, bd, IDESC_PV, (j > 0 || kh > 0 || k > 0) ? 1u : 0u);
+              umma_ss_pair_elected(leader, tmem + TM_O + n2 * 128, ad, bd, IDESC_PV, (!pend_first || kh > 0 || k > 0) ? 1u : 0u);
             }
           }
           umma_commit_pair_elected(leader, BAR_VEMPTY(kh), 3);
         }
         umma_commit_pair_elected(leader, BAR_ODONE, 3);
-        TRACE(5, j);
+        if (pend_last) umma_commit_pair_elected(leader, BAR_OLAST, 3);      // one phase per item, for the epilogue
+        TRACE(5, t);
         return true;
       };
-      for (int j = 0; ok && j < n_tiles; ++j) {
-        const uint32_t stm = tmem + ((j & 1) ? TM_S1 : TM_S0);
-        TRACE(0, j);
-#pragma unroll
-        for (int gk = 0; gk < NKG; ++gk) {
-          ok = mbar_wait(BAR_KFULL(gk), j & 1, abort_flag);
-          if (gk == 0) TRACE(1, j);
-          if (!ok) { if (leader) fail(ERR_WAIT_KV_FULL); break; }
-          tc_fence_after();
-#pragma unroll
-          for (int pos = piece_begin(gk); pos < piece_begin(gk + 1); ++pos) {
-            const int c = pos == 0 ? 8 : pos - 1;               // the rope chunk goes first
-#pragma unroll
-            for (int k = 0; k < 4; ++k) {
-              const uint64_t ad = desc_add(qd0, (c * QCH + k * 32) >> 4);
-              const uint64_t bd = desc_add(kd0, (c * KCH + k * 32) >> 4);
-              umma_ss_pair_elected(leader, stm, ad, bd, IDESC_S, (c != 8 || k > 0) ? 1u : 0u);
+      for (long long idx = pair_id; ok && idx < p.n_items; idx += n_pairs) {
+        const Item it = make_item(p, idx);
+        if (it.n_tiles == 0) continue;
+        for (int j = 0; ok && j < it.n_tiles; ++j, ++jt) {
+          // In the middle of an item S of tile j goes before P V of tile j - 1.  At an item boundary the
+          // last P V of the previous item goes first: nothing else can run until the new query tile is in.
+          const bool pv_first = (j == 0);
+          if (pv_first) {
+            if (pending) ok = issue_pending_pv();
+            if (ok) {
+              ok = mbar_wait(BAR_Q, n_item & 1, abort_flag);
+              if (!ok && leader) fail(ERR_WAIT_Q);
             }
+            if (!ok) break;
           }
-          umma_commit_pair_elected(leader, BAR_KEMPTY(gk), 3);
+          const uint32_t stm = tmem + ((jt & 1) ? TM_S1 : TM_S0);
+          TRACE(0, jt);
+#pragma unroll
+          for (int gk = 0; gk < NKG; ++gk) {
+            ok = mbar_wait(BAR_KFULL(gk), jt & 1, abort_flag);
+            if (gk == 0) TRACE(1, jt);
+            if (!ok) { if (leader) fail(ERR_WAIT_KV_FULL); break; }
+            tc_fence_after();
+#pragma unroll
+            for (int pos = piece_begin(gk); pos < piece_begin(gk + 1); ++pos) {
+              const int c = pos == 0 ? 8 : pos - 1;               // the rope chunk goes first
+#pragma unroll
+              for (int k = 0; k < 4; ++k) {
+                const uint64_t ad = desc_add(qd0, (c * QCH + k * 32) >> 4);
+                const uint64_t bd = desc_add(kd0, (c * KCH + k * 32) >> 4);
+                umma_ss_pair_elected(leader, stm, ad, bd, IDESC_S, (c != 8 || k > 0) ? 1u : 0u);
+              }
+            }
+            umma_commit_pair_elected(leader, BAR_KEMPTY(gk), 3);
+          }
+          if (!ok) break;
+          umma_commit_pair_elected(leader, (jt & 1) ? BAR_SFULL1 : BAR_SFULL0, 3);
+          if (j + 1 == it.n_tiles) umma_commit_pair_elected(leader, BAR_QFREE, 3);     // last S of the item is in flight
+          TRACE(2, jt);
+          if (!pv_first && pending) ok = issue_pending_pv();
+          pending = true; pend_t = jt; pend_first = (j == 0); pend_last = (j + 1 == it.n_tiles); pend_item = n_item;
         }
-        if (!ok) break;
-        umma_commit_pair_elected(leader, (j & 1) ? BAR_SFULL1 : BAR_SFULL0, 3);
-        TRACE(2, j);
-        if (j >= 1) ok = issue_pv(j - 1);
+        ++n_item;
       }
-      if (ok) issue_pv(n_tiles - 1);
+      if (ok && pending) issue_pending_pv();
     }
-    // =============================================== relay (odd CTA): "P of this CTA is complete" -> even CTA
+    // =============================================== relay (odd CTA): "P complete" / "O read out" -> even CTA
     // A release-arrive on a barrier of the other CTA stalls its thread for 1000-2000 cycles.  The odd CTA's
-    // softmax threads therefore arrive on a barrier of their own CTA and this otherwise idle thread forwards
-    // one arrival per tile (its acquire on the local barrier and release on the remote one chain the ordering).
-    if (rank == 1 && lane == 0 && n_tiles > 0) {
-      const uint32_t pfull_addr = mapa_u32(BAR_PFULL, 0);
-      for (int j = 0; j < n_tiles; ++j) {
-        if (!mbar_wait(BAR_PLOCAL, j & 1, abort_flag)) { fail(ERR_WAIT_P_FULL); break; }
-        mbar_arrive_cluster_relaxed(pfull_addr);
+    // softmax threads therefore arrive on barriers of their own CTA and this otherwise idle thread forwards
+    // one relaxed arrival per tile and one per item: it has observed the threads' arrivals (acquire), their
+    // writes of P (followed by a proxy fence) and reads of O (followed by tcgen05.wait) are complete, and the
+    // consumer is this SM's own tensor core, started by an instruction that the even CTA issues afterwards.
+    if (rank == 1 && lane == 0 && !*abort_flag) {
+      const uint32_t pfull_addr = mapa_u32(BAR_PFULL, 0), ofree_addr = mapa_u32(BAR_OFREE, 0);
+      uint32_t jt = 0, n_item = 0;
+      bool good = true;
+      for (long long idx = pair_id; good && idx < p.n_items; idx += n_pairs) {
+        const Item it = make_item(p, idx);
+        if (it.n_tiles == 0) continue;
+        for (int j = 0; j < it.n_tiles; ++j, ++jt) {
+          if (!mbar_wait(BAR_PLOCAL, jt & 1, abort_flag)) { fail(ERR_WAIT_P_FULL); good = false; break; }
+          mbar_arrive_cluster_relaxed(pfull_addr);
+        }
+        if (!good) break;
+        if (!mbar_wait(BAR_OLOCAL, n_item & 1, abort_flag)) { fail(ERR_WAIT_O_DONE); break; }
+        mbar_arrive_cluster_relaxed(ofree_addr);
+        ++n_item;
       }
     }
   } else {
@@ -276,27 +352,33 @@ attn_tc2_kernel(const __grid_constant__ Tc2Params p) {
     const uint32_t lane_base = (uint32_t)(quarter * 32) << 16;
     const int rg = row0 + rl;
     const int tl = rg / p.HB, hl = rg % p.HB;
+    volatile int* fail_word = reinterpret_cast<volatile int*>(smem + OFF_MISC + 16);   // [3], softmax threads only
+    if (ln < 3) fail_word[ln] = 0;
+    asm volatile("bar.sync 1, 128;" ::: "memory");
+    // All 128 threads execute exactly one named barrier per tile and one per item, whatever happens: a
+    // thread whose wait expired marks the fail word before the barrier and everybody leaves after it.
+    bool ok = !*abort_flag;
+    uint32_t jt = 0, n_item = 0;                 // tiles / non-empty items of this pair so far
+    for (long long idx = pair_id; ok && idx < p.n_items; idx += n_pairs) {
+    const Item it = make_item(p, idx);
+    const int b = it.b, head0 = it.head0, t0 = it.t0, nA = it.nA, n_tiles = it.n_tiles;
+    const int n_a_lo = it.n_a_lo, n_a_hi = it.n_a_hi, first_lo = it.first_lo;
     const int t_row = t0 + tl;
-    const bool row_valid = t_row < p.q_len;
+    const bool row_valid = t_row <= it.t1;
     int n_a_row, bias_rows, first_row;
     if (p.decode) { n_a_row = n_a_hi; bias_rows = min(p.n_rep_bias, n_a_row); first_row = 0; }
     else { n_a_row = reps_visible(min(t_row, p.q_len - 1), p.w, p.g); bias_rows = n_a_row; first_row = n_a_row * p.g; }
     float m_ref = -INFINITY, l_sum = 0.f;
-    volatile int* fail_word = reinterpret_cast<volatile int*>(smem + OFF_MISC + 16);   // [2], softmax threads only
-    if (ln < 2) fail_word[ln] = 0;
-    asm volatile("bar.sync 1, 128;" ::: "memory");
-    // All 128 threads execute exactly one named barrier per tile, whatever happens: a thread whose
-    // wait expired marks the tile's fail word before the barrier and everybody leaves after it.
-    bool ok = !*abort_flag;
-    for (int j = 0; j < n_tiles; ++j) {
-      if (ln == 0) TRACE(8, j);
+    bool all_left = false;                       // every one of the 128 threads left the tile loop at a barrier
+    for (int j = 0; j < n_tiles; ++j, ++jt) {
+      if (ln == 0) TRACE(8, jt);
       if (ok) {
-        ok = mbar_wait((j & 1) ? BAR_SFULL1 : BAR_SFULL0, (j >> 1) & 1, abort_flag);
+        ok = mbar_wait((jt & 1) ? BAR_SFULL1 : BAR_SFULL0, (jt >> 1) & 1, abort_flag);
         if (!ok && lane == 0) fail(ERR_WAIT_S_FULL);
       }
-      if (ln == 0) TRACE(9, j);
+      if (ln == 0) TRACE(9, jt);
       ok = __all_sync(0xffffffffu, ok);
-      const uint32_t stm = tmem + lane_base + ((j & 1) ? TM_S1 : TM_S0);
+      const uint32_t stm = tmem + lane_base + ((jt & 1) ? TM_S1 : TM_S0);
       uint32_t sr[2][32];
       float tmax = -INFINITY;
       bool plain = false;
@@ -339,18 +421,18 @@ attn_tc2_kernel(const __grid_constant__ Tc2Params p) {
           }
         }
       } else {
-        fail_word[j & 1] = 1;
+        fail_word[jt & 1] = 1;
       }
       // the two key halves of a row live in different warps: combine their maxima
-      red[(j & 1) * 128 + ln] = tmax;
+      red[(jt & 1) * 128 + ln] = tmax;
       asm volatile("bar.sync 1, 128;" ::: "memory");
-      if (fail_word[j & 1]) { ok = false; break; }          // uniform over the 128 threads
-      tmax = fmaxf(tmax, red[(j & 1) * 128 + (ln ^ 64)]);
+      if (fail_word[jt & 1]) { ok = false; all_left = true; break; }          // uniform over the 128 threads
+      tmax = fmaxf(tmax, red[(jt & 1) * 128 + (ln ^ 64)]);
       bool need = false;
       float factor = 1.f;
       if (j == 0) m_ref = tmax;
       else if (tmax > m_ref + RESCALE_THRESHOLD) { need = true; factor = exp2f(m_ref - tmax); }
-      if (ln == 0) TRACE(10, j);
+      if (ln == 0) TRACE(10, jt);
       // The probabilities depend only on S and the (new) reference maximum: compute and pack them
       // while P V of the previous tile is still running, then wait, rescale O if needed, and store.
       const float m_new = need ? tmax : m_ref;
@@ -368,13 +450,13 @@ attn_tc2_kernel(const __grid_constant__ Tc2Params p) {
       }
       if (j >= 1) {
         // P (one buffer) and O are free once P_{j-1} V_{j-1} has completed
-        ok = mbar_wait(BAR_ODONE, (j - 1) & 1, abort_flag);
+        ok = mbar_wait(BAR_ODONE, (jt - 1) & 1, abort_flag);
         if (!ok && lane == 0) fail(ERR_WAIT_O_DONE);
         ok = __all_sync(0xffffffffu, ok);
         if (!ok) continue;                                   // reported at the next tile's barrier
         tc_fence_after();
       }
-      if (ln == 0) TRACE(11, j);
+      if (ln == 0) TRACE(11, jt);
       if (__any_sync(0xffffffffu, need)) {
 #pragma unroll
         for (int q = 0; q < 8; ++q) {
@@ -399,19 +481,22 @@ attn_tc2_kernel(const __grid_constant__ Tc2Params p) {
       fence_proxy_async_smem();                   // P is read by the tensor core (async proxy)
       tc_fence_before();
       mbar_arrive(rank == 0 ? BAR_PFULL : BAR_PLOCAL);
-      if (ln == 0) TRACE(12, j);
+      if (ln == 0) TRACE(12, jt);
     }
-    // ---- epilogue
-    if (ok && n_tiles > 0) {
-      ok = mbar_wait(BAR_ODONE, (n_tiles - 1) & 1, abort_flag);
+    if (all_left) break;
+    // ---- epilogue of the item (a warp whose last wait expired still takes the barrier below)
+    if (n_tiles > 0) {
+      if (ok) ok = mbar_wait(BAR_OLAST, n_item & 1, abort_flag);
       ok = __all_sync(0xffffffffu, ok);
       if (!ok && lane == 0) fail(ERR_WAIT_O_DONE);
+      if (!ok) fail_word[2] = 1;
+      // total row sum = sum over both key halves
+      red[2 * 128 + ln] = l_sum;
+      asm volatile("bar.sync 1, 128;" ::: "memory");
+      if (fail_word[2]) { ok = false; break; }                 // uniform over the 128 threads
     }
-    // total row sum = sum over both key halves
-    red[ln] = l_sum;
-    asm volatile("bar.sync 1, 128;" ::: "memory");
-    const float l_tot = l_sum + red[ln ^ 64];
-    if (ok) {
+    const float l_tot = n_tiles > 0 ? l_sum + red[2 * 128 + (ln ^ 64)] : 0.f;
+    {
       tc_fence_after();
       const float inv = (n_tiles > 0 && l_tot > 0.f) ? 1.f / l_tot : 0.f;
       const size_t orow = ((size_t)b * p.q_len + t_row) * p.H + head0 + hl;
@@ -423,6 +508,11 @@ attn_tc2_kernel(const __grid_constant__ Tc2Params p) {
         else {
 #pragma unroll
           for (int i = 0; i < 32; ++i) o[i] = 0;
+        }
+        if (q == 7 && n_tiles > 0) {
+          // every column of O is in registers: the next item may overwrite the accumulator
+          tc_fence_before();
+          mbar_arrive(rank == 0 ? BAR_OFREE : BAR_OLOCAL);
         }
         if (row_valid) {
           // TMEM columns [0,128): output columns 128*half + c ; [128,256): 256 + 128*half + (c-128)
@@ -442,6 +532,8 @@ attn_tc2_kernel(const __grid_constant__ Tc2Params p) {
       if (p.lse && row_valid && half == 0)
         p.lse[orow] = (n_tiles > 0 && l_tot > 0.f) ? (m_ref + log2f(l_tot)) * 0.6931471805599453f : -INFINITY;
     }
+    if (n_tiles > 0) ++n_item;
+    }   // items
     tc_fence_before();
   }
   // ---- teardown
@@ -468,6 +560,32 @@ bool attn_tc2_supported(const AttnProblem& a) {
   return H >= 1 && (128 % H) == 0;      // each CTA of the pair takes whole tokens
 }
 
+// CTA pairs that can be resident at once on the current device (one CTA per SM by shared memory): the size
+// of the persistent grid.  Asked from the occupancy calculator once per device; half the SM count otherwise.
+static int resident_pairs() {
+  static int cached[64];
+  int dev = 0;
+  if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) dev = 0;
+  if (cached[dev] > 0) return cached[dev];
+  int n = 0;
+  cudaLaunchConfig_t cfg;
+  memset(&cfg, 0, sizeof(cfg));
+  cfg.gridDim = dim3(2 * 1024); cfg.blockDim = dim3(pair::THREADS); cfg.dynamicSmemBytes = pair::SMEM_BYTES;
+  cudaLaunchAttribute attr;
+  attr.id = cudaLaunchAttributeClusterDimension;
+  attr.val.clusterDim.x = 2; attr.val.clusterDim.y = 1; attr.val.clusterDim.z = 1;
+  cfg.attrs = &attr; cfg.numAttrs = 1;
+  if (cudaFuncSetAttribute(attn_tc2_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, pair::SMEM_BYTES) != cudaSuccess ||
+      cudaOccupancyMaxActiveClusters(&n, attn_tc2_kernel, &cfg) != cudaSuccess || n <= 0) {
+    cudaGetLastError();
+    int sms = 0;
+    if (cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || sms < 2) sms = 2;
+    n = sms / 2;
+  }
+  cached[dev] = n;
+  return n;
+}
+
 int attn_tc2_launch(const AttnProblem& a) {
   using namespace pair;
   if (!attn_tc2_supported(a)) return LCA_ERR_UNSUPPORTED_SHAPE;
@@ -479,6 +597,8 @@ int attn_tc2_launch(const AttnProblem& a) {
   p.B = a.batch; p.q_len = a.q_len; p.H = H; p.L = a.seq_len; p.g = a.group_size; p.w = a.window;
   p.cap = a.cache_row_capacity; p.n_rep_bias = a.n_rep_bias; p.decode = a.decode;
   p.n_tok_tiles = (a.q_len + p.TB - 1) / p.TB;
+  p.n_head_blocks = H >= 128 ? H / 128 : 1;
+  p.n_items = (long long)p.n_tok_tiles * p.n_head_blocks * a.batch;
   p.scale_log2 = a.softmax_scale * 1.4426950408889634f;
   p.bias_log2 = a.rep_logit_bias * 1.4426950408889634f;
   p.out = (bf16*)a.out; p.lse = a.lse; p.cache_rows = a.cache_rows;
@@ -496,7 +616,9 @@ int attn_tc2_launch(const AttnProblem& a) {
   if (!ok) return LCA_ERR_CUDA;
   if (cudaFuncSetAttribute(attn_tc2_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM_BYTES) != cudaSuccess)
     return LCA_ERR_CUDA;
-  dim3 grid(2 * p.n_tok_tiles, H >= 128 ? H / 128 : 1, a.batch);
+  const long long n_pairs = p.n_items < resident_pairs() ? p.n_items : resident_pairs();
+  if (n_pairs <= 0) return LCA_OK;
+  dim3 grid((unsigned)(2 * n_pairs));
   attn_tc2_kernel<<<grid, THREADS, SMEM_BYTES, a.stream>>>(p);
   note_launch();
   return cudaGetLastError() == cudaSuccess ? LCA_OK : LCA_ERR_CUDA;
