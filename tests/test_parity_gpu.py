@@ -210,6 +210,54 @@ def test_mla_decode_matches_oracle_and_prefill_row(B):
         np.testing.assert_allclose(lse[b].cpu().numpy(), refs[b][1], atol=2e-3, rtol=1e-4)
 
 
+def test_mla_many_query_tiles_per_cta_pair(B):
+    # 128 heads: one token per 128-row tile, so 2000 work items for the ~74 resident CTA pairs of the persistent
+    # kernel -- about 27 items per pair, of 1 to 8 key tiles each: item boundaries, the per-item barriers
+    # wrapping many times, tile counts of both parities.  Sampled rows, every head.
+    cfg = I.scaled(I.CONFIGS["mla_1k"], seq_len=2000, n_q_heads=128, group_size=16, window=300, n_needles=8)
+    inp = I.make_mla_inputs(cfg, "cpu")
+    p, cond, out, lse = run_mla(B, cfg, to_dev(inp), want_scores=False)
+    L = cfg.seq_len
+    rows = np.unique(np.concatenate([np.arange(0, L, 13), np.arange(0, 40), np.arange(L - 160, L)]))
+    ref = Hh.oracle_mla(inp, cfg.group_size, cfg.window, cfg.softmax_scale, rows=rows)
+    Hh.check_condense(one_seq(cond), ref["cond"])
+    Hh.check_outputs(out[0][torch.from_numpy(rows).to(DEV)], ref["out"], "mla many items per pair")
+    np.testing.assert_allclose(lse[0].cpu().numpy()[rows], ref["lse"], atol=2e-3, rtol=1e-4)
+    assert B.lca_last_device_status() == 0
+
+
+def test_mla_decode_more_sequences_than_cta_pairs_with_empty_caches(B):
+    # 100 sequences x 128 heads = 100 work items: some CTA pairs take two.  Row counts span several key-tile
+    # counts; two sequences have an empty cache (no item work: zero output, lse = -inf).
+    H, nb, cap = 128, 100, 700
+    gen = torch.Generator().manual_seed(77)
+    cache_sem = torch.randn((nb, cap, 1, 512), generator=gen).bfloat16()
+    cache_pos = torch.randn((nb, cap, 1, 64), generator=gen).bfloat16()
+    q_sem = torch.randn((nb, H, 512), generator=gen).bfloat16()
+    q_pos = torch.randn((nb, H, 64), generator=gen).bfloat16()
+    rows = torch.randint(1, cap + 1, (nb,), generator=gen, dtype=torch.int32)
+    rows[5] = 0; rows[93] = 0; rows[7] = cap; rows[8] = 128; rows[9] = 129; rows[10] = 1
+    n_rep = 40
+    cfg = I.scaled(I.CONFIGS["mla_decode"], batch=nb, seq_len=4096, n_q_heads=H, group_size=64, window=256)
+    p = B.params_from_config(cfg, batch=nb)
+    out, lse = B.decode_attention(p, q_sem.to(DEV), q_pos.to(DEV), cache_sem.to(DEV), cache_pos.to(DEV),
+                                  rows.to(DEV), n_rep, want_lse=True)
+    torch.cuda.synchronize()
+    assert B.lca_last_device_status() == 0
+    for b in list(range(0, nb, 9)) + [5, 7, 8, 9, 10, 93]:
+        n = int(rows[b])
+        if n == 0:
+            assert torch.count_nonzero(out[b]) == 0
+            assert torch.isinf(lse[b]).all() and (lse[b] < 0).all()
+            continue
+        cs = O.bits_to_f64(Hh.bits(cache_sem[b, :n, 0]))
+        cp = O.bits_to_f64(Hh.bits(cache_pos[b, :n, 0]))
+        ro, rl = O.mla_decode(O.torch_bf16_to_f64(q_sem[b]), O.torch_bf16_to_f64(q_pos[b]), cs, cp,
+                              min(n_rep, n), Hh.f32(cfg.softmax_scale))
+        Hh.check_outputs(out[b], ro, f"decode seq {b} rows {n}")
+        np.testing.assert_allclose(lse[b].cpu().numpy(), rl, atol=2e-3, rtol=1e-4)
+
+
 def test_dense_window_is_plain_causal_attention(B):
     # window >= L: the dense-MLA comparison run through the same entry point (Eq. 5), every row.
     cfg = I.scaled(I.CONFIGS["mla_1k"], seq_len=600, n_q_heads=16, window=600)
