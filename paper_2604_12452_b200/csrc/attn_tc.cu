@@ -62,6 +62,11 @@ struct Plan1 {
   static_assert(2 * BN + NV * 64 <= 512, "TMEM budget");
 };
 
+#ifndef LCA_TC1_POLY_OF_4
+#define LCA_TC1_POLY_OF_4 1
+#endif
+constexpr int POLY_OF_4 = LCA_TC1_POLY_OF_4;   // exponentials out of every four that go to the FMA pipe (interior tiles)
+
 template <int NK_SEM, int NK_POS, int NV, bool V_IN_K, int STAGES>
 __global__ void __launch_bounds__(320, 1)
 attn_tc1_kernel(const __grid_constant__ TcParams p) {
@@ -322,12 +327,26 @@ attn_tc1_kernel(const __grid_constant__ TcParams p) {
       float rs0 = 0.f, rs1 = 0.f;
       uint32_t pk[32];
       const float e_mul = plain ? p.scale_log2 : 1.f;       // sr holds raw products (plain) or scaled logits
+      if (plain) {
+        // Interior tile: every logit is finite.  POLY_OF_4 of every four exponentials are evaluated on the
+        // FMA pipe, the others on the special-function unit, so that the two pipes share the 16384 per tile.
 #pragma unroll
-      for (int i = 0; i < 32; ++i) {
-        const float p0 = exp2f(fmaf(__uint_as_float(sr[i >> 4][(2 * i) & 31]), e_mul, -m_use));
-        const float p1 = exp2f(fmaf(__uint_as_float(sr[i >> 4][(2 * i + 1) & 31]), e_mul, -m_use));
-        rs0 += p0; rs1 += p1;
-        pk[i] = pack_bf16x2(p0, p1);
+        for (int i = 0; i < 32; ++i) {
+          const float a0 = fmaf(__uint_as_float(sr[i >> 4][(2 * i) & 31]), e_mul, -m_use);
+          const float a1 = fmaf(__uint_as_float(sr[i >> 4][(2 * i + 1) & 31]), e_mul, -m_use);
+          const float p0 = ((2 * i) & 3) < POLY_OF_4 ? exp2_fma(a0) : exp2f(a0);
+          const float p1 = ((2 * i + 1) & 3) < POLY_OF_4 ? exp2_fma(a1) : exp2f(a1);
+          rs0 += p0; rs1 += p1;
+          pk[i] = pack_bf16x2(p0, p1);
+        }
+      } else {
+#pragma unroll
+        for (int i = 0; i < 32; ++i) {
+          const float p0 = exp2f(fmaf(__uint_as_float(sr[i >> 4][(2 * i) & 31]), e_mul, -m_use));
+          const float p1 = exp2f(fmaf(__uint_as_float(sr[i >> 4][(2 * i + 1) & 31]), e_mul, -m_use));
+          rs0 += p0; rs1 += p1;
+          pk[i] = pack_bf16x2(p0, p1);
+        }
       }
       l_sum += rs0 + rs1;
       tmem_st32(stm + 32 * half, pk);     // P columns 32*half .. 32*half+31 = keys 64*half .. 64*half+63

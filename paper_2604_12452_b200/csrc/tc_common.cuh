@@ -263,6 +263,21 @@ __device__ __forceinline__ void umma_commit_pair_elected(uint32_t leader, uint32
       ::"r"(bar), "h"(cta_mask), "r"(leader) : "memory");
 }
 
+// 2^t for finite t <= ~100 on the FMA / ALU pipes instead of the special-function unit (which delivers
+// 16 results per clock per SM and is the busiest pipe of a d = 128 attention tile).  t is split into
+// round(t) + f with the 1.5 * 2^23 trick, 2^f on [-0.5, 0.5] is a cubic (relative error 7.5e-5, fifty
+// times below the rounding of a bf16 probability), and round(t) is added to the exponent field.
+// Arguments below -126 are clamped (result ~1e-38 instead of a smaller number or 0).
+__device__ __forceinline__ float exp2_fma(float t) {
+  t = fmaxf(t, -126.f);
+  const float r = t + 12582912.f;                   // low mantissa bits of r = round(t)
+  const float f = t - (r - 12582912.f);
+  float p = fmaf(f, 0.055171601474285126f, 0.2426111102104187f);
+  p = fmaf(f, p, 0.6932610273361206f);
+  p = fmaf(f, p, 0.9999280571937561f);
+  return __int_as_float(__float_as_int(p) + (__float_as_int(r) << 23));
+}
+
 __device__ __forceinline__ uint32_t pack_bf16x2(float lo, float hi) {
   __nv_bfloat162 v = __floats2bfloat162_rn(lo, hi);
   return *reinterpret_cast<uint32_t*>(&v);
