@@ -280,9 +280,10 @@ def run_ours(args, cfg, rank, world, local_rank):
     value = whole_job_value(L * cfg.batch, world, ms_per_step)
 
     # ---- end to end: pinned host buffers; every step copies its inputs host -> device, runs the two
-    # entry points and copies its output device -> host.  Two streams with their own device buffers
-    # take alternate steps, so the upload of one step overlaps the download of the previous one (PCIe
-    # is full duplex); the timed region covers all copies of all steps.
+    # entry points and copies its output device -> host.  Up to three streams with their own device
+    # buffers take the steps in turn, so the upload of one step overlaps the kernels of the previous
+    # one and the download of the one before (PCIe is full duplex); the timed region covers all
+    # copies of all steps.
     e2e = None
     if not args.no_e2e:
         try:
@@ -290,8 +291,11 @@ def run_ours(args, cfg, rank, world, local_rank):
             n_e2e = max(2, args.e2e_steps)
             h2d = sum(v.numel() * v.element_size() for v in host.values())
             d2h = out.numel() * out.element_size()
+            per_set = h2d + d2h + sum(v.numel() * v.element_size() for v in cache.values() if torch.is_tensor(v))
+            free_bytes = torch.cuda.mem_get_info(dev)[0]
+            n_sets = 3 if free_bytes > 2 * per_set + (8 << 30) else 2
             sets = []
-            for i in range(2):
+            for i in range(n_sets):
                 dev_in = inp if i == 0 else {kname: torch.empty_like(v) for kname, v in inp.items()}
                 sets.append(dict(
                     stream=torch.cuda.Stream(), inp=dev_in, out=out if i == 0 else torch.empty_like(out),
@@ -317,7 +321,7 @@ def run_ours(args, cfg, rank, world, local_rank):
             for st in sets:
                 st["stream"].wait_event(e0)
             for i in range(n_e2e):
-                e2e_step(sets[i % 2])
+                e2e_step(sets[i % n_sets])
             for st in sets:
                 torch.cuda.current_stream().wait_stream(st["stream"])
             e1.record()
@@ -325,7 +329,7 @@ def run_ours(args, cfg, rank, world, local_rank):
             t_e2e = max_over_ranks(e0.elapsed_time(e1) / n_e2e, dist, dev)
             e2e = dict(value=whole_job_value(L * cfg.batch, world, t_e2e), unit=UNIT, h2d_bytes_per_step=h2d,
                        d2h_bytes_per_step=d2h, steps=n_e2e, ms_per_step=t_e2e,
-                       note="two streams take alternate steps: uploads overlap the previous step's download")
+                       note=f"{n_sets} streams take the steps in turn: uploads overlap the kernels and the downloads of earlier steps")
             del host, sets
             torch.cuda.empty_cache()
         except RuntimeError as ex:      # e.g. not enough pinnable host memory on this machine
@@ -541,7 +545,7 @@ def main():
                     help="mla_128k is the benchmark; mla_1k / mla_32k run the same step on configs 1 / 2; mla_decode and "
                          "gqa_64k print the side measurements of configs 4 / 5 on their own (used for profiling)")
     ap.add_argument("--attn-impl", type=int, default=0, help="0 auto, 1 scalar kernel, 2 tensor-core kernel")
-    ap.add_argument("--e2e-steps", type=int, default=6)
+    ap.add_argument("--e2e-steps", type=int, default=9)
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-extras", action="store_true", help="skip the decode / GQA / dense-comparison side measurements")
