@@ -35,6 +35,7 @@ struct TcParams {
   bf16* out; float* lse; const int32_t* cache_rows;
   int B, q_len, Hq, Hkv, L, g, w, cap, n_rep_bias, decode;
   int HB, TB, n_tok_tiles, d_out;
+  int out_wide;                   // out is 32-byte aligned: 256-bit stores
   float scale_log2, bias_log2;
 };
 
@@ -378,15 +379,14 @@ attn_tc1_kernel(const __grid_constant__ TcParams p) {
           for (int i = 0; i < 32; ++i) o[i] = 0;
         }
         if (row_valid && hl < p.HB && head0 + hl < p.Hq) {
-          uint4* d4 = reinterpret_cast<uint4*>(dst + q * 32);
+          // 32 bytes per store: every lane writes whole sectors of its own row
 #pragma unroll
-          for (int v = 0; v < 4; ++v) {
-            uint4 w;
-            w.x = pack_bf16x2(__uint_as_float(o[8 * v + 0]) * inv, __uint_as_float(o[8 * v + 1]) * inv);
-            w.y = pack_bf16x2(__uint_as_float(o[8 * v + 2]) * inv, __uint_as_float(o[8 * v + 3]) * inv);
-            w.z = pack_bf16x2(__uint_as_float(o[8 * v + 4]) * inv, __uint_as_float(o[8 * v + 5]) * inv);
-            w.w = pack_bf16x2(__uint_as_float(o[8 * v + 6]) * inv, __uint_as_float(o[8 * v + 7]) * inv);
-            d4[v] = w;
+          for (int v = 0; v < 2; ++v) {
+            uint32_t w[8];
+#pragma unroll
+            for (int e = 0; e < 8; ++e)
+              w[e] = pack_bf16x2(__uint_as_float(o[16 * v + 2 * e]) * inv, __uint_as_float(o[16 * v + 2 * e + 1]) * inv);
+            st_global_32B(dst + q * 32 + 16 * v, w, p.out_wide != 0);
           }
         }
       }
@@ -480,6 +480,7 @@ int attn_tc_launch(const AttnProblem& a) {
   p.scale_log2 = a.softmax_scale * 1.4426950408889634f;
   p.bias_log2 = a.rep_logit_bias * 1.4426950408889634f;
   p.out = (bf16*)a.out; p.lse = a.lse; p.cache_rows = a.cache_rows;
+  p.out_wide = (reinterpret_cast<uintptr_t>(a.out) & 31u) == 0;
   const long long qrows = (long long)a.batch * a.q_len;
   bool ok = make_tensor_map_3d(&p.q_sem, nullptr, 0, 0, 0, 0, 0);
   ok = ok && make_tensor_map_3d(&p.q_pos, a.q_pos, a.d_pos, a.n_q_heads, qrows, p.HB, p.TB);

@@ -74,6 +74,7 @@ struct Tc2Params {
   bf16* out; float* lse; const int32_t* cache_rows;
   int B, q_len, H, L, g, w, cap, n_rep_bias, decode;
   int HB, TB, n_tok_tiles, n_head_blocks;
+  int out_wide;                   // out is 32-byte aligned: 256-bit stores
   long long n_items;              // query tiles x head blocks x batch
   float scale_log2, bias_log2;
 };
@@ -517,15 +518,14 @@ attn_tc2_kernel(const __grid_constant__ Tc2Params p) {
         if (row_valid) {
           // TMEM columns [0,128): output columns 128*half + c ; [128,256): 256 + 128*half + (c-128)
           const int col = (q >> 2) * 256 + 128 * half + (q & 3) * 32;
-          uint4* d4 = reinterpret_cast<uint4*>(dst + col);
+          // 32 bytes per store: every lane writes whole sectors of its own row
 #pragma unroll
-          for (int v = 0; v < 4; ++v) {
-            uint4 w;
-            w.x = pack_bf16x2(__uint_as_float(o[8 * v + 0]) * inv, __uint_as_float(o[8 * v + 1]) * inv);
-            w.y = pack_bf16x2(__uint_as_float(o[8 * v + 2]) * inv, __uint_as_float(o[8 * v + 3]) * inv);
-            w.z = pack_bf16x2(__uint_as_float(o[8 * v + 4]) * inv, __uint_as_float(o[8 * v + 5]) * inv);
-            w.w = pack_bf16x2(__uint_as_float(o[8 * v + 6]) * inv, __uint_as_float(o[8 * v + 7]) * inv);
-            d4[v] = w;
+          for (int v = 0; v < 2; ++v) {
+            uint32_t w[8];
+#pragma unroll
+            for (int e = 0; e < 8; ++e)
+              w[e] = pack_bf16x2(__uint_as_float(o[16 * v + 2 * e]) * inv, __uint_as_float(o[16 * v + 2 * e + 1]) * inv);
+            st_global_32B(dst + col + 16 * v, w, p.out_wide != 0);
           }
         }
       }
@@ -602,6 +602,7 @@ int attn_tc2_launch(const AttnProblem& a) {
   p.scale_log2 = a.softmax_scale * 1.4426950408889634f;
   p.bias_log2 = a.rep_logit_bias * 1.4426950408889634f;
   p.out = (bf16*)a.out; p.lse = a.lse; p.cache_rows = a.cache_rows;
+  p.out_wide = (reinterpret_cast<uintptr_t>(a.out) & 31u) == 0;
   const int hbc = p.HB >= 64 ? 64 : p.HB, tbc = 64 / hbc;
   const long long qrows = (long long)a.batch * a.q_len, krows = (long long)a.batch * a.seq_len,
                   crows = (long long)a.batch * a.cache_row_capacity;

@@ -278,6 +278,19 @@ __device__ __forceinline__ float exp2_fma(float t) {
   return __int_as_float(__float_as_int(p) + (__float_as_int(r) << 23));
 }
 
+// 32 bytes to global memory: one 256-bit store (sm_100; a whole sector per lane) where the address is
+// 32-byte aligned (`wide`, decided once per launch from the base pointer), else two 128-bit stores.
+__device__ __forceinline__ void st_global_32B(void* p, const uint32_t (&v)[8], bool wide) {
+  if (wide) {
+    asm volatile("st.global.v8.b32 [%0], {%1, %2, %3, %4, %5, %6, %7, %8};"
+                 ::"l"(p), "r"(v[0]), "r"(v[1]), "r"(v[2]), "r"(v[3]), "r"(v[4]), "r"(v[5]), "r"(v[6]), "r"(v[7]) : "memory");
+  } else {
+    uint4* q = reinterpret_cast<uint4*>(p);
+    q[0] = make_uint4(v[0], v[1], v[2], v[3]);
+    q[1] = make_uint4(v[4], v[5], v[6], v[7]);
+  }
+}
+
 __device__ __forceinline__ uint32_t pack_bf16x2(float lo, float hi) {
   __nv_bfloat162 v = __floats2bfloat162_rn(lo, hi);
   return *reinterpret_cast<uint32_t*>(&v);

@@ -93,6 +93,11 @@ def bf16_ulp_distance(a_bits: np.ndarray, b_bits: np.ndarray) -> np.ndarray:
     return np.abs(key(a_bits) - key(b_bits))
 
 
+def bits_t(t: torch.Tensor) -> torch.Tensor:
+    """bf16 tensor -> its bit patterns as int16 (for exact comparisons on the device)."""
+    return t.contiguous().view(torch.int16)
+
+
 def check_outputs(got: torch.Tensor, ref: np.ndarray, what: str = ""):
     """max-abs <= ATOL + RTOL*|ref| element-wise and mean-abs <= MEAN_ATOL + MEAN_RTOL*mean|ref|;
     returns the stats.  The relative terms only matter where outputs exceed unit scale (rows that

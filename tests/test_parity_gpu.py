@@ -172,6 +172,36 @@ def test_gqa_small_cases_match_oracle_on_every_row(B, L, Hq, Hkv, g, w):
     np.testing.assert_allclose(lse[0].cpu().numpy(), ref["lse"], atol=2e-3, rtol=1e-4)
 
 
+def test_output_pointer_aligned_to_16_bytes_only(B):
+    # The ABI promises 16-byte alignment, the tensor-core kernels store 32 bytes at a time where they can:
+    # an output buffer that starts 16 bytes into an allocation must give the same bits as an aligned one.
+    def shifted(shape):
+        n = int(np.prod(shape))
+        raw = torch.zeros(n + 8, dtype=torch.bfloat16, device=DEV)
+        view = raw[8:].view(shape)
+        assert view.data_ptr() % 32 == 16
+        return view
+
+    cfg = I.scaled(I.CONFIGS["mla_1k"], seq_len=300, n_q_heads=16, group_size=16, window=64)
+    d = to_dev(I.make_mla_inputs(cfg, "cpu"))
+    p = B.params_from_config(cfg, batch=1)
+    cond = B.condense(p, d["q_sem"][300 - 16:], d["q_pos"][300 - 16:], d["ckv"], d["kr"])
+    args = (p, d["q_sem"], d["q_pos"], d["ckv"], d["kr"], cond["cache_sem"], cond["cache_pos"])
+    ref, _ = B.prefill_attention(*args)
+    out, _ = B.prefill_attention(*args, out=shifted((1, 300, 16, 512)))
+    assert torch.equal(Hh.bits_t(out), Hh.bits_t(ref))
+
+    cfg = I.scaled(I.CONFIGS["gqa_64k"], seq_len=260, n_q_heads=8, n_kv_heads=2, group_size=16, window=40)
+    d = to_dev(I.make_gqa_inputs(cfg, "cpu"))
+    p = B.params_from_config(cfg, batch=1)
+    cond = B.condense(p, None, d["q"][260 - 16:], d["v"], d["k"])
+    args = (p, None, d["q"], d["v"], d["k"], cond["cache_sem"], cond["cache_pos"])
+    ref, _ = B.prefill_attention(*args)
+    out, _ = B.prefill_attention(*args, out=shifted((1, 260, 8, 128)))
+    assert torch.equal(Hh.bits_t(out), Hh.bits_t(ref))
+    assert B.lca_last_device_status() == 0
+
+
 def test_mla_decode_matches_oracle_and_prefill_row(B):
     # contexts of different lengths share one cache buffer (capacity = longest + 1 appended row)
     cfg = I.scaled(I.CONFIGS["mla_decode"], batch=3, seq_len=1500, n_q_heads=128, group_size=64, window=256)
