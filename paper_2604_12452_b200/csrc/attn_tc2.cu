@@ -408,18 +408,23 @@ attn_tc2_kernel(const __grid_constant__ Tc2Params p) {
           }
           tmax = fmaxf(fmaxf(t0m, t1m), fmaxf(t2m, t3m)) * p.scale_log2;
         } else {
+          // boundary tile: scale, bias and mask with selects only (per-element branches cost ~25 cycles
+          // each here), four short maximum chains
+          const float bias = (isA && p.bias_log2 != 0.f) ? p.bias_log2 : 0.f;
+          const int lo_m = need_mask ? lo : -(1 << 30), hi_m = need_mask ? hi : (1 << 30);
+          float tm[4] = {-INFINITY, -INFINITY, -INFINITY, -INFINITY};
 #pragma unroll
           for (int q = 0; q < 2; ++q) {
 #pragma unroll
             for (int i = 0; i < 32; ++i) {
               const int c = q * 32 + i;
-              float s = __uint_as_float(sr[q][i]) * p.scale_log2;
-              if (isA && p.bias_log2 != 0.f && c < blim) s += p.bias_log2;
-              if (need_mask && (c < lo || c > hi)) s = -INFINITY;
+              float s = fmaf(__uint_as_float(sr[q][i]), p.scale_log2, c < blim ? bias : 0.f);
+              s = ((c >= lo_m) & (c <= hi_m)) ? s : -INFINITY;
               sr[q][i] = __float_as_uint(s);
-              tmax = fmaxf(tmax, s);
+              tm[i & 3] = fmaxf(tm[i & 3], s);
             }
           }
+          tmax = fmaxf(fmaxf(tm[0], tm[1]), fmaxf(tm[2], tm[3]));
         }
       } else {
         fail_word[jt & 1] = 1;
