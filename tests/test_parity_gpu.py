@@ -151,6 +151,21 @@ def test_mla_batched_sequences_are_independent(B):
         Hh.check_outputs(out[b], ref["out"], f"batch {b}")
 
 
+@pytest.mark.parametrize("H", [1, 2, 8, 32, 64, 256])
+def test_mla_head_counts_of_the_pair_kernel(B, H):
+    # Every way a 128-row tile of the CTA-pair kernel splits into tokens x heads: H < 128 puts 128 / H tokens in
+    # a tile (H = 1: 64 tokens per CTA), H = 256 two head blocks per token.  Every row, tensor-core path forced.
+    L, g, w = 333, 16, 50
+    cfg = I.scaled(I.CONFIGS["mla_1k"], seq_len=L, n_q_heads=H, group_size=g, window=w, n_needles=4)
+    inp = I.make_mla_inputs(cfg, "cpu")
+    p, cond, out, lse = run_mla(B, cfg, to_dev(inp), impl=2, want_scores=False)
+    ref = Hh.oracle_mla(inp, g, w, cfg.softmax_scale, rows=np.arange(L))
+    Hh.check_condense(one_seq(cond), ref["cond"])
+    Hh.check_outputs(out[0], ref["out"], f"mla H={H}")
+    np.testing.assert_allclose(lse[0].cpu().numpy(), ref["lse"], atol=2e-3, rtol=1e-4)
+    assert B.lca_last_device_status() == 0
+
+
 GQA_SMALL = [(1024, 32, 8, 64, 128), (515, 8, 2, 16, 40), (96, 4, 4, 64, 64), (260, 32, 8, 64, 0)]
 
 
