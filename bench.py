@@ -293,7 +293,8 @@ def run_ours(args, cfg, rank, world, local_rank):
             d2h = out.numel() * out.element_size()
             per_set = h2d + d2h + sum(v.numel() * v.element_size() for v in cache.values() if torch.is_tensor(v))
             free_bytes = torch.cuda.mem_get_info(dev)[0]
-            n_sets = 3 if free_bytes > 2 * per_set + (8 << 30) else 2
+            # a third set costs another pinned output buffer per rank: only where few ranks share the host
+            n_sets = 3 if (free_bytes > 2 * per_set + (8 << 30) and world <= 2) else 2
             sets = []
             for i in range(n_sets):
                 dev_in = inp if i == 0 else {kname: torch.empty_like(v) for kname, v in inp.items()}
