@@ -63,6 +63,8 @@ constexpr int SMEM_BYTES = OFF_BAR + 512 + 3 * 128 * 4;     // 231424
 constexpr int TM_S0 = 0, TM_S1 = 64, TM_O = 128, TM_COLS = 512;
 constexpr int THREADS = 224;            // warps: 0 K/Q loads, 1 MMA + TMEM, 2-5 softmax, 6 V loads
 constexpr float RESCALE_THRESHOLD = 8.0f;
+constexpr int L2_AHEAD = 0;              // decode: the key tile is requested into L2 this many tiles ahead of its load
+                                        // (0 = the tile about to be loaded, before the wait for the buffer: measured best)
 static_assert(SMEM_BYTES <= 232448, "shared memory budget of one SM");
 }  // namespace pair
 
@@ -193,6 +195,13 @@ attn_tc2_kernel(const __grid_constant__ Tc2Params p) {
           const int row = (isA ? it.b * p.cap + j * BN : it.b * p.L + it.first_lo + (j - it.nA) * BN) + 64 * (int)rank;
           const CUtensorMap* ms = isA ? &p.c_sem : &p.k_sem;
           const CUtensorMap* mp = isA ? &p.c_pos : &p.k_pos;
+          if (p.decode && j + L2_AHEAD < it.n_tiles) {
+            // Decode: every sequence streams its own cache from HBM (in prefill the pairs share the stream through
+            // L2).  Ask for the key rows into L2 before waiting for the buffer, so that the load below finds them there.
+            const int rowa = row + L2_AHEAD * BN;
+            for (int c = 0; c < 8; c += KBOX) tma_prefetch_l2_3d(&p.c_sem, 0, rowa, c);
+            tma_prefetch_l2_3d(&p.c_pos, 0, 0, rowa);
+          }
           for (int gk = 0; gk < NKG; ++gk) {
             if (!mbar_wait(BAR_KEMPTY(gk), (jt & 1) ^ 1, abort_flag)) { fail(ERR_WAIT_KV_EMPTY); good = false; break; }
             const int pos0 = piece_begin(gk), pos1 = piece_begin(gk + 1);
