@@ -475,12 +475,13 @@ int condense_take_status() {
 
 // ------------------------------------------------------------------------------ local window
 // Copies, for every sequence, one contiguous block of `bytes16` 16-byte words.
-__global__ void copy_blocks_kernel(const uint4* __restrict__ src, uint4* __restrict__ dst,
-                                   size_t src_batch_stride16, size_t dst_batch_stride16,
-                                   size_t src_off16, size_t dst_off16, size_t n16) {
-  const uint4* s = src + (size_t)blockIdx.y * src_batch_stride16 + src_off16;
-  uint4* d = dst + (size_t)blockIdx.y * dst_batch_stride16 + dst_off16;
-  for (size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x; i < n16;
+// Two block copies per sequence in one launch (blockIdx.z: the semantic and the positional part).
+struct CopySeg { const uint4* src; uint4* dst; size_t src_batch_stride16, dst_batch_stride16, src_off16, dst_off16, n16; };
+__global__ void copy_blocks_kernel(const CopySeg a, const CopySeg b) {
+  const CopySeg& c = blockIdx.z == 0 ? a : b;
+  const uint4* s = c.src + (size_t)blockIdx.y * c.src_batch_stride16 + c.src_off16;
+  uint4* d = c.dst + (size_t)blockIdx.y * c.dst_batch_stride16 + c.dst_off16;
+  for (size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x; i < c.n16;
        i += (size_t)gridDim.x * blockDim.x)
     d[i] = s[i];
 }
@@ -576,14 +577,13 @@ int condense_launch(const CondenseLaunch& c) {
     // rows L-k..L-1 of each sequence -> cache rows m..m+k-1 (one contiguous block per sequence)
     const size_t row_sem = (size_t)Hkv * p->d_sem * sizeof(bf16) / 16;
     const size_t row_pos = (size_t)Hkv * p->d_pos * sizeof(bf16) / 16;
-    const unsigned blocks = 148 * 4;
-    copy_blocks_kernel<<<dim3(blocks, B), 256, 0, c.stream>>>(
-        (const uint4*)c.kv_sem, (uint4*)c.cache_sem, (size_t)p->seq_len * row_sem, (size_t)(m + k) * row_sem,
-        (size_t)(p->seq_len - k) * row_sem, (size_t)m * row_sem, (size_t)k * row_sem);
-    copy_blocks_kernel<<<dim3(blocks, B), 256, 0, c.stream>>>(
-        (const uint4*)c.kv_pos, (uint4*)c.cache_pos, (size_t)p->seq_len * row_pos, (size_t)(m + k) * row_pos,
-        (size_t)(p->seq_len - k) * row_pos, (size_t)m * row_pos, (size_t)k * row_pos);
-    note_launch(2);
+    const unsigned blocks = 148 * 2;
+    const CopySeg sem = {(const uint4*)c.kv_sem, (uint4*)c.cache_sem, (size_t)p->seq_len * row_sem, (size_t)(m + k) * row_sem,
+                         (size_t)(p->seq_len - k) * row_sem, (size_t)m * row_sem, (size_t)k * row_sem};
+    const CopySeg pos = {(const uint4*)c.kv_pos, (uint4*)c.cache_pos, (size_t)p->seq_len * row_pos, (size_t)(m + k) * row_pos,
+                         (size_t)(p->seq_len - k) * row_pos, (size_t)m * row_pos, (size_t)k * row_pos};
+    copy_blocks_kernel<<<dim3(blocks, B, 2), 256, 0, c.stream>>>(sem, pos);
+    note_launch();
   }
   return cudaGetLastError() == cudaSuccess ? LCA_OK : LCA_ERR_CUDA;
 }
