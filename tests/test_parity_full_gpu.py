@@ -118,3 +118,23 @@ def test_config4_batched_condense_and_decode_full_size(B):
                               O.bits_to_f64(Hh.bits(dpos[b, :, 0])), m, Hh.f32(cfg.softmax_scale))
         Hh.check_outputs(out[b], ro, f"decode seq {b}")
         np.testing.assert_allclose(lse[b].cpu().numpy(), rl, atol=2e-3, rtol=1e-4)
+
+
+def test_attention_is_bit_reproducible_at_full_size(B):
+    # The kernels are deterministic (fixed tile order, no atomics in the data path), so two launches on the same
+    # inputs must agree in every bit of the 16.8 M x 512 outputs of config 3: a missed ordering between the
+    # softmax threads, the relay signal and the tensor core would show up here as a difference.
+    cfg = I.CONFIGS["mla_128k"]
+    L, g = cfg.seq_len, cfg.group_size
+    inp = I.make_mla_inputs(cfg, DEV)
+    p = B.params_from_config(cfg, batch=1)
+    cond = B.condense(p, inp["q_sem"][L - g:], inp["q_pos"][L - g:], inp["ckv"], inp["kr"])
+    args = (p, inp["q_sem"], inp["q_pos"], inp["ckv"], inp["kr"], cond["cache_sem"], cond["cache_pos"])
+    out1, lse1 = B.prefill_attention(*args, want_lse=True)
+    out2, lse2 = B.prefill_attention(*args, want_lse=True)
+    torch.cuda.synchronize()
+    assert B.lca_last_device_status() == 0
+    step = 8192                                     # compare in slices: no second full-size temporary
+    for t in range(0, L, step):
+        assert torch.equal(Hh.bits_t(out1[0, t:t + step]), Hh.bits_t(out2[0, t:t + step])), f"tokens {t}..{t + step}"
+    assert torch.equal(lse1, lse2)
