@@ -97,13 +97,13 @@ __device__ inline void cp_async16(void* smem_dst, const void* gmem_src) {
   asm volatile("cp.async.cg.shared.global [%0], [%1], 16;\n" ::"r"(s), "l"(gmem_src) : "memory");
 }
 
-// Persistent CTAs, one per SM; group index = (b * Hkv + hk) * m + j.  Two shared-memory stages:
+// Persistent CTAs (as many per SM as shared memory allows, at most two by registers); group index = (b * Hkv + hk) * m + j.  Two shared-memory stages:
 // while a group is scored and pooled, the next one streams in with 16-byte cp.async copies, so
 // every history byte is read from HBM once and the loads never wait for the arithmetic.
 // A stage holds the g tokens [g][d_sem] and [g][d_pos] in bf16 and the summary query in fp64.
 // Scores stay in fp64 (the arg-max must follow the exact scores); the group softmax and the
 // pooling run in fp32, c_rep is rounded once to bf16.
-__global__ void __launch_bounds__(CONDENSE_THREADS, 1)
+__global__ void __launch_bounds__(CONDENSE_THREADS, 2)
 condense_kernel(CondenseArgs a) {
   extern __shared__ __align__(16) unsigned char smem_raw[];
   const int g = a.g, d_sem = a.d_sem, d_pos = a.d_pos;
@@ -569,7 +569,15 @@ int condense_launch(const CondenseLaunch& c) {
       size_t smem = condense_smem_bytes(p);
       if (cudaFuncSetAttribute(condense_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) != cudaSuccess)
         return LCA_ERR_CUDA;
-      condense_kernel<<<dim3((unsigned)ctas), CONDENSE_THREADS, smem, c.stream>>>(a);
+      // as many resident CTAs per SM as shared memory and registers allow: a group is little work between
+      // block-wide barriers, so several CTAs per SM overlap each other's phases
+      int per_sm = 1;
+      if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, condense_kernel, CONDENSE_THREADS, smem) != cudaSuccess || per_sm < 1) {
+        cudaGetLastError();
+        per_sm = 1;
+      }
+      const long long resident = (long long)sms * per_sm;
+      condense_kernel<<<dim3((unsigned)(a.n_groups < resident ? a.n_groups : resident)), CONDENSE_THREADS, smem, c.stream>>>(a);
     }
     note_launch();
   }
