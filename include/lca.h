@@ -152,7 +152,8 @@ int lca_condense_static_scratch(const lca_params* p, const void* q_tail_sem, con
  *   kv_sem, kv_pos, cache_sem, cache_pos: as for lca_condense (the cache may be NULL when m = 0)
  *   out [B, L, H, d_sem] bf16: softmax-weighted sum of the sem vectors (latent space for MLA)
  *   lse_opt [B, L, H] fp32 or NULL: natural-log sum-exp of the logits of each row
- * fp32 softmax and accumulation, bf16 tensor-core products. */
+ * fp32 softmax and accumulation, bf16 tensor-core products.  `out` may be aligned to 16 bytes only;
+ * where it is aligned to 32 bytes the tensor-core kernels store 32 bytes per instruction. */
 int lca_prefill_attention(const lca_params* p, const void* q_sem, const void* q_pos,
                           const void* kv_sem, const void* kv_pos, const void* cache_sem,
                           const void* cache_pos, void* out, float* lse_opt, void* ws,
