@@ -473,7 +473,7 @@ attn_tc2_kernel(const __grid_constant__ Tc2Params p) {
       }
       if (ln == 0) TRACE(11, jt);
       if (__any_sync(0xffffffffu, need)) {
-#pragma unroll
+#pragma unroll 1                                   // rare path: kept small (the kernel is sensitive to its code size)
         for (int q = 0; q < 8; ++q) {
           uint32_t o[32];
           tmem_ld32(tmem + lane_base + TM_O + q * 32, o);
@@ -516,7 +516,7 @@ attn_tc2_kernel(const __grid_constant__ Tc2Params p) {
       const float inv = (n_tiles > 0 && l_tot > 0.f) ? 1.f / l_tot : 0.f;
       const size_t orow = ((size_t)b * p.q_len + t_row) * p.H + head0 + hl;
       bf16* dst = p.out + orow * 512;
-#pragma unroll
+#pragma unroll 1                                   // once per item: kept small
       for (int q = 0; q < 8; ++q) {
         uint32_t o[32];
         if (n_tiles > 0) { tmem_ld32(tmem + lane_base + TM_O + q * 32, o); tmem_wait_ld(); }
