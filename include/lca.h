@@ -107,8 +107,9 @@ size_t lca_workspace_bytes(const lca_params* p, int32_t which);
  *   anchor_idx [B, m, n_kv_heads] int32 out: absolute token index of I_j (lowest index on ties).
  *   scores_opt [B, n_kv_heads, m*g] fp64 out or NULL: the importance scores s_i the kernel used.
  *   ws / ws_bytes: >= lca_workspace_bytes(p, LCA_WS_CONDENSE).
- * Scores, the group softmax and the pooling are evaluated in fp64 (the kernel is HBM-bound),
- * so anchors follow the fp64 scores and c_rep is rounded once, to bf16. */
+ * The summary query and the importance scores are evaluated in fp64, so the arg-max anchors
+ * follow the exact scores (lowest index on exact ties); the group softmax (Eq. 6) and the
+ * pooling (Eq. 7) are fp32, and c_rep is rounded once, to bf16 (nearest even). */
 int lca_condense(const lca_params* p, const void* q_tail_sem, const void* q_tail_pos,
                  int64_t q_tail_batch_stride, const float* qbar_opt, const void* kv_sem,
                  const void* kv_pos, void* cache_sem, void* cache_pos, int32_t* anchor_idx,
@@ -209,6 +210,15 @@ int64_t lca_launch_count(void);
  * current device: 0 = none expired.  Synchronises `stream`.  Returns LCA_OK or
  * LCA_ERR_DEVICE_TIMEOUT / LCA_ERR_CUDA. */
 int lca_last_device_status(void* stream);
+
+/* Self-test of the time-out mechanism (the paper has no counterpart).  Every device-side wait of
+ * the tensor-core kernels gives up after a fixed number of SM cycles, records a code in the status
+ * word that lca_last_device_status reads, and the kernel returns in an orderly way.  This call
+ * launches a one-thread kernel that waits, with the same routine and a limit of `limit_cycles`
+ * (1 .. 1e8), on a barrier nobody ever arrives on: afterwards lca_last_device_status returns
+ * LCA_ERR_DEVICE_TIMEOUT once, and the next ordinary call works as usual.  Nothing faults, traps or
+ * waits longer than the limit. */
+int lca_selftest_bounded_wait(int64_t limit_cycles, void* stream);
 
 const char* lca_status_string(int status);
 int lca_version(void);

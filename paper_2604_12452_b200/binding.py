@@ -23,6 +23,7 @@ LCA_VARIANT_MLA, LCA_VARIANT_GQA = 0, 1
 LCA_WS_CONDENSE, LCA_WS_PREFILL, LCA_WS_DECODE, LCA_WS_UPDATE = 0, 1, 2, 3
 LCA_STATIC_SCRATCH_BYTES = 1 << 20
 LCA_ERR_STATIC_SCRATCH_EXCEEDED = -7
+LCA_ERR_DEVICE_TIMEOUT = -6
 ATTN_AUTO, ATTN_SCALAR, ATTN_TENSOR = 0, 1, 2
 REDUCE_DEFAULT, REDUCE_MAXPOOL, REDUCE_MEANPOOL, REDUCE_WEIGHTED, REDUCE_MAXSEL = 0, 1, 2, 3, 4
 
@@ -70,6 +71,8 @@ def _load() -> C.CDLL:
     lib.lca_decode_attention.argtypes = [P, vp, vp, vp, vp, vp, i32, i32, vp, vp, vp, sz, vp]
     lib.lca_decode_update.restype = C.c_int
     lib.lca_decode_update.argtypes = [P, vp, vp, i64, vp, vp, vp, i32, vp, vp, vp, vp, sz, vp]
+    lib.lca_selftest_bounded_wait.restype = C.c_int
+    lib.lca_selftest_bounded_wait.argtypes = [i64, vp]
     lib.lca_last_device_status.restype = C.c_int
     lib.lca_last_device_status.argtypes = [vp]
     return lib
@@ -171,6 +174,10 @@ def lca_decode_update(params, q_tail_sem, q_tail_pos, q_tail_batch_stride, qbar_
     return int(_lib.lca_decode_update(C.byref(params), _ptr(q_tail_sem), _ptr(q_tail_pos), int(q_tail_batch_stride),
                                       _ptr(qbar_opt), _ptr(cache_sem), _ptr(cache_pos), int(cache_row_capacity),
                                       _ptr(n_rep), _ptr(cache_rows), _ptr(anchor_out), _ptr(ws), wsb, _stream(stream)))
+
+
+def lca_selftest_bounded_wait(limit_cycles: int, stream=None) -> int:
+    return int(_lib.lca_selftest_bounded_wait(int(limit_cycles), _stream(stream)))
 
 
 def lca_last_device_status(stream=None) -> int:

@@ -29,27 +29,15 @@ using namespace tc;
 
 static __device__ int g_tc2_status = 0;
 
-#ifdef LCA_TC2_TRACE
-// Debug build only: per-phase clock64 stamps of one CTA pair (block 0), read back by a test script.
-static __device__ long long g_trace[8192];
-#define TRACE(slot, j) do { if (blockIdx.x < 2 && blockIdx.y == 0 && blockIdx.z == 0 && (j) < 60) g_trace[(int)rank * 4096 + (j) * 16 + (slot)] = clock64(); } while (0)
-#else
-#define TRACE(slot, j) do { } while (0)
-#endif
-
 namespace pair {
 constexpr int BN = 128;                 // keys per tile (64 per CTA for S)
 constexpr int NKC = 9;                  // 64-column key chunks: 8 latent + 1 rope
 // The key part of a tile is one buffer, filled and released in NKG pieces, so that the refill of a piece
 // starts while S = Q K^T still reads the others.  S takes the chunks in the order rope, latent 0..7; piece p
 // covers positions [piece_begin(p), piece_begin(p + 1)) of that order.
-#ifndef LCA_TC2_NKG
-#define LCA_TC2_NKG 2
-#endif
-constexpr int NKG = LCA_TC2_NKG;
-static_assert(NKG >= 1 && NKG <= 3, "pieces of the key buffer");
-__host__ __device__ constexpr int piece_begin(int p) { return NKG == 1 ? 9 * p : NKG == 2 ? (p == 0 ? 0 : p == 1 ? 5 : 9) : 3 * p; }
-constexpr int KBOX = NKG == 1 ? 8 : NKG == 2 ? 4 : 1;   // latent column chunks brought by one TMA request of the key part
+constexpr int NKG = 2;                  // two pieces: rope chunk + latent chunks 0-3, latent chunks 4-7
+__host__ __device__ constexpr int piece_begin(int p) { return p == 0 ? 0 : p == 1 ? 5 : 9; }
+constexpr int KBOX = 4;                 // latent column chunks brought by one TMA request of the key part
 constexpr int VBOX = 2;                 // column chunks brought by one request of the value part
 constexpr int QCH = 64 * 128;           // bytes of one query chunk  (64 rows)
 constexpr int KCH = 64 * 128;           // bytes of one key chunk    (64 keys)
@@ -63,8 +51,6 @@ constexpr int SMEM_BYTES = OFF_BAR + 512 + 3 * 128 * 4;     // 231424
 constexpr int TM_S0 = 0, TM_S1 = 64, TM_O = 128, TM_COLS = 512;
 constexpr int THREADS = 224;            // warps: 0 K/Q loads, 1 MMA + TMEM, 2-5 softmax, 6 V loads
 constexpr float RESCALE_THRESHOLD = 8.0f;
-constexpr int L2_AHEAD = 0;              // decode: the key tile is requested into L2 this many tiles ahead of its load
-                                        // (0 = the tile about to be loaded, before the wait for the buffer: measured best)
 static_assert(SMEM_BYTES <= 232448, "shared memory budget of one SM");
 }  // namespace pair
 
@@ -111,6 +97,11 @@ __device__ __forceinline__ Item make_item(const Tc2Params& p, long long idx) {
   return it;
 }
 
+// Decode only: tile j of the item contains cache rows at or behind the sequence's valid row count.
+__device__ __forceinline__ bool ragged_decode_tile(const Tc2Params& p, const Item& it, int j) {
+  return p.decode && (j + 1) * pair::BN > it.n_a_hi;
+}
+
 __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(pair::THREADS, 1)
 attn_tc2_kernel(const __grid_constant__ Tc2Params p) {
   using namespace pair;
@@ -129,6 +120,7 @@ attn_tc2_kernel(const __grid_constant__ Tc2Params p) {
   auto BAR_KEMPTY = [&](int c) { return bars + 40 + 72 + 8 * c; };      // NKG (room for 9)
   auto BAR_VFULL = [&](int h) { return bars + 40 + 144 + 8 * h; };      // 2
   auto BAR_VEMPTY = [&](int h) { return bars + 40 + 160 + 8 * h; };     // 2
+  auto BAR_VLOC = [&](int h) { return bars + 40 + 16 + 8 * h; };        // 2: odd CTA, value part of a ragged decode tile
   const uint32_t BAR_PLOCAL = bars + 224;        // odd CTA: its 128 softmax threads -> its relay thread
   const uint32_t BAR_QFREE = bars + 216;         // last S of an item done: the query tile may be replaced
   const uint32_t BAR_OLAST = bars + 232;         // last P V of an item done: O is complete
@@ -147,7 +139,7 @@ attn_tc2_kernel(const __grid_constant__ Tc2Params p) {
   if (threadIdx.x == 0) {
     mbar_init(BAR_Q, 1);
     for (int c = 0; c < NKG; ++c) { mbar_init(BAR_KFULL(c), 1); mbar_init(BAR_KEMPTY(c), 1); }
-    for (int h = 0; h < 2; ++h) { mbar_init(BAR_VFULL(h), 1); mbar_init(BAR_VEMPTY(h), 1); }
+    for (int h = 0; h < 2; ++h) { mbar_init(BAR_VFULL(h), 1); mbar_init(BAR_VEMPTY(h), 1); mbar_init(BAR_VLOC(h), 1); }
     mbar_init(BAR_SFULL0, 1); mbar_init(BAR_SFULL1, 1);
     mbar_init(BAR_PFULL, 129); mbar_init(BAR_ODONE, 1);     // 128 threads of the even CTA + the odd CTA's relay
     mbar_init(BAR_PLOCAL, 128);
@@ -195,12 +187,11 @@ attn_tc2_kernel(const __grid_constant__ Tc2Params p) {
           const int row = (isA ? it.b * p.cap + j * BN : it.b * p.L + it.first_lo + (j - it.nA) * BN) + 64 * (int)rank;
           const CUtensorMap* ms = isA ? &p.c_sem : &p.k_sem;
           const CUtensorMap* mp = isA ? &p.c_pos : &p.k_pos;
-          if (p.decode && j + L2_AHEAD < it.n_tiles) {
+          if (p.decode) {
             // Decode: every sequence streams its own cache from HBM (in prefill the pairs share the stream through
             // L2).  Ask for the key rows into L2 before waiting for the buffer, so that the load below finds them there.
-            const int rowa = row + L2_AHEAD * BN;
-            for (int c = 0; c < 8; c += KBOX) tma_prefetch_l2_3d(&p.c_sem, 0, rowa, c);
-            tma_prefetch_l2_3d(&p.c_pos, 0, 0, rowa);
+            for (int c = 0; c < 8; c += KBOX) tma_prefetch_l2_3d(&p.c_sem, 0, row, c);
+            tma_prefetch_l2_3d(&p.c_pos, 0, 0, row);
           }
           for (int gk = 0; gk < NKG; ++gk) {
             if (!mbar_wait(BAR_KEMPTY(gk), (jt & 1) ^ 1, abort_flag)) { fail(ERR_WAIT_KV_EMPTY); good = false; break; }
@@ -224,10 +215,21 @@ attn_tc2_kernel(const __grid_constant__ Tc2Params p) {
           const bool isA = j < it.nA;
           const int row = isA ? it.b * p.cap + j * BN : it.b * p.L + it.first_lo + (j - it.nA) * BN;
           const CUtensorMap* mv = isA ? &p.c_val : &p.k_val;
+          // Decode, last tile of a sequence whose valid rows end inside it: the rows behind them may hold anything
+          // (0 x NaN would reach O), so the softmax threads of each CTA zero them in their own value buffers before
+          // they release P.  They must see the data land first: the odd CTA's copies then complete on a barrier of
+          // its own, and the even CTA's barrier expects the even CTA's bytes only.
+          const bool ragged = ragged_decode_tile(p, it, j);
           for (int kh = 0; kh < 2; ++kh) {            // keys [64*kh, 64*kh+64) of the tile
             if (!mbar_wait(BAR_VEMPTY(kh), (jt & 1) ^ 1, abort_flag)) { fail(ERR_WAIT_KV_EMPTY); good = false; break; }
-            if (rank == 0) mbar_expect_tx(BAR_VFULL(kh), 2 * 4 * VCH);
-            const uint32_t v_bar = mapa_u32(BAR_VFULL(kh), 0);
+            uint32_t v_bar;
+            if (ragged && rank == 1) {
+              mbar_expect_tx(BAR_VLOC(kh), 4 * VCH);
+              v_bar = BAR_VLOC(kh);
+            } else {
+              if (rank == 0) mbar_expect_tx(BAR_VFULL(kh), (ragged ? 1 : 2) * 4 * VCH);
+              v_bar = mapa_u32(BAR_VFULL(kh), 0);
+            }
             // output columns of this CTA: [128*rank, +128) of the first 256, then of the second 256
             for (int i = 0; i < 4; i += VBOX) {
               const int chunk = (i >> 1) * 4 + 2 * (int)rank + (i & 1);
@@ -257,13 +259,11 @@ attn_tc2_kernel(const __grid_constant__ Tc2Params p) {
       auto issue_pending_pv = [&]() -> bool {
         const uint32_t t = pend_t;
         pending = false;
-        TRACE(3, t);
         if (pend_first && pend_item > 0) {
           // O of the previous item has been read out by the epilogue threads of both CTAs
           if (!mbar_wait(BAR_OFREE, (pend_item - 1) & 1, abort_flag)) { if (leader) fail(ERR_WAIT_O_DONE); return false; }
         }
         if (!mbar_wait(BAR_PFULL, t & 1, abort_flag)) { if (leader) fail(ERR_WAIT_P_FULL); return false; }
-        TRACE(4, t);
 #pragma unroll
         for (int kh = 0; kh < 2; ++kh) {
           if (!mbar_wait(BAR_VFULL(kh), t & 1, abort_flag)) { if (leader) fail(ERR_WAIT_KV_FULL); return false; }
@@ -282,7 +282,6 @@ attn_tc2_kernel(const __grid_constant__ Tc2Params p) {
         }
         umma_commit_pair_elected(leader, BAR_ODONE, 3);
         if (pend_last) umma_commit_pair_elected(leader, BAR_OLAST, 3);      // one phase per item, for the epilogue
-        TRACE(5, t);
         return true;
       };
       for (long long idx = pair_id; ok && idx < p.n_items; idx += n_pairs) {
@@ -301,11 +300,9 @@ attn_tc2_kernel(const __grid_constant__ Tc2Params p) {
             if (!ok) break;
           }
           const uint32_t stm = tmem + ((jt & 1) ? TM_S1 : TM_S0);
-          TRACE(0, jt);
 #pragma unroll
           for (int gk = 0; gk < NKG; ++gk) {
             ok = mbar_wait(BAR_KFULL(gk), jt & 1, abort_flag);
-            if (gk == 0) TRACE(1, jt);
             if (!ok) { if (leader) fail(ERR_WAIT_KV_FULL); break; }
             tc_fence_after();
 #pragma unroll
@@ -323,7 +320,6 @@ attn_tc2_kernel(const __grid_constant__ Tc2Params p) {
           if (!ok) break;
           umma_commit_pair_elected(leader, (jt & 1) ? BAR_SFULL1 : BAR_SFULL0, 3);
           if (j + 1 == it.n_tiles) umma_commit_pair_elected(leader, BAR_QFREE, 3);     // last S of the item is in flight
-          TRACE(2, jt);
           if (!pv_first && pending) ok = issue_pending_pv();
           pending = true; pend_t = jt; pend_first = (j == 0); pend_last = (j + 1 == it.n_tiles); pend_item = n_item;
         }
@@ -368,7 +364,7 @@ attn_tc2_kernel(const __grid_constant__ Tc2Params p) {
     // All 128 threads execute exactly one named barrier per tile and one per item, whatever happens: a
     // thread whose wait expired marks the fail word before the barrier and everybody leaves after it.
     bool ok = !*abort_flag;
-    uint32_t jt = 0, n_item = 0;                 // tiles / non-empty items of this pair so far
+    uint32_t jt = 0, n_item = 0, n_ragged = 0;   // tiles / non-empty items / ragged decode tiles of this pair so far
     for (long long idx = pair_id; ok && idx < p.n_items; idx += n_pairs) {
     const Item it = make_item(p, idx);
     const int b = it.b, head0 = it.head0, t0 = it.t0, nA = it.nA, n_tiles = it.n_tiles;
@@ -381,12 +377,10 @@ attn_tc2_kernel(const __grid_constant__ Tc2Params p) {
     float m_ref = -INFINITY, l_sum = 0.f;
     bool all_left = false;                       // every one of the 128 threads left the tile loop at a barrier
     for (int j = 0; j < n_tiles; ++j, ++jt) {
-      if (ln == 0) TRACE(8, jt);
       if (ok) {
         ok = mbar_wait((jt & 1) ? BAR_SFULL1 : BAR_SFULL0, (jt >> 1) & 1, abort_flag);
         if (!ok && lane == 0) fail(ERR_WAIT_S_FULL);
       }
-      if (ln == 0) TRACE(9, jt);
       ok = __all_sync(0xffffffffu, ok);
       const uint32_t stm = tmem + lane_base + ((jt & 1) ? TM_S1 : TM_S0);
       uint32_t sr[2][32];
@@ -447,7 +441,6 @@ attn_tc2_kernel(const __grid_constant__ Tc2Params p) {
       float factor = 1.f;
       if (j == 0) m_ref = tmax;
       else if (tmax > m_ref + RESCALE_THRESHOLD) { need = true; factor = exp2f(m_ref - tmax); }
-      if (ln == 0) TRACE(10, jt);
       // The probabilities depend only on S and the (new) reference maximum: compute and pack them
       // while P V of the previous tile is still running, then wait, rescale O if needed, and store.
       const float m_new = need ? tmax : m_ref;
@@ -471,7 +464,6 @@ attn_tc2_kernel(const __grid_constant__ Tc2Params p) {
         if (!ok) continue;                                   // reported at the next tile's barrier
         tc_fence_after();
       }
-      if (ln == 0) TRACE(11, jt);
       if (__any_sync(0xffffffffu, need)) {
 #pragma unroll 1                                   // rare path: kept small (the kernel is sensitive to its code size)
         for (int q = 0; q < 8; ++q) {
@@ -485,6 +477,24 @@ attn_tc2_kernel(const __grid_constant__ Tc2Params p) {
         tmem_wait_st();
       }
       if (need) { l_sum *= factor; m_ref = tmax; }
+      if (ragged_decode_tile(p, it, j)) {
+        // rows >= first_bad of this tile are not part of the sequence: zero them in this CTA's value buffers
+        // (their probabilities are exactly 0, but 0 x NaN is not)
+        bool vok = true;
+#pragma unroll
+        for (int kh = 0; kh < 2; ++kh)
+          vok = vok && mbar_wait(rank == 0 ? BAR_VFULL(kh) : BAR_VLOC(kh), (rank == 0 ? jt : n_ragged) & 1, abort_flag);
+        if (!vok && lane == 0) fail(ERR_WAIT_KV_FULL);
+        ok = __all_sync(0xffffffffu, vok);
+        if (!ok) continue;                                   // reported at the next tile's barrier
+        ++n_ragged;
+        const int first_bad = n_a_hi - j * BN;               // 1 .. 127
+        for (int x = ln; x < (BN - first_bad) * 32; x += 128) {
+          const int kr = first_bad + (x >> 5), chunk = (x >> 3) & 3, piece = x & 7;
+          const uint32_t a = sV + ((kr >> 6) * 4 + chunk) * VCH + (kr & 63) * 128 + piece * 16;
+          asm volatile("st.shared.v4.b32 [%0], {%1, %1, %1, %1};" ::"r"(a), "r"(0) : "memory");
+        }
+      }
       const uint32_t prow = sP + half * PCH + rl * 128;
 #pragma unroll
       for (int s8 = 0; s8 < 8; ++s8) {             // 16-byte slot s8 holds keys 8*s8 .. 8*s8+7
@@ -496,7 +506,6 @@ attn_tc2_kernel(const __grid_constant__ Tc2Params p) {
       fence_proxy_async_smem();                   // P is read by the tensor core (async proxy)
       tc_fence_before();
       mbar_arrive(rank == 0 ? BAR_PFULL : BAR_PLOCAL);
-      if (ln == 0) TRACE(12, jt);
     }
     if (all_left) break;
     // ---- epilogue of the item (a warp whose last wait expired still takes the barrier below)
@@ -638,12 +647,6 @@ int attn_tc2_launch(const AttnProblem& a) {
   note_launch();
   return cudaGetLastError() == cudaSuccess ? LCA_OK : LCA_ERR_CUDA;
 }
-
-#ifdef LCA_TC2_TRACE
-extern "C" int lca_debug_read_trace(long long* dst) {
-  return cudaMemcpyFromSymbol(dst, g_trace, sizeof(long long) * 8192) == cudaSuccess ? 0 : -1;
-}
-#endif
 
 int attn_tc2_take_status() {
   int st = 0;

@@ -217,6 +217,11 @@ int lca_decode_update(const lca_params* p, const void* q_tail_sem, const void* q
                        cache_row_capacity, n_rep, cache_rows, anchor_out, ws, (cudaStream_t)stream);
 }
 
+int lca_selftest_bounded_wait(int64_t limit_cycles, void* stream) {
+  if (limit_cycles < 1 || limit_cycles > 100000000ll) return LCA_ERR_INVALID_ARG;     // at most ~50 ms
+  return bounded_wait_selftest_launch((long long)limit_cycles, (cudaStream_t)stream);
+}
+
 int lca_last_device_status(void* stream) {
   const int st = attn_tc_device_status((cudaStream_t)stream);      // synchronises the stream
   const int cst = condense_take_status();

@@ -85,5 +85,6 @@ bool attn_tc_supported(const AttnProblem& a);   // tensor-core (tcgen05) kernels
 size_t attn_tc_workspace_bytes(const AttnProblem& a);
 int attn_tc_launch(const AttnProblem& a);
 int attn_tc_device_status(cudaStream_t stream);
+int bounded_wait_selftest_launch(long long limit_cycles, cudaStream_t stream);
 
 }  // namespace lca

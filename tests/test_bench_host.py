@@ -13,7 +13,7 @@ import bench  # noqa: E402
 from paper_2604_12452_b200 import inputs as I  # noqa: E402
 
 
-def test_key_visits_matches_brute_force_and_survey_counts():
+def test_key_visits_matches_brute_force_and_the_quoted_counts():
     def brute(L, g, w):
         n = 0
         for t in range(1, L + 1):

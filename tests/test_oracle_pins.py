@@ -35,35 +35,34 @@ def np_dense_causal(q, key, val, scale):
     return out
 
 
-def np_alg1_literal(qbar, q_last, C, KR, w, g, scale, bias=0.0):
-    """Alg. 1 as printed, for ONE sequence prefix and its LAST query (all heads).
-    q_last [H, dc+dr]; C [t, dc]; KR [t, dr].  Independent of the oracle's indexing helpers:
-    the fused matrices K_fused / V_fused are materialised explicitly."""
-    t = C.shape[0]
-    if t < w + g:
-        m = 0
-    else:
-        m = (t - w) // g
+def np_fused_context_attention(qbar, q_last, C, KR, w, g, scale, bias=0.0):
+    """LCA for ONE sequence prefix and its LAST query (all heads), written from the definitions of
+    Sec. 4.2 / Eq. 6-10 with whole-array numpy operations (the oracle loops over tokens): the distant
+    history is folded into an [m, g, .] block, the group softmax, the pooled latents and the anchors
+    come out of that block at once, and the fused key / value matrices of Eq. 9-10 are materialised
+    before a single softmax.  q_last [H, dc+dr]; C [t, dc]; KR [t, dr]."""
+    t, dc = C.shape
+    m = (t - w) // g if t >= w + g else 0
     K = np.concatenate([C, KR], axis=1)
-    reps_k, reps_v = [], []
-    for j in range(1, m + 1):
-        G = list(range((j - 1) * g, j * g))          # 0-based members of G_j
-        s = np.array([qbar @ K[i] * scale for i in G])
-        a = np_softmax(s)
-        c_rep = sum(a[x] * C[i] for x, i in enumerate(G))
-        I = G[int(np.argmax(s))]
-        reps_k.append(np.concatenate([c_rep, KR[I]]))
-        reps_v.append(c_rep)
-    k = t - m * g                                     # = w + (t-w) mod g when m > 0
-    K_loc, V_loc = K[t - k:], C[t - k:]
-    K_f = np.concatenate([np.array(reps_k).reshape(m, K.shape[1]), K_loc], axis=0)
-    V_f = np.concatenate([np.array(reps_v).reshape(m, C.shape[1]), V_loc], axis=0)
-    out = np.zeros((q_last.shape[0], C.shape[1]))
-    for h in range(q_last.shape[0]):
-        logit = K_f @ q_last[h] * scale
-        logit[:m] += bias
-        out[h] = np_softmax(logit) @ V_f
-    return out
+    hist = K[: m * g].reshape(m, g, K.shape[1])                              # G_1 .. G_m
+    s = hist @ qbar * scale                                           # importance scores, [m, g]
+    e = np.exp(s - s.max(axis=1, keepdims=True, initial=-np.inf))
+    alpha = e / e.sum(axis=1, keepdims=True)                          # Eq. 6
+    c_rep = np.einsum("mg,mgc->mc", alpha, C[: m * g].reshape(m, g, dc))      # Eq. 7
+    anchor = (s.argmax(axis=1) if m else np.zeros(0, int)) + g * np.arange(m)     # Eq. 8 (first maximum)
+    k_rep = np.concatenate([c_rep, KR[anchor.astype(int)]], axis=1)
+    K_f = np.concatenate([k_rep, K[m * g:]], axis=0)                  # Eq. 9: every token after the groups
+    V_f = np.concatenate([c_rep, C[m * g:]], axis=0)
+    logits = q_last @ K_f.T * scale                                   # Eq. 10
+    logits[:, :m] += bias
+    p = np.exp(logits - logits.max(axis=1, keepdims=True))
+    return (p / p.sum(axis=1, keepdims=True)) @ V_f
+
+
+def np_summary_query(qs, qp, n):
+    """Mean over the last n positions and all heads of [q_latent | q_rope] (Alg. 1, first step)."""
+    q = np.concatenate([qs, qp], axis=-1)
+    return q[q.shape[0] - n:].reshape(-1, q.shape[-1]).mean(axis=0)
 
 
 def rand_mla(rng, L, H, dc, dr):
@@ -165,10 +164,11 @@ def test_every_row_is_alg1_on_its_prefix(g, w):
     qs, qp, C, KR = rand_mla(rng, L, H, dc, dr)
     scale = 0.4
     for bias in (0.0, math.log(g)):
-        qbar, _, out, _ = oracle_full_prefill(qs, qp, C, KR, g, w, scale, bias)
+        _, _, out, _ = oracle_full_prefill(qs, qp, C, KR, g, w, scale, bias)
+        qbar = np_summary_query(qs, qp, min(L, g))          # not the oracle's: [latent | rope] order is part of the pin
         q = np.concatenate([qs, qp], -1)
         for t in range(1, L + 1):
-            ref = np_alg1_literal(qbar, q[t - 1], C[:t], KR[:t], w, g, scale, bias)
+            ref = np_fused_context_attention(qbar, q[t - 1], C[:t], KR[:t], w, g, scale, bias)
             np.testing.assert_allclose(out[t - 1], ref, rtol=0, atol=1e-12, err_msg=f"t={t}")
 
 
@@ -178,6 +178,19 @@ def test_summary_query_is_mean_of_last_rows_and_heads():
     np.testing.assert_allclose(O.summary_query(q[-4:]), q[-4:].reshape(-1, 7).mean(0), atol=1e-15)
     # a single head with a single row is returned untouched
     np.testing.assert_array_equal(O.summary_query(q[-1:, :1]), q[-1, 0])
+
+
+def test_mla_summary_query_is_latent_part_then_rope_part():
+    # Alg. 1 first step on the absorbed query [q_latent | q_rope]: d_c != d_R, so a swapped concatenation,
+    # a mean over the wrong axis or a dropped head cannot pass.
+    rng = RNG(41)
+    n, H, dc, dr = 5, 3, 7, 2
+    qs, qp = rng.standard_normal((n, H, dc)), rng.standard_normal((n, H, dr)) + 10.0
+    got = O.mla_summary_query(qs, qp)
+    assert got.shape == (dc + dr,)
+    np.testing.assert_allclose(got, np.concatenate([qs, qp], -1).mean((0, 1)), atol=1e-14)
+    np.testing.assert_allclose(got[:dc], qs.reshape(-1, dc).mean(0), atol=1e-14)
+    assert (got[dc:] > 5.0).all()                       # the rope part (shifted by 10) sits at the end
 
 
 def test_alpha_is_a_distribution_and_pooling_is_convex():
@@ -292,8 +305,10 @@ def test_decode_equals_prefill_row_of_longer_sequence():
                                       KR[cs["anchor"]], g, w, scale)
     np.testing.assert_allclose(out_d, out_p[0], atol=1e-12)
     np.testing.assert_allclose(lse_d, lse_p[0], atol=1e-12)
-    # and the last prefill row is Alg. 1 as printed on the whole sequence
-    ref = np_alg1_literal(qbar, np.concatenate([qs[L - 1], qp[L - 1]], -1), C[:L], KR[:L], w, g, scale)
+    # and the last prefill row is Alg. 1 on the whole sequence (summary query restated in numpy)
+    np.testing.assert_allclose(qbar, np_summary_query(qs[:L], qp[:L], g), atol=1e-15)
+    ref = np_fused_context_attention(np_summary_query(qs[:L], qp[:L], g), np.concatenate([qs[L - 1], qp[L - 1]], -1),
+                                     C[:L], KR[:L], w, g, scale)
     out_last, _ = O.mla_prefill_rows(qs[L - 1:L], qp[L - 1:L], np.array([L - 1]), C[:L], KR[:L],
                                      cs["pooled"], KR[cs["anchor"]], g, w, scale)
     np.testing.assert_allclose(out_last[0], ref, atol=1e-12)
@@ -409,6 +424,46 @@ def test_gqa_with_group_one_is_textbook_mha():
     for h in range(Hq):
         ref = np_dense_causal(q[:, h:h + 1], k[:, h // 2], v[:, h // 2], scale)
         np.testing.assert_allclose(out[:, h], ref[:, 0], atol=1e-12)
+
+
+def test_gqa_decode_maps_each_query_head_to_its_kv_head():
+    # Sec. 5.4 decode: query head h reads KV head h // (Hq / Hkv).  Three query heads per KV head and
+    # keys / values that differ strongly per KV head, so a wrong mapping (h % Hkv, transposed cache,
+    # shared head) fails; the bias applies to the leading n_rep rows only.
+    rng = RNG(42)
+    rows, Hq, Hkv, d, n_rep, scale, bias = 23, 6, 2, 5, 4, 0.37, 0.6
+    q = rng.standard_normal((Hq, d))
+    ck = rng.standard_normal((rows, Hkv, d)) + np.array([0.0, 3.0])[None, :, None]
+    cv = rng.standard_normal((rows, Hkv, d)) * np.array([1.0, -2.0])[None, :, None]
+    out, lse = O.gqa_decode(q, ck, cv, n_rep, scale, bias)
+    assert out.shape == (Hq, d) and lse.shape == (Hq,)
+    for h in range(Hq):
+        kv = h // (Hq // Hkv)
+        lg = ck[:, kv] @ q[h] * scale
+        lg[:n_rep] += bias
+        np.testing.assert_allclose(out[h], np_softmax(lg) @ cv[:, kv], atol=1e-13)
+        assert abs(lse[h] - np.log(np.exp(lg).sum())) < 1e-12
+
+
+def test_gqa_decode_equals_last_prefill_row():
+    # Decoding the last token against the cache [representatives ; last k tokens] of the same sequence
+    # is the last row of the prefill (Sec. 4.3 / 5.4), for every query head.
+    rng = RNG(43)
+    L, Hq, Hkv, d, g, w, scale = 31, 6, 2, 4, 4, 5, 0.5
+    q = rng.standard_normal((L, Hq, d))
+    k = rng.standard_normal((L, Hkv, d)) + np.array([0.0, 1.5])[None, :, None]
+    v = rng.standard_normal((L, Hkv, d))
+    qbar = O.gqa_summary_query(q[-g:], Hkv)
+    cs = O.gqa_condense(qbar, k, v, g, w, scale)
+    m, kk = cs["m"], cs["k"]
+    assert m > 0
+    k_rep = np.stack([k[cs["anchor"][:, h], h] for h in range(Hkv)], axis=1)
+    cache_k = np.concatenate([k_rep, k[L - kk:]], axis=0)
+    cache_v = np.concatenate([cs["v_rep"], v[L - kk:]], axis=0)
+    out_d, lse_d = O.gqa_decode(q[-1], cache_k, cache_v, m, scale, 0.3)
+    out_p, lse_p = O.gqa_prefill_rows(q[-1:], np.array([L - 1]), k, v, k_rep, cs["v_rep"], g, w, scale, 0.3)
+    np.testing.assert_allclose(out_d, out_p[0], atol=1e-12)
+    np.testing.assert_allclose(lse_d, lse_p[0], atol=1e-12)
 
 
 def test_gqa_condense_selects_keys_and_pools_values():

@@ -61,6 +61,29 @@ def test_config3_mla_128k_full_size(B):
     check_mla_full(B, "mla_128k", n_uniform=24)
 
 
+def test_long_context_256k_with_the_paper_default_group_and_window(B):
+    # The scaling run's shape (V2-Lite-like layer, g = 16, w = 1024) at 262144 tokens: 16320 representatives, query
+    # rows far beyond 2^17, the cache compared in full, sampled rows (the last one included) on every head.
+    cfg = I.scaled(I.CONFIGS["mla_32k"], name="v2lite_256k", seq_len=262144, group_size=16, window=1024, needle_every=4096)
+    L, g, w = cfg.seq_len, cfg.group_size, cfg.window
+    inp = I.make_mla_inputs(cfg, DEV)
+    p = B.params_from_config(cfg, batch=1)
+    cond = B.condense(p, inp["q_sem"][L - g:], inp["q_pos"][L - g:], inp["ckv"], inp["kr"])
+    assert cond["m"] == (L - w) // g == 16320
+    out, lse = B.prefill_attention(p, inp["q_sem"], inp["q_pos"], inp["ckv"], inp["kr"], cond["cache_sem"],
+                                   cond["cache_pos"], want_lse=True)
+    torch.cuda.synchronize()
+    assert B.lca_last_device_status() == 0
+    rows = Hh.sample_positions(L, g, w, extra=[131071, 131072, 131073, 200000, L - 17, L - 16], n_uniform=24, seed=9)
+    assert rows[-1] == L - 1
+    idx = torch.from_numpy(rows).to(DEV)
+    ref = Hh.oracle_mla_sampled(inp["ckv"].cpu(), inp["kr"].cpu(), inp["q_sem"][L - g:].cpu(), inp["q_pos"][L - g:].cpu(),
+                                inp["q_sem"][idx].cpu(), inp["q_pos"][idx].cpu(), rows, g, w, cfg.softmax_scale)
+    Hh.check_condense(one_seq(cond), ref["cond"])
+    Hh.check_outputs(out[0][idx], ref["out"], "256k sampled rows")
+    np.testing.assert_allclose(lse[0][idx].cpu().numpy(), ref["lse"], atol=2e-3, rtol=1e-4)
+
+
 def test_config5_gqa_64k_full_size(B):
     cfg = I.CONFIGS["gqa_64k"]
     L, g, w = cfg.seq_len, cfg.group_size, cfg.window

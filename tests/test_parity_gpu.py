@@ -447,3 +447,74 @@ def test_gqa_decode_matches_oracle(B):
         for b in range(3):
             Hh.check_outputs(out[b], refs[b][0], f"gqa decode seq {b} impl {impl}")
             np.testing.assert_allclose(lse[b].cpu().numpy(), refs[b][1], atol=2e-3, rtol=1e-4)
+
+
+def test_decode_ignores_non_finite_rows_behind_the_valid_count(B):
+    # Capacity rows at or behind cache_rows[b] may hold anything (here NaN and Inf bit patterns): they must not reach
+    # the output (probability 0 times NaN is NaN).  Ragged counts, a count on a tile boundary, empty caches; the MLA
+    # shape (CTA-pair kernel) and the GQA shape (one-CTA kernel).
+    gen = torch.Generator().manual_seed(123)
+    nb, cap, H = 6, 300, 128
+    counts = [300, 299, 129, 128, 1, 0]
+    cache_sem = torch.randn((nb, cap, 1, 512), generator=gen).bfloat16()
+    cache_pos = torch.randn((nb, cap, 1, 64), generator=gen).bfloat16()
+    q_sem = torch.randn((nb, H, 512), generator=gen).bfloat16()
+    q_pos = torch.randn((nb, H, 64), generator=gen).bfloat16()
+    poisoned_sem, poisoned_pos = cache_sem.clone(), cache_pos.clone()
+    for b, n in enumerate(counts):
+        poisoned_sem[b, n:] = float("nan")
+        poisoned_pos[b, n:] = float("inf") if b % 2 else float("nan")
+    cfg = I.scaled(I.CONFIGS["mla_decode"], batch=nb, seq_len=4096, n_q_heads=H)
+    p = B.params_from_config(cfg, batch=nb)
+    rows = torch.tensor(counts, dtype=torch.int32, device=DEV)
+    out, lse = B.decode_attention(p, q_sem.to(DEV), q_pos.to(DEV), poisoned_sem.to(DEV), poisoned_pos.to(DEV), rows, 17,
+                                  want_lse=True)
+    assert B.lca_last_device_status() == 0
+    assert torch.isfinite(out.float()).all()
+    for b, n in enumerate(counts):
+        if n == 0:
+            assert torch.count_nonzero(out[b]) == 0
+            continue
+        ro, rl = O.mla_decode(O.torch_bf16_to_f64(q_sem[b]), O.torch_bf16_to_f64(q_pos[b]),
+                              O.bits_to_f64(Hh.bits(cache_sem[b, :n, 0])), O.bits_to_f64(Hh.bits(cache_pos[b, :n, 0])),
+                              min(17, n), Hh.f32(cfg.softmax_scale))
+        Hh.check_outputs(out[b], ro, f"mla decode, {n} valid rows, NaN behind")
+        np.testing.assert_allclose(lse[b].cpu().numpy(), rl, atol=2e-3, rtol=1e-4)
+
+    Hq, Hkv, d = 32, 8, 128
+    ck = torch.randn((nb, cap, Hkv, d), generator=gen).bfloat16()
+    cv = torch.randn((nb, cap, Hkv, d), generator=gen).bfloat16()
+    q = torch.randn((nb, Hq, d), generator=gen).bfloat16()
+    pk, pv = ck.clone(), cv.clone()
+    for b, n in enumerate(counts):
+        pk[b, n:] = float("nan")
+        pv[b, n:] = float("nan")
+    cfg = I.scaled(I.CONFIGS["gqa_64k"], batch=nb, seq_len=4096)
+    p = B.params_from_config(cfg, batch=nb)
+    out, _ = B.decode_attention(p, None, q.to(DEV), pv.to(DEV), pk.to(DEV), rows, 17)
+    assert B.lca_last_device_status() == 0
+    assert torch.isfinite(out.float()).all()
+    for b, n in enumerate(counts):
+        if n == 0:
+            assert torch.count_nonzero(out[b]) == 0
+            continue
+        ro, _ = O.gqa_decode(O.torch_bf16_to_f64(q[b]), O.bits_to_f64(Hh.bits(ck[b, :n])), O.bits_to_f64(Hh.bits(cv[b, :n])),
+                             min(17, n), Hh.f32(cfg.softmax_scale))
+        Hh.check_outputs(out[b], ro, f"gqa decode, {n} valid rows, NaN behind")
+
+
+def test_a_bounded_device_wait_that_expires_is_reported_and_harmless(B):
+    # The library's own self-test kernel waits, with the routine every tensor-core kernel uses, on a barrier nobody
+    # arrives on; after ~1e5 cycles it gives up, records the code and returns.  The status is reported once, and the
+    # next ordinary call works.
+    assert B.lca_last_device_status() == 0
+    assert B.lca_selftest_bounded_wait(0) == -1 and B.lca_selftest_bounded_wait(10 ** 12) == -1      # limit out of range
+    assert B.lca_selftest_bounded_wait(100_000) == 0
+    assert B.lca_last_device_status() == B.LCA_ERR_DEVICE_TIMEOUT
+    assert B.lca_last_device_status() == 0
+    cfg = I.scaled(I.CONFIGS["mla_1k"], seq_len=300, n_q_heads=16, group_size=16, window=64)
+    inp = I.make_mla_inputs(cfg, "cpu")
+    p, cond, out, _ = run_mla(B, cfg, to_dev(inp), want_scores=False)
+    assert B.lca_last_device_status() == 0
+    ref = Hh.oracle_mla(inp, cfg.group_size, cfg.window, cfg.softmax_scale, rows=np.arange(cfg.seq_len))
+    Hh.check_outputs(out[0], ref["out"], "after an expired wait")

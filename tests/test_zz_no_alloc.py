@@ -35,7 +35,7 @@ def _outputs(B, p, dev):
                 anchor_idx=torch.full((p.batch, max(m, 1), p.n_kv_heads), -1, dtype=torch.int32, device=dev)), m
 
 
-def _both_ways(B, cfg, want_scores):
+def _both_ways(B, cfg, want_scores, first_call_on_device=False):
     inp = {k: v.to(DEV) for k, v in I.make_mla_inputs(cfg, "cpu").items()}
     p = B.params_from_config(cfg, batch=1)
     L, g = cfg.seq_len, cfg.group_size
@@ -49,10 +49,16 @@ def _both_ways(B, cfg, want_scores):
     assert B.lca_condense(p, tail_sem, tail_pos, n, None, inp["ckv"], inp["kr"], ref["cache_sem"], ref["cache_pos"],
                           ref["anchor_idx"], sc_ref, ws) == 0
     before = B.lca_launch_count()
+    torch.cuda.synchronize()
+    free_before = torch.cuda.mem_get_info()[0]          # the driver's count of free device bytes
     assert B.lca_condense_static_scratch(p, tail_sem, tail_pos, n, None, inp["ckv"], inp["kr"], got["cache_sem"],
                                          got["cache_pos"], got["anchor_idx"], sc_got) == 0
     assert B.lca_launch_count() > before
     torch.cuda.synchronize()
+    if not first_call_on_device:
+        # nothing was allocated or freed behind the caller's back (the very first call may page in the
+        # library's kernels, which the driver accounts to the context, so it is left out)
+        assert torch.cuda.mem_get_info()[0] == free_before
     # same kernels, same arithmetic, only the scratch lives elsewhere: the tolerance of the other
     # condense tests (bit-exact anchors and copies, c_rep within one bf16 ulp) tightens to equality
     for key in ref:
@@ -65,7 +71,7 @@ def test_static_scratch_condense_matches_lca_condense_twice_in_a_row(B):
     big = I.scaled(I.CONFIGS["mla_1k"], seq_len=2048, n_q_heads=128, group_size=64, window=256)
     small = I.scaled(I.CONFIGS["mla_1k"], seq_len=777, n_q_heads=16, group_size=16, window=100)
     assert 0 < B.lca_workspace_bytes(B.params_from_config(big, batch=1), B.LCA_WS_CONDENSE) <= B.LCA_STATIC_SCRATCH_BYTES
-    _both_ways(B, big, want_scores=True)       # first call on this device: looks the array up
+    _both_ways(B, big, want_scores=True, first_call_on_device=True)       # first call on this device: looks the array up
     _both_ways(B, small, want_scores=False)    # second call: the array still holds the first call's data
 
 
