@@ -484,9 +484,10 @@ def measure_decode_config(B, dev, batch, peaks, warmup=3, iters=5):
                 online_update=upd)
 
 
-def measure_gqa_config(B, dev, peaks, warmup=3, iters=5):
-    """Config 5: GQA variant (pool V, select K per KV head): condense + prefill attention."""
-    cfg = I.CONFIGS["gqa_64k"]
+def measure_gqa_config(B, dev, peaks, warmup=3, iters=5, seq_len=None):
+    """Config 5: GQA variant (pool V, select K per KV head): condense + prefill attention.
+    `seq_len` shortens the sequence (profiler captures of the same kernels on a small case)."""
+    cfg = I.CONFIGS["gqa_64k"] if not seq_len else I.scaled(I.CONFIGS["gqa_64k"], seq_len=seq_len)
     L, g = cfg.seq_len, cfg.group_size
     inp = I.make_gqa_inputs(cfg, dev)
     p = B.params_from_config(cfg, batch=1)
@@ -573,6 +574,7 @@ def main():
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-extras", action="store_true", help="skip the decode / GQA / dense-comparison side measurements")
     ap.add_argument("--decode-batch", type=int, default=64)
+    ap.add_argument("--seq-len", type=int, default=0, help="gqa_64k only: a shorter sequence of the same shape (small profiler captures)")
     ap.add_argument("--ref-rows", type=int, default=24, help="query rows in the oracle's bounded sample")
     ap.add_argument("--ref-heads", type=int, default=16, help="heads per sampled row in the oracle's sample")
     args = ap.parse_args()
@@ -602,7 +604,7 @@ def main():
             peaks = measured_peaks()
             dev = f"cuda:{local_rank}"
             res = (measure_decode_config(B, dev, args.decode_batch, peaks, args.warmup, args.steps) if args.config == "mla_decode"
-                   else measure_gqa_config(B, dev, peaks, args.warmup, args.steps))
+                   else measure_gqa_config(B, dev, peaks, args.warmup, args.steps, args.seq_len))
             print(json.dumps(dict(metric="side_measurement", config=dict(workload=res["workload"]), n_gpus=1, steps=args.steps,
                                   warmup=args.warmup, data="synthetic", result=res, gpu_launches=None)))
         return

@@ -197,6 +197,18 @@ int lca_decode_update(const lca_params* p, const void* q_tail_sem, const void* q
                       int32_t* cache_rows, int32_t* anchor_out, void* ws, size_t ws_bytes,
                       void* stream);
 
+/* Value up-projection of the latent attention output (Alg. 1: v = c W^UV; Sec. 4.3: in the absorbed
+ * form the attention result lives in the latent space and W^UV is applied to it once per query and
+ * head):   out_v[t, h, :] = attn_latent[t, h, :] . W^UV[h]
+ *   attn_latent [n_tokens, n_heads, d_latent] bf16: `out` of lca_prefill_attention / lca_decode_attention
+ *                                                   (n_tokens = batch * seq_len, or batch for decode)
+ *   w_uv        [n_heads, d_latent, d_v] bf16 (d_v contiguous)
+ *   out_v       [n_tokens, n_heads, d_v] bf16 (products in bf16 on the tensor cores, fp32 sums, one rounding)
+ * Built for d_latent = 512, d_v = 128 (DeepSeek-V2 / V3); other sizes return LCA_ERR_UNSUPPORTED_SHAPE.
+ * Needs no workspace.  n_tokens = 0 is a no-op. */
+int lca_latent_to_value(const void* attn_latent, const void* w_uv, void* out_v, int64_t n_tokens,
+                        int32_t n_heads, int32_t d_latent, int32_t d_v, void* stream);
+
 /* Which attention implementation lca_prefill_attention / lca_decode_attention use:
  *   0 = automatic (tensor-core kernels where the shape is supported, else the scalar kernel),
  *   1 = force the scalar (CUDA-core) kernel, 2 = force the tensor-core kernel (unsupported

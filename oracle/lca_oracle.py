@@ -235,6 +235,13 @@ def mla_decode(q_sem, q_pos, cache_sem, cache_pos, n_rep, scale, rep_logit_bias=
     return decode_rows(q, ckey, cs, n_rep, scale, rep_logit_bias)
 
 
+def latent_to_value(attn_latent: np.ndarray, w_uv: np.ndarray) -> np.ndarray:
+    """Value up-projection of the latent attention output (Alg. 1: v = c W^UV, applied after the
+    attention in the absorbed form of Sec. 4.3): attn_latent [..., H, d_c], w_uv [H, d_c, d_v] ->
+    [..., H, d_v], one matrix product per head."""
+    return np.einsum("...hc,hcv->...hv", _f64(attn_latent), _f64(w_uv))
+
+
 # ------------------------------------------------------------------------------ GQA flavour
 def gqa_summary_query(q_tail: np.ndarray, n_kv_heads: int) -> np.ndarray:
     """q_tail [n, Hq, d] -> q_bar [Hkv, d]: mean over positions and the Hq/Hkv heads of each KV head."""

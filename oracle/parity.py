@@ -50,6 +50,7 @@ def mla_pipeline(ckv, kr, q_tail_sem, q_tail_pos, g, w, scale, q_rows_sem=None, 
         out, lse = O.mla_prefill_rows(O.torch_bf16_to_f64(qs), O.torch_bf16_to_f64(qp), rows, ckv64, kr64,
                                       rep_sem, rep_pos, g, w, f32(scale), f32(rep_logit_bias))
         res.update(rows=rows, out=out, lse=lse)
+    res["vmax"] = np.abs(ckv64).max(axis=0)            # largest |value| per latent column (needle rows included)
     return res
 
 
@@ -68,6 +69,8 @@ def gqa_pipeline(q_tail, k, v, g, w, scale, q_rows=None, rows=None, rep_logit_bi
         out, lse = O.gqa_prefill_rows(O.torch_bf16_to_f64(q_rows), rows, k64, v64, k_rep, v_rep, g, w,
                                       f32(scale), f32(rep_logit_bias))
         res.update(rows=rows, out=out, lse=lse)
+    hq = O.torch_bf16_to_f64(q_tail).shape[1]
+    res["vmax"] = np.repeat(np.abs(v64).max(axis=0), hq // hkv, axis=0)      # [Hq, d]: per query head, its KV head's columns
     return res
 
 
@@ -80,18 +83,40 @@ def bf16_ulp_distance(a_bits: np.ndarray, b_bits: np.ndarray) -> np.ndarray:
     return np.abs(key(a_bits) - key(b_bits))
 
 
-def output_stats(got, ref: np.ndarray) -> dict:
-    """Raw error figures of an attention output (`got`: torch tensor on any device, or numpy)."""
+def output_bound(ref: np.ndarray, vmax=None) -> np.ndarray:
+    """Element-wise error bound of an attention output computed with bf16 probabilities.
+
+    The kernels round the softmax weights to bf16 before P V and normalise by the sum of the rounded
+    weights, so the result is a convex combination with every weight perturbed by at most 2^-9
+    relative: the error in column c is at most 2^-9 sum_i p_i |v_ic - out_c| <= 2^-9 (vmax_c + |out_c|),
+    vmax_c = the largest |value| of that column; the bf16 store of the result adds 2^-9 |out_c| (half an
+    ulp at the top of a binade, 2^-8 at the bottom).  For values of unit scale (N(0,1): vmax ~ 4.6) that
+    is below the 2e-2 stated for the method; it grows with the values (x4 "needle" rows: vmax ~ 17).
+    The bound returned is the larger of the stated 2e-2 and the derived one.  Without `vmax` only the
+    output rounding is scaled: max(2e-2, 2^-7 |ref|)."""
+    aref = np.abs(ref)
+    if vmax is None:
+        return np.maximum(2e-2, 2.0 ** -7 * aref)
+    return np.maximum(2e-2, 2.0 ** -9 * (np.asarray(vmax) + aref) + 2.0 ** -8 * aref)
+
+
+def output_stats(got, ref: np.ndarray, vmax=None) -> dict:
+    """Raw error figures of an attention output (`got`: torch tensor on any device, or numpy) and the
+    worst ratio to output_bound."""
     g = got.detach().float().cpu().numpy() if hasattr(got, "detach") else np.asarray(got)
     g = g.astype(np.float64)
     if g.size == 0:
         return dict(n=0, max_abs=0.0, mean_abs=0.0, max_ref=0.0, mean_ref=0.0, finite=True, n_above_2e2=0,
-                    worst_over_ulp_bound=0.0)
+                    max_abs_unit_scale=0.0, worst_over_bound=0.0)
     err = np.abs(g - ref)
     aref = np.abs(ref)
+    # elements whose column holds only values of unit scale (|v| <= 5: no x4 needle of any size) and whose result
+    # is of unit scale (|ref| <= 1.5): there the derived bound is below 2e-2, which must then hold as stated
+    unit = aref <= 1.5 if vmax is None else (aref <= 1.5) & (np.broadcast_to(np.asarray(vmax), ref.shape) <= 5.0)
     return dict(n=int(err.size), max_abs=float(err.max()), mean_abs=float(err.mean()), max_ref=float(aref.max()),
                 mean_ref=float(aref.mean()), finite=bool(np.isfinite(g).all()), n_above_2e2=int((err > 2e-2).sum()),
-                worst_over_ulp_bound=float((err / np.maximum(2e-2, 2.0 ** -7 * aref)).max()))
+                max_abs_unit_scale=float(err[unit].max()) if unit.any() else 0.0,
+                worst_over_bound=float((err / output_bound(ref, vmax)).max()))
 
 
 def near_ties(scores: np.ndarray, g: int, rel: float = 1e-6) -> int:

@@ -71,6 +71,8 @@ def _load() -> C.CDLL:
     lib.lca_decode_attention.argtypes = [P, vp, vp, vp, vp, vp, i32, i32, vp, vp, vp, sz, vp]
     lib.lca_decode_update.restype = C.c_int
     lib.lca_decode_update.argtypes = [P, vp, vp, i64, vp, vp, vp, i32, vp, vp, vp, vp, sz, vp]
+    lib.lca_latent_to_value.restype = C.c_int
+    lib.lca_latent_to_value.argtypes = [vp, vp, vp, i64, i32, i32, i32, vp]
     lib.lca_selftest_bounded_wait.restype = C.c_int
     lib.lca_selftest_bounded_wait.argtypes = [i64, vp]
     lib.lca_last_device_status.restype = C.c_int
@@ -176,6 +178,11 @@ def lca_decode_update(params, q_tail_sem, q_tail_pos, q_tail_batch_stride, qbar_
                                       _ptr(n_rep), _ptr(cache_rows), _ptr(anchor_out), _ptr(ws), wsb, _stream(stream)))
 
 
+def lca_latent_to_value(attn_latent, w_uv, out_v, n_tokens, n_heads, d_latent, d_v, stream=None) -> int:
+    return int(_lib.lca_latent_to_value(_ptr(attn_latent), _ptr(w_uv), _ptr(out_v), int(n_tokens), int(n_heads),
+                                        int(d_latent), int(d_v), _stream(stream)))
+
+
 def lca_selftest_bounded_wait(limit_cycles: int, stream=None) -> int:
     return int(_lib.lca_selftest_bounded_wait(int(limit_cycles), _stream(stream)))
 
@@ -267,6 +274,16 @@ def decode_attention(params: LcaParams, q_sem, q_pos, cache_sem, cache_pos, cach
                               ws, stream=stream)
     _check(st, "lca_decode_attention")
     return out, lse
+
+
+def latent_to_value(attn_latent: torch.Tensor, w_uv: torch.Tensor, out=None, stream=None):
+    """out_v[..., h, :] = attn_latent[..., h, :] @ w_uv[h]  (attn_latent [..., H, d_latent], w_uv [H, d_latent, d_v])."""
+    H, d_latent, d_v = w_uv.shape
+    n_tokens = attn_latent.numel() // (H * d_latent)
+    if out is None:
+        out = torch.empty(attn_latent.shape[:-1] + (d_v,), dtype=torch.bfloat16, device=attn_latent.device)
+    _check(lca_latent_to_value(attn_latent, w_uv, out, n_tokens, H, d_latent, d_v, stream=stream), "lca_latent_to_value")
+    return out
 
 
 def decode_update(params: LcaParams, q_tail_sem, q_tail_pos, cache_sem, cache_pos, n_rep, cache_rows,

@@ -21,6 +21,8 @@ SOURCES = {
     "attn_simt.cu": ["--use_fast_math"],
     "attn_tc.cu": ["--use_fast_math"],
     "attn_tc2.cu": ["--use_fast_math"],
+    "attn_gqa2.cu": ["--use_fast_math"],
+    "gemm_uv.cu": ["--use_fast_math"],
 }
 
 

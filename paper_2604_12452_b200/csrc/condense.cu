@@ -267,8 +267,17 @@ constexpr int SEM_BYTES = G * DS * 2, POS_BYTES = G * DP * 2, STAGE_BYTES = SEM_
 constexpr int OFF_Q = STAGES * STAGE_BYTES;                 // double[DK]
 constexpr int OFF_S = OFF_Q + DK * 8;                       // double[2][G] scores
 constexpr int OFF_A = OFF_S + 2 * G * 8;                    // float[2][G] alpha
-constexpr int OFF_BAR = OFF_A + 2 * G * 4;                  // mbarriers: full[3] free[3] ready[2] afree[2], then flags
+constexpr int OFF_S32 = OFF_A + 2 * G * 4;                  // float[2][G] fp32 products q_bar . k_i (before the scale)
+constexpr int OFF_ABS = OFF_S32 + 2 * G * 4;                // float[2][G] sum_c |q_bar_c| |k_ic|: scale of their rounding error
+constexpr int OFF_BAR = OFF_ABS + 2 * G * 4;                // mbarriers: full[3] free[3] ready[2] afree[2], then flags
 constexpr int SMEM_BYTES = OFF_BAR + 128;
+// An fp32 product sum of this kernel passes through at most 15 roundings (9 multiply-adds per chain, the
+// chain pair, 5 shuffle levels) and q_bar itself is rounded once to fp32: |s32_i - s_i| <= 16 u A_i (1 + 16 u),
+// u = 2^-24, A_i = sum_c |q_bar_c| |k_ic|, and the fp32 A_i is at least A_i (1 - 16 u).  A group whose two largest
+// fp32 products differ by more than 48 u max_i A_i (twice 20 u A: the bound with a quarter of slack, plus the
+// rounding of the difference) therefore has the same arg-max in exact arithmetic; any other group (exact ties
+// included) is scored again in fp64.
+constexpr float MARGIN_FACTOR = 48.0f * 5.9604644775390625e-08f;
 static_assert(SMEM_BYTES <= 232448, "shared memory budget of one SM");
 constexpr long long WAIT_CYCLES = 2000000000ll;
 }  // namespace fast
@@ -291,6 +300,42 @@ __device__ __forceinline__ void cond_arrive(unsigned bar) {
   asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar) : "memory");
 }
 
+// The exact scores of a score warp's four tokens (warp w: tokens w, w + 16, w + 32, w + 48) in fp64, q_bar read from
+// shared memory.  Kept out of line: it runs for the rare groups whose fp32 arg-max is not provably the exact one (and
+// for every group when the caller asked for the scores), and its registers should not weigh on the fp32 path.
+__device__ __noinline__ void score_tokens_fp64(const unsigned char* t_sem, const unsigned char* t_pos, const double* s_q,
+                                               double* s_out, int warp, int lane, double scale) {
+  using namespace fast;
+  double part[4];
+#pragma unroll
+  for (int tt = 0; tt < 4; ++tt) {
+    const int i = warp + SCORE_WARPS * tt;
+    const uint4 v0 = *reinterpret_cast<const uint4*>(t_sem + (size_t)i * (DS * 2) + 16 * lane);
+    const uint4 v1 = *reinterpret_cast<const uint4*>(t_sem + (size_t)i * (DS * 2) + 512 + 16 * lane);
+    const unsigned vp = *reinterpret_cast<const unsigned*>(t_pos + (size_t)i * (DP * 2) + 4 * lane);
+    const unsigned w[9] = {v0.x, v0.y, v0.z, v0.w, v1.x, v1.y, v1.z, v1.w, vp};
+    double acc0 = 0.0, acc1 = 0.0;
+#pragma unroll
+    for (int k = 0; k < 9; ++k) {
+      const int c0 = k < 4 ? 8 * lane + 2 * k : k < 8 ? 256 + 8 * lane + 2 * (k - 4) : DS + 2 * lane;
+      acc0 = fma(s_q[c0], (double)__uint_as_float(w[k] << 16), acc0);
+      acc1 = fma(s_q[c0 + 1], (double)__uint_as_float(w[k] & 0xffff0000u), acc1);
+    }
+    part[tt] = acc0 + acc1;
+  }
+  // transposed reduction: lanes 0, 8, 16, 24 end up with the sums of tokens 0..3
+  const bool up16 = (lane & 16) != 0, up8 = (lane & 8) != 0;
+  const double k0 = up16 ? part[2] : part[0], k1 = up16 ? part[3] : part[1];
+  const double g0 = up16 ? part[0] : part[2], g1 = up16 ? part[1] : part[3];
+  const double b0 = k0 + __shfl_xor_sync(0xffffffffu, g0, 16);
+  const double b1 = k1 + __shfl_xor_sync(0xffffffffu, g1, 16);
+  double c = (up8 ? b1 : b0) + __shfl_xor_sync(0xffffffffu, up8 ? b0 : b1, 8);
+  c += __shfl_xor_sync(0xffffffffu, c, 4);
+  c += __shfl_xor_sync(0xffffffffu, c, 2);
+  c += __shfl_xor_sync(0xffffffffu, c, 1);
+  if ((lane & 7) == 0) s_out[warp + SCORE_WARPS * (lane >> 3)] = c * scale;
+}
+
 __global__ void __launch_bounds__(fast::THREADS, 1)
 condense_mla64_kernel(CondenseArgs a) {
   using namespace fast;
@@ -298,6 +343,8 @@ condense_mla64_kernel(CondenseArgs a) {
   double* s_q = reinterpret_cast<double*>(smem + OFF_Q);
   double* s_s = reinterpret_cast<double*>(smem + OFF_S);
   float* s_a = reinterpret_cast<float*>(smem + OFF_A);
+  float* s_s32 = reinterpret_cast<float*>(smem + OFF_S32);
+  float* s_abs = reinterpret_cast<float*>(smem + OFF_ABS);
   const unsigned bar0 = (unsigned)__cvta_generic_to_shared(smem + OFF_BAR);
   auto BAR_FULL = [&](int st) { return bar0 + 8 * st; };
   auto BAR_FREE = [&](int st) { return bar0 + 24 + 8 * st; };
@@ -346,7 +393,12 @@ condense_mla64_kernel(CondenseArgs a) {
     }
   } else if (warp < SCORE_WARPS) {
     // ===================================================== scores, arg-max, softmax
-    double q[18];
+    // The products q_bar . k_i are taken in fp32 together with A_i = sum |q_bar_c| |k_ic|.  Where the two largest
+    // products of a group are further apart than the rounding error A_i allows (MARGIN_FACTOR), the fp32 arg-max
+    // is the exact one; otherwise, and whenever the caller asked for the scores, the group is scored in fp64.
+    float q[18];
+    const bool exact_all = a.scores != nullptr;
+    const float scale32 = (float)a.scale;
     long long cur_b = -1;
     for (long long it = 0; it < n_mine; ++it) {
       const int st = (int)(it % STAGES), p = (int)(it & 1);
@@ -359,18 +411,18 @@ condense_mla64_kernel(CondenseArgs a) {
         for (int x = tid; x < DK; x += 32 * SCORE_WARPS) s_q[x] = qb[x];
         asm volatile("bar.sync 1, 512;" ::: "memory");
 #pragma unroll
-        for (int i = 0; i < 8; ++i) { q[i] = s_q[8 * lane + i]; q[8 + i] = s_q[256 + 8 * lane + i]; }
-        q[16] = s_q[DS + 2 * lane]; q[17] = s_q[DS + 2 * lane + 1];
+        for (int i = 0; i < 8; ++i) { q[i] = (float)s_q[8 * lane + i]; q[8 + i] = (float)s_q[256 + 8 * lane + i]; }
+        q[16] = (float)s_q[DS + 2 * lane]; q[17] = (float)s_q[DS + 2 * lane + 1];
       }
       bool ok = cond_wait(BAR_FULL(st), (unsigned)((it / STAGES) & 1), s_abort);
       if (ok && it >= 2) ok = cond_wait(BAR_AFREE(p), (unsigned)(((it >> 1) - 1) & 1), s_abort);
       const unsigned char* t_sem = smem + (size_t)st * STAGE_BYTES;
       const unsigned char* t_pos = t_sem + SEM_BYTES;
-      if (ok) {
-        // the warp's four tokens together: 4 x 18 independent multiply-add chains, then one
-        // transposed reduction (lanes 0, 8, 16, 24 end up with the sums of tokens 0..3)
-        static_assert(G / SCORE_WARPS == 4, "four tokens per score warp");
-        double part[4];
+      static_assert(G / SCORE_WARPS == 4, "four tokens per score warp");
+      if (ok && !exact_all) {
+        // the warp's four tokens together: 4 x 4 independent multiply-add chains, then one transposed
+        // reduction of the eight sums (lanes 0, 4, ... 28 end up with one of them each)
+        float v[8];
 #pragma unroll
         for (int tt = 0; tt < 4; ++tt) {
           const int i = warp + SCORE_WARPS * tt;
@@ -378,41 +430,77 @@ condense_mla64_kernel(CondenseArgs a) {
           const uint4 v1 = *reinterpret_cast<const uint4*>(t_sem + (size_t)i * (DS * 2) + 512 + 16 * lane);
           const unsigned vp = *reinterpret_cast<const unsigned*>(t_pos + (size_t)i * (DP * 2) + 4 * lane);
           const unsigned w[9] = {v0.x, v0.y, v0.z, v0.w, v1.x, v1.y, v1.z, v1.w, vp};
-          double acc0 = 0.0, acc1 = 0.0;
+          float acc0 = 0.f, acc1 = 0.f, abs0 = 0.f, abs1 = 0.f;
 #pragma unroll
           for (int k = 0; k < 9; ++k) {
-            acc0 = fma(q[2 * k], (double)__uint_as_float(w[k] << 16), acc0);
-            acc1 = fma(q[2 * k + 1], (double)__uint_as_float(w[k] & 0xffff0000u), acc1);
+            const float lo = __uint_as_float(w[k] << 16), hi = __uint_as_float(w[k] & 0xffff0000u);
+            acc0 = fmaf(q[2 * k], lo, acc0);
+            acc1 = fmaf(q[2 * k + 1], hi, acc1);
+            abs0 = fmaf(fabsf(q[2 * k]), fabsf(lo), abs0);        // |.| is an operand modifier of the multiply-add
+            abs1 = fmaf(fabsf(q[2 * k + 1]), fabsf(hi), abs1);
           }
-          part[tt] = acc0 + acc1;
+          v[tt] = acc0 + acc1;
+          v[4 + tt] = abs0 + abs1;
         }
-        const bool up16 = (lane & 16) != 0, up8 = (lane & 8) != 0;
-        const double k0 = up16 ? part[2] : part[0], k1 = up16 ? part[3] : part[1];
-        const double g0 = up16 ? part[0] : part[2], g1 = up16 ? part[1] : part[3];
-        const double b0 = k0 + __shfl_xor_sync(0xffffffffu, g0, 16);
-        const double b1 = k1 + __shfl_xor_sync(0xffffffffu, g1, 16);
-        double c = (up8 ? b1 : b0) + __shfl_xor_sync(0xffffffffu, up8 ? b0 : b1, 8);
-        c += __shfl_xor_sync(0xffffffffu, c, 4);
+        const bool up16 = (lane & 16) != 0, up8 = (lane & 8) != 0, up4 = (lane & 4) != 0;
+        float r[4], t2[2];
+#pragma unroll
+        for (int i = 0; i < 4; ++i) r[i] = (up16 ? v[4 + i] : v[i]) + __shfl_xor_sync(0xffffffffu, up16 ? v[i] : v[4 + i], 16);
+#pragma unroll
+        for (int i = 0; i < 2; ++i) t2[i] = (up8 ? r[2 + i] : r[i]) + __shfl_xor_sync(0xffffffffu, up8 ? r[i] : r[2 + i], 8);
+        float c = (up4 ? t2[1] : t2[0]) + __shfl_xor_sync(0xffffffffu, up4 ? t2[0] : t2[1], 4);
         c += __shfl_xor_sync(0xffffffffu, c, 2);
         c += __shfl_xor_sync(0xffffffffu, c, 1);
-        if ((lane & 7) == 0) s_s[p * G + warp + SCORE_WARPS * (lane >> 3)] = c * a.scale;
+        // lane bit 4: products (0) or absolute sums (1); bits 3, 2: which of the warp's four tokens
+        if ((lane & 3) == 0) (up16 ? s_abs : s_s32)[p * G + warp + SCORE_WARPS * ((lane >> 2) & 3)] = c;
       }
       // one thread samples the abort flag before the barrier, so that all score warps leave in
       // the same iteration (a warp whose own wait expired skips the work and is caught next time)
       if (tid == 0) s_stop[p] = *s_abort;
       asm volatile("bar.sync 1, 512;" ::: "memory");
       if (s_stop[p]) break;
-      if (warp == 0) {
-        const double sa = s_s[p * G + lane], sb = s_s[p * G + lane + 32];
-        double best = sa; int besti = lane;
-        if (sb > best) { best = sb; besti = lane + 32; }
+      // every warp takes the same decision from the same numbers: largest and second largest product
+      // (a repeated maximum counts twice) and the largest absolute sum of the group
+      bool exact = exact_all;
+      float m1 = 0.f;
+      int i1 = 0;
+      if (!exact_all) {
+        const float sa = s_s32[p * G + lane], sb = s_s32[p * G + lane + 32];
+        float m2;
+        if (sb > sa) { m1 = sb; i1 = lane + 32; m2 = sa; } else { m1 = sa; i1 = lane; m2 = sb; }
+        float am = fmaxf(s_abs[p * G + lane], s_abs[p * G + lane + 32]);
 #pragma unroll
         for (int o = 16; o > 0; o >>= 1) {
-          const double ob = __shfl_xor_sync(0xffffffffu, best, o);
-          const int oi = __shfl_xor_sync(0xffffffffu, besti, o);
-          if (ob > best || (ob == best && oi < besti)) { best = ob; besti = oi; }
+          const float om1 = __shfl_xor_sync(0xffffffffu, m1, o), om2 = __shfl_xor_sync(0xffffffffu, m2, o);
+          const int oi = __shfl_xor_sync(0xffffffffu, i1, o);
+          am = fmaxf(am, __shfl_xor_sync(0xffffffffu, am, o));
+          m2 = fmaxf(fminf(m1, om1), fmaxf(m2, om2));
+          if (om1 > m1 || (om1 == m1 && oi < i1)) { m1 = om1; i1 = oi; }
         }
-        const float ea = expf((float)(sa - best)), eb = expf((float)(sb - best));
+        exact = !(m1 - m2 > MARGIN_FACTOR * am);          // also taken when a value is not finite
+      }
+      if (exact) {
+        score_tokens_fp64(t_sem, t_pos, s_q, s_s + p * G, warp, lane, a.scale);
+        asm volatile("bar.sync 1, 512;" ::: "memory");    // uniform: every score warp took the same decision
+      }
+      if (warp == 0) {
+        float ea, eb;
+        int besti;
+        if (exact) {
+          const double sa = s_s[p * G + lane], sb = s_s[p * G + lane + 32];
+          double best = sa; besti = lane;
+          if (sb > best) { best = sb; besti = lane + 32; }
+#pragma unroll
+          for (int o = 16; o > 0; o >>= 1) {
+            const double ob = __shfl_xor_sync(0xffffffffu, best, o);
+            const int oi = __shfl_xor_sync(0xffffffffu, besti, o);
+            if (ob > best || (ob == best && oi < besti)) { best = ob; besti = oi; }
+          }
+          ea = expf((float)(sa - best)); eb = expf((float)(sb - best));
+        } else {
+          besti = i1;
+          ea = expf((s_s32[p * G + lane] - m1) * scale32); eb = expf((s_s32[p * G + lane + 32] - m1) * scale32);
+        }
         const float inv = 1.f / warp_sum(ea + eb);
         s_a[p * G + lane] = ea * inv; s_a[p * G + lane + 32] = eb * inv;
         if (lane == 0) s_anchor[p] = besti;

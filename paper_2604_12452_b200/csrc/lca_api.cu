@@ -217,6 +217,15 @@ int lca_decode_update(const lca_params* p, const void* q_tail_sem, const void* q
                        cache_row_capacity, n_rep, cache_rows, anchor_out, ws, (cudaStream_t)stream);
 }
 
+int lca_latent_to_value(const void* attn_latent, const void* w_uv, void* out_v, int64_t n_tokens,
+                        int32_t n_heads, int32_t d_latent, int32_t d_v, void* stream) {
+  if (n_tokens < 0 || n_heads <= 0 || d_latent <= 0 || d_v <= 0) return LCA_ERR_INVALID_ARG;
+  if (n_tokens == 0) return LCA_OK;
+  if (!attn_latent || !w_uv || !out_v) return LCA_ERR_INVALID_ARG;
+  if (!aligned16(attn_latent) || !aligned16(w_uv) || !aligned16(out_v)) return LCA_ERR_MISALIGNED;
+  return latent_to_value_launch(attn_latent, w_uv, out_v, n_tokens, n_heads, d_latent, d_v, (cudaStream_t)stream);
+}
+
 int lca_selftest_bounded_wait(int64_t limit_cycles, void* stream) {
   if (limit_cycles < 1 || limit_cycles > 100000000ll) return LCA_ERR_INVALID_ARG;     // at most ~50 ms
   return bounded_wait_selftest_launch((long long)limit_cycles, (cudaStream_t)stream);
@@ -224,9 +233,9 @@ int lca_selftest_bounded_wait(int64_t limit_cycles, void* stream) {
 
 int lca_last_device_status(void* stream) {
   const int st = attn_tc_device_status((cudaStream_t)stream);      // synchronises the stream
-  const int cst = condense_take_status();
-  if (cst < 0) return LCA_ERR_CUDA;
-  if (cst > 0) return LCA_ERR_DEVICE_TIMEOUT;
+  const int cst = condense_take_status(), ust = latent_to_value_take_status();
+  if (cst < 0 || ust < 0) return LCA_ERR_CUDA;
+  if (cst > 0 || ust > 0) return LCA_ERR_DEVICE_TIMEOUT;
   return st;
 }
 

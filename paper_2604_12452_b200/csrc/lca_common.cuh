@@ -86,5 +86,8 @@ size_t attn_tc_workspace_bytes(const AttnProblem& a);
 int attn_tc_launch(const AttnProblem& a);
 int attn_tc_device_status(cudaStream_t stream);
 int bounded_wait_selftest_launch(long long limit_cycles, cudaStream_t stream);
+int latent_to_value_launch(const void* latent, const void* w_uv, void* out, long long n_tokens, int n_heads,
+                           int d_latent, int d_v, cudaStream_t stream);
+int latent_to_value_take_status();
 
 }  // namespace lca

@@ -12,15 +12,15 @@ from oracle import lca_oracle as O
 from oracle import parity as P
 
 # Outputs (bf16 inputs, bf16 tensor-core products, fp32 accumulation and softmax, bf16 result):
-#   every element   |err| <= max(ATOL, RTOL * |ref|)
+#   every element   |err| <= max(ATOL, derived bound)      (oracle/parity.py: output_bound)
 #   the mean        mean|err| <= max(MEAN_ATOL, MEAN_RTOL * mean|ref|)
-# ATOL / MEAN_ATOL are the bounds stated for outputs of unit scale.  The relative arms only take
-# over where the stored result cannot do better: above |ref| = 2.56 one bf16 ulp of the output
-# (2^-7 relative at the bottom of a binade) exceeds ATOL (rows locked onto a x4 "needle" token
-# reach |out| ~ 16, ulp 0.125), and the rounding of the stored output alone has a mean of about
-# 0.7 * 2^-9 of the mean magnitude.
+# ATOL / MEAN_ATOL are the bounds stated for the method (values of unit scale); elements of unit scale
+# (|ref| <= 1.5 and every value of their column within 5) must meet ATOL as it stands.  The derived bound follows
+# the arithmetic -- bf16 weights, normaliser over the rounded weights, bf16 store:
+# 2^-9 (vmax_c + |ref|) + 2^-8 |ref| -- and only exceeds ATOL where the values or the result are large
+# (rows that attend to a x4 needle token reach |out| ~ 16, one bf16 ulp = 0.125).  The rounding of the
+# stored output alone has a mean of about 0.7 * 2^-9 of the mean magnitude.
 ATOL = 2e-2
-RTOL = 2.0 ** -7
 MEAN_ATOL = 2e-3
 MEAN_RTOL = 2.0 ** -9
 
@@ -66,15 +66,19 @@ def bits_t(t: torch.Tensor) -> torch.Tensor:
     return t.contiguous().view(torch.int16)
 
 
-def check_outputs(got: torch.Tensor, ref: np.ndarray, what: str = ""):
+def check_outputs(got: torch.Tensor, ref, what: str = "", vmax=None):
     """Apply the output gate stated at the top of this file; returns the raw statistics (and appends
-    them to the file named by LCA_PARITY_LOG, if set, before any assertion)."""
-    st = P.output_stats(got, ref)
+    them to the file named by LCA_PARITY_LOG, if set, before any assertion).  `ref` is the oracle's
+    output array, or the dict of an oracle pipeline (its "out" and "vmax" are used)."""
+    if isinstance(ref, dict):
+        ref, vmax = ref["out"], ref["vmax"][None] if vmax is None else vmax
+    st = P.output_stats(got, ref, vmax)
     if os.environ.get("LCA_PARITY_LOG"):
         with open(os.environ["LCA_PARITY_LOG"], "a") as f:
             f.write(json.dumps(dict(what=what, **st)) + "\n")
     assert st["finite"], f"{what}: non-finite output"
-    assert st["worst_over_ulp_bound"] <= 1.0, f"{what}: {st}"
+    assert st["max_abs_unit_scale"] <= ATOL, f"{what}: {st}"
+    assert st["worst_over_bound"] <= 1.0, f"{what}: {st}"
     assert st["mean_abs"] <= max(MEAN_ATOL, MEAN_RTOL * st["mean_ref"]), f"{what}: {st}"
     return st
 

@@ -283,8 +283,23 @@ def test_absorbed_form_equals_unabsorbed_form():
                 vs.append(C[i] @ WUV[h])
             qh = np.concatenate([q_nope[p, h], q_rope[p, h]])
             ref = np_softmax(np.array(ks) @ qh * scale) @ np.array(vs)
-            np.testing.assert_allclose(out_lat[p, h] @ WUV[h], ref, atol=1e-11)
+            np.testing.assert_allclose(O.latent_to_value(out_lat[p], WUV)[h], ref, atol=1e-11)
     assert m == (L - w) // g
+
+
+def test_latent_to_value_is_one_matrix_product_per_head():
+    # explicit loops, non-square shapes and heads that differ: a transposed W^UV, a shared head or a wrong
+    # contraction axis cannot pass
+    rng = RNG(44)
+    T, H, dc, dv = 3, 2, 5, 4
+    x = rng.standard_normal((T, H, dc))
+    W = rng.standard_normal((H, dc, dv)) * np.array([1.0, -3.0])[:, None, None]
+    got = O.latent_to_value(x, W)
+    assert got.shape == (T, H, dv)
+    for t in range(T):
+        for h in range(H):
+            for v in range(dv):
+                assert abs(got[t, h, v] - sum(x[t, h, c] * W[h, c, v] for c in range(dc))) < 1e-13
 
 
 def test_decode_equals_prefill_row_of_longer_sequence():

@@ -79,7 +79,7 @@ def test_mla_small_cases_match_oracle_on_every_row(B, L, H, g, w, ns):
     if ref["cond"]["m"]:
         sc = cond["scores"][0, 0].cpu().numpy()
         np.testing.assert_allclose(sc, ref["cond"]["scores"], rtol=0, atol=1e-12)
-    Hh.check_outputs(out[0], ref["out"], f"mla L={L} H={H} g={g} w={w}")
+    Hh.check_outputs(out[0], ref, f"mla L={L} H={H} g={g} w={w}")
     np.testing.assert_allclose(lse[0].cpu().numpy(), ref["lse"], atol=2e-3, rtol=1e-4)
 
 
@@ -92,7 +92,7 @@ def test_mla_stress_peaky_queries_and_exact_ties(B):
     alpha = ref["cond"]["alpha"].reshape(-1, cfg.group_size)
     assert alpha.max() > 0.5
     Hh.check_condense(one_seq(cond), ref["cond"])
-    Hh.check_outputs(out[0], ref["out"], "mla stress")
+    Hh.check_outputs(out[0], ref, "mla stress")
 
 
 def test_mla_zero_queries_give_mean_pooling(B):
@@ -105,7 +105,7 @@ def test_mla_zero_queries_give_mean_pooling(B):
     m = ref["cond"]["m"]
     assert np.array_equal(ref["cond"]["anchor"], np.arange(m) * cfg.group_size)
     Hh.check_condense(one_seq(cond), ref["cond"])
-    Hh.check_outputs(out[0], ref["out"], "mla q=0")
+    Hh.check_outputs(out[0], ref, "mla q=0")
 
 
 def test_mla_rep_logit_bias_and_supplied_summary_query(B):
@@ -120,7 +120,7 @@ def test_mla_rep_logit_bias_and_supplied_summary_query(B):
     ref = Hh.oracle_mla(inp, cfg.group_size, cfg.window, cfg.softmax_scale, rows=np.arange(cfg.seq_len),
                         rep_logit_bias=bias, qbar=qbar32[0, 0].double().numpy())
     Hh.check_condense(one_seq(cond), ref["cond"])
-    Hh.check_outputs(out[0], ref["out"], "mla bias=ln g")
+    Hh.check_outputs(out[0], ref, "mla bias=ln g")
 
 
 def test_mla_batched_sequences_are_independent(B):
@@ -148,7 +148,7 @@ def test_mla_batched_sequences_are_independent(B):
         for key in ("cache_sem", "cache_pos", "anchor_idx"):
             r[key] = cond[key][b]
         Hh.check_condense(r, ref["cond"])
-        Hh.check_outputs(out[b], ref["out"], f"batch {b}")
+        Hh.check_outputs(out[b], ref, f"batch {b}")
 
 
 @pytest.mark.parametrize("H", [1, 2, 8, 32, 64, 256])
@@ -161,7 +161,7 @@ def test_mla_head_counts_of_the_pair_kernel(B, H):
     p, cond, out, lse = run_mla(B, cfg, to_dev(inp), impl=2, want_scores=False)
     ref = Hh.oracle_mla(inp, g, w, cfg.softmax_scale, rows=np.arange(L))
     Hh.check_condense(one_seq(cond), ref["cond"])
-    Hh.check_outputs(out[0], ref["out"], f"mla H={H}")
+    Hh.check_outputs(out[0], ref, f"mla H={H}")
     np.testing.assert_allclose(lse[0].cpu().numpy(), ref["lse"], atol=2e-3, rtol=1e-4)
     assert B.lca_last_device_status() == 0
 
@@ -183,7 +183,7 @@ def test_gqa_small_cases_match_oracle_on_every_row(B, L, Hq, Hkv, g, w):
     assert B.lca_last_device_status() == 0
     ref = Hh.oracle_gqa(inp, g, w, cfg.softmax_scale, rows=np.arange(L))
     Hh.check_condense(one_seq(cond), ref["cond"], kind="gqa")
-    Hh.check_outputs(out[0], ref["out"], f"gqa L={L}")
+    Hh.check_outputs(out[0], ref, f"gqa L={L}")
     np.testing.assert_allclose(lse[0].cpu().numpy(), ref["lse"], atol=2e-3, rtol=1e-4)
 
 
@@ -266,7 +266,7 @@ def test_mla_many_query_tiles_per_cta_pair(B):
     rows = np.unique(np.concatenate([np.arange(0, L, 13), np.arange(0, 40), np.arange(L - 160, L)]))
     ref = Hh.oracle_mla(inp, cfg.group_size, cfg.window, cfg.softmax_scale, rows=rows)
     Hh.check_condense(one_seq(cond), ref["cond"])
-    Hh.check_outputs(out[0][torch.from_numpy(rows).to(DEV)], ref["out"], "mla many items per pair")
+    Hh.check_outputs(out[0][torch.from_numpy(rows).to(DEV)], ref, "mla many items per pair")
     np.testing.assert_allclose(lse[0].cpu().numpy()[rows], ref["lse"], atol=2e-3, rtol=1e-4)
     assert B.lca_last_device_status() == 0
 
@@ -310,7 +310,7 @@ def test_dense_window_is_plain_causal_attention(B):
     p, cond, out, _ = run_mla(B, cfg, to_dev(inp))
     assert cond["m"] == 0 and cond["k"] == 600
     ref = Hh.oracle_mla(inp, cfg.group_size, cfg.window, cfg.softmax_scale, rows=np.arange(600))
-    Hh.check_outputs(out[0], ref["out"], "dense")
+    Hh.check_outputs(out[0], ref, "dense")
 
 
 def test_launches_are_counted(B):
@@ -517,4 +517,69 @@ def test_a_bounded_device_wait_that_expires_is_reported_and_harmless(B):
     p, cond, out, _ = run_mla(B, cfg, to_dev(inp), want_scores=False)
     assert B.lca_last_device_status() == 0
     ref = Hh.oracle_mla(inp, cfg.group_size, cfg.window, cfg.softmax_scale, rows=np.arange(cfg.seq_len))
-    Hh.check_outputs(out[0], ref["out"], "after an expired wait")
+    Hh.check_outputs(out[0], ref, "after an expired wait")
+
+
+@pytest.mark.parametrize("T,H", [(300, 16), (128, 1), (1, 128), (1000, 3)])
+def test_latent_to_value_matches_oracle(B, T, H):
+    # out_v[t, h] = latent[t, h] W^UV[h]: several token tiles and a ragged last one, one head to many;
+    # bf16 products, fp32 sums of 512 terms, one rounding of the result
+    gen = torch.Generator().manual_seed(1000 + T)
+    x = torch.randn((T, H, 512), generator=gen).bfloat16()
+    W = (torch.randn((H, 512, 128), generator=gen) / 512 ** 0.5).bfloat16()
+    W[H // 2] *= -2.0
+    got = B.latent_to_value(x.to(DEV), W.to(DEV))
+    torch.cuda.synchronize()
+    assert B.lca_last_device_status() == 0
+    ref = O.latent_to_value(O.torch_bf16_to_f64(x), O.torch_bf16_to_f64(W))
+    ulp = Hh.bf16_ulp_distance(Hh.bits(got), O.round_bf16_bits(ref))
+    err = np.abs(got.float().cpu().numpy().astype(np.float64) - ref)
+    # fp32 accumulation of 512 terms: absolute error <= 512 * 2^-24 * sum |x||w| (~1e-4 here), else one bf16 ulp
+    assert ((ulp <= 1) | (err <= 2e-4)).all(), f"max ulp {ulp.max()}, max err {err.max()}"
+    assert (ulp > 0).mean() < 0.02
+
+
+def test_absorbed_attention_plus_value_projection_equals_unabsorbed_attention(B):
+    # Alg. 1 builds k_rep = [c_rep W^UK, k^R_I] and v_rep = c_rep W^UV; the library works in the latent space with
+    # q_latent = q_nope W^UK^T and applies W^UV to the attention result.  Against a numpy restatement of the
+    # un-absorbed form on the same bf16 inputs (the representatives taken from the device cache).
+    rng = np.random.default_rng(77)
+    L, H, g, w, dn = 300, 16, 16, 40, 128
+    scale = 1.0 / (dn + 64) ** 0.5
+    cfg = I.scaled(I.CONFIGS["mla_1k"], seq_len=L, n_q_heads=H, group_size=g, window=w, n_needles=0, softmax_scale=scale)
+    inp = I.make_mla_inputs(cfg, "cpu")
+    WUK = torch.from_numpy(rng.standard_normal((H, 512, dn)) / 512 ** 0.5).bfloat16()
+    WUV = torch.from_numpy(rng.standard_normal((H, 512, 128)) / 512 ** 0.5).bfloat16()
+    q_nope = torch.from_numpy(rng.standard_normal((L, H, dn))).bfloat16()
+    q_lat = torch.einsum("lhn,hcn->lhc", q_nope.float(), WUK.float()).bfloat16()        # absorbed query, as the model would feed it
+    inp["q_sem"] = q_lat
+    d = to_dev(inp)
+    p = B.params_from_config(cfg, batch=1)
+    cond = B.condense(p, d["q_sem"][L - g:], d["q_pos"][L - g:], d["ckv"], d["kr"])
+    out, _ = B.prefill_attention(p, d["q_sem"], d["q_pos"], d["ckv"], d["kr"], cond["cache_sem"], cond["cache_pos"])
+    out_v = B.latent_to_value(out, WUV.to(DEV))
+    torch.cuda.synchronize()
+    assert B.lca_last_device_status() == 0
+    m = cond["m"]
+    C, KR = O.torch_bf16_to_f64(inp["ckv"]), O.torch_bf16_to_f64(inp["kr"])
+    c_rep = O.bits_to_f64(Hh.bits(cond["cache_sem"][0, :m, 0]))
+    kr_rep = O.bits_to_f64(Hh.bits(cond["cache_pos"][0, :m, 0]))
+    wuk, wuv = O.torch_bf16_to_f64(WUK), O.torch_bf16_to_f64(WUV)
+    qn, qr = O.torch_bf16_to_f64(q_nope), O.torch_bf16_to_f64(inp["q_pos"])
+    rows = [0, 5, w + g - 2, w + g - 1, w + g, 150, L - 1]
+    ref = np.zeros((len(rows), H, 128))
+    for x, t in enumerate(rows):
+        mt = 0 if t + 1 < w + g else (t + 1 - w) // g
+        sem = np.concatenate([c_rep[:mt], C[mt * g:t + 1]], 0)          # representatives, then the tokens after them
+        pos = np.concatenate([kr_rep[:mt], KR[mt * g:t + 1]], 0)
+        for h in range(H):
+            keys = np.concatenate([sem @ wuk[h], pos], 1)               # k = [c W^UK, k^R]   (un-absorbed, per head)
+            vals = sem @ wuv[h]                                         # v = c W^UV
+            lg = keys @ np.concatenate([qn[t, h], qr[t, h]]) * Hh.f32(scale)
+            e = np.exp(lg - lg.max())
+            ref[x, h] = (e / e.sum()) @ vals
+    got = out_v[0][torch.tensor(rows, device=DEV)]
+    # the device saw q_latent rounded to bf16 (logits shift by ~3e-3), then two bf16 roundings (latent output,
+    # projected output) on values of unit scale
+    st = Hh.check_outputs(got, ref, "absorbed attention + W^UV vs un-absorbed attention")
+    assert st["max_abs"] < 2e-2
