@@ -87,6 +87,8 @@ def _ptr(x):
     if x is None:
         return None
     if isinstance(x, torch.Tensor):
+        if not x.is_contiguous():
+            raise ValueError("the LCA entry points take dense row-major tensors: call .contiguous() first")
         return C.c_void_p(x.data_ptr())
     return C.c_void_p(int(x))
 

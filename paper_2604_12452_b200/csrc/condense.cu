@@ -38,17 +38,29 @@ __global__ void qbar_partial_kernel(const bf16* __restrict__ q_sem, const bf16* 
 #pragma unroll
   for (int i = 0; i < 8; ++i) acc[i] = 0.0;
   if (rl < row_lanes) {
-#pragma unroll 8
-    for (int r = r0 + rl; r < r1; r += row_lanes) {
-      const int pos = r / rep, head = hk * rep + r % rep;
-      const size_t row = ((size_t)b * batch_stride_rows + pos) * Hq + head;
-      const bf16* src = (pc < sem_pieces) ? q_sem + row * d_sem + 8 * pc : q_pos + row * d_pos + 8 * (pc - sem_pieces);
-      const uint4 v = *reinterpret_cast<const uint4*>(src);
-      const unsigned w[4] = {v.x, v.y, v.z, v.w};
+    // eight rows per step: all eight loads are issued before the first one is used (the kernel is bound by memory
+    // latency otherwise); rows behind the end of the chunk contribute exact zeros, the order of the sums is fixed
+    for (int r = r0 + rl; r < r1; r += 8 * row_lanes) {
+      uint4 v[8];
 #pragma unroll
-      for (int i = 0; i < 4; ++i) {
-        acc[2 * i] += (double)__uint_as_float(w[i] << 16);
-        acc[2 * i + 1] += (double)__uint_as_float(w[i] & 0xffff0000u);
+      for (int u = 0; u < 8; ++u) {
+        const int rr = r + u * row_lanes;
+        v[u] = make_uint4(0u, 0u, 0u, 0u);
+        if (rr < r1) {
+          const int pos = rr / rep, head = hk * rep + rr % rep;
+          const size_t row = ((size_t)b * batch_stride_rows + pos) * Hq + head;
+          const bf16* src = (pc < sem_pieces) ? q_sem + row * d_sem + 8 * pc : q_pos + row * d_pos + 8 * (pc - sem_pieces);
+          v[u] = *reinterpret_cast<const uint4*>(src);
+        }
+      }
+#pragma unroll
+      for (int u = 0; u < 8; ++u) {
+        const unsigned w[4] = {v[u].x, v[u].y, v[u].z, v[u].w};
+#pragma unroll
+        for (int i = 0; i < 4; ++i) {
+          acc[2 * i] += (double)__uint_as_float(w[i] << 16);
+          acc[2 * i + 1] += (double)__uint_as_float(w[i] & 0xffff0000u);
+        }
       }
     }
 #pragma unroll
@@ -247,38 +259,39 @@ condense_kernel(CondenseArgs a) {
 }
 
 // ----------------------------------------------------- condense, MLA shape with g = 64 (the fast path)
-// Same arithmetic as condense_kernel for d_sem = 512, d_pos = 64, g = 64 and one KV stream, laid
-// out for the instruction budget HBM speed leaves (about 3000 cycles per group and SM).  The
-// float-to-double conversions of the scores (one per key element, on the slow conversion unit)
-// take most of that budget, so nothing else may wait for them: the CTA is split into roles that
-// work on different groups at the same time.
-//   * one producer thread fetches a group (64 KB + 8 KB of contiguous memory) with two bulk
-//     copies (cp.async.bulk) into one of three stages, completion on an mbarrier per stage;
-//   * sixteen score warps: warp w takes tokens w, w+16, ...; lane l holds the 18 components of q_bar
-//     it needs in registers (columns 8l..8l+7 and 256+8l..256+8l+7 of the latent part, 2l, 2l+1
-//     of the rope part) and reads its share of a token with two 16-byte and one 4-byte load;
-//     fp64 multiply-adds, warp-shuffle reduction; warp 0 then takes the arg-max and the softmax;
-//   * four pool warps, one group behind: four output columns per thread, fp32, alpha read four
-//     tokens at a time; they also copy the anchor's rope row and write index and scores.
+// Same results as condense_kernel for d_sem = 512, d_pos = 64, g = 64 and one KV stream, laid out for the
+// instruction budget HBM speed leaves (about 3000 issue cycles per group and SM, for 73 KB of input).  The
+// CTA is split into roles that work on different groups at the same time and meet only through mbarriers:
+//   * one producer thread fetches a group (64 KB + 8 KB of contiguous memory) with two bulk copies
+//     (cp.async.bulk) into one of three stages;
+//   * sixteen score warps: warp w takes tokens w, w+16, w+32, w+48; lane l holds the 18 components of q_bar
+//     it needs in registers (columns 8l..8l+7 and 256+8l..256+8l+7 of the latent part, 2l, 2l+1 of the rope
+//     part) as fp32, reads its share of a token with two 16-byte and one 4-byte load, and forms the product
+//     sum in fp32 together with max_c |k_ic|; one transposed shuffle reduction per four tokens;
+//   * one arbiter warp takes the group's arg-max and softmax from those 64 sums.  An fp32 sum of this kernel
+//     passes through at most 15 roundings (9 multiply-adds per chain, the chain pair, 5 shuffle levels) and
+//     q_bar is rounded once to fp32, so |s32_i - s_i| <= 16 u (1 + 16 u) sum_c |q_c| |k_ic| <= 16 u (1 + 16 u)
+//     |q_bar|_1 max_c |k_ic| with u = 2^-24.  Where the two largest sums of a group are further apart than
+//     MARGIN_FACTOR |q_bar|_1 max_ic |k_ic| (twice that bound with a quarter of slack and the rounding of |q_bar|_1
+//     and of the difference), the fp32 arg-max is the arg-max of the exact scores.  Every other group (about one
+//     in a thousand; exact ties included) is scored again by the arbiter warp in fp64, and so is every group when
+//     the caller asked for the scores: anchors always follow the fp64 scores, lowest index on ties;
+//   * four pool warps, one group behind: four output columns per thread, fp32 pairs, alpha read four tokens at
+//     a time; they also copy the anchor's rope row and write the anchor index.
 namespace fast {
 constexpr int G = 64, DS = 512, DP = 64, DK = DS + DP, STAGES = 3;
-constexpr int SCORE_WARPS = 16, POOL_WARPS = 4, THREADS = 32 * (SCORE_WARPS + POOL_WARPS + 1);
+constexpr int SCORE_WARPS = 16, POOL_WARPS = 4;
+constexpr int WARP_ARBITER = SCORE_WARPS, WARP_POOL0 = SCORE_WARPS + 1, WARP_PRODUCER = WARP_POOL0 + POOL_WARPS;
+constexpr int THREADS = 32 * (WARP_PRODUCER + 1);
 constexpr int SEM_BYTES = G * DS * 2, POS_BYTES = G * DP * 2, STAGE_BYTES = SEM_BYTES + POS_BYTES;
-constexpr int OFF_Q = STAGES * STAGE_BYTES;                 // double[DK]
-constexpr int OFF_S = OFF_Q + DK * 8;                       // double[2][G] scores
-constexpr int OFF_A = OFF_S + 2 * G * 8;                    // float[2][G] alpha
-constexpr int OFF_S32 = OFF_A + 2 * G * 4;                  // float[2][G] fp32 products q_bar . k_i (before the scale)
-constexpr int OFF_ABS = OFF_S32 + 2 * G * 4;                // float[2][G] sum_c |q_bar_c| |k_ic|: scale of their rounding error
-constexpr int OFF_BAR = OFF_ABS + 2 * G * 4;                // mbarriers: full[3] free[3] ready[2] afree[2], then flags
+constexpr int OFF_A = STAGES * STAGE_BYTES;                 // float[2][G] alpha
+constexpr int OFF_S32 = OFF_A + 2 * G * 4;                  // float[2][G] fp32 sums q_bar . k_i (before the scale)
+constexpr int OFF_NRM = OFF_S32 + 2 * G * 4;                // float[2][G] max_c |k_ic|
+constexpr int OFF_BAR = OFF_NRM + 2 * G * 4;                // mbarriers: full[3] free[3] scored[2] ready[2] afree[2], then flags
 constexpr int SMEM_BYTES = OFF_BAR + 128;
-// An fp32 product sum of this kernel passes through at most 15 roundings (9 multiply-adds per chain, the
-// chain pair, 5 shuffle levels) and q_bar itself is rounded once to fp32: |s32_i - s_i| <= 16 u A_i (1 + 16 u),
-// u = 2^-24, A_i = sum_c |q_bar_c| |k_ic|, and the fp32 A_i is at least A_i (1 - 16 u).  A group whose two largest
-// fp32 products differ by more than 48 u max_i A_i (twice 20 u A: the bound with a quarter of slack, plus the
-// rounding of the difference) therefore has the same arg-max in exact arithmetic; any other group (exact ties
-// included) is scored again in fp64.
 constexpr float MARGIN_FACTOR = 48.0f * 5.9604644775390625e-08f;
 static_assert(SMEM_BYTES <= 232448, "shared memory budget of one SM");
+static_assert(G / SCORE_WARPS == 4, "four tokens per score warp");
 constexpr long long WAIT_CYCLES = 2000000000ll;
 }  // namespace fast
 
@@ -299,17 +312,32 @@ __device__ __forceinline__ bool cond_wait(unsigned bar, unsigned parity, volatil
 __device__ __forceinline__ void cond_arrive(unsigned bar) {
   asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar) : "memory");
 }
+__device__ __forceinline__ float f32_max3_abs(float acc, float a, float b) {     // max(acc, |a|, |b|)
+  return fmaxf(fmaxf(acc, fabsf(a)), fabsf(b));
+}
+__device__ __forceinline__ unsigned long long f32x2(float lo, float hi) {
+  unsigned long long r;
+  asm("mov.b64 %0, {%1, %2};" : "=l"(r) : "f"(lo), "f"(hi));
+  return r;
+}
+__device__ __forceinline__ unsigned long long fma_f32x2(unsigned long long a, unsigned long long b, unsigned long long c) {
+  unsigned long long r;
+  asm("fma.rn.f32x2 %0, %1, %2, %3;" : "=l"(r) : "l"(a), "l"(b), "l"(c));
+  return r;
+}
 
-// The exact scores of a score warp's four tokens (warp w: tokens w, w + 16, w + 32, w + 48) in fp64, q_bar read from
-// shared memory.  Kept out of line: it runs for the rare groups whose fp32 arg-max is not provably the exact one (and
-// for every group when the caller asked for the scores), and its registers should not weigh on the fp32 path.
-__device__ __noinline__ void score_tokens_fp64(const unsigned char* t_sem, const unsigned char* t_pos, const double* s_q,
-                                               double* s_out, int warp, int lane, double scale) {
+// The exact scores of one group by one warp (the arbiter), q_bar in fp64 from global memory: token by token,
+// lane l takes the same 18 columns as in the fp32 pass; every lane ends up with the scores of tokens l and l + 32.
+__device__ __noinline__ void score_group_fp64(const unsigned char* t_sem, const unsigned char* t_pos, const double* qbar,
+                                              int lane, double scale, double& s_lo, double& s_hi) {
   using namespace fast;
-  double part[4];
+  double q[18];
 #pragma unroll
-  for (int tt = 0; tt < 4; ++tt) {
-    const int i = warp + SCORE_WARPS * tt;
+  for (int i = 0; i < 8; ++i) { q[i] = qbar[8 * lane + i]; q[8 + i] = qbar[256 + 8 * lane + i]; }
+  q[16] = qbar[DS + 2 * lane]; q[17] = qbar[DS + 2 * lane + 1];
+  s_lo = 0.0; s_hi = 0.0;
+#pragma unroll 1
+  for (int i = 0; i < G; ++i) {
     const uint4 v0 = *reinterpret_cast<const uint4*>(t_sem + (size_t)i * (DS * 2) + 16 * lane);
     const uint4 v1 = *reinterpret_cast<const uint4*>(t_sem + (size_t)i * (DS * 2) + 512 + 16 * lane);
     const unsigned vp = *reinterpret_cast<const unsigned*>(t_pos + (size_t)i * (DP * 2) + 4 * lane);
@@ -317,42 +345,29 @@ __device__ __noinline__ void score_tokens_fp64(const unsigned char* t_sem, const
     double acc0 = 0.0, acc1 = 0.0;
 #pragma unroll
     for (int k = 0; k < 9; ++k) {
-      const int c0 = k < 4 ? 8 * lane + 2 * k : k < 8 ? 256 + 8 * lane + 2 * (k - 4) : DS + 2 * lane;
-      acc0 = fma(s_q[c0], (double)__uint_as_float(w[k] << 16), acc0);
-      acc1 = fma(s_q[c0 + 1], (double)__uint_as_float(w[k] & 0xffff0000u), acc1);
+      acc0 = fma(q[2 * k], (double)__uint_as_float(w[k] << 16), acc0);
+      acc1 = fma(q[2 * k + 1], (double)__uint_as_float(w[k] & 0xffff0000u), acc1);
     }
-    part[tt] = acc0 + acc1;
+    const double c = warp_sum(acc0 + acc1) * scale;       // the same value in every lane (xor butterfly)
+    if ((i & 31) == lane) { if (i < 32) s_lo = c; else s_hi = c; }
   }
-  // transposed reduction: lanes 0, 8, 16, 24 end up with the sums of tokens 0..3
-  const bool up16 = (lane & 16) != 0, up8 = (lane & 8) != 0;
-  const double k0 = up16 ? part[2] : part[0], k1 = up16 ? part[3] : part[1];
-  const double g0 = up16 ? part[0] : part[2], g1 = up16 ? part[1] : part[3];
-  const double b0 = k0 + __shfl_xor_sync(0xffffffffu, g0, 16);
-  const double b1 = k1 + __shfl_xor_sync(0xffffffffu, g1, 16);
-  double c = (up8 ? b1 : b0) + __shfl_xor_sync(0xffffffffu, up8 ? b0 : b1, 8);
-  c += __shfl_xor_sync(0xffffffffu, c, 4);
-  c += __shfl_xor_sync(0xffffffffu, c, 2);
-  c += __shfl_xor_sync(0xffffffffu, c, 1);
-  if ((lane & 7) == 0) s_out[warp + SCORE_WARPS * (lane >> 3)] = c * scale;
 }
 
 __global__ void __launch_bounds__(fast::THREADS, 1)
 condense_mla64_kernel(CondenseArgs a) {
   using namespace fast;
   extern __shared__ __align__(128) unsigned char smem[];
-  double* s_q = reinterpret_cast<double*>(smem + OFF_Q);
-  double* s_s = reinterpret_cast<double*>(smem + OFF_S);
   float* s_a = reinterpret_cast<float*>(smem + OFF_A);
   float* s_s32 = reinterpret_cast<float*>(smem + OFF_S32);
-  float* s_abs = reinterpret_cast<float*>(smem + OFF_ABS);
+  float* s_nrm = reinterpret_cast<float*>(smem + OFF_NRM);
   const unsigned bar0 = (unsigned)__cvta_generic_to_shared(smem + OFF_BAR);
   auto BAR_FULL = [&](int st) { return bar0 + 8 * st; };
   auto BAR_FREE = [&](int st) { return bar0 + 24 + 8 * st; };
-  auto BAR_READY = [&](int p) { return bar0 + 48 + 8 * p; };      // alpha / anchor of parity p written
-  auto BAR_AFREE = [&](int p) { return bar0 + 64 + 8 * p; };      // ... and consumed
-  volatile int* s_anchor = reinterpret_cast<volatile int*>(smem + OFF_BAR + 80);   // [2]
-  volatile int* s_abort = reinterpret_cast<volatile int*>(smem + OFF_BAR + 88);
-  volatile int* s_stop = reinterpret_cast<volatile int*>(smem + OFF_BAR + 96);     // [2]
+  auto BAR_SCORED = [&](int p) { return bar0 + 48 + 8 * p; };     // sums of parity p written by the score warps
+  auto BAR_READY = [&](int p) { return bar0 + 64 + 8 * p; };      // alpha / anchor of parity p written
+  auto BAR_AFREE = [&](int p) { return bar0 + 80 + 8 * p; };      // ... and consumed
+  volatile int* s_anchor = reinterpret_cast<volatile int*>(smem + OFF_BAR + 96);   // [2]
+  volatile int* s_abort = reinterpret_cast<volatile int*>(smem + OFF_BAR + 104);
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
 
   if (tid == 0) {
@@ -361,6 +376,7 @@ condense_mla64_kernel(CondenseArgs a) {
       asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(BAR_FREE(st)), "r"(POOL_WARPS) : "memory");
     }
     for (int p = 0; p < 2; ++p) {
+      asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(BAR_SCORED(p)), "r"(SCORE_WARPS) : "memory");
       asm volatile("mbarrier.init.shared::cta.b64 [%0], 1;" ::"r"(BAR_READY(p)) : "memory");
       asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(BAR_AFREE(p)), "r"(POOL_WARPS) : "memory");
     }
@@ -372,7 +388,7 @@ condense_mla64_kernel(CondenseArgs a) {
   const long long first = blockIdx.x, stride = gridDim.x;
   const long long n_mine = first < a.n_groups ? (a.n_groups - first + stride - 1) / stride : 0;
 
-  if (warp == SCORE_WARPS + POOL_WARPS) {
+  if (warp == WARP_PRODUCER) {
     // ===================================================== producer
     if (lane == 0) {
       for (long long it = 0; it < n_mine; ++it) {
@@ -392,125 +408,125 @@ condense_mla64_kernel(CondenseArgs a) {
       }
     }
   } else if (warp < SCORE_WARPS) {
-    // ===================================================== scores, arg-max, softmax
-    // The products q_bar . k_i are taken in fp32 together with A_i = sum |q_bar_c| |k_ic|.  Where the two largest
-    // products of a group are further apart than the rounding error A_i allows (MARGIN_FACTOR), the fp32 arg-max
-    // is the exact one; otherwise, and whenever the caller asked for the scores, the group is scored in fp64.
+    // ===================================================== fp32 product sums and max |k| of four tokens per warp
     float q[18];
-    const bool exact_all = a.scores != nullptr;
-    const float scale32 = (float)a.scale;
     long long cur_b = -1;
     for (long long it = 0; it < n_mine; ++it) {
       const int st = (int)(it % STAGES), p = (int)(it & 1);
       const long long grp = first + it * stride;
       const long long b = grp / a.m;
-      if (b != cur_b) {                                   // uniform over the score warps; rare
+      if (b != cur_b) {                                   // rare: the next sequence's summary query
         cur_b = b;
-        asm volatile("bar.sync 1, 512;" ::: "memory");    // nobody still reads the old q_bar
         const double* qb = a.qbar + (size_t)b * DK;
-        for (int x = tid; x < DK; x += 32 * SCORE_WARPS) s_q[x] = qb[x];
-        asm volatile("bar.sync 1, 512;" ::: "memory");
 #pragma unroll
-        for (int i = 0; i < 8; ++i) { q[i] = (float)s_q[8 * lane + i]; q[8 + i] = (float)s_q[256 + 8 * lane + i]; }
-        q[16] = (float)s_q[DS + 2 * lane]; q[17] = (float)s_q[DS + 2 * lane + 1];
+        for (int i = 0; i < 8; ++i) { q[i] = (float)qb[8 * lane + i]; q[8 + i] = (float)qb[256 + 8 * lane + i]; }
+        q[16] = (float)qb[DS + 2 * lane]; q[17] = (float)qb[DS + 2 * lane + 1];
       }
-      bool ok = cond_wait(BAR_FULL(st), (unsigned)((it / STAGES) & 1), s_abort);
-      if (ok && it >= 2) ok = cond_wait(BAR_AFREE(p), (unsigned)(((it >> 1) - 1) & 1), s_abort);
+      if (!cond_wait(BAR_FULL(st), (unsigned)((it / STAGES) & 1), s_abort)) break;
+      if (it >= 2 && !cond_wait(BAR_AFREE(p), (unsigned)(((it >> 1) - 1) & 1), s_abort)) break;
       const unsigned char* t_sem = smem + (size_t)st * STAGE_BYTES;
       const unsigned char* t_pos = t_sem + SEM_BYTES;
-      static_assert(G / SCORE_WARPS == 4, "four tokens per score warp");
-      if (ok && !exact_all) {
-        // the warp's four tokens together: 4 x 4 independent multiply-add chains, then one transposed
-        // reduction of the eight sums (lanes 0, 4, ... 28 end up with one of them each)
-        float v[8];
+      float v[8];                                         // sums of the four tokens, then their max |k|
 #pragma unroll
-        for (int tt = 0; tt < 4; ++tt) {
-          const int i = warp + SCORE_WARPS * tt;
-          const uint4 v0 = *reinterpret_cast<const uint4*>(t_sem + (size_t)i * (DS * 2) + 16 * lane);
-          const uint4 v1 = *reinterpret_cast<const uint4*>(t_sem + (size_t)i * (DS * 2) + 512 + 16 * lane);
-          const unsigned vp = *reinterpret_cast<const unsigned*>(t_pos + (size_t)i * (DP * 2) + 4 * lane);
-          const unsigned w[9] = {v0.x, v0.y, v0.z, v0.w, v1.x, v1.y, v1.z, v1.w, vp};
-          float acc0 = 0.f, acc1 = 0.f, abs0 = 0.f, abs1 = 0.f;
+      for (int tt = 0; tt < 4; ++tt) {
+        const int i = warp + SCORE_WARPS * tt;
+        const uint4 v0 = *reinterpret_cast<const uint4*>(t_sem + (size_t)i * (DS * 2) + 16 * lane);
+        const uint4 v1 = *reinterpret_cast<const uint4*>(t_sem + (size_t)i * (DS * 2) + 512 + 16 * lane);
+        const unsigned vp = *reinterpret_cast<const unsigned*>(t_pos + (size_t)i * (DP * 2) + 4 * lane);
+        const unsigned w[9] = {v0.x, v0.y, v0.z, v0.w, v1.x, v1.y, v1.z, v1.w, vp};
+        float acc0 = 0.f, acc1 = 0.f, kmax = 0.f;
 #pragma unroll
-          for (int k = 0; k < 9; ++k) {
-            const float lo = __uint_as_float(w[k] << 16), hi = __uint_as_float(w[k] & 0xffff0000u);
-            acc0 = fmaf(q[2 * k], lo, acc0);
-            acc1 = fmaf(q[2 * k + 1], hi, acc1);
-            abs0 = fmaf(fabsf(q[2 * k]), fabsf(lo), abs0);        // |.| is an operand modifier of the multiply-add
-            abs1 = fmaf(fabsf(q[2 * k + 1]), fabsf(hi), abs1);
-          }
-          v[tt] = acc0 + acc1;
-          v[4 + tt] = abs0 + abs1;
+        for (int k = 0; k < 9; ++k) {
+          const float lo = __uint_as_float(w[k] << 16), hi = __uint_as_float(w[k] & 0xffff0000u);
+          acc0 = fmaf(q[2 * k], lo, acc0);
+          acc1 = fmaf(q[2 * k + 1], hi, acc1);
+          kmax = f32_max3_abs(kmax, lo, hi);
         }
-        const bool up16 = (lane & 16) != 0, up8 = (lane & 8) != 0, up4 = (lane & 4) != 0;
-        float r[4], t2[2];
-#pragma unroll
-        for (int i = 0; i < 4; ++i) r[i] = (up16 ? v[4 + i] : v[i]) + __shfl_xor_sync(0xffffffffu, up16 ? v[i] : v[4 + i], 16);
-#pragma unroll
-        for (int i = 0; i < 2; ++i) t2[i] = (up8 ? r[2 + i] : r[i]) + __shfl_xor_sync(0xffffffffu, up8 ? r[i] : r[2 + i], 8);
-        float c = (up4 ? t2[1] : t2[0]) + __shfl_xor_sync(0xffffffffu, up4 ? t2[0] : t2[1], 4);
-        c += __shfl_xor_sync(0xffffffffu, c, 2);
-        c += __shfl_xor_sync(0xffffffffu, c, 1);
-        // lane bit 4: products (0) or absolute sums (1); bits 3, 2: which of the warp's four tokens
-        if ((lane & 3) == 0) (up16 ? s_abs : s_s32)[p * G + warp + SCORE_WARPS * ((lane >> 2) & 3)] = c;
+        v[tt] = acc0 + acc1;
+        v[4 + tt] = kmax;
       }
-      // one thread samples the abort flag before the barrier, so that all score warps leave in
-      // the same iteration (a warp whose own wait expired skips the work and is caught next time)
-      if (tid == 0) s_stop[p] = *s_abort;
-      asm volatile("bar.sync 1, 512;" ::: "memory");
-      if (s_stop[p]) break;
-      // every warp takes the same decision from the same numbers: largest and second largest product
-      // (a repeated maximum counts twice) and the largest absolute sum of the group
-      bool exact = exact_all;
-      float m1 = 0.f;
-      int i1 = 0;
-      if (!exact_all) {
-        const float sa = s_s32[p * G + lane], sb = s_s32[p * G + lane + 32];
-        float m2;
-        if (sb > sa) { m1 = sb; i1 = lane + 32; m2 = sa; } else { m1 = sa; i1 = lane; m2 = sb; }
-        float am = fmaxf(s_abs[p * G + lane], s_abs[p * G + lane + 32]);
+      // transposed reduction over the warp: lanes with bit 4 clear add up the sums, the others take the maxima;
+      // bits 3 and 2 select the token; lanes 0, 4, ..., 28 end up with one result each
+      const bool up16 = (lane & 16) != 0, up8 = (lane & 8) != 0, up4 = (lane & 4) != 0;
+      auto comb = [&](float x, float y) { return up16 ? fmaxf(x, y) : x + y; };
+      float r[4], t2[2];
+#pragma unroll
+      for (int i = 0; i < 4; ++i) r[i] = comb(up16 ? v[4 + i] : v[i], __shfl_xor_sync(0xffffffffu, up16 ? v[i] : v[4 + i], 16));
+#pragma unroll
+      for (int i = 0; i < 2; ++i) t2[i] = comb(up8 ? r[2 + i] : r[i], __shfl_xor_sync(0xffffffffu, up8 ? r[i] : r[2 + i], 8));
+      float c = comb(up4 ? t2[1] : t2[0], __shfl_xor_sync(0xffffffffu, up4 ? t2[0] : t2[1], 4));
+      c = comb(c, __shfl_xor_sync(0xffffffffu, c, 2));
+      c = comb(c, __shfl_xor_sync(0xffffffffu, c, 1));
+      if ((lane & 3) == 0) (up16 ? s_nrm : s_s32)[p * G + warp + SCORE_WARPS * ((lane >> 2) & 3)] = c;
+      __syncwarp();
+      if (lane == 0) cond_arrive(BAR_SCORED(p));
+    }
+  } else if (warp == WARP_ARBITER) {
+    // ===================================================== arg-max (fp32 where provably exact, else fp64) and softmax
+    const bool exact_all = a.scores != nullptr;
+    const float scale32 = (float)a.scale;
+    long long cur_b = -1;
+    float q_l1 = 0.f;                                     // |q_bar|_1 of the current sequence (fp32 values, fp32 sum)
+    for (long long it = 0; it < n_mine; ++it) {
+      const int st = (int)(it % STAGES), p = (int)(it & 1);
+      const long long grp = first + it * stride;
+      const int j = (int)(grp % a.m);
+      const long long b = grp / a.m;
+      const double* qb = a.qbar + (size_t)b * DK;
+      if (b != cur_b) {
+        cur_b = b;
+        float t = 0.f;
+        for (int x = lane; x < DK; x += 32) t += fabsf((float)qb[x]);
+        q_l1 = warp_sum(t);
+      }
+      if (!cond_wait(BAR_SCORED(p), (unsigned)((it >> 1) & 1), s_abort)) break;
+      const float sa = s_s32[p * G + lane], sb = s_s32[p * G + lane + 32];
+      float m1, m2;
+      int i1;
+      if (sb > sa) { m1 = sb; i1 = lane + 32; m2 = sa; } else { m1 = sa; i1 = lane; m2 = sb; }
+      float km = fmaxf(s_nrm[p * G + lane], s_nrm[p * G + lane + 32]);
+#pragma unroll
+      for (int o = 16; o > 0; o >>= 1) {
+        const float om1 = __shfl_xor_sync(0xffffffffu, m1, o), om2 = __shfl_xor_sync(0xffffffffu, m2, o);
+        const int oi = __shfl_xor_sync(0xffffffffu, i1, o);
+        km = fmaxf(km, __shfl_xor_sync(0xffffffffu, km, o));
+        m2 = fmaxf(fminf(m1, om1), fmaxf(m2, om2));       // a repeated maximum counts twice
+        if (om1 > m1 || (om1 == m1 && oi < i1)) { m1 = om1; i1 = oi; }
+      }
+      const bool exact = exact_all || !(m1 - m2 > MARGIN_FACTOR * q_l1 * km);   // also taken when a value is not finite
+      float ea, eb;
+      int besti;
+      if (exact) {
+        if (!cond_wait(BAR_FULL(st), (unsigned)((it / STAGES) & 1), s_abort)) break;    // complete; makes the tile visible here
+        const unsigned char* t_sem = smem + (size_t)st * STAGE_BYTES;
+        double da, db;
+        score_group_fp64(t_sem, t_sem + SEM_BYTES, qb, lane, a.scale, da, db);
+        double best = da; besti = lane;
+        if (db > best) { best = db; besti = lane + 32; }
 #pragma unroll
         for (int o = 16; o > 0; o >>= 1) {
-          const float om1 = __shfl_xor_sync(0xffffffffu, m1, o), om2 = __shfl_xor_sync(0xffffffffu, m2, o);
-          const int oi = __shfl_xor_sync(0xffffffffu, i1, o);
-          am = fmaxf(am, __shfl_xor_sync(0xffffffffu, am, o));
-          m2 = fmaxf(fminf(m1, om1), fmaxf(m2, om2));
-          if (om1 > m1 || (om1 == m1 && oi < i1)) { m1 = om1; i1 = oi; }
+          const double ob = __shfl_xor_sync(0xffffffffu, best, o);
+          const int oi = __shfl_xor_sync(0xffffffffu, besti, o);
+          if (ob > best || (ob == best && oi < besti)) { best = ob; besti = oi; }
         }
-        exact = !(m1 - m2 > MARGIN_FACTOR * am);          // also taken when a value is not finite
-      }
-      if (exact) {
-        score_tokens_fp64(t_sem, t_pos, s_q, s_s + p * G, warp, lane, a.scale);
-        asm volatile("bar.sync 1, 512;" ::: "memory");    // uniform: every score warp took the same decision
-      }
-      if (warp == 0) {
-        float ea, eb;
-        int besti;
-        if (exact) {
-          const double sa = s_s[p * G + lane], sb = s_s[p * G + lane + 32];
-          double best = sa; besti = lane;
-          if (sb > best) { best = sb; besti = lane + 32; }
-#pragma unroll
-          for (int o = 16; o > 0; o >>= 1) {
-            const double ob = __shfl_xor_sync(0xffffffffu, best, o);
-            const int oi = __shfl_xor_sync(0xffffffffu, besti, o);
-            if (ob > best || (ob == best && oi < besti)) { best = ob; besti = oi; }
-          }
-          ea = expf((float)(sa - best)); eb = expf((float)(sb - best));
-        } else {
-          besti = i1;
-          ea = expf((s_s32[p * G + lane] - m1) * scale32); eb = expf((s_s32[p * G + lane + 32] - m1) * scale32);
+        ea = expf((float)(da - best)); eb = expf((float)(db - best));
+        if (a.scores) {
+          double* sc = a.scores + ((size_t)b * a.m + j) * G;
+          sc[lane] = da; sc[lane + 32] = db;
         }
-        const float inv = 1.f / warp_sum(ea + eb);
-        s_a[p * G + lane] = ea * inv; s_a[p * G + lane + 32] = eb * inv;
-        if (lane == 0) s_anchor[p] = besti;
-        __syncwarp();
-        if (lane == 0) cond_arrive(BAR_READY(p));
+      } else {
+        besti = i1;
+        ea = expf((sa - m1) * scale32); eb = expf((sb - m1) * scale32);
       }
+      const float inv = 1.f / warp_sum(ea + eb);
+      s_a[p * G + lane] = ea * inv; s_a[p * G + lane + 32] = eb * inv;
+      if (lane == 0) s_anchor[p] = besti;
+      __syncwarp();
+      if (lane == 0) cond_arrive(BAR_READY(p));
     }
   } else {
     // ===================================================== pooling and outputs, one group behind
-    const int pt = tid - 32 * SCORE_WARPS;                // 0..127: output columns 4 pt .. 4 pt + 3
+    const int pt = tid - 32 * WARP_POOL0;                 // 0..127: output columns 4 pt .. 4 pt + 3
     for (long long it = 0; it < n_mine; ++it) {
       const int st = (int)(it % STAGES), p = (int)(it & 1);
       const long long grp = first + it * stride;
@@ -521,7 +537,7 @@ condense_mla64_kernel(CondenseArgs a) {
       const unsigned char* t_sem = smem + (size_t)st * STAGE_BYTES;
       const unsigned char* t_pos = t_sem + SEM_BYTES;
       const size_t out_row = (size_t)b * a.cache_rows + j;
-      float a0 = 0.f, a1 = 0.f, a2 = 0.f, a3 = 0.f;
+      unsigned long long acc01 = f32x2(0.f, 0.f), acc23 = f32x2(0.f, 0.f);
       const uint2* col = reinterpret_cast<const uint2*>(t_sem) + pt;
       const float* al_base = s_a + p * G;
 #pragma unroll 2
@@ -531,11 +547,15 @@ condense_mla64_kernel(CondenseArgs a) {
 #pragma unroll
         for (int u = 0; u < 4; ++u) {
           const uint2 w = col[(i + u) * (DS / 4)];
-          a0 = fmaf(alv[u], __uint_as_float(w.x << 16), a0); a1 = fmaf(alv[u], __uint_as_float(w.x & 0xffff0000u), a1);
-          a2 = fmaf(alv[u], __uint_as_float(w.y << 16), a2); a3 = fmaf(alv[u], __uint_as_float(w.y & 0xffff0000u), a3);
+          const unsigned long long al2 = f32x2(alv[u], alv[u]);
+          acc01 = fma_f32x2(al2, f32x2(__uint_as_float(w.x << 16), __uint_as_float(w.x & 0xffff0000u)), acc01);
+          acc23 = fma_f32x2(al2, f32x2(__uint_as_float(w.y << 16), __uint_as_float(w.y & 0xffff0000u)), acc23);
         }
       }
       {
+        float a0, a1, a2, a3;
+        asm("mov.b64 {%0, %1}, %2;" : "=f"(a0), "=f"(a1) : "l"(acc01));
+        asm("mov.b64 {%0, %1}, %2;" : "=f"(a2), "=f"(a3) : "l"(acc23));
         const bf162 lo = __floats2bfloat162_rn(a0, a1), hi = __floats2bfloat162_rn(a2, a3);
         uint2 o;
         o.x = *reinterpret_cast<const unsigned*>(&lo); o.y = *reinterpret_cast<const unsigned*>(&hi);
@@ -545,7 +565,6 @@ condense_mla64_kernel(CondenseArgs a) {
       if (pt < DP / 8)
         reinterpret_cast<uint4*>(a.cache_pos + out_row * DP)[pt] = reinterpret_cast<const uint4*>(t_pos + (size_t)ia * (DP * 2))[pt];
       if (pt == 32) a.anchor[(size_t)b * a.m + j] = j * G + ia;
-      if (a.scores && pt >= 64) a.scores[((size_t)b * a.m + j) * G + (pt - 64)] = s_s[p * G + pt - 64];
       __syncwarp();
       if (lane == 0) { cond_arrive(BAR_AFREE(p)); cond_arrive(BAR_FREE(st)); }
     }

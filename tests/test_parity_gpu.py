@@ -551,7 +551,7 @@ def test_absorbed_attention_plus_value_projection_equals_unabsorbed_attention(B)
     WUK = torch.from_numpy(rng.standard_normal((H, 512, dn)) / 512 ** 0.5).bfloat16()
     WUV = torch.from_numpy(rng.standard_normal((H, 512, 128)) / 512 ** 0.5).bfloat16()
     q_nope = torch.from_numpy(rng.standard_normal((L, H, dn))).bfloat16()
-    q_lat = torch.einsum("lhn,hcn->lhc", q_nope.float(), WUK.float()).bfloat16()        # absorbed query, as the model would feed it
+    q_lat = torch.einsum("lhn,hcn->lhc", q_nope.float(), WUK.float()).bfloat16().contiguous()   # absorbed query, as the model would feed it
     inp["q_sem"] = q_lat
     d = to_dev(inp)
     p = B.params_from_config(cfg, batch=1)
