@@ -56,7 +56,8 @@ enum { LCA_VARIANT_MLA = 0, LCA_VARIANT_GQA = 1 };
  *   WEIGHTED sum_i alpha_i x_i with the Eq. 6 weights    MAXSEL    the vector of the arg-max token (Eq. 8)
  * DEFAULT is the method itself: WEIGHTED for the semantic part (Eq. 7), MAXSEL for the positional part. */
 enum { LCA_REDUCE_DEFAULT = 0, LCA_REDUCE_MAXPOOL = 1, LCA_REDUCE_MEANPOOL = 2, LCA_REDUCE_WEIGHTED = 3, LCA_REDUCE_MAXSEL = 4 };
-enum { LCA_WS_CONDENSE = 0, LCA_WS_PREFILL = 1, LCA_WS_DECODE = 2, LCA_WS_UPDATE = 3 };
+enum { LCA_WS_CONDENSE = 0, LCA_WS_PREFILL = 1, LCA_WS_DECODE = 2, LCA_WS_UPDATE = 3,
+       LCA_WS_CONDENSE_VARLEN = 4, LCA_WS_PREFILL_VARLEN = 5 };
 
 /* Problem statement = the REQUIRE line of Alg. 1 (L, C^KV, K^R, Q, w, g) plus the head layout.
  *   MLA: n_kv_heads = 1, d_sem = d_c (512), d_pos = d_R (64); logits use [sem | pos], values = sem.
@@ -159,6 +160,31 @@ int lca_prefill_attention(const lca_params* p, const void* q_sem, const void* q_
                           const void* kv_sem, const void* kv_pos, const void* cache_sem,
                           const void* cache_pos, void* out, float* lse_opt, void* ws,
                           size_t ws_bytes, void* stream);
+
+/* Batches of sequences of different lengths (Alg. 1 takes one L per sequence: a batch is `batch` independent runs,
+ * each with its own L_b, m_b = floor((L_b - w)/g) and k_b).  The sequences are packed one after the other, without
+ * padding, in every tensor:
+ *   q_sem / q_pos  [T, H, d]          T = sum of L_b           kv_sem / kv_pos [T, n_kv_heads, d]
+ *   cache_sem / cache_pos [R, n_kv_heads, d]   R = sum of (m_b + k_b), each sequence in the layout stated at the top
+ *   anchor_idx [M, n_kv_heads]        M = sum of m_b (token indices count from the start of their own sequence)
+ *   out [T, H, d_sem], lse_opt [T, H]
+ * seq_lens [batch] is a HOST array of positive lengths; p->seq_len is ignored, except that lca_workspace_bytes(p,
+ * LCA_WS_CONDENSE_VARLEN / LCA_WS_PREFILL_VARLEN) sizes the workspace for sequences of at most p->seq_len tokens.
+ * lca_varlen_layout fills the prefix sums (batch + 1 entries each, any of them may be NULL): first token row, first
+ * cache row and first anchor_idx row of every sequence, totals in the last entry.  Host only.
+ * lca_condense_varlen takes the WHOLE packed query tensors and averages the last min(n_summary_q, L_b) positions of
+ * each sequence (or uses qbar_opt [batch, n_kv_heads, dk]); it does not return the scores.  Results are those of one
+ * call per sequence, bit for bit.  The calls copy a few small tables to the device from pageable host memory, which
+ * orders the host behind earlier work of `stream`. */
+int lca_varlen_layout(const lca_params* p, const int32_t* seq_lens, int64_t* token_offsets,
+                      int64_t* cache_row_offsets, int64_t* group_offsets);
+int lca_condense_varlen(const lca_params* p, const int32_t* seq_lens, const void* q_sem, const void* q_pos,
+                        const float* qbar_opt, const void* kv_sem, const void* kv_pos, void* cache_sem,
+                        void* cache_pos, int32_t* anchor_idx, void* ws, size_t ws_bytes, void* stream);
+int lca_prefill_attention_varlen(const lca_params* p, const int32_t* seq_lens, const void* q_sem,
+                                 const void* q_pos, const void* kv_sem, const void* kv_pos,
+                                 const void* cache_sem, const void* cache_pos, void* out, float* lse_opt,
+                                 void* ws, size_t ws_bytes, void* stream);
 
 /* Decode attention (Sec. 4.3): one new query per sequence attends to every valid row of that
  * sequence's condensed cache (the caller has appended the new token's own row).

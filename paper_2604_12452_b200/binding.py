@@ -21,6 +21,7 @@ from . import build as _build
 LCA_OK = 0
 LCA_VARIANT_MLA, LCA_VARIANT_GQA = 0, 1
 LCA_WS_CONDENSE, LCA_WS_PREFILL, LCA_WS_DECODE, LCA_WS_UPDATE = 0, 1, 2, 3
+LCA_WS_CONDENSE_VARLEN, LCA_WS_PREFILL_VARLEN = 4, 5
 LCA_STATIC_SCRATCH_BYTES = 1 << 20
 LCA_ERR_STATIC_SCRATCH_EXCEEDED = -7
 LCA_ERR_DEVICE_TIMEOUT = -6
@@ -71,6 +72,13 @@ def _load() -> C.CDLL:
     lib.lca_decode_attention.argtypes = [P, vp, vp, vp, vp, vp, i32, i32, vp, vp, vp, sz, vp]
     lib.lca_decode_update.restype = C.c_int
     lib.lca_decode_update.argtypes = [P, vp, vp, i64, vp, vp, vp, i32, vp, vp, vp, vp, sz, vp]
+    pi32, pi64 = C.POINTER(i32), C.POINTER(i64)
+    lib.lca_varlen_layout.restype = C.c_int
+    lib.lca_varlen_layout.argtypes = [P, pi32, pi64, pi64, pi64]
+    lib.lca_condense_varlen.restype = C.c_int
+    lib.lca_condense_varlen.argtypes = [P, pi32, vp, vp, vp, vp, vp, vp, vp, vp, vp, sz, vp]
+    lib.lca_prefill_attention_varlen.restype = C.c_int
+    lib.lca_prefill_attention_varlen.argtypes = [P, pi32, vp, vp, vp, vp, vp, vp, vp, vp, vp, sz, vp]
     lib.lca_latent_to_value.restype = C.c_int
     lib.lca_latent_to_value.argtypes = [vp, vp, vp, i64, i32, i32, i32, vp]
     lib.lca_selftest_bounded_wait.restype = C.c_int
@@ -180,6 +188,36 @@ def lca_decode_update(params, q_tail_sem, q_tail_pos, q_tail_batch_stride, qbar_
                                       _ptr(n_rep), _ptr(cache_rows), _ptr(anchor_out), _ptr(ws), wsb, _stream(stream)))
 
 
+def _lens(seq_lens):
+    return (C.c_int32 * len(seq_lens))(*[int(x) for x in seq_lens])
+
+
+def lca_varlen_layout(params, seq_lens):
+    """(token_offsets, cache_row_offsets, group_offsets): lists of batch + 1 prefix sums."""
+    n = params.batch + 1
+    tok, cache, grp = (C.c_int64 * n)(), (C.c_int64 * n)(), (C.c_int64 * n)()
+    st = _lib.lca_varlen_layout(C.byref(params), _lens(seq_lens), tok, cache, grp)
+    if st != LCA_OK:
+        raise LcaError(st, "lca_varlen_layout")
+    return list(tok), list(cache), list(grp)
+
+
+def lca_condense_varlen(params, seq_lens, q_sem, q_pos, qbar_opt, kv_sem, kv_pos, cache_sem, cache_pos, anchor_idx,
+                        ws, ws_bytes=None, stream=None) -> int:
+    wsb = _nbytes(ws) if ws_bytes is None else int(ws_bytes)
+    return int(_lib.lca_condense_varlen(C.byref(params), _lens(seq_lens), _ptr(q_sem), _ptr(q_pos), _ptr(qbar_opt),
+                                        _ptr(kv_sem), _ptr(kv_pos), _ptr(cache_sem), _ptr(cache_pos), _ptr(anchor_idx),
+                                        _ptr(ws), wsb, _stream(stream)))
+
+
+def lca_prefill_attention_varlen(params, seq_lens, q_sem, q_pos, kv_sem, kv_pos, cache_sem, cache_pos, out, lse_opt,
+                                 ws, ws_bytes=None, stream=None) -> int:
+    wsb = _nbytes(ws) if ws_bytes is None else int(ws_bytes)
+    return int(_lib.lca_prefill_attention_varlen(C.byref(params), _lens(seq_lens), _ptr(q_sem), _ptr(q_pos), _ptr(kv_sem),
+                                                 _ptr(kv_pos), _ptr(cache_sem), _ptr(cache_pos), _ptr(out), _ptr(lse_opt),
+                                                 _ptr(ws), wsb, _stream(stream)))
+
+
 def lca_latent_to_value(attn_latent, w_uv, out_v, n_tokens, n_heads, d_latent, d_v, stream=None) -> int:
     return int(_lib.lca_latent_to_value(_ptr(attn_latent), _ptr(w_uv), _ptr(out_v), int(n_tokens), int(n_heads),
                                         int(d_latent), int(d_v), _stream(stream)))
@@ -275,6 +313,41 @@ def decode_attention(params: LcaParams, q_sem, q_pos, cache_sem, cache_pos, cach
     st = lca_decode_attention(params, q_sem, q_pos, cache_sem, cache_pos, cache_rows, cap, n_rep, out, lse,
                               ws, stream=stream)
     _check(st, "lca_decode_attention")
+    return out, lse
+
+
+def condense_varlen(params: LcaParams, seq_lens, q_sem, q_pos, kv_sem, kv_pos, qbar: Optional[torch.Tensor] = None,
+                    stream=None):
+    """Packed batch of sequences of different lengths: allocate the packed cache and run lca_condense_varlen.
+    Returns dict(cache_sem, cache_pos, anchor_idx, token_offsets, cache_row_offsets, group_offsets)."""
+    dev = kv_sem.device
+    p = LcaParams.from_buffer_copy(params)
+    p.batch, p.seq_len = len(seq_lens), max(seq_lens)
+    tok, cache, grp = lca_varlen_layout(p, seq_lens)
+    Hkv = p.n_kv_heads
+    out = dict(cache_sem=torch.empty((cache[-1], Hkv, p.d_sem), dtype=torch.bfloat16, device=dev),
+               cache_pos=torch.empty((cache[-1], Hkv, p.d_pos), dtype=torch.bfloat16, device=dev),
+               anchor_idx=torch.empty((max(grp[-1], 1), Hkv), dtype=torch.int32, device=dev))
+    ws = workspace(p, LCA_WS_CONDENSE_VARLEN, dev)
+    st = lca_condense_varlen(p, seq_lens, q_sem, q_pos, qbar, kv_sem, kv_pos, out["cache_sem"], out["cache_pos"],
+                             out["anchor_idx"], ws, stream=stream)
+    _check(st, "lca_condense_varlen")
+    out.update(token_offsets=tok, cache_row_offsets=cache, group_offsets=grp, ws=ws)
+    return out
+
+
+def prefill_attention_varlen(params: LcaParams, seq_lens, q_sem, q_pos, kv_sem, kv_pos, cache_sem, cache_pos,
+                             want_lse: bool = False, stream=None):
+    dev = kv_sem.device
+    p = LcaParams.from_buffer_copy(params)
+    p.batch, p.seq_len = len(seq_lens), max(seq_lens)
+    T, H = sum(seq_lens), p.n_q_heads
+    out = torch.empty((T, H, p.d_sem), dtype=torch.bfloat16, device=dev)
+    lse = torch.empty((T, H), dtype=torch.float32, device=dev) if want_lse else None
+    ws = workspace(p, LCA_WS_PREFILL_VARLEN, dev)
+    st = lca_prefill_attention_varlen(p, seq_lens, q_sem, q_pos, kv_sem, kv_pos, cache_sem, cache_pos, out, lse, ws,
+                                      stream=stream)
+    _check(st, "lca_prefill_attention_varlen")
     return out, lse
 
 

@@ -52,6 +52,7 @@ struct Gqa2Params {
   int HB, TB, n_blocks;                   // heads and tokens per sub-tile, 2*TB-token blocks per sequence
   int out_wide;
   float scale_log2, bias_log2;
+  SeqTab tab;                             // ragged batch (tok_off != nullptr): q_len, L and cap are unused
 };
 
 template <bool WANT_LSE>
@@ -77,10 +78,18 @@ attn_gqa2_kernel(const __grid_constant__ Gqa2Params p) {
   const int warp = __shfl_sync(0xffffffffu, (int)(threadIdx.x >> 5), 0), lane = threadIdx.x & 31;
 
   // ---- which rows, which key tiles (the same arithmetic in every role)
-  const int blk = p.n_blocks - 1 - (int)blockIdx.x;          // heaviest (latest) blocks first
   const int hk = blockIdx.y, b = blockIdx.z;
+  int q_len = p.q_len, qbase = b * p.q_len, kbase = b * p.L, cbase = b * p.cap, n_blocks = p.n_blocks;
+  if (p.tab.tok_off) {                                       // ragged batch: this sequence's rows and length
+    qbase = kbase = p.tab.tok_off[b];
+    q_len = p.tab.tok_off[b + 1] - qbase;
+    cbase = p.tab.cache_off[b];
+    n_blocks = (q_len + 2 * p.TB - 1) / (2 * p.TB);
+  }
+  const int blk = n_blocks - 1 - (int)blockIdx.x;            // heaviest (latest) blocks first
+  if (blk < 0) return;                                       // the grid covers the longest sequence (whole CTA leaves)
   const int t0 = blk * 2 * p.TB;                             // first token of the block
-  const int t1 = min(t0 + 2 * p.TB, p.q_len) - 1;            // last valid token
+  const int t1 = min(t0 + 2 * p.TB, q_len) - 1;              // last valid token
   const int head0 = hk * p.HB;
   const int n_a_lo = reps_visible(t0, p.w, p.g), n_a_hi = reps_visible(t1, p.w, p.g);
   const int first_lo = n_a_lo * p.g;
@@ -121,13 +130,13 @@ attn_gqa2_kernel(const __grid_constant__ Gqa2Params p) {
       prefetch_tmap(&p.q); prefetch_tmap(&p.k); prefetch_tmap(&p.v);
       mbar_expect_tx(BAR_Q, Q_BYTES);
       for (int r = 0; r < 2; ++r) {
-        const int qrow = b * p.q_len + t0 + r * p.TB;
+        const int qrow = qbase + t0 + r * p.TB;
         for (int c = 0; c < 2; ++c) tma_load_3d(sQ + (r * 2 + c) * QCH, &p.q, c * 64, head0, qrow, BAR_Q);
       }
       for (int j = 0; j < n_tiles; ++j) {
         const int s = j % STAGES, round = j / STAGES;
         const bool isA = j < nA;
-        const int row = isA ? b * p.cap + j * BN : b * p.L + first_lo + (j - nA) * BN;
+        const int row = isA ? cbase + j * BN : kbase + first_lo + (j - nA) * BN;
         const CUtensorMap* mk = isA ? &p.ck : &p.k;
         const CUtensorMap* mv = isA ? &p.cv : &p.v;
         if (!mbar_wait(BAR_KEMPTY(s), (round & 1) ^ 1, abort_flag)) { fail(ERR_WAIT_KV_EMPTY); break; }
@@ -211,8 +220,8 @@ attn_gqa2_kernel(const __grid_constant__ Gqa2Params p) {
     const uint32_t s_tm = tmem + lane_base + TM_S + 128 * r, o_tm = tmem + lane_base + TM_O + 128 * r;
     const int tl = row / p.HB, hl = row % p.HB;
     const int t_row = t0 + r * p.TB + tl;
-    const bool row_valid = t_row < p.q_len;
-    const int n_a_row = reps_visible(min(t_row, p.q_len - 1), p.w, p.g);
+    const bool row_valid = t_row < q_len;
+    const int n_a_row = reps_visible(min(t_row, q_len - 1), p.w, p.g);
     const int first_row = n_a_row * p.g;
     float m_ref = -INFINITY, l_sum = 0.f;
     bool ok = true;
@@ -334,7 +343,7 @@ attn_gqa2_kernel(const __grid_constant__ Gqa2Params p) {
     if (ok) {
       tc_fence_after();
       const float inv = l_sum > 0.f ? 1.f / l_sum : 0.f;
-      const size_t orow = ((size_t)b * p.q_len + t_row) * p.Hq + head0 + hl;
+      const size_t orow = ((size_t)qbase + t_row) * p.Hq + head0 + hl;
       bf16* dst = p.out + orow * 128;
 #pragma unroll 1
       for (int q = 0; q < 4; ++q) {
@@ -392,8 +401,13 @@ int attn_gqa2_launch(const AttnProblem& a) {
   p.bias_log2 = a.rep_logit_bias * 1.4426950408889634f;
   p.out = (bf16*)a.out; p.lse = a.lse;
   p.out_wide = (reinterpret_cast<uintptr_t>(a.out) & 31u) == 0;
-  const long long qrows = (long long)a.batch * a.q_len, krows = (long long)a.batch * a.seq_len,
-                  crows = (long long)a.batch * a.cache_row_capacity;
+  long long qrows = (long long)a.batch * a.q_len, krows = (long long)a.batch * a.seq_len,
+            crows = (long long)a.batch * a.cache_row_capacity;
+  if (a.h_tok_off) {
+    p.tab = a.tab;
+    qrows = krows = a.h_tok_off[a.batch];
+    crows = a.h_cache_off[a.batch];
+  }
   bool ok = make_tensor_map_3d(&p.q, a.q_pos, 128, a.n_q_heads, qrows, p.HB, p.TB);
   ok = ok && make_tensor_map_3d(&p.k, a.kv_pos, 128, a.n_kv_heads, krows, 1, BN);
   ok = ok && make_tensor_map_3d(&p.v, a.kv_sem, 128, a.n_kv_heads, krows, 1, BN);

@@ -15,6 +15,8 @@ struct SimtArgs {
   bf16* out; float* lse;
   int B, q_len, Hq, Hkv, decode, L, g, w, cap, n_rep_bias;
   float scale, bias;
+  SeqTab tab;              // ragged prefill batch (tok_off != nullptr): q_len, L and cap are unused
+  long long n_rows;        // query rows of the launch (tokens x heads)
 };
 
 template <int D_SEM, int D_POS, bool SEM_IN_LOGIT>
@@ -24,11 +26,17 @@ attn_simt_kernel(SimtArgs a) {
   constexpr int PP = D_POS / 64;   // pos part
   const int lane = threadIdx.x & 31;
   const long long row = (long long)blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5);
-  const long long n_rows = (long long)a.B * a.q_len * a.Hq;
-  if (row >= n_rows) return;
+  if (row >= a.n_rows) return;
   const int h = (int)(row % a.Hq);
-  const int t = (int)((row / a.Hq) % a.q_len);
-  const int b = (int)(row / ((long long)a.Hq * a.q_len));
+  int t = (int)((row / a.Hq) % a.q_len);
+  int b = (int)(row / ((long long)a.Hq * a.q_len));
+  size_t kbase = (size_t)b * a.L, cbase = (size_t)b * a.cap;       // first token row / cache row of the sequence
+  if (a.tab.tok_off) {
+    const long long tok = row / a.Hq;
+    b = seq_of(a.tab.tok_off, a.tab.B, tok);
+    t = (int)(tok - a.tab.tok_off[b]);
+    kbase = (size_t)a.tab.tok_off[b]; cbase = (size_t)a.tab.cache_off[b];
+  }
   const int hk = h / (a.Hq / a.Hkv);
 
   float qs[2 * PS > 0 ? 2 * PS : 1], qp[2 * PP > 0 ? 2 * PP : 1];
@@ -70,11 +78,11 @@ attn_simt_kernel(SimtArgs a) {
     const bf16 *ks, *kp;
     float add = 0.f;
     if (x < n_a) {
-      size_t r = ((size_t)b * a.cap + x) * a.Hkv + hk;
+      size_t r = (cbase + x) * a.Hkv + hk;
       ks = a.cache_sem + r * D_SEM; kp = a.cache_pos + r * D_POS;
       if (x < bias_rows) add = a.bias;
     } else {
-      size_t r = ((size_t)b * a.L + (b_first + x - n_a)) * a.Hkv + hk;
+      size_t r = (kbase + (b_first + x - n_a)) * a.Hkv + hk;
       ks = a.kv_sem + r * D_SEM; kp = a.kv_pos + r * D_POS;
     }
     float2 v[PS];
@@ -119,7 +127,9 @@ int attn_simt_launch(const AttnProblem& p) {
   a.B = p.batch; a.q_len = p.q_len; a.Hq = p.n_q_heads; a.Hkv = p.n_kv_heads; a.decode = p.decode;
   a.L = p.seq_len; a.g = p.group_size; a.w = p.window; a.cap = p.cache_row_capacity;
   a.n_rep_bias = p.n_rep_bias; a.scale = p.softmax_scale; a.bias = p.rep_logit_bias;
-  const long long rows = (long long)p.batch * p.q_len * p.n_q_heads;
+  const long long rows = p.h_tok_off ? (long long)p.h_tok_off[p.batch] * p.n_q_heads : (long long)p.batch * p.q_len * p.n_q_heads;
+  a.tab = p.h_tok_off ? p.tab : SeqTab{};
+  a.n_rows = rows;
   if (rows == 0) return LCA_OK;
   const unsigned blocks = (unsigned)((rows + 3) / 4);
   if (p.variant == LCA_VARIANT_MLA && p.d_sem == 512 && p.d_pos == 64)

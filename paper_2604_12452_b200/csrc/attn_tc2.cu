@@ -19,7 +19,9 @@
 // tokens) down in a fixed stride.  Barriers and tensor memory are set up once; the query tile of the
 // next item is fetched as soon as the last S product of the current one has completed, and its first
 // products run while the softmax threads still normalise and store the current output.
+#include <algorithm>
 #include <cstring>
+#include <vector>
 
 #include "lca_common.cuh"
 #include "tc_common.cuh"
@@ -64,24 +66,41 @@ struct Tc2Params {
   int HB, TB, n_tok_tiles, n_head_blocks;
   int out_wide;                   // out is 32-byte aligned: 256-bit stores
   long long n_items;              // query tiles x head blocks x batch
+  // ragged prefill batch: (sequence, token tile) of every entry, heaviest first, and the sequences' first rows;
+  // item idx is head block idx % n_head_blocks of entry idx / n_head_blocks.  nullptr: uniform batch.
+  const int2* entries;
+  SeqTab tab;
   float scale_log2, bias_log2;
 };
 
 // One work item = one tile of 128 query rows; the same arithmetic in every role of both CTAs.
 struct Item {
-  int b, head0, t0, t1;
+  int b, head0, t0, t1, len;      // sequence, first head, first / last token of the tile, length of the sequence
+  int qbase, kbase, cbase;        // row of the sequence's first token in the query / token arrays, of its first cache row
   int n_a_lo, n_a_hi, first_lo, nA, n_tiles;
 };
 __device__ __forceinline__ Item make_item(const Tc2Params& p, long long idx) {
   Item it;
-  // heaviest query tiles (latest tokens) first; batch and head block vary fastest
-  const long long per_tile = (long long)p.n_head_blocks * p.B;
-  const int tile = p.n_tok_tiles - 1 - (int)(idx / per_tile);
-  const int rem = (int)(idx % per_tile);
-  it.b = rem / p.n_head_blocks;
-  it.head0 = (rem % p.n_head_blocks) * p.HB;
+  int tile;
+  if (p.entries) {
+    const int2 e = p.entries[idx / p.n_head_blocks];
+    it.b = e.x; tile = e.y;
+    it.head0 = (int)(idx % p.n_head_blocks) * p.HB;
+    it.qbase = it.kbase = p.tab.tok_off[it.b];
+    it.len = p.tab.tok_off[it.b + 1] - it.qbase;
+    it.cbase = p.tab.cache_off[it.b];
+  } else {
+    // heaviest query tiles (latest tokens) first; batch and head block vary fastest
+    const long long per_tile = (long long)p.n_head_blocks * p.B;
+    tile = p.n_tok_tiles - 1 - (int)(idx / per_tile);
+    const int rem = (int)(idx % per_tile);
+    it.b = rem / p.n_head_blocks;
+    it.head0 = (rem % p.n_head_blocks) * p.HB;
+    it.len = p.q_len;
+    it.qbase = it.b * p.q_len; it.kbase = it.b * p.L; it.cbase = it.b * p.cap;
+  }
   it.t0 = tile * p.TB;
-  it.t1 = min(it.t0 + p.TB, p.q_len) - 1;
+  it.t1 = min(it.t0 + p.TB, it.len) - 1;
   int nB;
   if (p.decode) {
     it.n_a_hi = it.n_a_lo = min(max(p.cache_rows[it.b], 0), p.cap);
@@ -178,13 +197,13 @@ attn_tc2_kernel(const __grid_constant__ Tc2Params p) {
         // the query tile may be replaced once the last S of the previous item has completed
         if (!mbar_wait(BAR_QFREE, (n_item & 1) ^ 1, abort_flag)) { fail(ERR_WAIT_Q); break; }
         if (rank == 0) mbar_expect_tx(BAR_Q, 2 * Q_BYTES);
-        const int qtok = it.b * p.q_len + it.t0 + row0 / p.HB, qhead = it.head0 + row0 % p.HB;
+        const int qtok = it.qbase + it.t0 + row0 / p.HB, qhead = it.head0 + row0 % p.HB;
         for (int c = 0; c < 8; ++c) tma_load_3d_pair(sQ + c * QCH, &p.q_sem, c * 64, qhead, qtok, q_bar);
         tma_load_3d_pair(sQ + 8 * QCH, &p.q_pos, 0, qhead, qtok, q_bar);
         ++n_item;
         for (int j = 0; good && j < it.n_tiles; ++j, ++jt) {
           const bool isA = j < it.nA;
-          const int row = (isA ? it.b * p.cap + j * BN : it.b * p.L + it.first_lo + (j - it.nA) * BN) + 64 * (int)rank;
+          const int row = (isA ? it.cbase + j * BN : it.kbase + it.first_lo + (j - it.nA) * BN) + 64 * (int)rank;
           const CUtensorMap* ms = isA ? &p.c_sem : &p.k_sem;
           const CUtensorMap* mp = isA ? &p.c_pos : &p.k_pos;
           if (p.decode) {
@@ -213,7 +232,7 @@ attn_tc2_kernel(const __grid_constant__ Tc2Params p) {
         const Item it = make_item(p, idx);
         for (int j = 0; good && j < it.n_tiles; ++j, ++jt) {
           const bool isA = j < it.nA;
-          const int row = isA ? it.b * p.cap + j * BN : it.b * p.L + it.first_lo + (j - it.nA) * BN;
+          const int row = isA ? it.cbase + j * BN : it.kbase + it.first_lo + (j - it.nA) * BN;
           const CUtensorMap* mv = isA ? &p.c_val : &p.k_val;
           // Decode, last tile of a sequence whose valid rows end inside it: the rows behind them may hold anything
           // (0 x NaN would reach O), so the softmax threads of each CTA zero them in their own value buffers before
@@ -367,13 +386,13 @@ attn_tc2_kernel(const __grid_constant__ Tc2Params p) {
     uint32_t jt = 0, n_item = 0, n_ragged = 0;   // tiles / non-empty items / ragged decode tiles of this pair so far
     for (long long idx = pair_id; ok && idx < p.n_items; idx += n_pairs) {
     const Item it = make_item(p, idx);
-    const int b = it.b, head0 = it.head0, t0 = it.t0, nA = it.nA, n_tiles = it.n_tiles;
+    const int head0 = it.head0, t0 = it.t0, nA = it.nA, n_tiles = it.n_tiles;
     const int n_a_lo = it.n_a_lo, n_a_hi = it.n_a_hi, first_lo = it.first_lo;
     const int t_row = t0 + tl;
     const bool row_valid = t_row <= it.t1;
     int n_a_row, bias_rows, first_row;
     if (p.decode) { n_a_row = n_a_hi; bias_rows = min(p.n_rep_bias, n_a_row); first_row = 0; }
-    else { n_a_row = reps_visible(min(t_row, p.q_len - 1), p.w, p.g); bias_rows = n_a_row; first_row = n_a_row * p.g; }
+    else { n_a_row = reps_visible(min(t_row, it.len - 1), p.w, p.g); bias_rows = n_a_row; first_row = n_a_row * p.g; }
     float m_ref = -INFINITY, l_sum = 0.f, l_exact = 0.f;     // l_sum: rounded weights (normaliser); l_exact: for lse
     bool all_left = false;                       // every one of the 128 threads left the tile loop at a barrier
     for (int j = 0; j < n_tiles; ++j, ++jt) {
@@ -529,7 +548,7 @@ attn_tc2_kernel(const __grid_constant__ Tc2Params p) {
     {
       tc_fence_after();
       const float inv = (n_tiles > 0 && l_tot > 0.f) ? 1.f / l_tot : 0.f;
-      const size_t orow = ((size_t)b * p.q_len + t_row) * p.H + head0 + hl;
+      const size_t orow = ((size_t)it.qbase + t_row) * p.H + head0 + hl;
       bf16* dst = p.out + orow * 512;
 #pragma unroll 1                                   // once per item: kept small
       for (int q = 0; q < 8; ++q) {
@@ -582,6 +601,12 @@ attn_tc2_kernel(const __grid_constant__ Tc2Params p) {
 bool make_tensor_map_3d(CUtensorMap* map, const void* ptr, int d, int heads, long long rows, int box_heads, int box_rows);
 bool make_tensor_map_chunks(CUtensorMap* map, const void* ptr, int chunks, long long rows, int box_rows, int box_chunks);
 
+// Entries of a ragged batch behind the sequence table: one (sequence, tile) pair per token tile.
+size_t attn_tc2_ragged_workspace_bytes(int batch, int longest, int n_q_heads) {
+  const int TB = n_q_heads >= 128 ? 1 : 128 / n_q_heads;
+  return seq_table_bytes(batch) + (size_t)batch * ((size_t)(longest + TB - 1) / TB) * sizeof(int2);
+}
+
 bool attn_tc2_supported(const AttnProblem& a) {
   if (a.variant != LCA_VARIANT_MLA || a.d_sem != 512 || a.d_pos != 64 || a.n_kv_heads != 1) return false;
   const int H = a.n_q_heads;
@@ -628,13 +653,40 @@ int attn_tc2_launch(const AttnProblem& a) {
   p.n_tok_tiles = (a.q_len + p.TB - 1) / p.TB;
   p.n_head_blocks = H >= 128 ? H / 128 : 1;
   p.n_items = (long long)p.n_tok_tiles * p.n_head_blocks * a.batch;
+  long long qrows = (long long)a.batch * a.q_len, krows = (long long)a.batch * a.seq_len,
+            crows = (long long)a.batch * a.cache_row_capacity;
+  if (a.h_tok_off) {
+    // ragged batch: one entry per (sequence, token tile), heaviest (most key tiles) first, uploaded behind the table
+    std::vector<int2> entries;
+    std::vector<int> weight;
+    for (int b = 0; b < a.batch; ++b) {
+      const int len = a.h_tok_off[b + 1] - a.h_tok_off[b];
+      for (int tile = 0; tile * p.TB < len; ++tile) {
+        const int t0 = tile * p.TB, t1 = std::min(t0 + p.TB, len) - 1;
+        const int n_lo = reps_visible(t0, p.w, p.g), n_hi = reps_visible(t1, p.w, p.g);
+        entries.push_back(make_int2(b, tile));
+        weight.push_back((n_hi + BN - 1) / BN + (t1 - n_lo * p.g + BN) / BN);
+      }
+    }
+    std::vector<int> order(entries.size());
+    for (size_t i = 0; i < order.size(); ++i) order[i] = (int)i;
+    std::stable_sort(order.begin(), order.end(), [&](int x, int y) { return weight[x] > weight[y]; });
+    std::vector<int2> sorted(entries.size());
+    for (size_t i = 0; i < order.size(); ++i) sorted[i] = entries[order[i]];
+    int2* d_entries = reinterpret_cast<int2*>(static_cast<char*>(a.ws) + seq_table_bytes(a.batch));
+    if (!sorted.empty() &&
+        cudaMemcpyAsync(d_entries, sorted.data(), sorted.size() * sizeof(int2), cudaMemcpyHostToDevice, a.stream) != cudaSuccess)
+      return LCA_ERR_CUDA;
+    p.entries = d_entries; p.tab = a.tab;
+    p.n_items = (long long)sorted.size() * p.n_head_blocks;
+    qrows = krows = a.h_tok_off[a.batch];
+    crows = a.h_cache_off[a.batch];
+  }
   p.scale_log2 = a.softmax_scale * 1.4426950408889634f;
   p.bias_log2 = a.rep_logit_bias * 1.4426950408889634f;
   p.out = (bf16*)a.out; p.lse = a.lse; p.cache_rows = a.cache_rows;
   p.out_wide = (reinterpret_cast<uintptr_t>(a.out) & 31u) == 0;
   const int hbc = p.HB >= 64 ? 64 : p.HB, tbc = 64 / hbc;
-  const long long qrows = (long long)a.batch * a.q_len, krows = (long long)a.batch * a.seq_len,
-                  crows = (long long)a.batch * a.cache_row_capacity;
   bool ok = make_tensor_map_3d(&p.q_sem, a.q_sem, 512, H, qrows, hbc, tbc);
   ok = ok && make_tensor_map_3d(&p.q_pos, a.q_pos, 64, H, qrows, hbc, tbc);
   ok = ok && make_tensor_map_3d(&p.k_pos, a.kv_pos, 64, 1, krows, 1, 64);

@@ -22,12 +22,20 @@ static const int CONDENSE_THREADS = 512;
 // (8 columns) of the key dimension and every row_lanes-th row of the chunk, so that consecutive
 // threads read a whole query row and each thread has many independent loads in flight; the
 // row lanes are then added up through shared memory in a fixed order.
+// Ragged batch (tab.tok_off != nullptr): q_sem / q_pos are the whole packed query arrays and the tail of
+// sequence b is its last min(n_pos, L_b) positions.
 __global__ void qbar_partial_kernel(const bf16* __restrict__ q_sem, const bf16* __restrict__ q_pos,
                                     int64_t batch_stride_rows, int n_pos, int Hq, int Hkv, int d_sem,
-                                    int d_pos, int sem_in_logit, int row_lanes, double* __restrict__ partial) {
+                                    int d_pos, int sem_in_logit, int row_lanes, double* __restrict__ partial, SeqTab tab) {
   extern __shared__ double s_part[];                     // [row_lanes][dk]
   const int chunk = blockIdx.x, hk = blockIdx.y, b = blockIdx.z;
   const int rep = Hq / Hkv;
+  long long first_pos = (long long)b * batch_stride_rows;     // row (position) of the first averaged query
+  if (tab.tok_off) {
+    const int len = tab.tok_off[b + 1] - tab.tok_off[b];
+    n_pos = min(n_pos, len);
+    first_pos = (long long)tab.tok_off[b] + len - n_pos;
+  }
   const int n_rows = n_pos * rep;
   const int r0 = chunk * QBAR_ROWS_PER_CHUNK;
   const int r1 = min(n_rows, r0 + QBAR_ROWS_PER_CHUNK);
@@ -48,7 +56,7 @@ __global__ void qbar_partial_kernel(const bf16* __restrict__ q_sem, const bf16* 
         v[u] = make_uint4(0u, 0u, 0u, 0u);
         if (rr < r1) {
           const int pos = rr / rep, head = hk * rep + rr % rep;
-          const size_t row = ((size_t)b * batch_stride_rows + pos) * Hq + head;
+          const size_t row = ((size_t)first_pos + pos) * Hq + head;
           const bf16* src = (pc < sem_pieces) ? q_sem + row * d_sem + 8 * pc : q_pos + row * d_pos + 8 * (pc - sem_pieces);
           v[u] = *reinterpret_cast<const uint4*>(src);
         }
@@ -78,8 +86,12 @@ __global__ void qbar_partial_kernel(const bf16* __restrict__ q_sem, const bf16* 
 // Sum the chunk partials in chunk order and divide by the number of averaged rows.
 // grid (Hkv, B)
 __global__ void qbar_final_kernel(const double* __restrict__ partial, int nchunks, int dk,
-                                  double count, double* __restrict__ qbar) {
+                                  double count, double* __restrict__ qbar, SeqTab tab, int n_pos, int rep) {
   const size_t stream_id = (size_t)blockIdx.y * gridDim.x + blockIdx.x;
+  if (tab.tok_off) {
+    const int b = blockIdx.y;
+    count = (double)min(n_pos, tab.tok_off[b + 1] - tab.tok_off[b]) * (double)rep;
+  }
   const double* src = partial + stream_id * nchunks * dk;
   for (int c = threadIdx.x; c < dk; c += blockDim.x) {
     double s = 0.0;
@@ -100,9 +112,39 @@ struct CondenseArgs {
   bf16* cache_sem; bf16* cache_pos; int32_t* anchor; double* scores;
   int L, Hkv, d_sem, d_pos, g, m, cache_rows, sem_in_logit;
   int sem_reducer, pos_reducer;   // LCA_REDUCE_* with DEFAULT already resolved
-  long long n_groups;          // B * Hkv * m
+  long long n_groups;          // B * Hkv * m   (ragged batch: Hkv * sum of m_b)
   double scale;
+  SeqTab tab;                  // ragged batch: L, m and cache_rows above are unused
 };
+
+// Where group `grp` of the launch lives: uniform batch grp = (b * Hkv + hk) * m + j; ragged batch: the groups of
+// sequence b are grp_off[b] * Hkv + hk * m_b + j.
+struct GroupLoc { int b, hk, j; long long tok0, out_row, grp_row; };     // first token row, cache row, row of anchor_idx
+__device__ inline GroupLoc locate_group(const CondenseArgs& a, long long grp) {
+  GroupLoc l;
+  if (a.tab.tok_off) {
+    int lo = 0, hi = a.tab.B - 1;
+    while (lo < hi) {
+      const int mid = (lo + hi + 1) >> 1;
+      if ((long long)a.tab.grp_off[mid] * a.Hkv <= grp) lo = mid; else hi = mid - 1;
+    }
+    l.b = lo;
+    const int m_b = a.tab.grp_off[lo + 1] - a.tab.grp_off[lo];
+    const long long local = grp - (long long)a.tab.grp_off[lo] * a.Hkv;
+    l.hk = (int)(local / m_b); l.j = (int)(local % m_b);
+    l.tok0 = (long long)a.tab.tok_off[lo] + (long long)l.j * a.g;
+    l.out_row = (long long)a.tab.cache_off[lo] + l.j;
+    l.grp_row = (long long)a.tab.grp_off[lo] + l.j;
+  } else {
+    l.j = (int)(grp % a.m);
+    const long long bh = grp / a.m;
+    l.hk = (int)(bh % a.Hkv); l.b = (int)(bh / a.Hkv);
+    l.tok0 = (long long)l.b * a.L + (long long)l.j * a.g;
+    l.out_row = (long long)l.b * a.cache_rows + l.j;
+    l.grp_row = (long long)l.b * a.m + l.j;
+  }
+  return l;
+}
 
 __device__ inline void cp_async16(void* smem_dst, const void* gmem_src) {
   unsigned s = (unsigned)__cvta_generic_to_shared(smem_dst);
@@ -131,13 +173,13 @@ condense_kernel(CondenseArgs a) {
 
   auto stage_ptr = [&](int st) { return smem_raw + (size_t)st * stage_bytes; };
   auto prefetch = [&](long long grp, int st) {
-    const int j = (int)(grp % a.m);
-    const long long bh = grp / a.m;
-    const int hk = (int)(bh % a.Hkv), b = (int)(bh / a.Hkv);
+    const GroupLoc loc = locate_group(a, grp);
+    const int hk = loc.hk;
+    const long long bh = (long long)loc.b * a.Hkv + hk;
     bf16* t_sem = reinterpret_cast<bf16*>(stage_ptr(st));
     bf16* t_pos = t_sem + (size_t)g * d_sem;
     double* s_q = reinterpret_cast<double*>(t_pos + (size_t)g * d_pos);
-    const size_t tok0 = (size_t)b * a.L + (size_t)j * g;
+    const size_t tok0 = (size_t)loc.tok0;
     const bf16* gs = a.kv_sem + tok0 * row_stride_sem + (size_t)hk * d_sem;
     const bf16* gp = a.kv_pos + tok0 * row_stride_pos + (size_t)hk * d_pos;
     for (int x = tid; x < g * cps; x += blockDim.x) {
@@ -162,9 +204,8 @@ condense_kernel(CondenseArgs a) {
     asm volatile("cp.async.commit_group;\ncp.async.wait_group 1;\n" ::: "memory");
     __syncthreads();
 
-    const int j = (int)(grp % a.m);
-    const long long bh = grp / a.m;
-    const int hk = (int)(bh % a.Hkv), b = (int)(bh / a.Hkv);
+    const GroupLoc loc = locate_group(a, grp);
+    const int j = loc.j, hk = loc.hk;
     const bf16* t_sem = reinterpret_cast<const bf16*>(stage_ptr(st));
     const bf16* t_pos = t_sem + (size_t)g * d_sem;
     const double* s_q = reinterpret_cast<const double*>(t_pos + (size_t)g * d_pos);
@@ -223,7 +264,7 @@ condense_kernel(CondenseArgs a) {
 
     // 3. the representative: semantic part (Eq. 7 by default) and positional part (Eq. 8 by
     //    default), each reduced over the g tokens by the chosen operator, one column pair per thread
-    const size_t out_row = (size_t)b * a.cache_rows + j;
+    const size_t out_row = (size_t)loc.out_row;
     const int ia = s_anchor;
     auto reduce = [&](const bf16* tile, int d, int mode, bf16* dst, int tid0) {
       for (int pr = tid0; pr < d / 2; pr += blockDim.x) {
@@ -247,9 +288,9 @@ condense_kernel(CondenseArgs a) {
     reduce(t_pos, d_pos, a.pos_reducer, a.cache_pos + (out_row * a.Hkv + hk) * d_pos, blockDim.x - 1 - tid);
     {
       const int rt = blockDim.x - 1 - tid;
-      if (rt == 0) a.anchor[((size_t)b * a.m + j) * a.Hkv + hk] = j * g + ia;
+      if (rt == 0) a.anchor[(size_t)loc.grp_row * a.Hkv + hk] = j * g + ia;
       if (a.scores) {
-        double* sc = a.scores + (((size_t)b * a.Hkv + hk) * a.m + j) * g;
+        double* sc = a.scores + (((size_t)loc.b * a.Hkv + hk) * a.m + j) * g;
         for (int i = rt; i < g; i += blockDim.x) sc[i] = s_s[i];
       }
     }
@@ -395,9 +436,7 @@ condense_mla64_kernel(CondenseArgs a) {
         const int st = (int)(it % STAGES);
         if (it >= STAGES && !cond_wait(BAR_FREE(st), (unsigned)((it / STAGES - 1) & 1), s_abort)) break;
         const long long grp = first + it * stride;
-        const int j = (int)(grp % a.m);
-        const long long b = grp / a.m;
-        const size_t tok0 = (size_t)b * a.L + (size_t)j * G;
+        const size_t tok0 = (size_t)locate_group(a, grp).tok0;
         const unsigned dst = (unsigned)__cvta_generic_to_shared(smem + (size_t)st * STAGE_BYTES);
         const unsigned bar = BAR_FULL(st);
         asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(STAGE_BYTES) : "memory");
@@ -414,7 +453,7 @@ condense_mla64_kernel(CondenseArgs a) {
     for (long long it = 0; it < n_mine; ++it) {
       const int st = (int)(it % STAGES), p = (int)(it & 1);
       const long long grp = first + it * stride;
-      const long long b = grp / a.m;
+      const long long b = a.tab.tok_off ? seq_of(a.tab.grp_off, a.tab.B, grp) : grp / a.m;
       if (b != cur_b) {                                   // rare: the next sequence's summary query
         cur_b = b;
         const double* qb = a.qbar + (size_t)b * DK;
@@ -470,8 +509,7 @@ condense_mla64_kernel(CondenseArgs a) {
     for (long long it = 0; it < n_mine; ++it) {
       const int st = (int)(it % STAGES), p = (int)(it & 1);
       const long long grp = first + it * stride;
-      const int j = (int)(grp % a.m);
-      const long long b = grp / a.m;
+      const long long b = a.tab.tok_off ? seq_of(a.tab.grp_off, a.tab.B, grp) : grp / a.m;
       const double* qb = a.qbar + (size_t)b * DK;
       if (b != cur_b) {
         cur_b = b;
@@ -511,7 +549,7 @@ condense_mla64_kernel(CondenseArgs a) {
         }
         ea = expf((float)(da - best)); eb = expf((float)(db - best));
         if (a.scores) {
-          double* sc = a.scores + ((size_t)b * a.m + j) * G;
+          double* sc = a.scores + (size_t)grp * G;            // one KV stream: group grp of the launch is row grp
           sc[lane] = da; sc[lane + 32] = db;
         }
       } else {
@@ -530,13 +568,13 @@ condense_mla64_kernel(CondenseArgs a) {
     for (long long it = 0; it < n_mine; ++it) {
       const int st = (int)(it % STAGES), p = (int)(it & 1);
       const long long grp = first + it * stride;
-      const int j = (int)(grp % a.m);
-      const long long b = grp / a.m;
+      const GroupLoc loc = locate_group(a, grp);
+      const int j = loc.j;
       if (!cond_wait(BAR_READY(p), (unsigned)((it >> 1) & 1), s_abort)) break;
       if (!cond_wait(BAR_FULL(st), (unsigned)((it / STAGES) & 1), s_abort)) break;     // complete long ago
       const unsigned char* t_sem = smem + (size_t)st * STAGE_BYTES;
       const unsigned char* t_pos = t_sem + SEM_BYTES;
-      const size_t out_row = (size_t)b * a.cache_rows + j;
+      const size_t out_row = (size_t)loc.out_row;
       unsigned long long acc01 = f32x2(0.f, 0.f), acc23 = f32x2(0.f, 0.f);
       const uint2* col = reinterpret_cast<const uint2*>(t_sem) + pt;
       const float* al_base = s_a + p * G;
@@ -564,7 +602,7 @@ condense_mla64_kernel(CondenseArgs a) {
       const int ia = s_anchor[p];
       if (pt < DP / 8)
         reinterpret_cast<uint4*>(a.cache_pos + out_row * DP)[pt] = reinterpret_cast<const uint4*>(t_pos + (size_t)ia * (DP * 2))[pt];
-      if (pt == 32) a.anchor[(size_t)b * a.m + j] = j * G + ia;
+      if (pt == 32) a.anchor[grp] = j * G + ia;
       __syncwarp();
       if (lane == 0) { cond_arrive(BAR_AFREE(p)); cond_arrive(BAR_FREE(st)); }
     }
@@ -583,14 +621,24 @@ int condense_take_status() {
 // ------------------------------------------------------------------------------ local window
 // Copies, for every sequence, one contiguous block of `bytes16` 16-byte words.
 // Two block copies per sequence in one launch (blockIdx.z: the semantic and the positional part).
-struct CopySeg { const uint4* src; uint4* dst; size_t src_batch_stride16, dst_batch_stride16, src_off16, dst_off16, n16; };
-__global__ void copy_blocks_kernel(const CopySeg a, const CopySeg b) {
+struct CopySeg { const uint4* src; uint4* dst; size_t src_batch_stride16, dst_batch_stride16, src_off16, dst_off16, n16, row16; };
+// Ragged batch: the segment of sequence blockIdx.y (its last k tokens -> cache rows m .. m + k - 1) follows from the table.
+__global__ void copy_blocks_kernel(const CopySeg a, const CopySeg b, SeqTab tab, int g) {
   const CopySeg& c = blockIdx.z == 0 ? a : b;
-  const uint4* s = c.src + (size_t)blockIdx.y * c.src_batch_stride16 + c.src_off16;
-  uint4* d = c.dst + (size_t)blockIdx.y * c.dst_batch_stride16 + c.dst_off16;
-  for (size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x; i < c.n16;
-       i += (size_t)gridDim.x * blockDim.x)
-    d[i] = s[i];
+  size_t src_off = (size_t)blockIdx.y * c.src_batch_stride16 + c.src_off16;
+  size_t dst_off = (size_t)blockIdx.y * c.dst_batch_stride16 + c.dst_off16;
+  size_t n16 = c.n16;
+  if (tab.tok_off) {
+    const int s = blockIdx.y;
+    const int len = tab.tok_off[s + 1] - tab.tok_off[s], m = tab.grp_off[s + 1] - tab.grp_off[s], k = len - m * g;
+    src_off = (size_t)(tab.tok_off[s] + len - k) * c.row16;
+    dst_off = (size_t)(tab.cache_off[s] + m) * c.row16;
+    n16 = (size_t)k * c.row16;
+  }
+  const uint4* sp = c.src + src_off;
+  uint4* dp = c.dst + dst_off;
+  for (size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x; i < n16; i += (size_t)gridDim.x * blockDim.x)
+    dp[i] = sp[i];
 }
 
 // ------------------------------------------------------------------------------------- host
@@ -627,15 +675,17 @@ size_t condense_smem_bytes(const lca_params* p) {
 
 int condense_launch(const CondenseLaunch& c) {
   const lca_params* p = c.p;
+  const bool ragged = c.h_tok_off != nullptr;
   int64_t m, k;
-  partition(p->seq_len, p->window, p->group_size, &m, &k);
+  partition(p->seq_len, p->window, p->group_size, &m, &k);       // uniform batch; a ragged one takes them from the table
   const int dk = key_dim(p);
   const int sem_in_logit = p->variant == LCA_VARIANT_MLA;
   const int B = p->batch, Hkv = p->n_kv_heads;
+  const long long total_groups = ragged ? (long long)c.h_grp_off[B] : (long long)B * m;      // per KV stream
   double* qbar = reinterpret_cast<double*>(c.ws);
   double* partial = qbar + (size_t)B * Hkv * dk;
 
-  if (m > 0) {
+  if (total_groups > 0) {
     if (c.qbar_opt) {
       int n = B * Hkv * dk;
       qbar_widen_kernel<<<(n + 255) / 256, 256, 0, c.stream>>>(c.qbar_opt, qbar, n);
@@ -648,11 +698,13 @@ int condense_launch(const CondenseLaunch& c) {
       if (row_lanes < 1) row_lanes = 1;
       if (row_lanes > 16) row_lanes = 16;
       const int threads = ((pieces * row_lanes + 31) / 32) * 32;
+      const int n = ragged ? (p->n_summary_q > 0 ? p->n_summary_q : p->group_size) : n_summary(p);
       qbar_partial_kernel<<<grid, threads, (size_t)row_lanes * dk * sizeof(double), c.stream>>>(
-          (const bf16*)c.q_tail_sem, (const bf16*)c.q_tail_pos, c.q_tail_batch_stride, n_summary(p),
-          p->n_q_heads, Hkv, p->d_sem, p->d_pos, sem_in_logit, row_lanes, partial);
-      double count = (double)n_summary(p) * (double)(p->n_q_heads / Hkv);
-      qbar_final_kernel<<<dim3(Hkv, B), dk < 1024 ? ((dk + 31) / 32) * 32 : 1024, 0, c.stream>>>(partial, nch, dk, count, qbar);
+          (const bf16*)c.q_tail_sem, (const bf16*)c.q_tail_pos, c.q_tail_batch_stride, n,
+          p->n_q_heads, Hkv, p->d_sem, p->d_pos, sem_in_logit, row_lanes, partial, c.tab);
+      double count = (double)n * (double)(p->n_q_heads / Hkv);
+      qbar_final_kernel<<<dim3(Hkv, B), dk < 1024 ? ((dk + 31) / 32) * 32 : 1024, 0, c.stream>>>(partial, nch, dk, count, qbar, c.tab, n,
+                                                                                              p->n_q_heads / Hkv);
       note_launch(2);
     }
     CondenseArgs a;
@@ -662,7 +714,8 @@ int condense_launch(const CondenseLaunch& c) {
     a.L = p->seq_len; a.Hkv = Hkv; a.d_sem = p->d_sem; a.d_pos = p->d_pos; a.g = p->group_size;
     a.m = (int)m; a.cache_rows = (int)(m + k); a.sem_in_logit = sem_in_logit;
     a.scale = (double)p->softmax_scale;
-    a.n_groups = (long long)B * Hkv * m;
+    a.n_groups = total_groups * Hkv;
+    a.tab = c.tab;
     a.sem_reducer = p->sem_reducer == LCA_REDUCE_DEFAULT ? LCA_REDUCE_WEIGHTED : p->sem_reducer;
     a.pos_reducer = p->pos_reducer == LCA_REDUCE_DEFAULT ? LCA_REDUCE_MAXSEL : p->pos_reducer;
     int dev = 0, sms = 148;
@@ -688,16 +741,16 @@ int condense_launch(const CondenseLaunch& c) {
     }
     note_launch();
   }
-  if (k > 0) {
-    // rows L-k..L-1 of each sequence -> cache rows m..m+k-1 (one contiguous block per sequence)
+  if (ragged || k > 0) {
+    // the last k tokens of each sequence -> cache rows m..m+k-1 (one contiguous block per sequence)
     const size_t row_sem = (size_t)Hkv * p->d_sem * sizeof(bf16) / 16;
     const size_t row_pos = (size_t)Hkv * p->d_pos * sizeof(bf16) / 16;
-    const unsigned blocks = 148 * 2;
+    const unsigned blocks = B >= 148 ? 8 : 148 * 2;
     const CopySeg sem = {(const uint4*)c.kv_sem, (uint4*)c.cache_sem, (size_t)p->seq_len * row_sem, (size_t)(m + k) * row_sem,
-                         (size_t)(p->seq_len - k) * row_sem, (size_t)m * row_sem, (size_t)k * row_sem};
+                         (size_t)(p->seq_len - k) * row_sem, (size_t)m * row_sem, (size_t)k * row_sem, row_sem};
     const CopySeg pos = {(const uint4*)c.kv_pos, (uint4*)c.cache_pos, (size_t)p->seq_len * row_pos, (size_t)(m + k) * row_pos,
-                         (size_t)(p->seq_len - k) * row_pos, (size_t)m * row_pos, (size_t)k * row_pos};
-    copy_blocks_kernel<<<dim3(blocks, B, 2), 256, 0, c.stream>>>(sem, pos);
+                         (size_t)(p->seq_len - k) * row_pos, (size_t)m * row_pos, (size_t)k * row_pos, row_pos};
+    copy_blocks_kernel<<<dim3(blocks, B, 2), 256, 0, c.stream>>>(sem, pos, c.tab, p->group_size);
     note_launch();
   }
   return cudaGetLastError() == cudaSuccess ? LCA_OK : LCA_ERR_CUDA;
@@ -850,9 +903,9 @@ int update_launch(const lca_params* p, const void* q_tail_sem, const void* q_tai
     const int threads = ((pieces * row_lanes + 31) / 32) * 32;
     qbar_partial_kernel<<<dim3(nch, Hkv, B), threads, (size_t)row_lanes * dk * sizeof(double), stream>>>(
         (const bf16*)q_tail_sem, (const bf16*)q_tail_pos, q_tail_batch_stride, n, p->n_q_heads, Hkv, p->d_sem, p->d_pos,
-        sem_in_logit, row_lanes, partial);
+        sem_in_logit, row_lanes, partial, SeqTab{});
     qbar_final_kernel<<<dim3(Hkv, B), dk < 1024 ? ((dk + 31) / 32) * 32 : 1024, 0, stream>>>(
-        partial, nch, dk, (double)n * (double)(p->n_q_heads / Hkv), qbar);
+        partial, nch, dk, (double)n * (double)(p->n_q_heads / Hkv), qbar, SeqTab{}, n, p->n_q_heads / Hkv);
     note_launch(2);
   }
   UpdateArgs a;

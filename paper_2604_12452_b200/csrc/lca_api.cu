@@ -1,5 +1,6 @@
 // C-ABI entry points of the LCA library: host-side validation and dispatch to the kernels.
 #include <atomic>
+#include <vector>
 
 #include "lca_common.cuh"
 
@@ -31,6 +32,38 @@ static int check_params(const lca_params* p, bool need_partition) {
 static bool simt_shape_ok(const lca_params* p) {
   if (p->variant == LCA_VARIANT_MLA) return (p->d_sem == 512 || p->d_sem == 128) && p->d_pos == 64;
   return (p->d_sem == 128 && p->d_pos == 128) || (p->d_sem == 64 && p->d_pos == 64);
+}
+
+// Prefix sums of a ragged batch on the host: tokens, cache rows (m_b + k_b) and groups (m_b) before sequence b.
+struct HostSeqTable {
+  std::vector<int32_t> tok, cache, grp;
+  int longest = 0;
+};
+static int build_seq_table(const lca_params* p, const int32_t* seq_lens, HostSeqTable* t) {
+  const int B = p->batch;
+  t->tok.assign(B + 1, 0); t->cache.assign(B + 1, 0); t->grp.assign(B + 1, 0);
+  long long tok = 0, cache = 0, grp = 0;
+  for (int b = 0; b < B; ++b) {
+    if (seq_lens[b] <= 0) return LCA_ERR_INVALID_ARG;
+    int64_t m, k;
+    partition(seq_lens[b], p->window, p->group_size, &m, &k);
+    tok += seq_lens[b]; cache += m + k; grp += m;
+    if (tok > 0x7fffff00ll) return LCA_ERR_UNSUPPORTED_SHAPE;     // row coordinates are 32-bit
+    t->tok[b + 1] = (int32_t)tok; t->cache[b + 1] = (int32_t)cache; t->grp[b + 1] = (int32_t)grp;
+    if (seq_lens[b] > t->longest) t->longest = seq_lens[b];
+  }
+  return LCA_OK;
+}
+// Copies the three arrays to the start of `ws` (stream-ordered) and returns the device view.
+static int upload_seq_table(const HostSeqTable& t, int B, void* ws, cudaStream_t stream, SeqTab* tab) {
+  int32_t* d = static_cast<int32_t*>(ws);
+  const size_t n = (size_t)(B + 1) * sizeof(int32_t);
+  if (cudaMemcpyAsync(d, t.tok.data(), n, cudaMemcpyHostToDevice, stream) != cudaSuccess ||
+      cudaMemcpyAsync(d + (B + 1), t.cache.data(), n, cudaMemcpyHostToDevice, stream) != cudaSuccess ||
+      cudaMemcpyAsync(d + 2 * (B + 1), t.grp.data(), n, cudaMemcpyHostToDevice, stream) != cudaSuccess)
+    return LCA_ERR_CUDA;
+  tab->tok_off = d; tab->cache_off = d + (B + 1); tab->grp_off = d + 2 * (B + 1); tab->B = B;
+  return LCA_OK;
 }
 
 static int run_attention(const AttnProblem& a) {
@@ -85,6 +118,8 @@ int lca_partition(const lca_params* p, int32_t* m, int32_t* k) {
 size_t lca_workspace_bytes(const lca_params* p, int32_t which) {
   if (check_params(p, which != LCA_WS_DECODE && which != LCA_WS_UPDATE) != LCA_OK) return 0;
   if (which == LCA_WS_CONDENSE) return condense_workspace_bytes(p);
+  if (which == LCA_WS_CONDENSE_VARLEN) return seq_table_bytes(p->batch) + condense_workspace_bytes(p);
+  if (which == LCA_WS_PREFILL_VARLEN) return attn_tc2_ragged_workspace_bytes(p->batch, p->seq_len, p->n_q_heads);
   if (which == LCA_WS_UPDATE) return update_workspace_bytes(p);
   if (which == LCA_WS_PREFILL || which == LCA_WS_DECODE) {
     AttnProblem a = {};
@@ -123,6 +158,89 @@ int lca_condense(const lca_params* p, const void* q_tail_sem, const void* q_tail
   CondenseLaunch c = {p, q_tail_sem, q_tail_pos, q_tail_batch_stride, qbar_opt, kv_sem, kv_pos,
                       cache_sem, cache_pos, anchor_idx, scores_opt, ws, ws_bytes, (cudaStream_t)stream};
   return condense_launch(c);
+}
+
+int lca_varlen_layout(const lca_params* p, const int32_t* seq_lens, int64_t* token_offsets,
+                      int64_t* cache_row_offsets, int64_t* group_offsets) {
+  int st = check_params(p, false);
+  if (st != LCA_OK) return st;
+  if (p->group_size <= 0 || p->window < 0 || !seq_lens) return LCA_ERR_INVALID_ARG;
+  HostSeqTable t;
+  st = build_seq_table(p, seq_lens, &t);
+  if (st != LCA_OK) return st;
+  for (int b = 0; b <= p->batch; ++b) {
+    if (token_offsets) token_offsets[b] = t.tok[b];
+    if (cache_row_offsets) cache_row_offsets[b] = t.cache[b];
+    if (group_offsets) group_offsets[b] = t.grp[b];
+  }
+  return LCA_OK;
+}
+
+int lca_condense_varlen(const lca_params* p, const int32_t* seq_lens, const void* q_sem, const void* q_pos,
+                        const float* qbar_opt, const void* kv_sem, const void* kv_pos, void* cache_sem,
+                        void* cache_pos, int32_t* anchor_idx, void* ws, size_t ws_bytes, void* stream) {
+  int st = check_params(p, false);
+  if (st != LCA_OK) return st;
+  if (p->group_size <= 0 || p->window < 0 || p->n_summary_q < 0 || !seq_lens) return LCA_ERR_INVALID_ARG;
+  if (!kv_sem || !kv_pos || !cache_sem || !cache_pos) return LCA_ERR_INVALID_ARG;
+  HostSeqTable t;
+  st = build_seq_table(p, seq_lens, &t);
+  if (st != LCA_OK) return st;
+  lca_params q = *p;
+  q.seq_len = t.longest;                                   // sizes the summary-query scratch
+  if (t.grp[p->batch] > 0) {
+    if (!anchor_idx) return LCA_ERR_INVALID_ARG;
+    if (!qbar_opt) {
+      if (!q_pos || (p->variant == LCA_VARIANT_MLA && !q_sem)) return LCA_ERR_INVALID_ARG;
+      if (!aligned16(q_pos) || (q_sem && !aligned16(q_sem))) return LCA_ERR_MISALIGNED;
+    }
+    if (condense_smem_bytes(&q) > 227u * 1024u) return LCA_ERR_UNSUPPORTED_SHAPE;
+  }
+  if (!ws || !aligned16(ws)) return LCA_ERR_INVALID_ARG;
+  if (ws_bytes < seq_table_bytes(p->batch) + condense_workspace_bytes(&q)) return LCA_ERR_WORKSPACE_TOO_SMALL;
+  if (!aligned16(kv_sem) || !aligned16(kv_pos) || !aligned16(cache_sem) || !aligned16(cache_pos))
+    return LCA_ERR_MISALIGNED;
+  CondenseLaunch c = {&q, q_sem, q_pos, 0, qbar_opt, kv_sem, kv_pos, cache_sem, cache_pos, anchor_idx, nullptr,
+                      static_cast<char*>(ws) + seq_table_bytes(p->batch), ws_bytes - seq_table_bytes(p->batch),
+                      (cudaStream_t)stream};
+  c.h_tok_off = t.tok.data(); c.h_cache_off = t.cache.data(); c.h_grp_off = t.grp.data();
+  st = upload_seq_table(t, p->batch, ws, (cudaStream_t)stream, &c.tab);
+  if (st != LCA_OK) return st;
+  return condense_launch(c);
+}
+
+int lca_prefill_attention_varlen(const lca_params* p, const int32_t* seq_lens, const void* q_sem,
+                                 const void* q_pos, const void* kv_sem, const void* kv_pos,
+                                 const void* cache_sem, const void* cache_pos, void* out, float* lse_opt,
+                                 void* ws, size_t ws_bytes, void* stream) {
+  int st = check_params(p, false);
+  if (st != LCA_OK) return st;
+  if (p->group_size <= 0 || p->window < 0 || !seq_lens) return LCA_ERR_INVALID_ARG;
+  if (!q_pos || !kv_sem || !kv_pos || !out) return LCA_ERR_INVALID_ARG;
+  if (p->variant == LCA_VARIANT_MLA && !q_sem) return LCA_ERR_INVALID_ARG;
+  HostSeqTable t;
+  st = build_seq_table(p, seq_lens, &t);
+  if (st != LCA_OK) return st;
+  if (t.grp[p->batch] > 0 && (!cache_sem || !cache_pos)) return LCA_ERR_INVALID_ARG;
+  if (!aligned16(q_pos) || !aligned16(kv_sem) || !aligned16(kv_pos) || !aligned16(out) ||
+      (q_sem && !aligned16(q_sem)) || (cache_sem && !aligned16(cache_sem)) || (cache_pos && !aligned16(cache_pos)))
+    return LCA_ERR_MISALIGNED;
+  if (!simt_shape_ok(p)) return LCA_ERR_UNSUPPORTED_SHAPE;
+  if (!ws || !aligned16(ws)) return LCA_ERR_INVALID_ARG;
+  if (ws_bytes < attn_tc2_ragged_workspace_bytes(p->batch, t.longest, p->n_q_heads)) return LCA_ERR_WORKSPACE_TOO_SMALL;
+  AttnProblem a = {};
+  a.variant = p->variant; a.batch = p->batch; a.q_len = t.longest; a.n_q_heads = p->n_q_heads;
+  a.n_kv_heads = p->n_kv_heads; a.d_sem = p->d_sem; a.d_pos = p->d_pos; a.decode = 0;
+  a.seq_len = t.longest; a.group_size = p->group_size; a.window = p->window;
+  a.cache_rows = nullptr; a.cache_row_capacity = 0; a.n_rep_bias = 0;
+  a.softmax_scale = p->softmax_scale; a.rep_logit_bias = p->rep_logit_bias;
+  a.q_sem = q_sem; a.q_pos = q_pos; a.kv_sem = kv_sem; a.kv_pos = kv_pos;
+  a.cache_sem = cache_sem; a.cache_pos = cache_pos; a.out = out; a.lse = lse_opt;
+  a.ws = ws; a.ws_bytes = ws_bytes; a.stream = (cudaStream_t)stream;
+  a.h_tok_off = t.tok.data(); a.h_cache_off = t.cache.data();
+  st = upload_seq_table(t, p->batch, ws, (cudaStream_t)stream, &a.tab);
+  if (st != LCA_OK) return st;
+  return run_attention(a);
 }
 
 int lca_condense_static_scratch(const lca_params* p, const void* q_tail_sem, const void* q_tail_pos,

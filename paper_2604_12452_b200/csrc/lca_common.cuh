@@ -28,6 +28,28 @@ __host__ __device__ inline int reps_visible(int p, int w, int g) {
   return (t < w + g) ? 0 : (t - w) / g;
 }
 
+// Ragged batches (sequences of different lengths packed one after the other).  Device arrays of B + 1 prefix sums:
+// first token row, first cache row and first group of every sequence.  tok_off == nullptr means a uniform batch
+// (every sequence p->seq_len long), where the same quantities follow from the batch index by multiplication.
+struct SeqTab {
+  const int32_t* tok_off;
+  const int32_t* cache_off;
+  const int32_t* grp_off;
+  int B;
+};
+// Largest b in [0, B) with off[b] <= x (off is non-decreasing, off[0] = 0 <= x < off[B]).
+__device__ inline int seq_of(const int32_t* off, int B, long long x) {
+  int lo = 0, hi = B - 1;
+  while (lo < hi) {
+    const int mid = (lo + hi + 1) >> 1;
+    if ((long long)off[mid] <= x) lo = mid; else hi = mid - 1;
+  }
+  return lo;
+}
+
+// Bytes of the device copy of the three prefix arrays (at the start of the workspace of a ragged call).
+inline size_t seq_table_bytes(int B) { return ((size_t)3 * (B + 1) * sizeof(int32_t) + 15) / 16 * 16; }
+
 __device__ inline double warp_sum(double v) {
 #pragma unroll
   for (int o = 16; o > 0; o >>= 1) v += __shfl_xor_sync(0xffffffffu, v, o);
@@ -47,6 +69,9 @@ struct CondenseLaunch {
   const void* kv_sem; const void* kv_pos;
   void* cache_sem; void* cache_pos; int32_t* anchor_idx; double* scores_opt;
   void* ws; size_t ws_bytes; cudaStream_t stream;
+  // ragged batch: host prefix sums (B + 1 entries each) and their device copies; all null for a uniform batch
+  const int32_t* h_tok_off; const int32_t* h_cache_off; const int32_t* h_grp_off;
+  SeqTab tab;
 };
 size_t condense_workspace_bytes(const lca_params* p);
 int condense_launch(const CondenseLaunch& a);
@@ -79,12 +104,17 @@ struct AttnProblem {
   void* out; float* lse;                  // [B, q_len, H, d_sem], [B, q_len, H]
   void* ws; size_t ws_bytes;
   cudaStream_t stream;
+  // ragged prefill batch: host prefix sums (B + 1 entries) and their device copies; null for a uniform batch.
+  // q_len / seq_len then hold the longest sequence, cache_row_capacity is unused.
+  const int32_t* h_tok_off; const int32_t* h_cache_off;
+  SeqTab tab;
 };
 int attn_simt_launch(const AttnProblem& a);     // scalar kernel, every supported head shape
 bool attn_tc_supported(const AttnProblem& a);   // tensor-core (tcgen05) kernels
 size_t attn_tc_workspace_bytes(const AttnProblem& a);
 int attn_tc_launch(const AttnProblem& a);
 int attn_tc_device_status(cudaStream_t stream);
+size_t attn_tc2_ragged_workspace_bytes(int batch, int longest, int n_q_heads);
 int bounded_wait_selftest_launch(long long limit_cycles, cudaStream_t stream);
 int latent_to_value_launch(const void* latent, const void* w_uv, void* out, long long n_tokens, int n_heads,
                            int d_latent, int d_v, cudaStream_t stream);

@@ -47,6 +47,20 @@ def test_partition_matches_section_4_2(B):
     assert B.lca_partition(p) == (13, 168)
 
 
+def test_ragged_layout_is_the_partition_of_every_sequence(B):
+    # host-only helper: prefix sums of L_b, m_b + k_b and m_b (Sec. 4.2 per sequence)
+    p = B.make_params("mla", 4, 2000, 16, 1, 512, 64, 16, 64, 0.07)
+    tok, cache, grp = B.lca_varlen_layout(p, [1, 50, 777, 2000])
+    assert tok == [0, 1, 51, 828, 2828]
+    ms = [0, 0, (777 - 64) // 16, (2000 - 64) // 16]
+    ks = [1, 50, 777 - 16 * ms[2], 2000 - 16 * ms[3]]
+    assert grp == [0, 0, 0, ms[2], ms[2] + ms[3]]
+    assert cache == [0, 1, 51, 51 + ms[2] + ks[2], 51 + ms[2] + ks[2] + ms[3] + ks[3]]
+    with pytest.raises(B.LcaError):
+        B.lca_varlen_layout(p, [1, 0, 5, 7])               # lengths must be positive
+    assert B.lca_workspace_bytes(p, B.LCA_WS_PREFILL_VARLEN) > 0 and B.lca_workspace_bytes(p, B.LCA_WS_CONDENSE_VARLEN) > 0
+
+
 def test_invalid_calls_return_error_codes_without_launching(B):
     before = B.lca_launch_count()
     good = B.make_params("mla", 1, 1024, 4, 1, 512, 64, 64, 128, 0.07)

@@ -583,3 +583,57 @@ def test_absorbed_attention_plus_value_projection_equals_unabsorbed_attention(B)
     # projected output) on values of unit scale
     st = Hh.check_outputs(got, ref, "absorbed attention + W^UV vs un-absorbed attention")
     assert st["max_abs"] < 2e-2
+
+
+@pytest.mark.parametrize("kind", ["mla_generic", "mla_fast", "gqa"])
+def test_ragged_batch_equals_one_call_per_sequence_and_the_oracle(B, kind):
+    # Alg. 1 takes one L per sequence: four sequences of 1, 50, 777 and 2000 tokens packed into one call (no group,
+    # no group, 40-odd groups, 100-odd groups; the last tile of one sequence overlaps the first rows of the next)
+    # must give, bit for bit, what four single calls give, and match the oracle sequence by sequence.
+    lens = [1, 50, 777, 2000]
+    if kind == "gqa":
+        base = I.scaled(I.CONFIGS["gqa_64k"], n_q_heads=8, n_kv_heads=2, group_size=16, window=40, n_needles=2)
+        make = I.make_gqa_inputs
+        names = dict(q_sem=None, q_pos="q", kv_sem="v", kv_pos="k")
+    else:
+        g, w = (16, 64) if kind == "mla_generic" else (64, 128)
+        base = I.scaled(I.CONFIGS["mla_1k"], n_q_heads=16, group_size=g, window=w, n_needles=2)
+        make = I.make_mla_inputs
+        names = dict(q_sem="q_sem", q_pos="q_pos", kv_sem="ckv", kv_pos="kr")
+    g, w = base.group_size, base.window
+    seqs = [make(I.scaled(base, seq_len=L), "cpu", batch_index=b) for b, L in enumerate(lens)]
+    packed = {k: torch.cat([s_[k] for s_ in seqs]).to(DEV) for k in seqs[0]}
+    arg = lambda d, key: None if names[key] is None else d[names[key]]
+    p = B.params_from_config(I.scaled(base, seq_len=max(lens)), batch=len(lens))
+    cond = B.condense_varlen(p, lens, arg(packed, "q_sem"), arg(packed, "q_pos"), arg(packed, "kv_sem"), arg(packed, "kv_pos"))
+    out, lse = B.prefill_attention_varlen(p, lens, arg(packed, "q_sem"), arg(packed, "q_pos"), arg(packed, "kv_sem"),
+                                          arg(packed, "kv_pos"), cond["cache_sem"], cond["cache_pos"], want_lse=True)
+    torch.cuda.synchronize()
+    assert B.lca_last_device_status() == 0
+    tok, cro, gro = cond["token_offsets"], cond["cache_row_offsets"], cond["group_offsets"]
+    assert tok == [0, 1, 51, 828, 2828]
+    for b, L in enumerate(lens):
+        d = {k: v.to(DEV) for k, v in seqs[b].items()}
+        p1 = B.params_from_config(I.scaled(base, seq_len=L), batch=1)
+        n = min(L, g)
+        qs = arg(d, "q_sem")
+        one = B.condense(p1, None if qs is None else qs[L - n:], arg(d, "q_pos")[L - n:], arg(d, "kv_sem"), arg(d, "kv_pos"))
+        o1, l1 = B.prefill_attention(p1, qs, arg(d, "q_pos"), arg(d, "kv_sem"), arg(d, "kv_pos"), one["cache_sem"],
+                                     one["cache_pos"], want_lse=True)
+        m, k = one["m"], one["k"]
+        assert (cro[b + 1] - cro[b], gro[b + 1] - gro[b]) == (m + k, m)
+        assert torch.equal(Hh.bits_t(cond["cache_sem"][cro[b]:cro[b + 1]]), Hh.bits_t(one["cache_sem"][0]))
+        assert torch.equal(Hh.bits_t(cond["cache_pos"][cro[b]:cro[b + 1]]), Hh.bits_t(one["cache_pos"][0]))
+        if m:
+            assert torch.equal(cond["anchor_idx"][gro[b]:gro[b + 1]], one["anchor_idx"][0])
+        assert torch.equal(Hh.bits_t(out[tok[b]:tok[b + 1]]), Hh.bits_t(o1[0])), f"sequence {b}"
+        assert torch.equal(lse[tok[b]:tok[b + 1]], l1[0])
+        rows = np.arange(L) if L <= 777 else Hh.sample_positions(L, g, w, n_uniform=40, seed=b)
+        if kind == "gqa":
+            ref = Hh.oracle_gqa(seqs[b], g, w, base.softmax_scale, rows=rows)
+        else:
+            ref = Hh.oracle_mla(seqs[b], g, w, base.softmax_scale, rows=rows)
+        piece = dict(m=m, k=k, cache_sem=cond["cache_sem"][cro[b]:cro[b + 1]], cache_pos=cond["cache_pos"][cro[b]:cro[b + 1]],
+                     anchor_idx=cond["anchor_idx"][gro[b]:gro[b + 1]])
+        Hh.check_condense(piece, ref["cond"], kind="gqa" if kind == "gqa" else "mla")
+        Hh.check_outputs(out[tok[b]:tok[b + 1]][torch.from_numpy(rows).to(DEV)], ref, f"ragged {kind} sequence {b}")
