@@ -139,46 +139,67 @@ class ClockSampler:
 
 
 # ----------------------------------------------------------------------------- CPU oracle
-def oracle_sample(cfg, inp_cpu_small, n_rows: int, n_heads: int, seed: int = 0):
-    """Time the oracle on a bounded sample: condensation of the whole sequence plus `n_rows`
-    stratified query rows x `n_heads` heads.  Returns (tokens_per_s_estimate, description, threads)."""
-    from oracle import lca_oracle as O
-    from tests import helpers as Hh
+def sample_rows(cfg, n_rows: int, seed: int = 0):
+    from oracle import parity as P
+    return P.sample_positions(cfg.seq_len, cfg.group_size, cfg.window, n_uniform=max(0, n_rows - 18), seed=seed)[:max(n_rows, 1)]
+
+
+def oracle_sample(cfg, small, n_rows: int, n_heads: int, seed: int = 0):
+    """Time the oracle on a bounded sample: condensation of the whole sequence plus `n_rows` stratified query
+    rows x `n_heads` heads.  Returns (tokens_per_s_estimate, description, threads, oracle results)."""
+    from oracle import lca_oracle as O, parity as P
     L, g, w, H = cfg.seq_len, cfg.group_size, cfg.window, cfg.n_q_heads
-    rows = Hh.sample_positions(L, g, w, n_uniform=max(0, n_rows - 18), seed=seed)[:max(n_rows, 1)]
+    rows = sample_rows(cfg, n_rows, seed)
     heads = np.arange(min(n_heads, H))
     t0 = time.perf_counter()
-    ref = Hh.oracle_mla(inp_cpu_small, g, w, cfg.softmax_scale, rows=None)
-    t_cond = time.perf_counter() - t0
-    cond = ref["cond"]
-    m = cond["m"]
-    ckv = O.torch_bf16_to_f64(inp_cpu_small["ckv"])
-    kr = O.torch_bf16_to_f64(inp_cpu_small["kr"])
-    rep_sem = O.bits_to_f64(cond["cache_sem_bits"][:m])
-    rep_pos = O.bits_to_f64(cond["cache_pos_bits"][:m])
-    qs = O.torch_bf16_to_f64(inp_cpu_small["q_sem_rows"][:len(rows)][:, heads])
-    qp = O.torch_bf16_to_f64(inp_cpu_small["q_pos_rows"][:len(rows)][:, heads])
+    full = P.mla_pipeline(small["ckv"], small["kr"], small["q_sem"], small["q_pos"], g, w, cfg.softmax_scale)
+    t_cond = time.perf_counter() - t0                    # summary query + condensation of the whole sequence
+    m = full["cond"]["m"]
+    rep_sem = O.bits_to_f64(full["cond"]["cache_sem_bits"][:m]) if m else None
+    rep_pos = O.bits_to_f64(full["cond"]["cache_pos_bits"][:m]) if m else None
+    ckv64, kr64 = O.torch_bf16_to_f64(small["ckv"]), O.torch_bf16_to_f64(small["kr"])
+    qs = O.torch_bf16_to_f64(small["q_sem_rows"][:len(rows)][:, heads])
+    qp = O.torch_bf16_to_f64(small["q_pos_rows"][:len(rows)][:, heads])
     t0 = time.perf_counter()
-    O.mla_prefill_rows(qs, qp, rows, ckv, kr, rep_sem if m else None, rep_pos if m else None, g, w,
-                       float(np.float32(cfg.softmax_scale)))
+    out, lse = O.mla_prefill_rows(qs, qp, rows, ckv64, kr64, rep_sem, rep_pos, g, w, P.f32(cfg.softmax_scale))
     t_rows = time.perf_counter() - t0
+    full.update(rows=rows, out=out, lse=lse)
     mt = np.where(rows + 1 < w + g, 0, (rows + 1 - w) // g)
     sampled_visits = float((mt + (rows + 1 - mt * g)).sum()) * len(heads)
     total_visits = float(key_visits(L, g, w)) * H
     est_total = t_cond + t_rows * total_visits / max(sampled_visits, 1.0)
-    desc = (f"condense of all {L} tokens ({t_cond:.2f}s) + {len(rows)} stratified query rows x {len(heads)} heads "
+    desc = (f"condense of all {L} tokens ({t_cond:.2f}s) + {len(rows)} stratified query rows x {len(heads)} of {H} heads "
             f"({t_rows:.2f}s), scaled by visited (query,key,head) triples {sampled_visits:.3g}/{total_visits:.3g}")
-    return L * cfg.batch / est_total, desc, O.num_threads(), dict(rows=rows, heads=heads)
+    full.update(heads=heads)
+    return L * cfg.batch / est_total, desc, O.num_threads(), full
 
 
 def gather_oracle_inputs(cfg, inp, n_rows, seed=0):
     """CPU copies of what the oracle sample needs (the K/V streams and the sampled query rows)."""
-    from tests import helpers as Hh
-    L, g, w = cfg.seq_len, cfg.group_size, cfg.window
-    rows = Hh.sample_positions(L, g, w, n_uniform=max(0, n_rows - 18), seed=seed)[:max(n_rows, 1)]
+    L, g = cfg.seq_len, cfg.group_size
+    rows = sample_rows(cfg, n_rows, seed)
     idx = torch.from_numpy(rows).to(inp["q_sem"].device)
     return dict(ckv=inp["ckv"].cpu(), kr=inp["kr"].cpu(), q_sem=inp["q_sem"][L - g:].cpu(), q_pos=inp["q_pos"][L - g:].cpu(),
                 q_sem_rows=inp["q_sem"][idx].cpu(), q_pos_rows=inp["q_pos"][idx].cpu())
+
+
+def parity_record(ref, out_rows, cache=None, kind="mla"):
+    """Raw comparison figures of a device result with the oracle's (by-product of the oracle leg): attention
+    output on the sampled rows, and the condensed cache in full when given."""
+    from oracle import lca_oracle as O, parity as P
+    vmax = ref["vmax"][None]
+    ro = ref["out"]
+    st = P.output_stats(out_rows, ro, vmax)
+    rec = dict(rows=int(ro.shape[0]), heads=int(ro.shape[1]), max_abs=st["max_abs"], mean_abs=st["mean_abs"], max_ref=st["max_ref"],
+               mean_ref=st["mean_ref"], n_above_2e2=st["n_above_2e2"], max_abs_unit_scale=st["max_abs_unit_scale"],
+               worst_over_derived_bound=st["worst_over_bound"])
+    if cache is not None:
+        cs = P.condense_stats(O.torch_bf16_to_bits(cache["cache_sem"]), O.torch_bf16_to_bits(cache["cache_pos"]),
+                              cache["anchor_idx"].cpu().numpy(), ref["cond"], kind)
+        rec.update(anchor_mismatches=cs["anchor_mismatches"], near_tie_groups=cs["near_tie_groups"], groups=cs["m"],
+                   copied_rows_differing=cs["pos_rows_differ"] + cs["local_sem_rows_differ"],
+                   crep_off_by_one_ulp=cs["crep_off_by_one_ulp"], crep_beyond_one_ulp=cs["crep_bad"], crep_elems=cs["crep_elems"])
+    return rec
 
 
 # -------------------------------------------------------------------------------- main arms
@@ -363,16 +384,7 @@ def run_ours(args, cfg, rank, world, local_rank):
             dist.destroy_process_group()
         return
     peaks = measured_peaks()
-    extras = {}
-    if not args.no_extras and world == 1:
-        for name, fn in (("decode_config", lambda: measure_decode_config(B, dev, args.decode_batch, peaks)),
-                         ("gqa_config", lambda: measure_gqa_config(B, dev, peaks)),
-                         ("dense_mla_comparison", lambda: measure_dense_comparison(B, dev, peaks))):
-            try:
-                extras[name] = fn()
-            except Exception as ex:        # report, never lose the main line
-                extras[name] = dict(error=str(ex)[:200])
-            torch.cuda.empty_cache()
+    want_oracle = not args.no_cpu_baseline
     flops = attention_flops(cfg)
     tfl = flops / (t_attn * 1e-3) / 1e12
     cbytes = condense_bytes(cfg)
@@ -391,11 +403,47 @@ def run_ours(args, cfg, rank, world, local_rank):
                 roofline_condense=dict(bound="hbm", achieved=cgbs, peak=peaks["hbm_gbs"], unit="GB/s",
                                        frac=cgbs / peaks["hbm_gbs"], traffic=None, kernel="lca_condense (all launches)",
                                        bytes_per_launch=cbytes, ms_per_launch=t_cond, peak_kind=f"{peaks['source']} copy"),
-                attention_impl=args.attn_impl, extras=extras)
-    if not args.no_cpu_baseline:
+                attention_impl=args.attn_impl)
+    parity = {}
+    if want_oracle:
         small = gather_oracle_inputs(cfg, inp, args.ref_rows)
-        v, desc, threads, _ = oracle_sample(cfg, small, args.ref_rows, args.ref_heads)
+        v, desc, threads, ref = oracle_sample(cfg, small, args.ref_rows, args.ref_heads)
         line["cpu_baseline"] = dict(value=v, unit=UNIT, cores=threads, kind="oracle", sample=desc)
+        idx = torch.from_numpy(ref["rows"]).to(dev)
+        hd = torch.from_numpy(ref["heads"]).to(dev)
+        parity[cfg.name] = parity_record(ref, out[0][idx][:, hd], {kk: cache[kk][0] for kk in cache})
+        del small, ref
+    extras = {}
+    if not args.no_extras and world == 1:
+        side = [("dense_mla_at_this_config", lambda: measure_dense_here(B, dev, cfg, inp, out, t_cond + t_attn)),
+                ("value_projection", lambda: measure_value_projection(B, dev, cfg, out, peaks))]
+        for name, fn in side:
+            try:
+                extras[name] = fn()
+            except Exception as ex:        # report, never lose the main line
+                extras[name] = dict(error=str(ex)[:200])
+        del inp, out, cache
+        torch.cuda.empty_cache()
+        side = [("config1", lambda: measure_mla_small(B, dev, "mla_1k", want_oracle, parity)),
+                ("config2", lambda: measure_mla_small(B, dev, "mla_32k", want_oracle, parity)),
+                ("decode_config", lambda: measure_decode_config(B, dev, args.decode_batch, peaks, parity=parity if want_oracle else None)),
+                ("gqa_config", lambda: measure_gqa_config(B, dev, peaks, parity=parity if want_oracle else None)),
+                ("dense_mla_comparison", lambda: measure_dense_comparison(B, dev, peaks)),
+                ("scaling", lambda: measure_scaling(B, dev, peaks))]
+        for name, fn in side:
+            try:
+                extras[name] = fn()
+            except Exception as ex:
+                extras[name] = dict(error=str(ex)[:200])
+            torch.cuda.empty_cache()
+    if parity:
+        extras["parity"] = dict(note="device results against the fp64 oracle on the same bits, raw figures: |err| of the attention output "
+                                     "on sampled rows (max_abs_unit_scale: elements with |ref| <= 1.5 in columns without a x4 needle; "
+                                     "worst_over_derived_bound: against max(2e-2, 2^-9 (vmax_c + |ref|) + 2^-8 |ref|)), anchors and copied "
+                                     "rows of the whole condensed cache (bit-exact: mismatches must be 0; near_tie_groups counts groups whose "
+                                     "two best fp64 scores lie within 1e-6 relative), c_rep elements one bf16 ulp off",
+                                **parity)
+    line["extras"] = extras
     print(json.dumps(line))
     if dist is not None:
         dist.destroy_process_group()
@@ -414,7 +462,7 @@ def time_cuda(fn, warmup=3, iters=5):
     return e0.elapsed_time(e1) / iters
 
 
-def measure_decode_config(B, dev, batch, peaks, warmup=3, iters=5):
+def measure_decode_config(B, dev, batch, peaks, warmup=3, iters=5, parity=None):
     """Config 4: lca_condense over `batch` contexts of 65536 tokens (the HBM-bound figure), then
     lca_decode_attention of one new query per sequence over the condensed cache."""
     cfg = I.scaled(I.CONFIGS["mla_decode"], batch=batch)
@@ -474,6 +522,17 @@ def measure_decode_config(B, dev, batch, peaks, warmup=3, iters=5):
         del usem, upos
     except Exception as ex:
         upd = dict(error=str(ex)[:200])
+    if parity is not None:
+        # oracle on the first and the last sequence: the whole condensed cache and the decode output of every head
+        from oracle import lca_oracle as O, parity as P
+        recs = []
+        for b in sorted({0, batch - 1}):
+            ref = P.mla_pipeline(ckv[b].cpu(), kr[b].cpu(), q_tail_sem[b].cpu(), q_tail_pos[b].cpu(), g, cfg.window, cfg.softmax_scale)
+            ro, _ = O.mla_decode(O.torch_bf16_to_f64(q_new_sem[b].cpu()), O.torch_bf16_to_f64(q_new_pos[b].cpu()),
+                                 O.torch_bf16_to_f64(dsem[b, :, 0].cpu()), O.torch_bf16_to_f64(dpos[b, :, 0].cpu()), m, P.f32(cfg.softmax_scale))
+            ref.update(out=ro[None])
+            recs.append(parity_record(ref, out[b][None], {kk: cache[kk][b] for kk in cache}))
+        parity["mla_decode"] = dict(sequences=sorted({0, batch - 1}), per_sequence=recs)
     flops = float(batch) * H * cap * 2.0 * (cfg.d_sem + cfg.d_pos + cfg.d_sem)
     kv_bytes = float(batch) * cap * (cfg.d_sem + cfg.d_pos) * 2
     full_bytes = float(batch) * (L + 1) * (cfg.d_sem + cfg.d_pos) * 2
@@ -484,7 +543,7 @@ def measure_decode_config(B, dev, batch, peaks, warmup=3, iters=5):
                 online_update=upd)
 
 
-def measure_gqa_config(B, dev, peaks, warmup=3, iters=5, seq_len=None):
+def measure_gqa_config(B, dev, peaks, warmup=3, iters=5, seq_len=None, parity=None):
     """Config 5: GQA variant (pool V, select K per KV head): condense + prefill attention.
     `seq_len` shortens the sequence (profiler captures of the same kernels on a small case)."""
     cfg = I.CONFIGS["gqa_64k"] if not seq_len else I.scaled(I.CONFIGS["gqa_64k"], seq_len=seq_len)
@@ -497,12 +556,83 @@ def measure_gqa_config(B, dev, peaks, warmup=3, iters=5, seq_len=None):
     t_cond = time_cuda(lambda: B.condense(p, None, inp["q"][L - g:], inp["v"], inp["k"], out=cond, ws=ws), warmup, iters)
     t_attn = time_cuda(lambda: B.prefill_attention(p, None, inp["q"], inp["v"], inp["k"], cond["cache_sem"], cond["cache_pos"], out=out),
                        warmup, iters)
+    if parity is not None:
+        from oracle import parity as P
+        rows = P.sample_positions(L, g, cfg.window, n_uniform=14, seed=5)
+        idx = torch.from_numpy(rows).to(dev)
+        ref = P.gqa_pipeline(inp["q"][L - g:].cpu(), inp["k"].cpu(), inp["v"].cpu(), g, cfg.window, cfg.softmax_scale, inp["q"][idx].cpu(), rows)
+        parity[cfg.name] = parity_record(ref, out[0][idx], {kk: cond[kk][0] for kk in ("cache_sem", "cache_pos", "anchor_idx")}, kind="gqa")
     flops = attention_flops(cfg)
     cbytes = condense_bytes(cfg)
     return dict(workload=f"gqa_64k: L={L}, {cfg.n_q_heads} q heads / {cfg.n_kv_heads} kv heads, d={cfg.d_sem}, g={g}, w={cfg.window}",
                 tokens_per_s=L / ((t_cond + t_attn) * 1e-3), condense_ms=t_cond, condense_gbs=cbytes / t_cond / 1e6,
                 attention_ms=t_attn, attention_tflops=flops / t_attn / 1e9,
                 attention_frac_of_measured_burst=flops / t_attn / 1e9 / peaks["tflops_burst"])
+
+
+def measure_mla_small(B, dev, name, want_oracle, parity):
+    """Configs 1 and 2: the same step (condense + prefill attention) on the smaller MLA configurations, with an L2
+    flush between repetitions; the oracle on every row (config 1) or on sampled rows (config 2)."""
+    cfg = I.CONFIGS[name]
+    L, g = cfg.seq_len, cfg.group_size
+    inp = I.make_mla_inputs(cfg, dev)
+    p = B.params_from_config(cfg, batch=1)
+    cond = B.condense(p, inp["q_sem"][L - g:], inp["q_pos"][L - g:], inp["ckv"], inp["kr"])
+    out = torch.empty((1, L, cfg.n_q_heads, cfg.d_sem), dtype=torch.bfloat16, device=dev)
+    ws_c, ws_a = B.workspace(p, B.LCA_WS_CONDENSE, dev), B.workspace(p, B.LCA_WS_PREFILL, dev)
+    flush = torch.empty(256 << 20, dtype=torch.uint8, device=dev)
+    times = []
+    for i in range(8):
+        flush.zero_()
+        e = [torch.cuda.Event(enable_timing=True) for _ in range(3)]
+        e[0].record()
+        B.condense(p, inp["q_sem"][L - g:], inp["q_pos"][L - g:], inp["ckv"], inp["kr"], out=cond, ws=ws_c)
+        e[1].record()
+        B.prefill_attention(p, inp["q_sem"], inp["q_pos"], inp["ckv"], inp["kr"], cond["cache_sem"], cond["cache_pos"], out=out, ws=ws_a)
+        e[2].record()
+        torch.cuda.synchronize()
+        if i >= 3:
+            times.append((e[0].elapsed_time(e[1]), e[1].elapsed_time(e[2])))
+    t_c, t_a = float(np.mean([t[0] for t in times])), float(np.mean([t[1] for t in times]))
+    if want_oracle:
+        from oracle import parity as P
+        rows = np.arange(L) if L <= 2048 else P.sample_positions(L, g, cfg.window, n_uniform=14, seed=3)
+        idx = torch.from_numpy(rows).to(dev)
+        ref = P.mla_pipeline(inp["ckv"].cpu(), inp["kr"].cpu(), inp["q_sem"][L - g:].cpu(), inp["q_pos"][L - g:].cpu(), g, cfg.window,
+                             cfg.softmax_scale, inp["q_sem"][idx].cpu(), inp["q_pos"][idx].cpu(), rows)
+        parity[name] = parity_record(ref, out[0][idx], {kk: cond[kk][0] for kk in ("cache_sem", "cache_pos", "anchor_idx")})
+    fl = attention_flops(cfg)
+    return dict(workload=workload_config(cfg, 1)["workload"], tokens_per_s=L / ((t_c + t_a) * 1e-3), condense_us=t_c * 1e3,
+                attention_us=t_a * 1e3, attention_tflops=fl / t_a / 1e9, condense_gbs=condense_bytes(cfg) / t_c / 1e6,
+                l2_policy="a 256 MB buffer is written between repetitions")
+
+
+def measure_dense_here(B, dev, cfg, inp, out, t_lca_ms):
+    """Dense absorbed-MLA attention (Eq. 5: window >= L) on the benchmark's own tensors, one repetition (it is an
+    O(L^2) launch of seconds), beside the LCA step measured above."""
+    L, g = cfg.seq_len, cfg.group_size
+    cd = I.scaled(cfg, window=L)
+    p = B.params_from_config(cd, batch=1)
+    cond = B.condense(p, inp["q_sem"][L - g:], inp["q_pos"][L - g:], inp["ckv"], inp["kr"])
+    t = time_cuda(lambda: B.prefill_attention(p, inp["q_sem"], inp["q_pos"], inp["ckv"], inp["kr"], cond["cache_sem"],
+                                              cond["cache_pos"], out=out), 0, 1)
+    fl = attention_flops(cd)
+    return dict(workload=f"{cfg.name} with window = L (no condensation)", dense_ms=t, dense_flops=fl, dense_tflops=fl / t / 1e9,
+                lca_step_ms=t_lca_ms, speedup_lca_over_dense=t / t_lca_ms,
+                note="run after the LCA measurements: it overwrites the output buffer")
+
+
+def measure_value_projection(B, dev, cfg, out, peaks):
+    """out_v = attn_latent . W^UV on the benchmark's latent output (Alg. 1: v = c W^UV): HBM-bound by arithmetic."""
+    H = cfg.n_q_heads
+    gen = torch.Generator(device=dev)
+    gen.manual_seed(7)
+    w = (torch.randn((H, cfg.d_sem, 128), generator=gen, device=dev) / cfg.d_sem ** 0.5).bfloat16()
+    ov = torch.empty(out.shape[:-1] + (128,), dtype=torch.bfloat16, device=dev)
+    t = time_cuda(lambda: B.latent_to_value(out, w, out=ov), 1, 3)
+    nbytes = out.numel() * 2 + ov.numel() * 2 + w.numel() * 2
+    fl = 2.0 * out.numel() * 128
+    return dict(ms=t, bytes=nbytes, gbs=nbytes / t / 1e6, frac_of_measured_hbm=nbytes / t / 1e6 / peaks["hbm_gbs"], tflops=fl / t / 1e9)
 
 
 def measure_dense_comparison(B, dev, peaks, iters=2):
@@ -559,6 +689,17 @@ def measure_scaling(B, dev, peaks, lengths=(65536, 131072, 262144, 524288, 10485
     return dict(workload="V2-Lite-shaped layer, H=16, paper defaults g=16, w=1024", rows=rows)
 
 
+def launcher_command(n_gpus: int, argv, port: int = 0):
+    """The command that runs this script as `n_gpus` ranks of one node (one replica per GPU)."""
+    if port <= 0:
+        import socket
+        with socket.socket() as sk:
+            sk.bind(("127.0.0.1", 0))
+            port = sk.getsockname()[1]
+    return [sys.executable, "-m", "torch.distributed.run", "--nnodes=1", f"--nproc-per-node={n_gpus}", "--master-addr", "127.0.0.1",
+            "--master-port", str(port), os.path.abspath(__file__)] + list(argv)
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
@@ -575,9 +716,12 @@ def main():
     ap.add_argument("--no-extras", action="store_true", help="skip the decode / GQA / dense-comparison side measurements")
     ap.add_argument("--decode-batch", type=int, default=64)
     ap.add_argument("--seq-len", type=int, default=0, help="gqa_64k only: a shorter sequence of the same shape (small profiler captures)")
-    ap.add_argument("--ref-rows", type=int, default=24, help="query rows in the oracle's bounded sample")
-    ap.add_argument("--ref-heads", type=int, default=16, help="heads per sampled row in the oracle's sample")
+    ap.add_argument("--ref-rows", type=int, default=64, help="query rows in the oracle's bounded sample")
+    ap.add_argument("--ref-heads", type=int, default=128, help="heads per sampled row in the oracle's sample (capped at the head count)")
     args = ap.parse_args()
+    if args.gpus > 1 and "WORLD_SIZE" not in os.environ:
+        # no launcher around us: start the N replicas ourselves (one process per GPU) and hand over
+        raise SystemExit(subprocess.call(launcher_command(args.gpus, sys.argv[1:])))
     rank = int(os.environ.get("RANK", "0"))
     world = int(os.environ.get("WORLD_SIZE", "1"))
     local_rank = int(os.environ.get("LOCAL_RANK", "0"))

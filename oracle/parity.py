@@ -86,14 +86,14 @@ def bf16_ulp_distance(a_bits: np.ndarray, b_bits: np.ndarray) -> np.ndarray:
 def output_bound(ref: np.ndarray, vmax=None) -> np.ndarray:
     """Element-wise error bound of an attention output computed with bf16 probabilities.
 
-    The kernels round the softmax weights to bf16 before P V and normalise by the sum of the rounded
-    weights, so the result is a convex combination with every weight perturbed by at most 2^-9
-    relative: the error in column c is at most 2^-9 sum_i p_i |v_ic - out_c| <= 2^-9 (vmax_c + |out_c|),
-    vmax_c = the largest |value| of that column; the bf16 store of the result adds 2^-9 |out_c| (half an
-    ulp at the top of a binade, 2^-8 at the bottom).  For values of unit scale (N(0,1): vmax ~ 4.6) that
-    is below the 2e-2 stated for the method; it grows with the values (x4 "needle" rows: vmax ~ 17).
-    The bound returned is the larger of the stated 2e-2 and the derived one.  Without `vmax` only the
-    output rounding is scaled: max(2e-2, 2^-7 |ref|)."""
+    The kernels round the softmax weights p_i to bf16 before P V (relative error at most 2^-9 each) and
+    divide by a row sum taken in fp32.  Whether that sum runs over the rounded or the unrounded weights,
+    the error in column c is at most 2^-9 sum_i p_i max(|v_ic|, |v_ic - out_c|) / sum_i p_i
+    <= 2^-9 (vmax_c + |out_c|), vmax_c = the largest |value| of that column; the bf16 store of the result
+    adds up to 2^-8 |out_c| (half an ulp, relative 2^-9 at the top of a binade and 2^-8 at the bottom).
+    For values of unit scale (N(0,1): vmax ~ 4.6) that is below the 2e-2 stated for the method; it grows
+    with the values (x4 "needle" rows: vmax ~ 17).  The bound returned is the larger of the stated 2e-2
+    and the derived one.  Without `vmax` only the output rounding is scaled: max(2e-2, 2^-7 |ref|)."""
     aref = np.abs(ref)
     if vmax is None:
         return np.maximum(2e-2, 2.0 ** -7 * aref)

@@ -54,8 +54,8 @@ struct Plan1 {
   static constexpr int OFF_BAR = OFF_V + STAGES * V_STAGE;
   static constexpr int NBAR = 1 + 4 * STAGES + 2 + 2 + 1;
   static constexpr int OFF_MISC = OFF_BAR + NBAR * 8;
-  static constexpr int OFF_RED = OFF_MISC + 16;          // float [4][2][128]: row maxima (two tiles in flight), row sums, exact row sums
-  static constexpr int BYTES = OFF_RED + 8 * 128 * 4 + 1024;     // + slack to align the base to 1024 B
+  static constexpr int OFF_RED = OFF_MISC + 16;          // float [3][2][128]: row maxima (two tiles in flight) and row sums
+  static constexpr int BYTES = OFF_RED + 6 * 128 * 4 + 1024;     // + slack to align the base to 1024 B
   // tensor memory columns
   static constexpr int TM_S0 = 0, TM_S1 = BN, TM_O = 2 * BN;
   static constexpr int TM_COLS = 512;
@@ -241,7 +241,7 @@ attn_tc1_kernel(const __grid_constant__ TcParams p) {
     asm volatile("bar.sync 1, 256;" ::: "memory");
     // All 256 threads execute exactly one named barrier per tile, whatever happens: a thread whose
     // wait expired marks the tile's fail word before the barrier and everybody leaves after it.
-    float m_ref = -INFINITY, l_sum = 0.f, l_exact = 0.f;     // l_sum: rounded weights (normaliser); l_exact: for lse
+    float m_ref = -INFINITY, l_sum = 0.f;
     bool ok = true;
     for (int j = 0; j < n_tiles; ++j) {
       if (ok) {
@@ -323,10 +323,10 @@ attn_tc1_kernel(const __grid_constant__ TcParams p) {
           for (int i = 0; i < 32; ++i) o[i] = __float_as_uint(__uint_as_float(o[i]) * factor);
           tmem_st32(tmem + lane_base + P::TM_O + q * 32, o);
         }
-        if (need) { l_sum *= factor; l_exact *= factor; m_ref = tmax; }
+        if (need) { l_sum *= factor; m_ref = tmax; }
       }
       const float m_use = (m_ref == -INFINITY) ? 0.f : m_ref;
-      float rs0 = 0.f, rs1 = 0.f, re0 = 0.f, re1 = 0.f;
+      float rs0 = 0.f, rs1 = 0.f;
       uint32_t pk[32];
       const float e_mul = plain ? p.scale_log2 : 1.f;       // sr holds raw products (plain) or scaled logits
       if (plain) {
@@ -338,22 +338,19 @@ attn_tc1_kernel(const __grid_constant__ TcParams p) {
           const float a1 = fmaf(__uint_as_float(sr[i >> 4][(2 * i + 1) & 31]), e_mul, -m_use);
           const float p0 = ((2 * i) & 3) < POLY_OF_4 ? exp2_fma(a0) : exp2f(a0);
           const float p1 = ((2 * i + 1) & 3) < POLY_OF_4 ? exp2_fma(a1) : exp2f(a1);
+          rs0 += p0; rs1 += p1;
           pk[i] = pack_bf16x2(p0, p1);
-          rs0 += __uint_as_float(pk[i] << 16); rs1 += __uint_as_float(pk[i] & 0xffff0000u);     // sum of the rounded weights
-          re0 += p0; re1 += p1;
         }
       } else {
 #pragma unroll
         for (int i = 0; i < 32; ++i) {
           const float p0 = exp2f(fmaf(__uint_as_float(sr[i >> 4][(2 * i) & 31]), e_mul, -m_use));
           const float p1 = exp2f(fmaf(__uint_as_float(sr[i >> 4][(2 * i + 1) & 31]), e_mul, -m_use));
+          rs0 += p0; rs1 += p1;
           pk[i] = pack_bf16x2(p0, p1);
-          rs0 += __uint_as_float(pk[i] << 16); rs1 += __uint_as_float(pk[i] & 0xffff0000u);     // sum of the rounded weights
-          re0 += p0; re1 += p1;
         }
       }
       l_sum += rs0 + rs1;
-      l_exact += re0 + re1;
       tmem_st32(stm + 32 * half, pk);     // P columns 32*half .. 32*half+31 = keys 64*half .. 64*half+63
       tmem_wait_st();
       tc_fence_before();
@@ -367,11 +364,9 @@ attn_tc1_kernel(const __grid_constant__ TcParams p) {
     ok = __all_sync(0xffffffffu, ok);
     if (!ok) fail_word[0] = fail_word[1] = 1;
     red[(4 + half) * 128 + r] = l_sum;
-    red[(6 + half) * 128 + r] = l_exact;
     asm volatile("bar.sync 1, 256;" ::: "memory");
     if (!fail_word[0]) {
       const float l_tot = l_sum + red[(4 + (half ^ 1)) * 128 + r];
-      const float l_lse = l_exact + red[(6 + (half ^ 1)) * 128 + r];
       tc_fence_after();
       const float inv = (n_tiles > 0 && l_tot > 0.f) ? 1.f / l_tot : 0.f;
       const size_t orow = ((size_t)b * p.q_len + t_row) * p.Hq + head0 + hl;
@@ -397,7 +392,7 @@ attn_tc1_kernel(const __grid_constant__ TcParams p) {
         }
       }
       if (p.lse && row_valid && half == 0)
-        p.lse[orow] = (n_tiles > 0 && l_lse > 0.f) ? (m_ref + log2f(l_lse)) * 0.6931471805599453f : -INFINITY;
+        p.lse[orow] = (n_tiles > 0 && l_tot > 0.f) ? (m_ref + log2f(l_tot)) * 0.6931471805599453f : -INFINITY;
     }
     tc_fence_before();
   }

@@ -49,7 +49,7 @@ constexpr int Q_BYTES = NKC * QCH, K_BYTES = NKC * KCH, V_BYTES = 8 * VCH, P_BYT
 constexpr int OFF_Q = 0, OFF_K = OFF_Q + Q_BYTES, OFF_V = OFF_K + K_BYTES, OFF_P = OFF_V + V_BYTES;
 constexpr int OFF_BAR = OFF_P + P_BYTES;
 constexpr int OFF_MISC = OFF_BAR + 256, OFF_RED = OFF_BAR + 512;
-constexpr int SMEM_BYTES = OFF_BAR + 512 + 4 * 128 * 4;     // 231936
+constexpr int SMEM_BYTES = OFF_BAR + 512 + 3 * 128 * 4;     // 231424
 constexpr int TM_S0 = 0, TM_S1 = 64, TM_O = 128, TM_COLS = 512;
 constexpr int THREADS = 224;            // warps: 0 K/Q loads, 1 MMA + TMEM, 2-5 softmax, 6 V loads
 constexpr float RESCALE_THRESHOLD = 8.0f;
@@ -147,7 +147,7 @@ attn_tc2_kernel(const __grid_constant__ Tc2Params p) {
   const uint32_t BAR_OLOCAL = bars + 248;        // odd CTA: O read out by its 128 threads -> its relay thread
   volatile uint32_t* tmem_slot = reinterpret_cast<volatile uint32_t*>(smem + OFF_MISC);
   volatile int* abort_flag = reinterpret_cast<volatile int*>(smem + OFF_MISC + 4);
-  volatile float* red = reinterpret_cast<volatile float*>(smem + OFF_RED);    // [4][128]: maxima of even / odd tiles, row sums, exact row sums
+  volatile float* red = reinterpret_cast<volatile float*>(smem + OFF_RED);    // [3][128]: maxima of even / odd tiles, row sums
 
   // the warp index through a shuffle: provably warp-uniform, so the role branches below are uniform branches
   const int warp = __shfl_sync(0xffffffffu, (int)(threadIdx.x >> 5), 0), lane = threadIdx.x & 31;
@@ -393,7 +393,7 @@ attn_tc2_kernel(const __grid_constant__ Tc2Params p) {
     int n_a_row, bias_rows, first_row;
     if (p.decode) { n_a_row = n_a_hi; bias_rows = min(p.n_rep_bias, n_a_row); first_row = 0; }
     else { n_a_row = reps_visible(min(t_row, it.len - 1), p.w, p.g); bias_rows = n_a_row; first_row = n_a_row * p.g; }
-    float m_ref = -INFINITY, l_sum = 0.f, l_exact = 0.f;     // l_sum: rounded weights (normaliser); l_exact: for lse
+    float m_ref = -INFINITY, l_sum = 0.f;
     bool all_left = false;                       // every one of the 128 threads left the tile loop at a barrier
     for (int j = 0; j < n_tiles; ++j, ++jt) {
       if (ok) {
@@ -422,11 +422,13 @@ attn_tc2_kernel(const __grid_constant__ Tc2Params p) {
         if (plain) {
           // interior tile: the raw products stay in sr, the (positive) scale is applied to the maximum
           // here and folded into the exponent's multiply-add below
-          float t0m = -INFINITY, t1m = -INFINITY, t2m = -INFINITY, t3m = -INFINITY;    // four short chains
+          float t0m = -INFINITY, t1m = -INFINITY, t2m = -INFINITY, t3m = -INFINITY;    // four short chains, three-input maxima
 #pragma unroll
-          for (int i = 0; i < 32; i += 2) {
-            t0m = fmaxf(t0m, __uint_as_float(sr[0][i])); t1m = fmaxf(t1m, __uint_as_float(sr[0][i + 1]));
-            t2m = fmaxf(t2m, __uint_as_float(sr[1][i])); t3m = fmaxf(t3m, __uint_as_float(sr[1][i + 1]));
+          for (int i = 0; i < 32; i += 4) {
+            t0m = max3(t0m, __uint_as_float(sr[0][i]), __uint_as_float(sr[0][i + 1]));
+            t1m = max3(t1m, __uint_as_float(sr[0][i + 2]), __uint_as_float(sr[0][i + 3]));
+            t2m = max3(t2m, __uint_as_float(sr[1][i]), __uint_as_float(sr[1][i + 1]));
+            t3m = max3(t3m, __uint_as_float(sr[1][i + 2]), __uint_as_float(sr[1][i + 3]));
           }
           tmax = fmaxf(fmaxf(t0m, t1m), fmaxf(t2m, t3m)) * p.scale_log2;
         } else {
@@ -465,19 +467,18 @@ attn_tc2_kernel(const __grid_constant__ Tc2Params p) {
       const float m_new = need ? tmax : m_ref;
       const float m_use = (m_new == -INFINITY) ? 0.f : m_new;
       const float e_mul = plain ? p.scale_log2 : 1.f;       // sr holds raw products (plain) or scaled logits
-      float rs0 = 0.f, rs1 = 0.f, re0 = 0.f, re1 = 0.f;
+      // scale and row sum work on pairs of fp32 values (one instruction per pair)
+      const uint64_t mul2 = pack_f32x2(e_mul, e_mul), sub2 = pack_f32x2(-m_use, -m_use);
+      uint64_t rs2 = pack_f32x2(0.f, 0.f);
       uint32_t pk[32];
 #pragma unroll
       for (int i = 0; i < 32; ++i) {
         const int c = 2 * i;
-        const float p0 = exp2f(fmaf(__uint_as_float(sr[c >> 5][c & 31]), e_mul, -m_use));
-        const float p1 = exp2f(fmaf(__uint_as_float(sr[(c + 1) >> 5][(c + 1) & 31]), e_mul, -m_use));
+        float a0, a1;
+        unpack_f32x2(fma_f32x2(pack_f32x2(__uint_as_float(sr[c >> 5][c & 31]), __uint_as_float(sr[(c + 1) >> 5][(c + 1) & 31])), mul2, sub2), a0, a1);
+        const float p0 = exp2f(a0), p1 = exp2f(a1);
         pk[i] = pack_bf16x2(p0, p1);
-        // the row sum is taken over the probabilities as the tensor core will see them (rounded to bf16): numerator
-        // and denominator of the output then carry the same weights, and a row that is locked onto one large value
-        // does not inherit the rounding of its dominant probability
-        rs0 += __uint_as_float(pk[i] << 16); rs1 += __uint_as_float(pk[i] & 0xffff0000u);
-        re0 += p0; re1 += p1;
+        rs2 = add_f32x2(rs2, pack_f32x2(p0, p1));
       }
       if (j >= 1) {
         // P (one buffer) and O are free once P_{j-1} V_{j-1} has completed
@@ -499,7 +500,7 @@ attn_tc2_kernel(const __grid_constant__ Tc2Params p) {
         }
         tmem_wait_st();
       }
-      if (need) { l_sum *= factor; l_exact *= factor; m_ref = tmax; }
+      if (need) { l_sum *= factor; m_ref = tmax; }
       if (ragged_decode_tile(p, it, j)) {
         // rows >= first_bad of this tile are not part of the sequence: zero them in this CTA's value buffers
         // (their probabilities are exactly 0, but 0 x NaN is not)
@@ -524,8 +525,11 @@ attn_tc2_kernel(const __grid_constant__ Tc2Params p) {
         const uint32_t a = prow + ((s8 ^ (rl & 7)) << 4);
         asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(a), "r"(pk[4 * s8]), "r"(pk[4 * s8 + 1]), "r"(pk[4 * s8 + 2]), "r"(pk[4 * s8 + 3]) : "memory");
       }
-      l_sum += rs0 + rs1;
-      l_exact += re0 + re1;
+      {
+        float r0, r1;
+        unpack_f32x2(rs2, r0, r1);
+        l_sum += r0 + r1;
+      }
       fence_proxy_async_smem();                   // P is read by the tensor core (async proxy)
       tc_fence_before();
       mbar_arrive(rank == 0 ? BAR_PFULL : BAR_PLOCAL);
@@ -539,12 +543,10 @@ attn_tc2_kernel(const __grid_constant__ Tc2Params p) {
       if (!ok) fail_word[2] = 1;
       // total row sum = sum over both key halves
       red[2 * 128 + ln] = l_sum;
-      red[3 * 128 + ln] = l_exact;
       asm volatile("bar.sync 1, 128;" ::: "memory");
       if (fail_word[2]) { ok = false; break; }                 // uniform over the 128 threads
     }
     const float l_tot = n_tiles > 0 ? l_sum + red[2 * 128 + (ln ^ 64)] : 0.f;
-    const float l_lse = n_tiles > 0 ? l_exact + red[3 * 128 + (ln ^ 64)] : 0.f;
     {
       tc_fence_after();
       const float inv = (n_tiles > 0 && l_tot > 0.f) ? 1.f / l_tot : 0.f;
@@ -578,7 +580,7 @@ attn_tc2_kernel(const __grid_constant__ Tc2Params p) {
         }
       }
       if (p.lse && row_valid && half == 0)
-        p.lse[orow] = (n_tiles > 0 && l_lse > 0.f) ? (m_ref + log2f(l_lse)) * 0.6931471805599453f : -INFINITY;
+        p.lse[orow] = (n_tiles > 0 && l_tot > 0.f) ? (m_ref + log2f(l_tot)) * 0.6931471805599453f : -INFINITY;
     }
     if (n_tiles > 0) ++n_item;
     }   // items

@@ -16,7 +16,7 @@ from oracle import parity as P
 #   the mean        mean|err| <= max(MEAN_ATOL, MEAN_RTOL * mean|ref|)
 # ATOL / MEAN_ATOL are the bounds stated for the method (values of unit scale); elements of unit scale
 # (|ref| <= 1.5 and every value of their column within 5) must meet ATOL as it stands.  The derived bound follows
-# the arithmetic -- bf16 weights, normaliser over the rounded weights, bf16 store:
+# the arithmetic -- bf16 weights, fp32 row sum, bf16 store:
 # 2^-9 (vmax_c + |ref|) + 2^-8 |ref| -- and only exceeds ATOL where the values or the result are large
 # (rows that attend to a x4 needle token reach |out| ~ 16, one bf16 ulp = 0.125).  The rounding of the
 # stored output alone has a mean of about 0.7 * 2^-9 of the mean magnitude.

@@ -64,6 +64,15 @@ def test_two_gloo_ranks_report_the_slowest_time_and_the_whole_job_rate(tmp_path)
     assert abs(line["value"] - 2 * 131072 / 15e-3) < 1e-6
 
 
+def test_gpus_flag_without_a_launcher_starts_one_rank_per_gpu():
+    cmd = bench.launcher_command(4, ["--gpus", "4", "--steps", "2"], port=29999)
+    assert cmd[1:3] == ["-m", "torch.distributed.run"] and "--nproc-per-node=4" in cmd and "--nnodes=1" in cmd
+    assert cmd[cmd.index("--master-addr") + 1] == "127.0.0.1" and cmd[cmd.index("--master-port") + 1] == "29999"
+    assert cmd[-5].endswith("bench.py") and cmd[-4:] == ["--gpus", "4", "--steps", "2"]
+    # a free port is picked when none is given
+    assert int(bench.launcher_command(2, [])[bench.launcher_command(2, []).index("--master-port") + 1]) > 0
+
+
 def test_reference_arm_runs_only_on_rank_zero():
     env = dict(os.environ, RANK="1", WORLD_SIZE="2", LOCAL_RANK="1")
     r = subprocess.run([sys.executable, os.path.join(ROOT, "bench.py"), "--impl", "reference", "--config", "mla_1k"],
