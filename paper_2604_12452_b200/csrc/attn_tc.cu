@@ -469,7 +469,9 @@ int attn_gqa2_launch(const AttnProblem& a);
 int attn_gqa2_take_status();
 
 bool attn_tc_supported(const AttnProblem& a) { return gqa128_shape(a) || attn_tc2_supported(a); }
-size_t attn_tc_workspace_bytes(const AttnProblem&) { return 0; }
+size_t attn_tc_workspace_bytes(const AttnProblem& a) {
+  return (a.decode && attn_tc2_supported(a)) ? attn_tc2_decode_workspace_bytes(a.batch, a.n_q_heads) : 0;
+}
 
 int attn_tc_launch(const AttnProblem& a) {
   if (attn_tc2_supported(a)) return attn_tc2_launch(a);

@@ -71,13 +71,22 @@ struct Tc2Params {
   const int2* entries;
   SeqTab tab;
   float scale_log2, bias_log2;
+  // Split decode (few sequences): the key tiles of all (sequence, head block) units form one line that is cut into
+  // equal ranges, one per CTA pair; a range that does not hold a whole unit leaves an unnormalised partial result
+  // (O, row maximum, row sum) in `partial`, merged by decode_combine_kernel.  split = 0: one unit per work item.
+  int split;
+  float* partial;                 // [slots][PARTIAL_FLOATS]
 };
+constexpr int PARTIAL_FLOATS = 128 * 512 + 2 * 128;     // O of 128 rows, then (maximum, sum) per row
 
-// One work item = one tile of 128 query rows; the same arithmetic in every role of both CTAs.
+// One work item = one tile of 128 query rows (split decode: a range of its key tiles); the same arithmetic in every
+// role of both CTAs.
 struct Item {
   int b, head0, t0, t1, len;      // sequence, first head, first / last token of the tile, length of the sequence
   int qbase, kbase, cbase;        // row of the sequence's first token in the query / token arrays, of its first cache row
   int n_a_lo, n_a_hi, first_lo, nA, n_tiles;
+  int j0;                         // split decode: first key tile of the range (0 otherwise)
+  int slot;                       // split decode: >= 0 where the range is only a part of its unit
 };
 __device__ __forceinline__ Item make_item(const Tc2Params& p, long long idx) {
   Item it;
@@ -101,6 +110,7 @@ __device__ __forceinline__ Item make_item(const Tc2Params& p, long long idx) {
   }
   it.t0 = tile * p.TB;
   it.t1 = min(it.t0 + p.TB, it.len) - 1;
+  it.j0 = 0; it.slot = -1;
   int nB;
   if (p.decode) {
     it.n_a_hi = it.n_a_lo = min(max(p.cache_rows[it.b], 0), p.cap);
@@ -116,9 +126,92 @@ __device__ __forceinline__ Item make_item(const Tc2Params& p, long long idx) {
   return it;
 }
 
+// Key tiles of decode unit u = (sequence, head block), head block fastest.
+__device__ __forceinline__ int unit_tiles(const Tc2Params& p, int u) {
+  const int rows = min(max(p.cache_rows[u / p.n_head_blocks], 0), p.cap);
+  return (rows + pair::BN - 1) / pair::BN;
+}
+// Ranges (one per pair, `q` tiles long) that touch a unit of n > 0 tiles starting at tile `off` of the line.
+__device__ __forceinline__ int unit_ranges(long long off, int n, long long q) {
+  return (int)((off + n - 1) / q - off / q) + 1;
+}
+
+// The walk of one role over the work items of its CTA pair.  Every role of both CTAs runs the same walk.
+struct Walk {
+  long long idx, stride;          // one unit / tile per item: next item, number of pairs
+  long long cur, end, q, off;     // split decode: next tile of the line, end of this pair's range, range length,
+  int u, slot_base, n_units;      //   first tile of unit u, first partial slot of unit u
+  long long pair_id;
+};
+// Split decode: where the range of this pair starts, found once per CTA by one warp (units in chunks of 32, prefix
+// sums by shuffles) and left in shared memory for every role: {q, cur, end, off, u, slot_base}.
+__device__ __forceinline__ void split_start(const Tc2Params& p, long long pair_id, long long n_pairs, int lane, volatile int* dst) {
+  const int n_units = p.B * p.n_head_blocks;
+  int total = 0;
+  for (int u0 = 0; u0 < n_units; u0 += 32) {
+    const int n = u0 + lane < n_units ? unit_tiles(p, u0 + lane) : 0;
+    total += __reduce_add_sync(0xffffffffu, n);
+  }
+  const int q = total > 0 ? (int)((total + n_pairs - 1) / n_pairs) : 1;
+  const int cur = (int)min(pair_id * q, (long long)total), end = min(total, cur + q);
+  int off = 0, slot_base = 0, u_found = n_units, off_found = total, slot_found = 0;
+  for (int u0 = 0; u0 < n_units && u_found == n_units; u0 += 32) {
+    const int n = u0 + lane < n_units ? unit_tiles(p, u0 + lane) : 0;
+    int incl = n;                                            // inclusive prefix of the tile counts
+#pragma unroll
+    for (int o = 1; o < 32; o <<= 1) { const int t = __shfl_up_sync(0xffffffffu, incl, o); if (lane >= o) incl += t; }
+    const int my_off = off + incl - n;
+    const int r = n > 0 ? unit_ranges(my_off, n, q) : 0;
+    int rincl = r;                                           // inclusive prefix of the range counts
+#pragma unroll
+    for (int o = 1; o < 32; o <<= 1) { const int t = __shfl_up_sync(0xffffffffu, rincl, o); if (lane >= o) rincl += t; }
+    const bool holds = n > 0 && my_off <= cur && cur < my_off + n;
+    const unsigned who = __ballot_sync(0xffffffffu, holds);
+    if (who) {
+      const int src = __ffs(who) - 1;
+      u_found = u0 + src;
+      off_found = __shfl_sync(0xffffffffu, my_off, src);
+      slot_found = slot_base + __shfl_sync(0xffffffffu, rincl - r, src);
+    }
+    off += __shfl_sync(0xffffffffu, incl, 31);
+    slot_base += __shfl_sync(0xffffffffu, rincl, 31);
+  }
+  if (lane == 0) { dst[0] = q; dst[1] = cur; dst[2] = end; dst[3] = off_found; dst[4] = u_found; dst[5] = slot_found; }
+}
+__device__ __forceinline__ void walk_init(const Tc2Params& p, Walk& w, long long pair_id, long long n_pairs, const volatile int* start) {
+  w.idx = pair_id; w.stride = n_pairs; w.pair_id = pair_id;
+  if (!p.split) return;
+  w.n_units = p.B * p.n_head_blocks;
+  w.q = start[0]; w.cur = start[1]; w.end = start[2]; w.off = start[3]; w.u = start[4]; w.slot_base = start[5];
+}
+__device__ __forceinline__ bool walk_next(const Tc2Params& p, Walk& w, Item& it) {
+  if (!p.split) {
+    if (w.idx >= p.n_items) return false;
+    it = make_item(p, w.idx);
+    w.idx += w.stride;
+    return true;
+  }
+  if (w.cur >= w.end) return false;
+  int n = unit_tiles(p, w.u);
+  while (n == 0) { ++w.u; n = unit_tiles(p, w.u); }          // cur < total: a unit with tiles follows
+  const int j0 = (int)(w.cur - w.off);
+  const int j1 = (int)min((long long)n, j0 + (w.end - w.cur));
+  it.b = w.u / p.n_head_blocks;
+  it.head0 = (w.u % p.n_head_blocks) * p.HB;
+  it.len = 1; it.t0 = 0; it.t1 = 0;
+  it.qbase = it.b * p.q_len; it.kbase = 0; it.cbase = it.b * p.cap;
+  it.n_a_hi = it.n_a_lo = min(max(p.cache_rows[it.b], 0), p.cap);
+  it.first_lo = 0;
+  it.j0 = j0; it.nA = it.n_tiles = j1 - j0;
+  it.slot = (j0 == 0 && j1 == n) ? -1 : w.slot_base + (int)(w.pair_id - w.off / w.q);
+  w.cur += j1 - j0;
+  if (j1 == n) { w.slot_base += unit_ranges(w.off, n, w.q); w.off += n; ++w.u; }
+  return true;
+}
+
 // Decode only: tile j of the item contains cache rows at or behind the sequence's valid row count.
 __device__ __forceinline__ bool ragged_decode_tile(const Tc2Params& p, const Item& it, int j) {
-  return p.decode && (j + 1) * pair::BN > it.n_a_hi;
+  return p.decode && (it.j0 + j + 1) * pair::BN > it.n_a_hi;
 }
 
 __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(pair::THREADS, 1)
@@ -170,6 +263,8 @@ attn_tc2_kernel(const __grid_constant__ Tc2Params p) {
     tmem_alloc_pair(smem_u32((const void*)tmem_slot), TM_COLS);
     tmem_relinquish_pair();
   }
+  volatile int* split_state = reinterpret_cast<volatile int*>(smem + OFF_MISC + 32);   // [6], split decode only
+  if (p.split && warp == 0) split_start(p, pair_id, n_pairs, lane, split_state);
   tc_fence_before();
   __syncthreads();
   cluster_sync_all();                              // both CTAs' barriers are initialised
@@ -191,8 +286,10 @@ attn_tc2_kernel(const __grid_constant__ Tc2Params p) {
       const uint32_t q_bar = mapa_u32(BAR_Q, 0);
       uint32_t jt = 0, n_item = 0;
       bool good = true;
-      for (long long idx = pair_id; good && idx < p.n_items; idx += n_pairs) {
-        const Item it = make_item(p, idx);
+      Walk wk;
+      walk_init(p, wk, pair_id, n_pairs, split_state);
+      Item it;
+      while (good && walk_next(p, wk, it)) {
         if (it.n_tiles == 0) continue;             // nothing to attend to (decode with an empty cache): no loads, no phases
         // the query tile may be replaced once the last S of the previous item has completed
         if (!mbar_wait(BAR_QFREE, (n_item & 1) ^ 1, abort_flag)) { fail(ERR_WAIT_Q); break; }
@@ -203,7 +300,7 @@ attn_tc2_kernel(const __grid_constant__ Tc2Params p) {
         ++n_item;
         for (int j = 0; good && j < it.n_tiles; ++j, ++jt) {
           const bool isA = j < it.nA;
-          const int row = (isA ? it.cbase + j * BN : it.kbase + it.first_lo + (j - it.nA) * BN) + 64 * (int)rank;
+          const int row = (isA ? it.cbase + (it.j0 + j) * BN : it.kbase + it.first_lo + (j - it.nA) * BN) + 64 * (int)rank;
           const CUtensorMap* ms = isA ? &p.c_sem : &p.k_sem;
           const CUtensorMap* mp = isA ? &p.c_pos : &p.k_pos;
           if (p.decode) {
@@ -228,11 +325,13 @@ attn_tc2_kernel(const __grid_constant__ Tc2Params p) {
     if (lane == 0 && !*abort_flag) {
       uint32_t jt = 0;
       bool good = true;
-      for (long long idx = pair_id; good && idx < p.n_items; idx += n_pairs) {
-        const Item it = make_item(p, idx);
+      Walk wk;
+      walk_init(p, wk, pair_id, n_pairs, split_state);
+      Item it;
+      while (good && walk_next(p, wk, it)) {
         for (int j = 0; good && j < it.n_tiles; ++j, ++jt) {
           const bool isA = j < it.nA;
-          const int row = isA ? it.cbase + j * BN : it.kbase + it.first_lo + (j - it.nA) * BN;
+          const int row = isA ? it.cbase + (it.j0 + j) * BN : it.kbase + it.first_lo + (j - it.nA) * BN;
           const CUtensorMap* mv = isA ? &p.c_val : &p.k_val;
           // Decode, last tile of a sequence whose valid rows end inside it: the rows behind them may hold anything
           // (0 x NaN would reach O), so the softmax threads of each CTA zero them in their own value buffers before
@@ -303,8 +402,10 @@ attn_tc2_kernel(const __grid_constant__ Tc2Params p) {
         if (pend_last) umma_commit_pair_elected(leader, BAR_OLAST, 3);      // one phase per item, for the epilogue
         return true;
       };
-      for (long long idx = pair_id; ok && idx < p.n_items; idx += n_pairs) {
-        const Item it = make_item(p, idx);
+      Walk wk;
+      walk_init(p, wk, pair_id, n_pairs, split_state);
+      Item it;
+      while (ok && walk_next(p, wk, it)) {
         if (it.n_tiles == 0) continue;
         for (int j = 0; ok && j < it.n_tiles; ++j, ++jt) {
           // In the middle of an item S of tile j goes before P V of tile j - 1.  At an item boundary the
@@ -356,8 +457,10 @@ attn_tc2_kernel(const __grid_constant__ Tc2Params p) {
       const uint32_t pfull_addr = mapa_u32(BAR_PFULL, 0), ofree_addr = mapa_u32(BAR_OFREE, 0);
       uint32_t jt = 0, n_item = 0;
       bool good = true;
-      for (long long idx = pair_id; good && idx < p.n_items; idx += n_pairs) {
-        const Item it = make_item(p, idx);
+      Walk wk;
+      walk_init(p, wk, pair_id, n_pairs, split_state);
+      Item it;
+      while (good && walk_next(p, wk, it)) {
         if (it.n_tiles == 0) continue;
         for (int j = 0; j < it.n_tiles; ++j, ++jt) {
           if (!mbar_wait(BAR_PLOCAL, jt & 1, abort_flag)) { fail(ERR_WAIT_P_FULL); good = false; break; }
@@ -384,8 +487,10 @@ attn_tc2_kernel(const __grid_constant__ Tc2Params p) {
     // thread whose wait expired marks the fail word before the barrier and everybody leaves after it.
     bool ok = !*abort_flag;
     uint32_t jt = 0, n_item = 0, n_ragged = 0;   // tiles / non-empty items / ragged decode tiles of this pair so far
-    for (long long idx = pair_id; ok && idx < p.n_items; idx += n_pairs) {
-    const Item it = make_item(p, idx);
+    Walk wk;
+    walk_init(p, wk, pair_id, n_pairs, split_state);
+    Item it;
+    while (ok && walk_next(p, wk, it)) {
     const int head0 = it.head0, t0 = it.t0, nA = it.nA, n_tiles = it.n_tiles;
     const int n_a_lo = it.n_a_lo, n_a_hi = it.n_a_hi, first_lo = it.first_lo;
     const int t_row = t0 + tl;
@@ -406,7 +511,7 @@ attn_tc2_kernel(const __grid_constant__ Tc2Params p) {
       float tmax = -INFINITY;
       bool plain = false;
       const bool isA = j < nA;
-      const int tile_key0 = isA ? j * BN : first_lo + (j - nA) * BN;
+      const int tile_key0 = isA ? (it.j0 + j) * BN : first_lo + (j - nA) * BN;
       const int key0 = tile_key0 + 64 * half;     // first key of this thread's 64 columns
       if (ok) {
         tc_fence_after();
@@ -512,7 +617,7 @@ attn_tc2_kernel(const __grid_constant__ Tc2Params p) {
         ok = __all_sync(0xffffffffu, vok);
         if (!ok) continue;                                   // reported at the next tile's barrier
         ++n_ragged;
-        const int first_bad = n_a_hi - j * BN;               // 1 .. 127
+        const int first_bad = n_a_hi - (it.j0 + j) * BN;     // 1 .. 127
         for (int x = ln; x < (BN - first_bad) * 32; x += 128) {
           const int kr = first_bad + (x >> 5), chunk = (x >> 3) & 3, piece = x & 7;
           const uint32_t a = sV + ((kr >> 6) * 4 + chunk) * VCH + (kr & 63) * 128 + piece * 16;
@@ -565,9 +670,19 @@ attn_tc2_kernel(const __grid_constant__ Tc2Params p) {
           tc_fence_before();
           mbar_arrive(rank == 0 ? BAR_OFREE : BAR_OLOCAL);
         }
-        if (row_valid) {
-          // TMEM columns [0,128): output columns 128*half + c ; [128,256): 256 + 128*half + (c-128)
-          const int col = (q >> 2) * 256 + 128 * half + (q & 3) * 32;
+        // TMEM columns [0,128): output columns 128*half + c ; [128,256): 256 + 128*half + (c-128)
+        const int col = (q >> 2) * 256 + 128 * half + (q & 3) * 32;
+        if (row_valid && it.slot >= 0) {
+          // a part of the unit's key tiles: the unnormalised accumulator goes to the partial slot (fp32)
+          float* pd = p.partial + (size_t)it.slot * PARTIAL_FLOATS + (size_t)rg * 512 + col;
+#pragma unroll
+          for (int v = 0; v < 4; ++v) {
+            uint32_t w[8];
+#pragma unroll
+            for (int e = 0; e < 8; ++e) w[e] = o[8 * v + e];
+            st_global_32B(pd + 8 * v, w, true);
+          }
+        } else if (row_valid) {
           // 32 bytes per store: every lane writes whole sectors of its own row
 #pragma unroll
           for (int v = 0; v < 2; ++v) {
@@ -579,7 +694,10 @@ attn_tc2_kernel(const __grid_constant__ Tc2Params p) {
           }
         }
       }
-      if (p.lse && row_valid && half == 0)
+      if (row_valid && half == 0 && it.slot >= 0) {
+        float* ml = p.partial + (size_t)it.slot * PARTIAL_FLOATS + 128 * 512 + 2 * rg;
+        ml[0] = m_ref; ml[1] = l_tot;
+      } else if (p.lse && row_valid && half == 0)
         p.lse[orow] = (n_tiles > 0 && l_tot > 0.f) ? (m_ref + log2f(l_tot)) * 0.6931471805599453f : -INFINITY;
     }
     if (n_tiles > 0) ++n_item;
@@ -597,6 +715,62 @@ attn_tc2_kernel(const __grid_constant__ Tc2Params p) {
     tc_fence_after();
     tmem_dealloc_pair(tmem, TM_COLS);
   }
+}
+
+// Split decode, second step: one CTA of 128 threads per (unit, head): four output columns per thread.  Units whose
+// key tiles were all taken by one pair are complete already; units without any valid row get zeros (lse = -inf);
+// the others are merged from their partial results in range order:
+//     out = sum_s O_s 2^(m_s - M) / sum_s l_s 2^(m_s - M),   M = max_s m_s.
+__global__ void __launch_bounds__(128) decode_combine_kernel(const Tc2Params p, int n_pairs) {
+  const int u = blockIdx.x / p.HB, hl = blockIdx.x % p.HB, lane = threadIdx.x & 31;
+  const int n_units = p.B * p.n_head_blocks;
+  // every warp repeats the scan over the units (chunks of 32, prefix sums by shuffles): tiles before unit u, slots before it
+  int total = 0;
+  for (int u0 = 0; u0 < n_units; u0 += 32) total += __reduce_add_sync(0xffffffffu, u0 + lane < n_units ? unit_tiles(p, u0 + lane) : 0);
+  const int q = total > 0 ? (total + n_pairs - 1) / n_pairs : 1;
+  int off = 0, slot_base = 0, n = 0, my_slot = 0, n_seg = 0;
+  for (int u0 = 0; u0 <= u; u0 += 32) {
+    const int nn = u0 + lane < n_units ? unit_tiles(p, u0 + lane) : 0;
+    int incl = nn;
+#pragma unroll
+    for (int o = 1; o < 32; o <<= 1) { const int t = __shfl_up_sync(0xffffffffu, incl, o); if (lane >= o) incl += t; }
+    const int r = nn > 0 ? unit_ranges(off + incl - nn, nn, q) : 0;
+    int rincl = r;
+#pragma unroll
+    for (int o = 1; o < 32; o <<= 1) { const int t = __shfl_up_sync(0xffffffffu, rincl, o); if (lane >= o) rincl += t; }
+    if (u < u0 + 32) {
+      const int src = u - u0;
+      n = __shfl_sync(0xffffffffu, nn, src);
+      n_seg = __shfl_sync(0xffffffffu, r, src);
+      my_slot = slot_base + __shfl_sync(0xffffffffu, rincl - r, src);
+    }
+    off += __shfl_sync(0xffffffffu, incl, 31);
+    slot_base += __shfl_sync(0xffffffffu, rincl, 31);
+  }
+  if (n_seg == 1) return;
+  const int b = u / p.n_head_blocks, head0 = (u % p.n_head_blocks) * p.HB;
+  const int c4 = threadIdx.x;                               // columns 4 c4 .. 4 c4 + 3
+  const size_t orow = (size_t)b * p.H + head0 + hl;         // q_len = 1
+  const float* base = p.partial + (size_t)my_slot * PARTIAL_FLOATS;
+  float M = -INFINITY;
+  for (int sgm = 0; sgm < n_seg; ++sgm) M = fmaxf(M, base[(size_t)sgm * PARTIAL_FLOATS + 128 * 512 + 2 * hl]);
+  float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
+  float Lsum = 0.f;
+#pragma unroll 4
+  for (int sgm = 0; sgm < n_seg; ++sgm) {
+    const float* ps = base + (size_t)sgm * PARTIAL_FLOATS;
+    const float ms = ps[128 * 512 + 2 * hl], ls = ps[128 * 512 + 2 * hl + 1];
+    const float4 o = *reinterpret_cast<const float4*>(ps + (size_t)hl * 512 + 4 * c4);
+    const float f = (ms == -INFINITY) ? 0.f : exp2f(ms - M);
+    acc.x = fmaf(o.x, f, acc.x); acc.y = fmaf(o.y, f, acc.y); acc.z = fmaf(o.z, f, acc.z); acc.w = fmaf(o.w, f, acc.w);
+    Lsum = fmaf(ls, f, Lsum);
+  }
+  const float inv = Lsum > 0.f ? 1.f / Lsum : 0.f;
+  uint2 w;
+  w.x = pack_bf16x2(acc.x * inv, acc.y * inv); w.y = pack_bf16x2(acc.z * inv, acc.w * inv);
+  *reinterpret_cast<uint2*>(p.out + orow * 512 + 4 * c4) = w;
+  if (p.lse && c4 == 0) p.lse[orow] = Lsum > 0.f ? (M + log2f(Lsum)) * 0.6931471805599453f : -INFINITY;
+  (void)n;
 }
 
 // ----------------------------------------------------------------------------------- host
@@ -618,6 +792,21 @@ bool attn_tc2_supported(const AttnProblem& a) {
 
 // CTA pairs that can be resident at once on the current device (one CTA per SM by shared memory): the size
 // of the persistent grid.  Asked from the occupancy calculator once per device; half the SM count otherwise.
+static int resident_pairs();
+// Split decode is used while the (sequence, head block) units number at most half the resident CTA pairs: cutting the
+// line of key tiles into equal ranges costs a partial result per cut (256 KB written and read again) and a second
+// launch, about 30 us in all at 64 sequences x 40 tiles, which only pays where whole units would leave more than
+// half of the pairs idle.  The workspace holds one partial result per unit and per pair at most.
+static bool decode_splits(int batch, int n_q_heads) {
+  const int units = batch * (n_q_heads >= 128 ? n_q_heads / 128 : 1);
+  return 2 * units <= resident_pairs();
+}
+size_t attn_tc2_decode_workspace_bytes(int batch, int n_q_heads) {
+  if (!decode_splits(batch, n_q_heads)) return 0;
+  const size_t units = (size_t)batch * (n_q_heads >= 128 ? n_q_heads / 128 : 1);
+  return (units + (size_t)resident_pairs()) * PARTIAL_FLOATS * sizeof(float);
+}
+
 static int resident_pairs() {
   static int cached[64];
   int dev = 0;
@@ -635,7 +824,7 @@ static int resident_pairs() {
       cudaOccupancyMaxActiveClusters(&n, attn_tc2_kernel, &cfg) != cudaSuccess || n <= 0) {
     cudaGetLastError();
     int sms = 0;
-    if (cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || sms < 2) sms = 2;
+    if (cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || sms < 2) sms = 148;   // no device: a B200
     n = sms / 2;
   }
   cached[dev] = n;
@@ -700,11 +889,22 @@ int attn_tc2_launch(const AttnProblem& a) {
   if (!ok) return LCA_ERR_CUDA;
   if (cudaFuncSetAttribute(attn_tc2_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM_BYTES) != cudaSuccess)
     return LCA_ERR_CUDA;
-  const long long n_pairs = p.n_items < resident_pairs() ? p.n_items : resident_pairs();
+  long long n_pairs = p.n_items < resident_pairs() ? p.n_items : resident_pairs();
   if (n_pairs <= 0) return LCA_OK;
+  if (a.decode && decode_splits(a.batch, H)) {
+    // every pair takes an equal share of all key tiles; ranges that cut a unit leave partial results in the workspace
+    if (a.ws_bytes < attn_tc2_decode_workspace_bytes(a.batch, H)) return LCA_ERR_WORKSPACE_TOO_SMALL;
+    if (!a.ws || (reinterpret_cast<uintptr_t>(a.ws) & 31u)) return LCA_ERR_MISALIGNED;
+    p.split = 1; p.partial = static_cast<float*>(a.ws);
+    n_pairs = resident_pairs();
+  }
   dim3 grid((unsigned)(2 * n_pairs));
   attn_tc2_kernel<<<grid, THREADS, SMEM_BYTES, a.stream>>>(p);
   note_launch();
+  if (p.split) {
+    decode_combine_kernel<<<dim3((unsigned)(a.batch * p.n_head_blocks * p.HB)), 128, 0, a.stream>>>(p, (int)n_pairs);
+    note_launch();
+  }
   return cudaGetLastError() == cudaSuccess ? LCA_OK : LCA_ERR_CUDA;
 }
 

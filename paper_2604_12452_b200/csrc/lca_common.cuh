@@ -115,6 +115,7 @@ size_t attn_tc_workspace_bytes(const AttnProblem& a);
 int attn_tc_launch(const AttnProblem& a);
 int attn_tc_device_status(cudaStream_t stream);
 size_t attn_tc2_ragged_workspace_bytes(int batch, int longest, int n_q_heads);
+size_t attn_tc2_decode_workspace_bytes(int batch, int n_q_heads);     // MLA shape, CTA-pair kernel
 int bounded_wait_selftest_launch(long long limit_cycles, cudaStream_t stream);
 int latent_to_value_launch(const void* latent, const void* w_uv, void* out, long long n_tokens, int n_heads,
                            int d_latent, int d_v, cudaStream_t stream);

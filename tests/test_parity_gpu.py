@@ -637,3 +637,44 @@ def test_ragged_batch_equals_one_call_per_sequence_and_the_oracle(B, kind):
                      anchor_idx=cond["anchor_idx"][gro[b]:gro[b + 1]])
         Hh.check_condense(piece, ref["cond"], kind="gqa" if kind == "gqa" else "mla")
         Hh.check_outputs(out[tok[b]:tok[b + 1]][torch.from_numpy(rows).to(DEV)], ref, f"ragged {kind} sequence {b}")
+
+
+@pytest.mark.parametrize("nb,H,cap", [(1, 128, 5057), (8, 128, 2100), (3, 256, 900), (5, 16, 700), (37, 128, 600), (64, 128, 300)])
+def test_decode_key_ranges_split_over_cta_pairs_match_oracle(B, nb, H, cap):
+    # Few sequences: the key tiles of all sequences are cut into equal ranges, one per CTA pair, and a sequence's
+    # partial results are merged by a second kernel (one sequence of 40 tiles becomes 40 single-tile ranges; eight
+    # ragged ones share ranges; two head blocks per sequence; 16 heads use an eighth of a tile's rows; 37 sequences
+    # are the most that are still cut on 74 resident pairs).  64 sequences: whole sequences per work item, no merge.
+    # Ragged counts, an empty cache, lse.
+    gen = torch.Generator().manual_seed(nb * 1000 + H)
+    cache_sem = torch.randn((nb, cap, 1, 512), generator=gen).bfloat16()
+    cache_pos = torch.randn((nb, cap, 1, 64), generator=gen).bfloat16()
+    q_sem = torch.randn((nb, H, 512), generator=gen).bfloat16()
+    q_pos = torch.randn((nb, H, 64), generator=gen).bfloat16()
+    rows = torch.randint(1, cap + 1, (nb,), generator=gen, dtype=torch.int32)
+    rows[0] = cap
+    if nb > 2:
+        rows[1] = 0
+        rows[2] = 129
+    n_rep = 33
+    cfg = I.scaled(I.CONFIGS["mla_decode"], batch=nb, seq_len=4096, n_q_heads=H)
+    p = B.params_from_config(cfg, batch=nb)
+    out, lse = B.decode_attention(p, q_sem.to(DEV), q_pos.to(DEV), cache_sem.to(DEV), cache_pos.to(DEV), rows.to(DEV), n_rep,
+                                  want_lse=True)
+    out2, lse2 = B.decode_attention(p, q_sem.to(DEV), q_pos.to(DEV), cache_sem.to(DEV), cache_pos.to(DEV), rows.to(DEV), n_rep,
+                                    want_lse=True)
+    torch.cuda.synchronize()
+    assert B.lca_last_device_status() == 0
+    assert torch.equal(Hh.bits_t(out), Hh.bits_t(out2)) and torch.equal(lse, lse2)      # fixed merge order: reproducible
+    for b in sorted(set(list(range(0, nb, max(1, nb // 6))) + [0, min(1, nb - 1), min(2, nb - 1)])):
+        n = int(rows[b])
+        if n == 0:
+            assert torch.count_nonzero(out[b]) == 0
+            assert torch.isinf(lse[b]).all() and (lse[b] < 0).all()
+            continue
+        cs = O.bits_to_f64(Hh.bits(cache_sem[b, :n, 0]))
+        cp = O.bits_to_f64(Hh.bits(cache_pos[b, :n, 0]))
+        ro, rl = O.mla_decode(O.torch_bf16_to_f64(q_sem[b]), O.torch_bf16_to_f64(q_pos[b]), cs, cp, min(n_rep, n),
+                              Hh.f32(cfg.softmax_scale), 0.0)
+        Hh.check_outputs(out[b], ro, f"split decode nb={nb} H={H} seq {b} rows {n}")
+        np.testing.assert_allclose(lse[b].cpu().numpy(), rl, atol=2e-3, rtol=1e-4)
