@@ -35,7 +35,7 @@ METRIC = "lca_prefill_tokens_per_s"
 UNIT = "tokens/s"
 # dram__bytes_read.sum + dram__bytes_write.sum of attn_tc2_kernel at mla_32k (L=32768, H=16) divided by
 # L*H: the kernel reads every query row and writes every output row once, the key/value stream stays in L2.
-ATTN_DRAM_BYTES_PER_TOKEN_HEAD = (642.48e6 + 496.66e6) / (32768 * 16)
+ATTN_DRAM_BYTES_PER_TOKEN_HEAD = (642.909440e6 + 497.025536e6) / (32768 * 16)
 
 
 # ---------------------------------------------------------------------------- work counts
@@ -706,7 +706,7 @@ def main():
     ap.add_argument("--steps", type=int, default=5)
     ap.add_argument("--warmup", type=int, default=3)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
-    ap.add_argument("--config", default="mla_128k", choices=list(I.CONFIGS.keys()) + ["scaling"],
+    ap.add_argument("--config", default="mla_128k", choices=list(I.CONFIGS.keys()) + ["scaling", "value_projection"],
                     help="mla_128k is the benchmark; mla_1k / mla_32k run the same step on configs 1 / 2; mla_decode and "
                          "gqa_64k print the side measurements of configs 4 / 5 on their own (used for profiling)")
     ap.add_argument("--attn-impl", type=int, default=0, help="0 auto, 1 scalar kernel, 2 tensor-core kernel")
@@ -715,7 +715,7 @@ def main():
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-extras", action="store_true", help="skip the decode / GQA / dense-comparison side measurements")
     ap.add_argument("--decode-batch", type=int, default=64)
-    ap.add_argument("--seq-len", type=int, default=0, help="gqa_64k only: a shorter sequence of the same shape (small profiler captures)")
+    ap.add_argument("--seq-len", type=int, default=0, help="gqa_64k / value_projection: a shorter sequence of the same shape (small profiler captures)")
     ap.add_argument("--ref-rows", type=int, default=64, help="query rows in the oracle's bounded sample")
     ap.add_argument("--ref-heads", type=int, default=128, help="heads per sampled row in the oracle's sample (capped at the head count)")
     args = ap.parse_args()
@@ -741,6 +741,16 @@ def main():
             res = measure_scaling(B, f"cuda:{local_rank}", measured_peaks())
             print(json.dumps(dict(metric="side_measurement", config=dict(workload=res["workload"]), n_gpus=1, data="synthetic",
                                   result=res, gpu_launches=None)))
+        return
+    if args.config == "value_projection":
+        if rank == 0:
+            torch.cuda.set_device(local_rank)
+            dev = f"cuda:{local_rank}"
+            cfg = I.scaled(I.CONFIGS["mla_128k"], seq_len=args.seq_len or 16384)
+            lat = torch.randn((1, cfg.seq_len, cfg.n_q_heads, cfg.d_sem), device=dev).bfloat16()
+            res = measure_value_projection(B, dev, cfg, lat, measured_peaks())
+            print(json.dumps(dict(metric="side_measurement", config=dict(workload=f"value projection of {cfg.seq_len} tokens x {cfg.n_q_heads} heads"),
+                                  n_gpus=1, data="synthetic", result=res, gpu_launches=None)))
         return
     if args.config in ("mla_decode", "gqa_64k"):
         if rank == 0:
