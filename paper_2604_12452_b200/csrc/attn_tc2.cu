@@ -19,6 +19,12 @@
 // tokens) down in a fixed stride.  Barriers and tensor memory are set up once; the query tile of the
 // next item is fetched as soon as the last S product of the current one has completed, and its first
 // products run while the softmax threads still normalise and store the current output.
+//
+// The one software signal between the two CTAs ("P of the odd CTA is complete") is forwarded by a relay
+// thread with mbarrier.arrive.relaxed.cluster after it has acquired the local arrivals of the writers (whose
+// stores were followed by fence.proxy.async).  That the even CTA's next tcgen05.mma then sees the odd CTA's P
+// is an argument about the hardware's behaviour, not a guarantee of the PTX memory model; the test that runs the
+// 128K configuration twice and compares every output bit is its check and has to stay.
 #include <algorithm>
 #include <cstring>
 #include <vector>
