@@ -41,7 +41,7 @@ constexpr int SMEM_BYTES = OFF_MISC + 64 + 1024;      // + slack to align the ba
 constexpr int TM_S = 0, TM_O = 256, TM_COLS = 512;    // S_r buffer u at TM_S + 128 r + 64 u, O_r at TM_O + 128 r
 constexpr int THREADS = 320;
 constexpr float RESCALE_THRESHOLD = 8.0f; // log2 units
-constexpr int POLY_EVERY = 4;             // one exponential in POLY_EVERY of an interior tile goes to the FMA pipe (0: none)
+constexpr int POLY_EVERY = 8;             // one exponential in POLY_EVERY of an interior tile goes to the FMA pipe (0: none; measured at config 5: none 1134, 1 in 16 1178, 1 in 8 1201, 1 in 6 1161, 1 in 4 1134, 1 in 2 1102 TFLOP/s)
 static_assert(SMEM_BYTES <= 232448, "shared memory budget of one SM");
 }  // namespace gq
 
