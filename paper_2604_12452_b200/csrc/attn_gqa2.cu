@@ -70,8 +70,11 @@ attn_gqa2_kernel(const __grid_constant__ Gqa2Params p) {
   auto BAR_VEMPTY = [&](int s) { return bars + 8 * (1 + 3 * STAGES + s); };
   auto BAR_SFULL = [&](int r, int u) { return bars + 8 * (1 + 4 * STAGES + 2 * r + u); };   // S_r in buffer u is complete
   auto BAR_PFULL = [&](int r, int u) { return bars + 8 * (5 + 4 * STAGES + 2 * r + u); };   // P_r in buffer u has been written
-  auto BAR_ODONE = [&](int r) { return bars + 8 * (9 + 4 * STAGES + r); };                  // P_r V of the current tile is complete
-  static_assert(8 * (11 + 4 * STAGES) <= 256, "barrier block");
+  // P_r V of a tile is complete: one barrier per parity of the tile index, so that a waiter is never more than one
+  // phase behind its barrier (a parity wait cannot tell phases two apart; P V of tile j - 2 is known to be complete
+  // when S of tile j is, P V of tile j - 1 is not)
+  auto BAR_ODONE = [&](int r, int u) { return bars + 8 * (9 + 4 * STAGES + 2 * r + u); };
+  static_assert(8 * (13 + 4 * STAGES) <= 256, "barrier block");
   volatile uint32_t* tmem_slot = reinterpret_cast<volatile uint32_t*>(base_ptr + OFF_MISC);
   volatile int* abort_flag = reinterpret_cast<volatile int*>(base_ptr + OFF_MISC + 4);
 
@@ -104,8 +107,7 @@ attn_gqa2_kernel(const __grid_constant__ Gqa2Params p) {
       mbar_init(BAR_VFULL(s), 1); mbar_init(BAR_VEMPTY(s), 1);
     }
     for (int r = 0; r < 2; ++r) {
-      for (int u = 0; u < 2; ++u) { mbar_init(BAR_SFULL(r, u), 1); mbar_init(BAR_PFULL(r, u), 128); }
-      mbar_init(BAR_ODONE(r), 1);
+      for (int u = 0; u < 2; ++u) { mbar_init(BAR_SFULL(r, u), 1); mbar_init(BAR_PFULL(r, u), 128); mbar_init(BAR_ODONE(r, u), 1); }
     }
     *abort_flag = 0;
     fence_mbar_init();
@@ -172,7 +174,7 @@ attn_gqa2_kernel(const __grid_constant__ Gqa2Params p) {
       for (int k = 0; k < BN / 16; ++k)
         umma_ts_elected(leader, tmem + TM_O + 128 * r, tmem + TM_S + 128 * r + 64 * (j & 1) + k * 8, desc_add(vd0, (k * 2048) >> 4),
                         IDESC_PV, (j > 0 || k > 0) ? 1u : 0u);
-      umma_commit_elected(leader, BAR_ODONE(r));
+      umma_commit_elected(leader, BAR_ODONE(r, j & 1));
     };
     // S of the first two key tiles for both sub-tiles
     for (int j = 0; ok && j < 2 && j < n_tiles; ++j) {
@@ -285,7 +287,7 @@ attn_gqa2_kernel(const __grid_constant__ Gqa2Params p) {
       if (j == 0) m_ref = tmax;
       else if (tmax > m_ref + RESCALE_THRESHOLD) { need = true; factor = exp2f(m_ref - tmax); }
       if (__any_sync(0xffffffffu, need)) {
-        ok = mbar_wait(BAR_ODONE(r), (j - 1) & 1, abort_flag);       // P_r V of tile j - 1 has landed in O_r
+        ok = mbar_wait(BAR_ODONE(r, (j - 1) & 1), ((j - 1) >> 1) & 1, abort_flag);       // P_r V of tile j - 1 has landed in O_r
         if (!ok && lane == 0) fail(ERR_WAIT_O_DONE);
         ok = __all_sync(0xffffffffu, ok);
         if (!ok) break;
@@ -336,7 +338,7 @@ attn_gqa2_kernel(const __grid_constant__ Gqa2Params p) {
     }
     // ---- epilogue: O_r / l -> bf16 -> global
     if (ok) {
-      ok = mbar_wait(BAR_ODONE(r), (n_tiles - 1) & 1, abort_flag);
+      ok = mbar_wait(BAR_ODONE(r, (n_tiles - 1) & 1), ((n_tiles - 1) >> 1) & 1, abort_flag);
       if (!ok && lane == 0) fail(ERR_WAIT_O_DONE);
       ok = __all_sync(0xffffffffu, ok);
     }

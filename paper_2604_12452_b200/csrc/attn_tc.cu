@@ -351,6 +351,14 @@ attn_tc1_kernel(const __grid_constant__ TcParams p) {
         }
       }
       l_sum += rs0 + rs1;
+      if (j >= 1 && ok) {
+        // keep in step with the P V barrier (a parity wait only tells phases apart while the waiter is at most one
+        // phase behind): P V of tile j - 1 was issued before this tile's softmax began and is normally complete
+        ok = mbar_wait(BAR_ODONE, (j - 1) & 1, abort_flag);
+        if (!ok && lane == 0) fail(ERR_WAIT_O_DONE);
+        ok = __all_sync(0xffffffffu, ok);
+        if (!ok) continue;                                        // reported at the next tile's barrier
+      }
       tmem_st32(stm + 32 * half, pk);     // P columns 32*half .. 32*half+31 = keys 64*half .. 64*half+63
       tmem_wait_st();
       tc_fence_before();

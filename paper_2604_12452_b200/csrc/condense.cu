@@ -18,7 +18,8 @@ static const int CONDENSE_THREADS = 512;
 
 // ---------------------------------------------------------------------------- summary query
 // Partial sums of the query tail.  Rows of one KV head = (position, query head in its group);
-// a chunk is QBAR_ROWS_PER_CHUNK rows.  grid (nchunks, Hkv, B).  A thread owns one 16-byte piece
+// a chunk is QBAR_ROWS_PER_CHUNK rows and has its own partial sum; a CTA takes `chunks_per_cta` consecutive chunks one
+// after the other (the sums do not depend on that number).  grid (CTAs, Hkv, B).  A thread owns one 16-byte piece
 // (8 columns) of the key dimension and every row_lanes-th row of the chunk, so that consecutive
 // threads read a whole query row and each thread has many independent loads in flight; the
 // row lanes are then added up through shared memory in a fixed order.
@@ -26,9 +27,10 @@ static const int CONDENSE_THREADS = 512;
 // sequence b is its last min(n_pos, L_b) positions.
 __global__ void qbar_partial_kernel(const bf16* __restrict__ q_sem, const bf16* __restrict__ q_pos,
                                     int64_t batch_stride_rows, int n_pos, int Hq, int Hkv, int d_sem,
-                                    int d_pos, int sem_in_logit, int row_lanes, double* __restrict__ partial, SeqTab tab) {
+                                    int d_pos, int sem_in_logit, int row_lanes, double* __restrict__ partial, SeqTab tab,
+                                    int nchunks, int chunks_per_cta) {
   extern __shared__ double s_part[];                     // [row_lanes][dk]
-  const int chunk = blockIdx.x, hk = blockIdx.y, b = blockIdx.z;
+  const int hk = blockIdx.y, b = blockIdx.z;
   const int rep = Hq / Hkv;
   long long first_pos = (long long)b * batch_stride_rows;     // row (position) of the first averaged query
   if (tab.tok_off) {
@@ -37,11 +39,12 @@ __global__ void qbar_partial_kernel(const bf16* __restrict__ q_sem, const bf16* 
     first_pos = (long long)tab.tok_off[b] + len - n_pos;
   }
   const int n_rows = n_pos * rep;
-  const int r0 = chunk * QBAR_ROWS_PER_CHUNK;
-  const int r1 = min(n_rows, r0 + QBAR_ROWS_PER_CHUNK);
   const int dk = (sem_in_logit ? d_sem : 0) + d_pos;
   const int pieces = dk / 8, sem_pieces = sem_in_logit ? d_sem / 8 : 0;
   const int pc = threadIdx.x % pieces, rl = threadIdx.x / pieces;
+  for (int chunk = blockIdx.x * chunks_per_cta; chunk < min(nchunks, (int)(blockIdx.x + 1) * chunks_per_cta); ++chunk) {
+  const int r0 = chunk * QBAR_ROWS_PER_CHUNK;
+  const int r1 = min(n_rows, r0 + QBAR_ROWS_PER_CHUNK);
   double acc[8];
 #pragma unroll
   for (int i = 0; i < 8; ++i) acc[i] = 0.0;
@@ -75,11 +78,13 @@ __global__ void qbar_partial_kernel(const bf16* __restrict__ q_sem, const bf16* 
     for (int i = 0; i < 8; ++i) s_part[(size_t)rl * dk + 8 * pc + i] = acc[i];
   }
   __syncthreads();
-  double* dst = partial + (((size_t)b * Hkv + hk) * gridDim.x + chunk) * dk;
+  double* dst = partial + (((size_t)b * Hkv + hk) * nchunks + chunk) * dk;
   for (int c = threadIdx.x; c < dk; c += blockDim.x) {
     double sum = 0.0;
     for (int l = 0; l < row_lanes; ++l) sum += s_part[(size_t)l * dk + c];
     dst[c] = sum;
+  }
+  __syncthreads();                                       // s_part is reused by the next chunk
   }
 }
 
@@ -649,6 +654,11 @@ static int n_summary(const lca_params* p) {
 static int key_dim(const lca_params* p) {
   return (p->variant == LCA_VARIANT_MLA ? p->d_sem : 0) + p->d_pos;
 }
+// Chunks per CTA of a summary-query launch: one keeps the GPU busy when there are few rows; with many sequences four
+// amortise the start-up of a CTA (a CTA of one 64-row chunk reads 74 KB and is gone).
+static int qbar_chunks_per_cta(long long total_rows) {
+  return total_rows >= 256ll * 1024 ? 4 : 1;
+}
 static int qbar_chunks(const lca_params* p) {
   int rows = n_summary(p) * (p->n_q_heads / p->n_kv_heads);
   return (rows + QBAR_ROWS_PER_CHUNK - 1) / QBAR_ROWS_PER_CHUNK;
@@ -691,17 +701,20 @@ int condense_launch(const CondenseLaunch& c) {
       qbar_widen_kernel<<<(n + 255) / 256, 256, 0, c.stream>>>(c.qbar_opt, qbar, n);
       note_launch();
     } else {
-      const int nch = qbar_chunks(p);
-      dim3 grid(nch, Hkv, B);
+      const int n_req = ragged ? (p->n_summary_q > 0 ? p->n_summary_q : p->group_size) : n_summary(p);
+      const int rows_q = n_req * (p->n_q_heads / Hkv);
+      const int cpc = qbar_chunks_per_cta((long long)rows_q * Hkv * B);
+      const int nch = (rows_q + QBAR_ROWS_PER_CHUNK - 1) / QBAR_ROWS_PER_CHUNK;
+      dim3 grid((nch + cpc - 1) / cpc, Hkv, B);
       const int pieces = dk / 8;
       int row_lanes = 256 / pieces;
       if (row_lanes < 1) row_lanes = 1;
       if (row_lanes > 16) row_lanes = 16;
       const int threads = ((pieces * row_lanes + 31) / 32) * 32;
-      const int n = ragged ? (p->n_summary_q > 0 ? p->n_summary_q : p->group_size) : n_summary(p);
+      const int n = n_req;
       qbar_partial_kernel<<<grid, threads, (size_t)row_lanes * dk * sizeof(double), c.stream>>>(
           (const bf16*)c.q_tail_sem, (const bf16*)c.q_tail_pos, c.q_tail_batch_stride, n,
-          p->n_q_heads, Hkv, p->d_sem, p->d_pos, sem_in_logit, row_lanes, partial, c.tab);
+          p->n_q_heads, Hkv, p->d_sem, p->d_pos, sem_in_logit, row_lanes, partial, c.tab, nch, cpc);
       double count = (double)n * (double)(p->n_q_heads / Hkv);
       qbar_final_kernel<<<dim3(Hkv, B), dk < 1024 ? ((dk + 31) / 32) * 32 : 1024, 0, c.stream>>>(partial, nch, dk, count, qbar, c.tab, n,
                                                                                               p->n_q_heads / Hkv);
@@ -895,15 +908,16 @@ int update_launch(const lca_params* p, const void* q_tail_sem, const void* q_tai
   } else {
     const int n = p->n_summary_q > 0 ? p->n_summary_q : p->group_size;
     const int rows = n * (p->n_q_heads / Hkv);
+    const int cpc = qbar_chunks_per_cta((long long)rows * Hkv * B);
     const int nch = (rows + QBAR_ROWS_PER_CHUNK - 1) / QBAR_ROWS_PER_CHUNK;
     const int pieces = dk / 8;
     int row_lanes = 256 / pieces;
     if (row_lanes < 1) row_lanes = 1;
     if (row_lanes > 16) row_lanes = 16;
     const int threads = ((pieces * row_lanes + 31) / 32) * 32;
-    qbar_partial_kernel<<<dim3(nch, Hkv, B), threads, (size_t)row_lanes * dk * sizeof(double), stream>>>(
+    qbar_partial_kernel<<<dim3((nch + cpc - 1) / cpc, Hkv, B), threads, (size_t)row_lanes * dk * sizeof(double), stream>>>(
         (const bf16*)q_tail_sem, (const bf16*)q_tail_pos, q_tail_batch_stride, n, p->n_q_heads, Hkv, p->d_sem, p->d_pos,
-        sem_in_logit, row_lanes, partial, SeqTab{});
+        sem_in_logit, row_lanes, partial, SeqTab{}, nch, cpc);
     qbar_final_kernel<<<dim3(Hkv, B), dk < 1024 ? ((dk + 31) / 32) * 32 : 1024, 0, stream>>>(
         partial, nch, dk, (double)n * (double)(p->n_q_heads / Hkv), qbar, SeqTab{}, n, p->n_q_heads / Hkv);
     note_launch(2);

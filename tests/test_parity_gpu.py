@@ -678,3 +678,23 @@ def test_decode_key_ranges_split_over_cta_pairs_match_oracle(B, nb, H, cap):
                               Hh.f32(cfg.softmax_scale), 0.0)
         Hh.check_outputs(out[b], ro, f"split decode nb={nb} H={H} seq {b} rows {n}")
         np.testing.assert_allclose(lse[b].cpu().numpy(), rl, atol=2e-3, rtol=1e-4)
+
+
+def test_gqa_prefill_is_bit_reproducible_across_launches(B):
+    # Two softmax groups and the MMA warp of a CTA run at their own pace; every hand-off between them must be an
+    # ordering, not a coincidence of timing: four launches on the same inputs agree in every bit (sequence long
+    # enough for ~70 key tiles per block, 4096 CTAs in all).
+    cfg = I.scaled(I.CONFIGS["gqa_64k"], seq_len=8192, group_size=64, window=4096)
+    d = to_dev(I.make_gqa_inputs(cfg, "cpu"))
+    L, g = cfg.seq_len, cfg.group_size
+    p = B.params_from_config(cfg, batch=1)
+    cond = B.condense(p, None, d["q"][L - g:], d["v"], d["k"])
+    first = None
+    for _ in range(4):
+        out, lse = B.prefill_attention(p, None, d["q"], d["v"], d["k"], cond["cache_sem"], cond["cache_pos"], want_lse=True)
+        torch.cuda.synchronize()
+        if first is None:
+            first = (out.clone(), lse.clone())
+        else:
+            assert torch.equal(Hh.bits_t(out), Hh.bits_t(first[0])) and torch.equal(lse, first[1])
+    assert B.lca_last_device_status() == 0
