@@ -447,6 +447,20 @@ bool make_tensor_map_3d(CUtensorMap* map, const void* ptr, int d, int heads, lon
             CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
 
+// The same tensor with unswizzled boxes of whole rows: box {d, 1, box_rows} lands as a plain [box_rows][d] array
+// (the condensation kernels read their tiles with ordinary shared-memory loads).
+bool make_tensor_map_rows(CUtensorMap* map, const void* ptr, int d, int heads, long long rows, int box_rows) {
+  EncodeTiledFn fn = encode_fn();
+  if (!fn || !ptr) return false;
+  cuuint64_t dims[3] = {(cuuint64_t)d, (cuuint64_t)heads, (cuuint64_t)rows};
+  cuuint64_t strides[2] = {(cuuint64_t)d * 2, (cuuint64_t)d * 2 * heads};
+  cuuint32_t box[3] = {(cuuint32_t)d, 1, (cuuint32_t)box_rows};
+  cuuint32_t estr[3] = {1, 1, 1};
+  return fn(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 3, const_cast<void*>(ptr), dims, strides, box, estr,
+            CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_NONE, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+            CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+}
+
 // A [rows][64 * chunks] bf16 matrix seen as (64 columns, rows, 64-column chunks): one box then brings
 // several column chunks of the same rows, each landing as its own 128-byte-swizzled [rows][64] block
 // (chunk after chunk), in a single request instead of one request per chunk.

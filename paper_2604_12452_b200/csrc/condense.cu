@@ -9,6 +9,8 @@
 // are fp32 (the fp64 pipe could not keep up with HBM for both), c_rep is rounded once to bf16.
 #include <mutex>
 
+#include <cuda.h>
+
 #include "lca_common.cuh"
 
 namespace lca {
@@ -616,6 +618,242 @@ condense_mla64_kernel(CondenseArgs a) {
   if (tid == 0 && *s_abort) atomicCAS(&g_condense_status, 0, 1);
 }
 
+// ----------------------------------------------------- condense, GQA shape (head dimension 128) with g = 64
+// The role-split structure of condense_mla64_kernel for keys / values of 128 columns that are interleaved by KV head
+// in memory ([L, Hkv, 128]): a group of one KV head is 64 rows of 256 bytes, 256 Hkv bytes apart, fetched as two
+// tiled TMA boxes (keys 16 KB, values 16 KB) into one of six stages.  Four score warps (16 tokens each: eight tokens per
+// pass, a token's 128 columns over four lanes), the arbiter warp (arg-max: fp32 where the margin proves it, fp64
+// otherwise; softmax), one pool warp (four value columns per lane; anchor key row, index), one producer thread.
+// An fp32 sum passes through at most 19 roundings here (16 multiply-adds per chain, the chain pair, 2 shuffle levels).
+namespace gfast {
+constexpr int G = 64, D = 128, STAGES = 6;
+constexpr int SCORE_WARPS = 4;
+constexpr int WARP_ARBITER = SCORE_WARPS, WARP_POOL = SCORE_WARPS + 1, WARP_PRODUCER = SCORE_WARPS + 2;
+constexpr int THREADS = 32 * (WARP_PRODUCER + 1);
+constexpr int TILE_BYTES = G * D * 2, STAGE_BYTES = 2 * TILE_BYTES;         // keys, then values
+constexpr int OFF_A = STAGES * STAGE_BYTES;                 // float[2][G] alpha
+constexpr int OFF_S32 = OFF_A + 2 * G * 4, OFF_NRM = OFF_S32 + 2 * G * 4, OFF_BAR = OFF_NRM + 2 * G * 4;
+constexpr int SMEM_BYTES = OFF_BAR + 192;
+constexpr float MARGIN_FACTOR = 60.0f * 5.9604644775390625e-08f;
+static_assert(SMEM_BYTES <= 232448, "shared memory budget of one SM");
+}  // namespace gfast
+
+struct GqaCondenseMaps { CUtensorMap k, v; };
+
+__global__ void __launch_bounds__(gfast::THREADS, 1)
+condense_gqa64_kernel(CondenseArgs a, const __grid_constant__ GqaCondenseMaps maps) {
+  using namespace gfast;
+  extern __shared__ __align__(128) unsigned char smem[];
+  float* s_a = reinterpret_cast<float*>(smem + OFF_A);
+  float* s_s32 = reinterpret_cast<float*>(smem + OFF_S32);
+  float* s_nrm = reinterpret_cast<float*>(smem + OFF_NRM);
+  const unsigned bar0 = (unsigned)__cvta_generic_to_shared(smem + OFF_BAR);
+  auto BAR_FULL = [&](int st) { return bar0 + 8 * st; };
+  auto BAR_FREE = [&](int st) { return bar0 + 8 * (STAGES + st); };
+  auto BAR_SCORED = [&](int p) { return bar0 + 8 * (2 * STAGES + p); };
+  auto BAR_READY = [&](int p) { return bar0 + 8 * (2 * STAGES + 2 + p); };
+  auto BAR_AFREE = [&](int p) { return bar0 + 8 * (2 * STAGES + 4 + p); };
+  volatile int* s_anchor = reinterpret_cast<volatile int*>(smem + OFF_BAR + 8 * (2 * STAGES + 6));   // [2]
+  volatile int* s_abort = s_anchor + 2;
+  const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+
+  if (tid == 0) {
+    for (int st = 0; st < STAGES; ++st) {
+      asm volatile("mbarrier.init.shared::cta.b64 [%0], 1;" ::"r"(BAR_FULL(st)) : "memory");
+      asm volatile("mbarrier.init.shared::cta.b64 [%0], 1;" ::"r"(BAR_FREE(st)) : "memory");
+    }
+    for (int p = 0; p < 2; ++p) {
+      asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(BAR_SCORED(p)), "r"(SCORE_WARPS) : "memory");
+      asm volatile("mbarrier.init.shared::cta.b64 [%0], 1;" ::"r"(BAR_READY(p)) : "memory");
+      asm volatile("mbarrier.init.shared::cta.b64 [%0], 1;" ::"r"(BAR_AFREE(p)) : "memory");
+    }
+    *s_abort = 0;
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+  }
+  __syncthreads();
+
+  const long long first = blockIdx.x, stride = gridDim.x;
+  const long long n_mine = first < a.n_groups ? (a.n_groups - first + stride - 1) / stride : 0;
+
+  if (warp == WARP_PRODUCER) {
+    if (lane == 0) {
+      for (long long it = 0; it < n_mine; ++it) {
+        const int st = (int)(it % STAGES);
+        if (it >= STAGES && !cond_wait(BAR_FREE(st), (unsigned)((it / STAGES - 1) & 1), s_abort)) break;
+        const GroupLoc loc = locate_group(a, first + it * stride);
+        const unsigned dst = (unsigned)__cvta_generic_to_shared(smem + (size_t)st * STAGE_BYTES);
+        const unsigned bar = BAR_FULL(st);
+        asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(STAGE_BYTES) : "memory");
+        asm volatile("cp.async.bulk.tensor.3d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3, %4}], [%5];"
+                     ::"r"(dst), "l"(&maps.k), "r"(0), "r"(loc.hk), "r"((int)loc.tok0), "r"(bar) : "memory");
+        asm volatile("cp.async.bulk.tensor.3d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3, %4}], [%5];"
+                     ::"r"(dst + TILE_BYTES), "l"(&maps.v), "r"(0), "r"(loc.hk), "r"((int)loc.tok0), "r"(bar) : "memory");
+      }
+    }
+  } else if (warp < SCORE_WARPS) {
+    // ===================================================== fp32 product sums and max |k| of sixteen tokens per warp
+    const int tsub = lane >> 2, slice = lane & 3;           // token inside a pass of eight, 32-column slice
+    float q[32];
+    long long cur_stream = -1;
+    for (long long it = 0; it < n_mine; ++it) {
+      const int st = (int)(it % STAGES), p = (int)(it & 1);
+      const GroupLoc loc = locate_group(a, first + it * stride);
+      const long long stream = (long long)loc.b * a.Hkv + loc.hk;
+      if (stream != cur_stream) {                           // the next KV stream's summary query
+        cur_stream = stream;
+        const double* qb = a.qbar + (size_t)stream * D + 32 * slice;
+#pragma unroll
+        for (int i = 0; i < 32; ++i) q[i] = (float)qb[i];
+      }
+      if (!cond_wait(BAR_FULL(st), (unsigned)((it / STAGES) & 1), s_abort)) break;
+      if (it >= 2 && !cond_wait(BAR_AFREE(p), (unsigned)(((it >> 1) - 1) & 1), s_abort)) break;
+      const unsigned char* t_k = smem + (size_t)st * STAGE_BYTES;
+#pragma unroll
+      for (int pass = 0; pass < 2; ++pass) {
+        const int i = 16 * warp + 8 * pass + tsub;          // token of this lane
+        const uint4* src = reinterpret_cast<const uint4*>(t_k + (size_t)i * (D * 2) + 64 * slice);
+        float acc0 = 0.f, acc1 = 0.f, kmax = 0.f;
+#pragma unroll
+        for (int x = 0; x < 4; ++x) {
+          const uint4 v = src[x];
+          const unsigned w[4] = {v.x, v.y, v.z, v.w};
+#pragma unroll
+          for (int k = 0; k < 4; ++k) {
+            const float lo = __uint_as_float(w[k] << 16), hi = __uint_as_float(w[k] & 0xffff0000u);
+            acc0 = fmaf(q[8 * x + 2 * k], lo, acc0);
+            acc1 = fmaf(q[8 * x + 2 * k + 1], hi, acc1);
+            kmax = f32_max3_abs(kmax, lo, hi);
+          }
+        }
+        float sum = acc0 + acc1;
+        sum += __shfl_xor_sync(0xffffffffu, sum, 1); kmax = fmaxf(kmax, __shfl_xor_sync(0xffffffffu, kmax, 1));
+        sum += __shfl_xor_sync(0xffffffffu, sum, 2); kmax = fmaxf(kmax, __shfl_xor_sync(0xffffffffu, kmax, 2));
+        if (slice == 0) { s_s32[p * G + i] = sum; s_nrm[p * G + i] = kmax; }
+      }
+      __syncwarp();
+      if (lane == 0) cond_arrive(BAR_SCORED(p));
+    }
+  } else if (warp == WARP_ARBITER) {
+    // ===================================================== arg-max (fp32 where provably exact, else fp64) and softmax
+    const bool exact_all = a.scores != nullptr;
+    const float scale32 = (float)a.scale;
+    long long cur_stream = -1;
+    float q_l1 = 0.f;
+    for (long long it = 0; it < n_mine; ++it) {
+      const int st = (int)(it % STAGES), p = (int)(it & 1);
+      const GroupLoc loc = locate_group(a, first + it * stride);
+      const long long stream = (long long)loc.b * a.Hkv + loc.hk;
+      const double* qb = a.qbar + (size_t)stream * D;
+      if (stream != cur_stream) {
+        cur_stream = stream;
+        float t = 0.f;
+        for (int x = lane; x < D; x += 32) t += fabsf((float)qb[x]);
+        q_l1 = warp_sum(t);
+      }
+      if (!cond_wait(BAR_SCORED(p), (unsigned)((it >> 1) & 1), s_abort)) break;
+      const float sa = s_s32[p * G + lane], sb = s_s32[p * G + lane + 32];
+      float m1, m2;
+      int i1;
+      if (sb > sa) { m1 = sb; i1 = lane + 32; m2 = sa; } else { m1 = sa; i1 = lane; m2 = sb; }
+      float km = fmaxf(s_nrm[p * G + lane], s_nrm[p * G + lane + 32]);
+#pragma unroll
+      for (int o = 16; o > 0; o >>= 1) {
+        const float om1 = __shfl_xor_sync(0xffffffffu, m1, o), om2 = __shfl_xor_sync(0xffffffffu, m2, o);
+        const int oi = __shfl_xor_sync(0xffffffffu, i1, o);
+        km = fmaxf(km, __shfl_xor_sync(0xffffffffu, km, o));
+        m2 = fmaxf(fminf(m1, om1), fmaxf(m2, om2));
+        if (om1 > m1 || (om1 == m1 && oi < i1)) { m1 = om1; i1 = oi; }
+      }
+      const bool exact = exact_all || !(m1 - m2 > MARGIN_FACTOR * q_l1 * km);
+      float ea, eb;
+      int besti;
+      if (exact) {
+        if (!cond_wait(BAR_FULL(st), (unsigned)((it / STAGES) & 1), s_abort)) break;
+        const unsigned char* t_k = smem + (size_t)st * STAGE_BYTES;
+        // fp64 scores token by token: lane l takes columns 4 l .. 4 l + 3; lanes l and l + 32 keep the results
+        double qd[4];
+#pragma unroll
+        for (int i = 0; i < 4; ++i) qd[i] = qb[4 * lane + i];
+        double da = 0.0, db = 0.0;
+#pragma unroll 1
+        for (int i = 0; i < G; ++i) {
+          const uint2 v = *reinterpret_cast<const uint2*>(t_k + (size_t)i * (D * 2) + 8 * lane);
+          double acc = qd[0] * (double)__uint_as_float(v.x << 16);
+          acc = fma(qd[1], (double)__uint_as_float(v.x & 0xffff0000u), acc);
+          acc = fma(qd[2], (double)__uint_as_float(v.y << 16), acc);
+          acc = fma(qd[3], (double)__uint_as_float(v.y & 0xffff0000u), acc);
+          const double c = warp_sum(acc) * a.scale;
+          if ((i & 31) == lane) { if (i < 32) da = c; else db = c; }
+        }
+        double best = da; besti = lane;
+        if (db > best) { best = db; besti = lane + 32; }
+#pragma unroll
+        for (int o = 16; o > 0; o >>= 1) {
+          const double ob = __shfl_xor_sync(0xffffffffu, best, o);
+          const int oi = __shfl_xor_sync(0xffffffffu, besti, o);
+          if (ob > best || (ob == best && oi < besti)) { best = ob; besti = oi; }
+        }
+        ea = expf((float)(da - best)); eb = expf((float)(db - best));
+        if (a.scores) {
+          double* sc = a.scores + (((size_t)loc.b * a.Hkv + loc.hk) * a.m + loc.j) * G;
+          sc[lane] = da; sc[lane + 32] = db;
+        }
+      } else {
+        besti = i1;
+        ea = expf((sa - m1) * scale32); eb = expf((sb - m1) * scale32);
+      }
+      const float inv = 1.f / warp_sum(ea + eb);
+      s_a[p * G + lane] = ea * inv; s_a[p * G + lane + 32] = eb * inv;
+      if (lane == 0) s_anchor[p] = besti;
+      __syncwarp();
+      if (lane == 0) cond_arrive(BAR_READY(p));
+    }
+  } else if (warp == WARP_POOL) {
+    // ===================================================== pooling of the values and outputs, one group behind
+    for (long long it = 0; it < n_mine; ++it) {
+      const int st = (int)(it % STAGES), p = (int)(it & 1);
+      const GroupLoc loc = locate_group(a, first + it * stride);
+      if (!cond_wait(BAR_READY(p), (unsigned)((it >> 1) & 1), s_abort)) break;
+      if (!cond_wait(BAR_FULL(st), (unsigned)((it / STAGES) & 1), s_abort)) break;     // complete long ago
+      const unsigned char* t_k = smem + (size_t)st * STAGE_BYTES;
+      const uint2* col = reinterpret_cast<const uint2*>(t_k + TILE_BYTES) + lane;      // value columns 4 lane .. 4 lane + 3
+      const float* al_base = s_a + p * G;
+      unsigned long long acc01 = f32x2(0.f, 0.f), acc23 = f32x2(0.f, 0.f);
+#pragma unroll 4
+      for (int i = 0; i < G; i += 4) {
+        const float4 al = *reinterpret_cast<const float4*>(al_base + i);
+        const float alv[4] = {al.x, al.y, al.z, al.w};
+#pragma unroll
+        for (int u = 0; u < 4; ++u) {
+          const uint2 w = col[(i + u) * (D / 4)];
+          const unsigned long long al2 = f32x2(alv[u], alv[u]);
+          acc01 = fma_f32x2(al2, f32x2(__uint_as_float(w.x << 16), __uint_as_float(w.x & 0xffff0000u)), acc01);
+          acc23 = fma_f32x2(al2, f32x2(__uint_as_float(w.y << 16), __uint_as_float(w.y & 0xffff0000u)), acc23);
+        }
+      }
+      const size_t orow = (size_t)loc.out_row * a.Hkv + loc.hk;
+      {
+        float a0, a1, a2, a3;
+        asm("mov.b64 {%0, %1}, %2;" : "=f"(a0), "=f"(a1) : "l"(acc01));
+        asm("mov.b64 {%0, %1}, %2;" : "=f"(a2), "=f"(a3) : "l"(acc23));
+        const bf162 lo = __floats2bfloat162_rn(a0, a1), hi = __floats2bfloat162_rn(a2, a3);
+        uint2 o;
+        o.x = *reinterpret_cast<const unsigned*>(&lo); o.y = *reinterpret_cast<const unsigned*>(&hi);
+        *reinterpret_cast<uint2*>(a.cache_sem + orow * D + 4 * lane) = o;
+      }
+      const int ia = s_anchor[p];
+      reinterpret_cast<uint2*>(a.cache_pos + orow * D)[lane] = reinterpret_cast<const uint2*>(t_k + (size_t)ia * (D * 2))[lane];
+      if (lane == 0) a.anchor[(size_t)loc.grp_row * a.Hkv + loc.hk] = loc.j * G + ia;
+      __syncwarp();
+      if (lane == 0) { cond_arrive(BAR_AFREE(p)); cond_arrive(BAR_FREE(st)); }
+    }
+  }
+  __syncthreads();
+  if (tid == 0 && *s_abort) atomicCAS(&g_condense_status, 0, 1);
+}
+
+bool make_tensor_map_rows(CUtensorMap* map, const void* ptr, int d, int heads, long long rows, int box_rows);
+
 int condense_take_status() {
   int st = 0;
   if (cudaMemcpyFromSymbol(&st, g_condense_status, sizeof(int)) != cudaSuccess) return -1;
@@ -676,8 +914,15 @@ static bool condense_fast_shape(const lca_params* p) {
   return method && p->variant == LCA_VARIANT_MLA && p->d_sem == 512 && p->d_pos == 64 && p->group_size == 64 && p->n_kv_heads == 1;
 }
 
+static bool condense_gqa_fast_shape(const lca_params* p) {
+  const bool method = (p->sem_reducer == LCA_REDUCE_DEFAULT || p->sem_reducer == LCA_REDUCE_WEIGHTED) &&
+                      (p->pos_reducer == LCA_REDUCE_DEFAULT || p->pos_reducer == LCA_REDUCE_MAXSEL);
+  return method && p->variant == LCA_VARIANT_GQA && p->d_sem == 128 && p->d_pos == 128 && p->group_size == 64;
+}
+
 size_t condense_smem_bytes(const lca_params* p) {
   if (condense_fast_shape(p)) return fast::SMEM_BYTES;
+  if (condense_gqa_fast_shape(p)) return gfast::SMEM_BYTES;
   const size_t g = (size_t)p->group_size;
   const size_t stage = g * (size_t)(p->d_sem + p->d_pos) * sizeof(bf16) + (size_t)key_dim(p) * sizeof(double);
   return 2 * stage + g * (sizeof(double) + sizeof(float));
@@ -738,6 +983,15 @@ int condense_launch(const CondenseLaunch& c) {
       if (cudaFuncSetAttribute(condense_mla64_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, fast::SMEM_BYTES) != cudaSuccess)
         return LCA_ERR_CUDA;
       condense_mla64_kernel<<<dim3((unsigned)ctas), fast::THREADS, fast::SMEM_BYTES, c.stream>>>(a);
+    } else if (condense_gqa_fast_shape(p)) {
+      GqaCondenseMaps maps;
+      const long long rows = ragged ? (long long)c.h_tok_off[B] : (long long)B * p->seq_len;
+      if (!make_tensor_map_rows(&maps.k, c.kv_pos, 128, Hkv, rows, gfast::G) ||
+          !make_tensor_map_rows(&maps.v, c.kv_sem, 128, Hkv, rows, gfast::G))
+        return LCA_ERR_CUDA;
+      if (cudaFuncSetAttribute(condense_gqa64_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, gfast::SMEM_BYTES) != cudaSuccess)
+        return LCA_ERR_CUDA;
+      condense_gqa64_kernel<<<dim3((unsigned)ctas), gfast::THREADS, gfast::SMEM_BYTES, c.stream>>>(a, maps);
     } else {
       size_t smem = condense_smem_bytes(p);
       if (cudaFuncSetAttribute(condense_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) != cudaSuccess)
