@@ -1,16 +1,19 @@
-// Tensor-core attention over the condensed context (Eq. 10 at every prefix length; Sec. 4.3
-// decode) for sm_100a: TMA-staged 128-byte-swizzled tiles, tcgen05.mma with accumulators in
-// tensor memory, online softmax in fp32.
+// Tensor-core attention over the condensed context for grouped-query heads of dimension 128, one 128-row query tile
+// per CTA: TMA-staged 128-byte-swizzled tiles, tcgen05.mma with accumulators in tensor memory, online softmax in
+// fp32.  The library uses this kernel for GQA DECODE (Sec. 4.3, 5.4: one query token per sequence, so a CTA's tile
+// holds the query heads of one KV head); GQA prefill runs on attn_gqa2_kernel (two query tiles per CTA), the MLA shape
+// on attn_tc2_kernel (CTA pairs).  The tile walk below still covers the prefill case (representatives, then local
+// tokens) because it is the same code; this file also holds the tensor-map helpers and the dispatch of all three.
 //
 // One CTA owns a tile of 128 query rows = TB consecutive tokens x HB heads that share one
-// key/value stream.  It walks first the representative rows of the condensed cache that any of
-// its tokens may see, then the local tokens, in tiles of BN keys:
+// key/value stream.  It walks the rows of the condensed cache (prefill: the representatives any of
+// its tokens may see, then the local tokens) in tiles of BN keys:
 //     S  = Q K^T        (tcgen05.mma, A = Q and B = K tile from shared memory, D in TMEM)
-//     P  = exp2(S*c - m) with per-row masks only on boundary tiles (4 softmax warps, one row
-//          per thread, S read from TMEM, P written back to TMEM as packed bf16)
+//     P  = exp2(S*c - m) with per-row masks only on boundary tiles (two softmax threads per row,
+//          S read from TMEM, P written back to TMEM as packed bf16)
 //     O += P V          (tcgen05.mma, A = P from TMEM, B = V tile from shared memory)
 // Roles: warp 0 issues TMA loads, warp 1 owns TMEM and issues every MMA, warps 2..9 do the
-// softmax (two threads per row), the (rare) rescale of O when the running maximum grows by more than 2^8, and the
+// softmax, the (rare) rescale of O when the running maximum grows by more than 2^8, and the
 // epilogue.  Every wait is bounded; on expiry the CTA records a code in a global status word,
 // drains and returns.
 #include <cstring>

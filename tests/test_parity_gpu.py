@@ -698,3 +698,53 @@ def test_gqa_prefill_is_bit_reproducible_across_launches(B):
         else:
             assert torch.equal(Hh.bits_t(out), Hh.bits_t(first[0])) and torch.equal(lse, first[1])
     assert B.lca_last_device_status() == 0
+
+
+def test_random_shapes_match_oracle(B):
+    # Seeded sweep over shapes the other cases do not list: lengths around tile and group boundaries, group sizes that
+    # do not divide anything, windows from 0 to beyond the sequence, head counts of every tile split, summary lengths,
+    # bias on and off; MLA and GQA; prefill on every row and a decode of the last token against the resulting cache.
+    rng = np.random.default_rng(2604)
+    for case in range(14):
+        mla = case % 2 == 0
+        L = int(rng.choice([1, 2, 63, 64, 65, 127, 128, 129, 200, 255, 257, 400, 511, 640]))
+        g = int(rng.choice([1, 2, 3, 8, 16, 33, 64]))
+        w = int(rng.choice([0, 1, 7, 32, 64, 100, 300, 1000]))
+        ns = int(rng.choice([0, 1, 5, 64]))
+        bias = float(rng.choice([0.0, 0.5]))
+        if mla:
+            H = int(rng.choice([1, 2, 4, 8, 16, 32, 64, 128]))
+            cfg = I.scaled(I.CONFIGS["mla_1k"], seq_len=L, n_q_heads=H, group_size=g, window=w, n_needles=min(3, L))
+            inp = I.make_mla_inputs(cfg, "cpu")
+            d = to_dev(inp)
+            p = B.params_from_config(cfg, batch=1, n_summary_q=ns, rep_logit_bias=bias)
+            n = min(L, ns if ns > 0 else g)
+            cond = B.condense(p, d["q_sem"][L - n:], d["q_pos"][L - n:], d["ckv"], d["kr"])
+            out, lse = B.prefill_attention(p, d["q_sem"], d["q_pos"], d["ckv"], d["kr"], cond["cache_sem"], cond["cache_pos"], want_lse=True)
+            rows = torch.tensor([cond["m"] + cond["k"]], dtype=torch.int32, device=DEV)
+            dout, _ = B.decode_attention(p, d["q_sem"][L - 1].contiguous()[None], d["q_pos"][L - 1].contiguous()[None],
+                                         cond["cache_sem"], cond["cache_pos"], rows, cond["m"])
+            ref = Hh.oracle_mla(inp, g, w, cfg.softmax_scale, rows=np.arange(L), n_summary=ns, rep_logit_bias=bias)
+            kind = "mla"
+        else:
+            Hkv = int(rng.choice([1, 2, 4]))
+            Hq = Hkv * int(rng.choice([1, 2, 4, 8]))
+            cfg = I.scaled(I.CONFIGS["gqa_64k"], seq_len=L, n_q_heads=Hq, n_kv_heads=Hkv, group_size=g, window=w, n_needles=min(3, L))
+            inp = I.make_gqa_inputs(cfg, "cpu")
+            d = to_dev(inp)
+            p = B.params_from_config(cfg, batch=1, n_summary_q=ns, rep_logit_bias=bias)
+            n = min(L, ns if ns > 0 else g)
+            cond = B.condense(p, None, d["q"][L - n:], d["v"], d["k"])
+            out, lse = B.prefill_attention(p, None, d["q"], d["v"], d["k"], cond["cache_sem"], cond["cache_pos"], want_lse=True)
+            rows = torch.tensor([cond["m"] + cond["k"]], dtype=torch.int32, device=DEV)
+            dout, _ = B.decode_attention(p, None, d["q"][L - 1].contiguous()[None], cond["cache_sem"], cond["cache_pos"], rows, cond["m"])
+            ref = Hh.oracle_gqa(inp, g, w, cfg.softmax_scale, rows=np.arange(L), n_summary=ns, rep_logit_bias=bias)
+            kind = "gqa"
+        torch.cuda.synchronize()
+        what = f"case {case} {kind} L={L} g={g} w={w} ns={ns} bias={bias} heads={cfg.n_q_heads}/{cfg.n_kv_heads}"
+        assert B.lca_last_device_status() == 0, what
+        Hh.check_condense(one_seq(cond), ref["cond"], kind=kind)
+        Hh.check_outputs(out[0], ref, what)
+        np.testing.assert_allclose(lse[0].cpu().numpy(), ref["lse"], atol=2e-3, rtol=1e-4, err_msg=what)
+        # decoding the last token against the final cache is the last prefill row (Sec. 4.3)
+        Hh.check_outputs(dout[0], ref["out"][-1], what + " decode", vmax=ref["vmax"])
