@@ -332,3 +332,59 @@ def mla_decode_update(cache_sem_bits: np.ndarray, cache_pos_bits: np.ndarray, n_
     new_pos = np.concatenate([cache_pos_bits[:n_rep], cache_pos_bits[n_rep + ia:n_rep + ia + 1],
                               cache_pos_bits[n_rep + g:n_rows]], axis=0)
     return new_sem, new_pos, n_rep + 1, n_rows - (g - 1), ia
+
+
+# ------------------------------------------------------- ring layout of the decode cache
+# Sec. 4.3 keeps "the m representatives ... together with the w most recent latent vectors" and says
+# nothing about where they live.  The packed layout above moves every buffered token when a group is
+# condensed; the ring layout moves none:
+#   rows [0, R), R = w + g : token number n of the sequence (0-based from its start) at row n % R;
+#   rows [R, R + n_rep)    : the representatives in group order.
+# With n_rep representatives and n_tok tokens so far, the uncondensed tokens are n_rep*g .. n_tok-1.
+def ring_from_packed(cache_sem_bits: np.ndarray, cache_pos_bits: np.ndarray, n_rep: int, n_rows: int,
+                     g: int, w: int, capacity: int):
+    """Packed [representatives ; tokens in order] -> ring layout.  Returns (ring_sem_bits
+    [capacity, d], ring_pos_bits, n_tok); rows that hold nothing are zero."""
+    R = w + g
+    assert w % g == 0 and n_rows - n_rep <= R and R + n_rep <= capacity
+    ring_sem = np.zeros((capacity,) + cache_sem_bits.shape[1:], dtype=cache_sem_bits.dtype)
+    ring_pos = np.zeros((capacity,) + cache_pos_bits.shape[1:], dtype=cache_pos_bits.dtype)
+    first = n_rep * g
+    for i in range(n_rows - n_rep):
+        ring_sem[(first + i) % R] = cache_sem_bits[n_rep + i]
+        ring_pos[(first + i) % R] = cache_pos_bits[n_rep + i]
+    ring_sem[R:R + n_rep] = cache_sem_bits[:n_rep]
+    ring_pos[R:R + n_rep] = cache_pos_bits[:n_rep]
+    return ring_sem, ring_pos, first + (n_rows - n_rep)
+
+
+def ring_to_packed(ring_sem_bits: np.ndarray, ring_pos_bits: np.ndarray, n_rep: int, n_tok: int, g: int, w: int):
+    """The rows of a ring cache that take part, in the order [representatives ; tokens in order]
+    (what decode attends to).  Returns (cache_sem_bits, cache_pos_bits, n_rows)."""
+    R = w + g
+    first = n_rep * g
+    assert 0 <= n_tok - first <= R
+    rows = [R + j for j in range(n_rep)] + [n % R for n in range(first, n_tok)]
+    return ring_sem_bits[rows], ring_pos_bits[rows], len(rows)
+
+
+def mla_decode_update_ring(ring_sem_bits: np.ndarray, ring_pos_bits: np.ndarray, n_rep: int, n_tok: int,
+                           qbar: np.ndarray, g: int, w: int, scale: float):
+    """Sec. 4.3 online update on the ring layout, one sequence: when w + g tokens are uncondensed,
+    the earliest g of them (tokens n_rep*g .. n_rep*g + g - 1) become representative number n_rep
+    (scores of Sec. 4.2 with q_bar, Eq. 6, Eq. 7, Eq. 8), written to row R + n_rep; no other row
+    changes.  Returns (ring_sem_bits, ring_pos_bits, n_rep, anchor offset or -1)."""
+    R = w + g
+    first = n_rep * g
+    if n_tok - first < R or R + n_rep >= ring_sem_bits.shape[0]:
+        return ring_sem_bits, ring_pos_bits, n_rep, -1
+    rows = [(first + i) % R for i in range(g)]
+    grp_sem = bits_to_f64(ring_sem_bits[rows])
+    grp_pos = bits_to_f64(ring_pos_bits[rows])
+    r = condense_stream(np.concatenate([grp_sem, grp_pos], axis=1), grp_sem, qbar, g, 0, scale)   # one group
+    ia = int(r["anchor"][0])
+    ring_sem = ring_sem_bits.copy()
+    ring_pos = ring_pos_bits.copy()
+    ring_sem[R + n_rep] = round_bf16_bits(r["pooled"])[0]
+    ring_pos[R + n_rep] = ring_pos_bits[rows[ia]]
+    return ring_sem, ring_pos, n_rep + 1, ia

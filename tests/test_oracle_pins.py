@@ -569,6 +569,51 @@ def test_online_cache_update_waits_for_a_full_group_and_zero_query_gives_the_mea
     assert np.array_equal(p3[0], pos[0]) and np.array_equal(s3[1:], sem[g:]) and np.array_equal(p3[1:], pos[g:])
 
 
+def test_ring_layout_streaming_reproduces_alg1_on_the_longer_sequence():
+    """The ring layout of the decode cache (token n at row n % (w + g), representatives behind the ring) against
+    Alg. 1: start from the packed cache of a prefix, append tokens at their ring rows, update whenever w + g tokens
+    are uncondensed.  After every token the rows that take part, read in the order [representatives ; tokens], must
+    be the cache Alg. 1 builds from scratch on the longer sequence; the ring wraps several times on the way, and no
+    row other than the new representative's changes in an update."""
+    rng = RNG(23)
+    g, w, dc, dr = 4, 8, 8, 4
+    R = w + g
+    L0, T = w + 2 * g + 3, 4 * R + 5
+    import torch
+    C = torch.from_numpy(rng.standard_normal((L0 + T, dc))).bfloat16()
+    KR = torch.from_numpy(rng.standard_normal((L0 + T, dr))).bfloat16()
+    Cb, KRb = O.torch_bf16_to_bits(C), O.torch_bf16_to_bits(KR)
+    qbar = rng.standard_normal(dc + dr)
+    scale = 0.3
+    start = O.mla_condense(qbar, O.bits_to_f64(Cb[:L0]), O.bits_to_f64(KRb[:L0]), g, w, scale)
+    cap = R + (L0 + T) // g + 1
+    sem, pos, n_tok = O.ring_from_packed(start["cache_sem_bits"], start["cache_pos_bits"], start["m"],
+                                         start["m"] + start["k"], g, w, cap)
+    n_rep = start["m"]
+    assert n_tok == L0
+    back = O.ring_to_packed(sem, pos, n_rep, n_tok, g, w)
+    assert back[2] == start["m"] + start["k"]
+    assert np.array_equal(back[0], start["cache_sem_bits"]) and np.array_equal(back[1], start["cache_pos_bits"])
+    n_updates = 0
+    for t in range(L0, L0 + T):
+        sem[t % R], pos[t % R] = Cb[t], KRb[t]                             # the new token's row
+        n_tok += 1
+        before = (sem.copy(), pos.copy())
+        sem, pos, n_rep2, ia = O.mla_decode_update_ring(sem, pos, n_rep, n_tok, qbar, g, w, scale)
+        if ia >= 0:
+            n_updates += 1
+            changed = np.flatnonzero((sem != before[0]).any(axis=1) | (pos != before[1]).any(axis=1))
+            assert set(changed) <= {R + n_rep} and n_rep2 == n_rep + 1
+        else:
+            assert n_rep2 == n_rep and np.array_equal(sem, before[0]) and np.array_equal(pos, before[1])
+        n_rep = n_rep2
+        whole = O.mla_condense(qbar, O.bits_to_f64(Cb[:t + 1]), O.bits_to_f64(KRb[:t + 1]), g, w, scale)
+        psem, ppos, n_rows = O.ring_to_packed(sem, pos, n_rep, n_tok, g, w)
+        assert n_rep == whole["m"] and n_rows == whole["m"] + whole["k"]
+        assert np.array_equal(psem, whole["cache_sem_bits"]) and np.array_equal(ppos, whole["cache_pos_bits"])
+    assert n_updates == (L0 + T - w) // g - start["m"] and n_updates >= 4 * R // g
+
+
 def test_ablation_reducers_have_their_defining_properties():
     """Table 5 operators: the method's pair is the default; mean pooling is weighted pooling at a zero
     summary query; max selection returns a member of the group bit for bit; max pooling dominates every
