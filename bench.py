@@ -520,6 +520,38 @@ def measure_decode_config(B, dev, batch, peaks, warmup=3, iters=5, parity=None):
         upd = dict(us_per_update_all_sequences=min(times) * 1e3, amortised_us_per_token=min(times) * 1e3 / g,
                    note="every g-th decode step: summary query, condense the earliest g buffered tokens, move the window up")
         del usem, upos
+        # the same moment on the ring layout (token n at row n % (w + g), representatives behind the ring): nothing
+        # moves; timed with the query tails and with a summary query the caller kept up to date while decoding
+        R = cfg.window + g
+        cap_r = R + m + 8
+        rsem = torch.randn((batch, cap_r, 1, cfg.d_sem), generator=gen, device=dev).bfloat16()
+        rpos = torch.randn((batch, cap_r, 1, cfg.d_pos), generator=gen, device=dev).bfloat16()
+        qbar_ready = torch.randn((batch, 1, cfg.d_sem + cfg.d_pos), generator=gen, device=dev, dtype=torch.float32)
+        n_tok_full = torch.full((batch,), m * g + R, dtype=torch.int32, device=dev)
+        ring = {}
+        for name, qb in (("tails", None), ("ready_summary_query", qbar_ready)):
+            times = []
+            for _ in range(3):
+                n_rep_t = torch.full((batch,), m, dtype=torch.int32, device=dev)
+                torch.cuda.synchronize()
+                e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+                e0.record()
+                B.decode_update_ring(p, q_tail_sem, q_tail_pos, rsem, rpos, n_rep_t, n_tok_full, qbar=qb, ws=wsu)
+                e1.record()
+                torch.cuda.synchronize()
+                times.append(e0.elapsed_time(e1))
+                assert int(n_rep_t.min()) == m + 1
+            ring[name] = min(times) * 1e3
+        # decode over the ring one token after that update: g - 1 stale rows inside the ring are masked out
+        n_rep_t = torch.full((batch,), m + 1, dtype=torch.int32, device=dev)
+        n_tok_t = torch.full((batch,), m * g + R + 1, dtype=torch.int32, device=dev)
+        out_r = torch.empty_like(out)
+        t_ring_dec = time_cuda(lambda: B.decode_attention_ring(p, q_new_sem, q_new_pos, rsem, rpos, n_rep_t, n_tok_t, out=out_r, ws=wsd),
+                               warmup, iters)
+        upd["ring_layout"] = dict(us_per_update_all_sequences=ring["tails"], us_with_ready_summary_query=ring["ready_summary_query"],
+                                  amortised_us_per_token=ring["ready_summary_query"] / g, decode_us=t_ring_dec * 1e3,
+                                  note="lca_decode_update_ring / lca_decode_attention_ring: one new row per sequence, no row moves")
+        del rsem, rpos
     except Exception as ex:
         upd = dict(error=str(ex)[:200])
     if parity is not None:

@@ -223,6 +223,53 @@ int lca_decode_update(const lca_params* p, const void* q_tail_sem, const void* q
                       int32_t* cache_rows, int32_t* anchor_out, void* ws, size_t ws_bytes,
                       void* stream);
 
+/* ---- Ring layout of the decode cache -------------------------------------------------------
+ * Sec. 4.3 fixes what the cache holds while decoding (the m representatives and the most recent
+ * tokens) and how a group is condensed, not where the rows live.  In the packed layout above the
+ * representatives are followed by the tokens in order, so every update moves the whole window up
+ * by group_size - 1 rows.  In the ring layout nothing moves:
+ *   rows [0, R), R = window + group_size: the uncondensed tokens; token number n of the sequence
+ *                (0-based, counted from the start of the sequence) is at row n % R
+ *   rows [R, R + n_rep[b]): the representatives in group order
+ * State per sequence: n_rep[b] and n_tok[b] (tokens of the sequence so far); the uncondensed tokens
+ * are n_rep[b]*group_size .. n_tok[b]-1, at most R of them.  The caller writes the row of a new
+ * token at row n_tok[b] % R and then counts it in n_tok[b].  window must be a multiple of group_size
+ * (groups leave the ring whole), ring_row_capacity >= R + the representatives the sequence will have;
+ * buffers are [B, ring_row_capacity, n_kv_heads, d_sem | d_pos].  Rows that hold nothing yet must hold
+ * finite numbers (e.g. zeros), as for lca_decode_attention.
+ *
+ * lca_ring_from_packed: the step from a packed cache (lca_condense output, or a packed decode cache)
+ * to the ring layout: representatives to rows R.., token i of the packed tail to row
+ * (n_rep[b]*group_size + i) % R, n_tok_out[b] = n_rep[b]*group_size + packed_rows[b] - n_rep[b].
+ *   packed_rows [B], n_rep [B] int32 (device); packed_sem / packed_pos [B, packed_row_capacity, ...].
+ *   A sequence with more than R packed tokens, or more representatives than fit behind the ring, is
+ *   truncated to what fits (the caller sizes the buffers; nothing is written out of bounds). */
+int lca_ring_from_packed(const lca_params* p, const void* packed_sem, const void* packed_pos,
+                         const int32_t* packed_rows, const int32_t* n_rep, int32_t packed_row_capacity,
+                         void* ring_sem, void* ring_pos, int32_t ring_row_capacity, int32_t* n_tok_out,
+                         void* stream);
+
+/* lca_decode_attention over the ring layout: the query attends to the n_rep[b] representatives (each
+ * with rep_logit_bias) and to the uncondensed tokens n_rep[b]*g .. n_tok[b]-1 (the caller has written
+ * and counted the new token's own row).  Ring rows that still hold tokens of an already condensed
+ * group are left out.  Same arithmetic, outputs and workspace (LCA_WS_DECODE) as lca_decode_attention;
+ * n_rep, n_tok [B] int32 (device). */
+int lca_decode_attention_ring(const lca_params* p, const void* q_sem, const void* q_pos,
+                              const void* ring_sem, const void* ring_pos, const int32_t* n_rep,
+                              const int32_t* n_tok, int32_t ring_row_capacity, void* out, float* lse_opt,
+                              void* ws, size_t ws_bytes, void* stream);
+
+/* lca_decode_update over the ring layout: a sequence with window + group_size uncondensed tokens has
+ * its earliest group (ring rows (n_rep[b]*g) % R .. +g-1) condensed exactly as in lca_decode_update;
+ * the representative is written to row R + n_rep[b] and n_rep[b] grows by one.  No other row and no
+ * other counter changes (n_tok is read only).  A sequence whose representative region is full
+ * (R + n_rep[b] == ring_row_capacity) is left alone, anchor_out = -1.
+ * Summary-query arguments, anchor_out and workspace (LCA_WS_UPDATE) as for lca_decode_update. */
+int lca_decode_update_ring(const lca_params* p, const void* q_tail_sem, const void* q_tail_pos,
+                           int64_t q_tail_batch_stride, const float* qbar_opt, void* ring_sem,
+                           void* ring_pos, int32_t ring_row_capacity, int32_t* n_rep, const int32_t* n_tok,
+                           int32_t* anchor_out, void* ws, size_t ws_bytes, void* stream);
+
 /* Value up-projection of the latent attention output (Alg. 1: v = c W^UV; Sec. 4.3: in the absorbed
  * form the attention result lives in the latent space and W^UV is applied to it once per query and
  * head):   out_v[t, h, :] = attn_latent[t, h, :] . W^UV[h]

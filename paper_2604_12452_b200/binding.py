@@ -72,6 +72,12 @@ def _load() -> C.CDLL:
     lib.lca_decode_attention.argtypes = [P, vp, vp, vp, vp, vp, i32, i32, vp, vp, vp, sz, vp]
     lib.lca_decode_update.restype = C.c_int
     lib.lca_decode_update.argtypes = [P, vp, vp, i64, vp, vp, vp, i32, vp, vp, vp, vp, sz, vp]
+    lib.lca_ring_from_packed.restype = C.c_int
+    lib.lca_ring_from_packed.argtypes = [P, vp, vp, vp, vp, i32, vp, vp, i32, vp, vp]
+    lib.lca_decode_attention_ring.restype = C.c_int
+    lib.lca_decode_attention_ring.argtypes = [P, vp, vp, vp, vp, vp, vp, i32, vp, vp, vp, sz, vp]
+    lib.lca_decode_update_ring.restype = C.c_int
+    lib.lca_decode_update_ring.argtypes = [P, vp, vp, i64, vp, vp, vp, i32, vp, vp, vp, vp, sz, vp]
     pi32, pi64 = C.POINTER(i32), C.POINTER(i64)
     lib.lca_varlen_layout.restype = C.c_int
     lib.lca_varlen_layout.argtypes = [P, pi32, pi64, pi64, pi64]
@@ -186,6 +192,29 @@ def lca_decode_update(params, q_tail_sem, q_tail_pos, q_tail_batch_stride, qbar_
     return int(_lib.lca_decode_update(C.byref(params), _ptr(q_tail_sem), _ptr(q_tail_pos), int(q_tail_batch_stride),
                                       _ptr(qbar_opt), _ptr(cache_sem), _ptr(cache_pos), int(cache_row_capacity),
                                       _ptr(n_rep), _ptr(cache_rows), _ptr(anchor_out), _ptr(ws), wsb, _stream(stream)))
+
+
+def lca_ring_from_packed(params, packed_sem, packed_pos, packed_rows, n_rep, packed_row_capacity, ring_sem, ring_pos,
+                         ring_row_capacity, n_tok_out, stream=None) -> int:
+    return int(_lib.lca_ring_from_packed(C.byref(params), _ptr(packed_sem), _ptr(packed_pos), _ptr(packed_rows), _ptr(n_rep),
+                                         int(packed_row_capacity), _ptr(ring_sem), _ptr(ring_pos), int(ring_row_capacity),
+                                         _ptr(n_tok_out), _stream(stream)))
+
+
+def lca_decode_attention_ring(params, q_sem, q_pos, ring_sem, ring_pos, n_rep, n_tok, ring_row_capacity, out, lse_opt,
+                              ws, ws_bytes=None, stream=None) -> int:
+    wsb = _nbytes(ws) if ws_bytes is None else int(ws_bytes)
+    return int(_lib.lca_decode_attention_ring(C.byref(params), _ptr(q_sem), _ptr(q_pos), _ptr(ring_sem), _ptr(ring_pos),
+                                              _ptr(n_rep), _ptr(n_tok), int(ring_row_capacity), _ptr(out), _ptr(lse_opt),
+                                              _ptr(ws), wsb, _stream(stream)))
+
+
+def lca_decode_update_ring(params, q_tail_sem, q_tail_pos, q_tail_batch_stride, qbar_opt, ring_sem, ring_pos,
+                           ring_row_capacity, n_rep, n_tok, anchor_out, ws, ws_bytes=None, stream=None) -> int:
+    wsb = _nbytes(ws) if ws_bytes is None else int(ws_bytes)
+    return int(_lib.lca_decode_update_ring(C.byref(params), _ptr(q_tail_sem), _ptr(q_tail_pos), int(q_tail_batch_stride),
+                                           _ptr(qbar_opt), _ptr(ring_sem), _ptr(ring_pos), int(ring_row_capacity),
+                                           _ptr(n_rep), _ptr(n_tok), _ptr(anchor_out), _ptr(ws), wsb, _stream(stream)))
 
 
 def _lens(seq_lens):
@@ -372,4 +401,46 @@ def decode_update(params: LcaParams, q_tail_sem, q_tail_pos, cache_sem, cache_po
     st = lca_decode_update(params, q_tail_sem, q_tail_pos, n, qbar, cache_sem, cache_pos, cache_sem.shape[1], n_rep,
                            cache_rows, anchor, ws, stream=stream)
     _check(st, "lca_decode_update")
+    return anchor
+
+
+def ring_from_packed(params: LcaParams, packed_sem, packed_pos, packed_rows, n_rep, ring_row_capacity: int, stream=None):
+    """Allocate zeroed ring buffers and fill them from a packed cache.  Returns (ring_sem, ring_pos, n_tok [B] int32)."""
+    dev = packed_sem.device
+    B = params.batch
+    ring_sem = torch.zeros((B, ring_row_capacity) + tuple(packed_sem.shape[2:]), dtype=torch.bfloat16, device=dev)
+    ring_pos = torch.zeros((B, ring_row_capacity) + tuple(packed_pos.shape[2:]), dtype=torch.bfloat16, device=dev)
+    n_tok = torch.empty((B,), dtype=torch.int32, device=dev)
+    st = lca_ring_from_packed(params, packed_sem, packed_pos, packed_rows, n_rep, packed_sem.shape[1], ring_sem, ring_pos,
+                              ring_row_capacity, n_tok, stream=stream)
+    _check(st, "lca_ring_from_packed")
+    return ring_sem, ring_pos, n_tok
+
+
+def decode_attention_ring(params: LcaParams, q_sem, q_pos, ring_sem, ring_pos, n_rep, n_tok, out=None,
+                          want_lse: bool = False, ws=None, stream=None):
+    dev = ring_sem.device
+    B, H = params.batch, params.n_q_heads
+    if out is None:
+        out = torch.empty((B, H, params.d_sem), dtype=torch.bfloat16, device=dev)
+    lse = torch.empty((B, H), dtype=torch.float32, device=dev) if want_lse else None
+    if ws is None:
+        ws = workspace(params, LCA_WS_DECODE, dev)
+    st = lca_decode_attention_ring(params, q_sem, q_pos, ring_sem, ring_pos, n_rep, n_tok, ring_sem.shape[1], out, lse,
+                                   ws, stream=stream)
+    _check(st, "lca_decode_attention_ring")
+    return out, lse
+
+
+def decode_update_ring(params: LcaParams, q_tail_sem, q_tail_pos, ring_sem, ring_pos, n_rep, n_tok,
+                       qbar: Optional[torch.Tensor] = None, ws=None, stream=None):
+    """Run lca_decode_update_ring in place on the ring buffers and n_rep; returns anchor offsets [B, Hkv]."""
+    dev = ring_sem.device
+    anchor = torch.empty((params.batch, params.n_kv_heads), dtype=torch.int32, device=dev)
+    if ws is None:
+        ws = workspace(params, LCA_WS_UPDATE, dev)
+    n = params.n_summary_q if params.n_summary_q > 0 else params.group_size
+    st = lca_decode_update_ring(params, q_tail_sem, q_tail_pos, n, qbar, ring_sem, ring_pos, ring_sem.shape[1], n_rep,
+                                n_tok, anchor, ws, stream=stream)
+    _check(st, "lca_decode_update_ring")
     return anchor

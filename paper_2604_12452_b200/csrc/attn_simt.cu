@@ -11,11 +11,11 @@ struct SimtArgs {
   const bf16* q_sem; const bf16* q_pos;
   const bf16* kv_sem; const bf16* kv_pos;
   const bf16* cache_sem; const bf16* cache_pos;
-  const int32_t* cache_rows;
   bf16* out; float* lse;
-  int B, q_len, Hq, Hkv, decode, L, g, w, cap, n_rep_bias;
+  int B, q_len, Hq, Hkv, decode, L, g, w, cap;
   float scale, bias;
   SeqTab tab;              // ragged prefill batch (tok_off != nullptr): q_len, L and cap are unused
+  DecodeLayout dl;         // decode: which cache rows take part
   long long n_rows;        // query rows of the launch (tokens x heads)
 };
 
@@ -57,15 +57,16 @@ attn_simt_kernel(SimtArgs a) {
     }
   }
 
-  int n_a, b_first, b_last, bias_rows;
+  int n_a, b_first, b_last;
+  DecodeSpan sp;
   if (a.decode) {
-    n_a = min(max(a.cache_rows[b], 0), a.cap);
+    sp = decode_span(a.dl, b);
+    n_a = sp.rows_end;
     b_first = 0; b_last = -1;
-    bias_rows = min(a.n_rep_bias, n_a);
   } else {
     n_a = reps_visible(t, a.w, a.g);
     b_first = n_a * a.g; b_last = t;
-    bias_rows = n_a;
+    sp.rows_end = n_a; sp.inv_lo = sp.inv_hi = 0; sp.bias_lo = 0; sp.bias_hi = n_a;
   }
 
   float acc[2 * PS];
@@ -74,17 +75,20 @@ attn_simt_kernel(SimtArgs a) {
   float mx = -INFINITY, l = 0.f;
 
   const int n_total = n_a + (b_last - b_first + 1);
+  int n_seen = 0;
   for (int x = 0; x < n_total; ++x) {
     const bf16 *ks, *kp;
     float add = 0.f;
     if (x < n_a) {
+      if (x >= sp.inv_lo && x < sp.inv_hi) continue;       // ring layout: a condensed token that is still in its row
       size_t r = (cbase + x) * a.Hkv + hk;
       ks = a.cache_sem + r * D_SEM; kp = a.cache_pos + r * D_POS;
-      if (x < bias_rows) add = a.bias;
+      if (x >= sp.bias_lo && x < sp.bias_hi) add = a.bias;
     } else {
       size_t r = (kbase + (b_first + x - n_a)) * a.Hkv + hk;
       ks = a.kv_sem + r * D_SEM; kp = a.kv_pos + r * D_POS;
     }
+    ++n_seen;
     float2 v[PS];
 #pragma unroll
     for (int i = 0; i < PS; ++i) v[i] = __bfloat1622float2(reinterpret_cast<const bf162*>(ks)[lane + 32 * i]);
@@ -110,12 +114,12 @@ attn_simt_kernel(SimtArgs a) {
     }
     mx = mn;
   }
-  const float inv = n_total > 0 ? 1.f / l : 0.f;
+  const float inv = n_seen > 0 ? 1.f / l : 0.f;
   bf162* dst = reinterpret_cast<bf162*>(a.out + (size_t)row * D_SEM);
 #pragma unroll
   for (int i = 0; i < PS; ++i)
     dst[lane + 32 * i] = __floats2bfloat162_rn(acc[2 * i] * inv, acc[2 * i + 1] * inv);
-  if (a.lse && lane == 0) a.lse[row] = n_total > 0 ? mx + logf(l) : -INFINITY;
+  if (a.lse && lane == 0) a.lse[row] = n_seen > 0 ? mx + logf(l) : -INFINITY;
 }
 
 int attn_simt_launch(const AttnProblem& p) {
@@ -123,10 +127,11 @@ int attn_simt_launch(const AttnProblem& p) {
   a.q_sem = (const bf16*)p.q_sem; a.q_pos = (const bf16*)p.q_pos;
   a.kv_sem = (const bf16*)p.kv_sem; a.kv_pos = (const bf16*)p.kv_pos;
   a.cache_sem = (const bf16*)p.cache_sem; a.cache_pos = (const bf16*)p.cache_pos;
-  a.cache_rows = p.cache_rows; a.out = (bf16*)p.out; a.lse = p.lse;
+  a.out = (bf16*)p.out; a.lse = p.lse;
   a.B = p.batch; a.q_len = p.q_len; a.Hq = p.n_q_heads; a.Hkv = p.n_kv_heads; a.decode = p.decode;
   a.L = p.seq_len; a.g = p.group_size; a.w = p.window; a.cap = p.cache_row_capacity;
-  a.n_rep_bias = p.n_rep_bias; a.scale = p.softmax_scale; a.bias = p.rep_logit_bias;
+  a.scale = p.softmax_scale; a.bias = p.rep_logit_bias;
+  a.dl = DecodeLayout{p.cache_rows, p.ring_n_rep, p.ring_n_tok, p.cache_row_capacity, p.n_rep_bias, p.window + p.group_size, p.group_size};
   const long long rows = p.h_tok_off ? (long long)p.h_tok_off[p.batch] * p.n_q_heads : (long long)p.batch * p.q_len * p.n_q_heads;
   a.tab = p.h_tok_off ? p.tab : SeqTab{};
   a.n_rows = rows;

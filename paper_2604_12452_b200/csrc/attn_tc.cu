@@ -34,8 +34,9 @@ static constexpr float RESCALE_THRESHOLD = 8.0f;   // log2 units
 
 struct TcParams {
   CUtensorMap q_sem, q_pos, kv_sem, kv_pos, cache_sem, cache_pos;   // 3-D {d, heads, rows}
-  bf16* out; float* lse; const int32_t* cache_rows;
-  int B, q_len, Hq, Hkv, L, g, w, cap, n_rep_bias, decode;
+  bf16* out; float* lse;
+  DecodeLayout dl;                // decode: which rows of a sequence's cache take part (packed or ring layout)
+  int B, q_len, Hq, Hkv, L, g, w, cap, decode;
   int HB, TB, n_tok_tiles, d_out;
   int out_wide;                   // out is 32-byte aligned: 256-bit stores
   float scale_log2, bias_log2;
@@ -100,7 +101,7 @@ attn_tc1_kernel(const __grid_constant__ TcParams p) {
   const int hk = (p.Hkv == 1) ? 0 : hb;
   int nA, nB, first_lo, n_a_lo, n_a_hi;
   if (p.decode) {
-    n_a_hi = n_a_lo = min(max(p.cache_rows[b], 0), p.cap);
+    n_a_hi = n_a_lo = decode_span(p.dl, b).rows_end;
     first_lo = 0; nB = 0;
   } else {
     n_a_lo = reps_visible(t0, p.w, p.g);
@@ -235,9 +236,11 @@ attn_tc1_kernel(const __grid_constant__ TcParams p) {
     const int tl = r / p.HB, hl = r % p.HB;
     const int t_row = t0 + tl;
     const bool row_valid = t_row < p.q_len;
-    int n_a_row, bias_rows, first_row;
-    if (p.decode) { n_a_row = n_a_hi; bias_rows = min(p.n_rep_bias, n_a_row); first_row = 0; }
-    else { n_a_row = reps_visible(min(t_row, p.q_len - 1), p.w, p.g); bias_rows = n_a_row; first_row = n_a_row * p.g; }
+    int n_a_row, first_row;
+    // rows [inv_lo, inv_hi) of the cache part do not take part (ring layout); rows [bias_lo, bias_hi) are representatives
+    DecodeSpan sp = {};
+    if (p.decode) { sp = decode_span(p.dl, b); n_a_row = n_a_hi; first_row = 0; }
+    else { n_a_row = reps_visible(min(t_row, p.q_len - 1), p.w, p.g); sp.bias_hi = n_a_row; first_row = n_a_row * p.g; }
     volatile float* red = reinterpret_cast<volatile float*>(base_ptr + P::OFF_RED);          // [3][2][128]
     volatile int* fail_word = reinterpret_cast<volatile int*>(base_ptr + P::OFF_MISC + 8);   // [2]
     if (half == 0 && r < 2) fail_word[r] = 0;
@@ -268,8 +271,12 @@ attn_tc1_kernel(const __grid_constant__ TcParams p) {
         int lo, hi;                                  // visible columns of this thread: lo <= c <= hi
         if (isA) { lo = 0; hi = n_a_row - key0 - 1; need_mask = tile_key0 + BN > n_a_lo; }
         else { lo = first_row - key0; hi = t_row - key0; need_mask = (tile_key0 < n_a_hi * p.g) || (tile_key0 + BN - 1 > t0); }
-        const int blim = isA ? bias_rows - key0 : 0;  // columns < blim receive the bias
-        plain = !need_mask && !(isA && p.bias_log2 != 0.f);
+        bool tile_bias = false;
+        if (isA) {
+          need_mask = need_mask || (tile_key0 < sp.inv_hi && tile_key0 + BN > sp.inv_lo);
+          tile_bias = p.bias_log2 != 0.f && tile_key0 < sp.bias_hi && tile_key0 + BN > sp.bias_lo;
+        }
+        plain = !need_mask && !tile_bias;
         if (plain) {
           // interior tile: the raw products stay in sr, the (positive) scale is applied to the maximum
           // here and folded into the exponent's multiply-add below
@@ -283,16 +290,19 @@ attn_tc1_kernel(const __grid_constant__ TcParams p) {
         } else {
           // boundary tile: scale, bias and mask with selects only (per-element branches cost ~25 cycles
           // each here), four short maximum chains
-          const float bias = (isA && p.bias_log2 != 0.f) ? p.bias_log2 : 0.f;
+          const float bias = tile_bias ? p.bias_log2 : 0.f;
           const int lo_m = need_mask ? lo : -(1 << 30), hi_m = need_mask ? hi : (1 << 30);
+          // columns [blo, blo + bspan) receive the bias, columns [ilo, ilo + ispan) are left out (both empty outside the cache part)
+          const int blo = sp.bias_lo - key0, ilo = sp.inv_lo - key0;
+          const unsigned bspan = isA ? (unsigned)(sp.bias_hi - sp.bias_lo) : 0u, ispan = isA ? (unsigned)(sp.inv_hi - sp.inv_lo) : 0u;
           float tm[4] = {-INFINITY, -INFINITY, -INFINITY, -INFINITY};
 #pragma unroll
           for (int q = 0; q < 2; ++q) {
 #pragma unroll
             for (int i = 0; i < 32; ++i) {
               const int c = q * 32 + i;
-              float s = fmaf(__uint_as_float(sr[q][i]), p.scale_log2, c < blim ? bias : 0.f);
-              s = ((c >= lo_m) & (c <= hi_m)) ? s : -INFINITY;
+              float s = fmaf(__uint_as_float(sr[q][i]), p.scale_log2, (unsigned)(c - blo) < bspan ? bias : 0.f);
+              s = ((c >= lo_m) & (c <= hi_m) & !((unsigned)(c - ilo) < ispan)) ? s : -INFINITY;
               sr[q][i] = __float_as_uint(s);
               tm[i & 3] = fmaxf(tm[i & 3], s);
             }
@@ -507,11 +517,12 @@ int attn_tc_launch(const AttnProblem& a) {
   const int rep = a.n_q_heads / a.n_kv_heads;
   p.HB = rep; p.TB = ROWS / rep;
   p.B = a.batch; p.q_len = a.q_len; p.Hq = a.n_q_heads; p.Hkv = a.n_kv_heads; p.L = a.seq_len;
-  p.g = a.group_size; p.w = a.window; p.cap = a.cache_row_capacity; p.n_rep_bias = a.n_rep_bias;
+  p.g = a.group_size; p.w = a.window; p.cap = a.cache_row_capacity;
+  p.dl = DecodeLayout{a.cache_rows, a.ring_n_rep, a.ring_n_tok, a.cache_row_capacity, a.n_rep_bias, a.window + a.group_size, a.group_size};
   p.decode = a.decode; p.n_tok_tiles = (a.q_len + p.TB - 1) / p.TB; p.d_out = a.d_sem;
   p.scale_log2 = a.softmax_scale * 1.4426950408889634f;
   p.bias_log2 = a.rep_logit_bias * 1.4426950408889634f;
-  p.out = (bf16*)a.out; p.lse = a.lse; p.cache_rows = a.cache_rows;
+  p.out = (bf16*)a.out; p.lse = a.lse;
   p.out_wide = (reinterpret_cast<uintptr_t>(a.out) & 31u) == 0;
   const long long qrows = (long long)a.batch * a.q_len;
   bool ok = make_tensor_map_3d(&p.q_sem, nullptr, 0, 0, 0, 0, 0);

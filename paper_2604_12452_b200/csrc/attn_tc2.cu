@@ -67,8 +67,9 @@ struct Tc2Params {
   CUtensorMap k_pos, c_pos;       // rope keys of the tokens / of the condensed cache, box of 64 rows
   CUtensorMap k_sem, c_sem;       // latents seen as (64 columns, rows, chunks): box of 64 rows x KBOX chunks
   CUtensorMap k_val, c_val;       // the same memory, box of 64 rows x VBOX chunks
-  bf16* out; float* lse; const int32_t* cache_rows;
-  int B, q_len, H, L, g, w, cap, n_rep_bias, decode;
+  bf16* out; float* lse;
+  DecodeLayout dl;                // decode: which rows of a sequence's cache take part (packed or ring layout)
+  int B, q_len, H, L, g, w, cap, decode;
   int HB, TB, n_tok_tiles, n_head_blocks;
   int out_wide;                   // out is 32-byte aligned: 256-bit stores
   long long n_items;              // query tiles x head blocks x batch
@@ -119,7 +120,7 @@ __device__ __forceinline__ Item make_item(const Tc2Params& p, long long idx) {
   it.j0 = 0; it.slot = -1;
   int nB;
   if (p.decode) {
-    it.n_a_hi = it.n_a_lo = min(max(p.cache_rows[it.b], 0), p.cap);
+    it.n_a_hi = it.n_a_lo = decode_span(p.dl, it.b).rows_end;
     it.first_lo = 0; nB = 0;
   } else {
     it.n_a_lo = reps_visible(it.t0, p.w, p.g);
@@ -134,7 +135,7 @@ __device__ __forceinline__ Item make_item(const Tc2Params& p, long long idx) {
 
 // Key tiles of decode unit u = (sequence, head block), head block fastest.
 __device__ __forceinline__ int unit_tiles(const Tc2Params& p, int u) {
-  const int rows = min(max(p.cache_rows[u / p.n_head_blocks], 0), p.cap);
+  const int rows = decode_span(p.dl, u / p.n_head_blocks).rows_end;
   return (rows + pair::BN - 1) / pair::BN;
 }
 // Ranges (one per pair, `q` tiles long) that touch a unit of n > 0 tiles starting at tile `off` of the line.
@@ -206,7 +207,7 @@ __device__ __forceinline__ bool walk_next(const Tc2Params& p, Walk& w, Item& it)
   it.head0 = (w.u % p.n_head_blocks) * p.HB;
   it.len = 1; it.t0 = 0; it.t1 = 0;
   it.qbase = it.b * p.q_len; it.kbase = 0; it.cbase = it.b * p.cap;
-  it.n_a_hi = it.n_a_lo = min(max(p.cache_rows[it.b], 0), p.cap);
+  it.n_a_hi = it.n_a_lo = decode_span(p.dl, it.b).rows_end;
   it.first_lo = 0;
   it.j0 = j0; it.nA = it.n_tiles = j1 - j0;
   it.slot = (j0 == 0 && j1 == n) ? -1 : w.slot_base + (int)(w.pair_id - w.off / w.q);
@@ -220,6 +221,9 @@ __device__ __forceinline__ bool ragged_decode_tile(const Tc2Params& p, const Ite
   return p.decode && (it.j0 + j + 1) * pair::BN > it.n_a_hi;
 }
 
+// RING: decode over the ring layout of the cache (rows of condensed tokens inside the ring are masked out, the
+// representatives' bias applies from row R on); a separate instantiation so that the prefill code stays as it is.
+template <bool RING>
 __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(pair::THREADS, 1)
 attn_tc2_kernel(const __grid_constant__ Tc2Params p) {
   using namespace pair;
@@ -502,7 +506,8 @@ attn_tc2_kernel(const __grid_constant__ Tc2Params p) {
     const int t_row = t0 + tl;
     const bool row_valid = t_row <= it.t1;
     int n_a_row, bias_rows, first_row;
-    if (p.decode) { n_a_row = n_a_hi; bias_rows = min(p.n_rep_bias, n_a_row); first_row = 0; }
+    DecodeSpan sp = {};
+    if (p.decode) { sp = decode_span(p.dl, it.b); n_a_row = n_a_hi; bias_rows = sp.bias_hi; first_row = 0; }
     else { n_a_row = reps_visible(min(t_row, it.len - 1), p.w, p.g); bias_rows = n_a_row; first_row = n_a_row * p.g; }
     float m_ref = -INFINITY, l_sum = 0.f;
     bool all_left = false;                       // every one of the 128 threads left the tile loop at a barrier
@@ -529,7 +534,12 @@ attn_tc2_kernel(const __grid_constant__ Tc2Params p) {
         if (isA) { lo = 0; hi = n_a_row - key0 - 1; need_mask = tile_key0 + BN > n_a_lo; }
         else { lo = first_row - key0; hi = t_row - key0; need_mask = (tile_key0 < n_a_hi * p.g) || (tile_key0 + BN - 1 > t0); }
         const int blim = isA ? bias_rows - key0 : 0;
-        plain = !need_mask && !(isA && p.bias_log2 != 0.f);
+        bool tile_bias = isA && p.bias_log2 != 0.f;
+        if constexpr (RING) {
+          need_mask = need_mask || (tile_key0 < sp.inv_hi && tile_key0 + BN > sp.inv_lo);
+          tile_bias = tile_bias && tile_key0 < sp.bias_hi && tile_key0 + BN > sp.bias_lo;
+        }
+        plain = !need_mask && !tile_bias;
         if (plain) {
           // interior tile: the raw products stay in sr, the (positive) scale is applied to the maximum
           // here and folded into the exponent's multiply-add below
@@ -545,16 +555,25 @@ attn_tc2_kernel(const __grid_constant__ Tc2Params p) {
         } else {
           // boundary tile: scale, bias and mask with selects only (per-element branches cost ~25 cycles
           // each here), four short maximum chains
-          const float bias = (isA && p.bias_log2 != 0.f) ? p.bias_log2 : 0.f;
+          const float bias = tile_bias ? p.bias_log2 : 0.f;
           const int lo_m = need_mask ? lo : -(1 << 30), hi_m = need_mask ? hi : (1 << 30);
+          // ring layout: columns [ilo, ilo + ispan) are condensed tokens still in their rows, [blo, blo + bspan) representatives
+          const int ilo = sp.inv_lo - key0, blo = sp.bias_lo - key0;
+          const unsigned ispan = (unsigned)(sp.inv_hi - sp.inv_lo), bspan = (unsigned)(sp.bias_hi - sp.bias_lo);
           float tm[4] = {-INFINITY, -INFINITY, -INFINITY, -INFINITY};
 #pragma unroll
           for (int q = 0; q < 2; ++q) {
 #pragma unroll
             for (int i = 0; i < 32; ++i) {
               const int c = q * 32 + i;
-              float s = fmaf(__uint_as_float(sr[q][i]), p.scale_log2, c < blim ? bias : 0.f);
-              s = ((c >= lo_m) & (c <= hi_m)) ? s : -INFINITY;
+              float s;
+              if constexpr (RING) {
+                s = fmaf(__uint_as_float(sr[q][i]), p.scale_log2, (unsigned)(c - blo) < bspan ? bias : 0.f);
+                s = ((c >= lo_m) & (c <= hi_m) & !((unsigned)(c - ilo) < ispan)) ? s : -INFINITY;
+              } else {
+                s = fmaf(__uint_as_float(sr[q][i]), p.scale_log2, c < blim ? bias : 0.f);
+                s = ((c >= lo_m) & (c <= hi_m)) ? s : -INFINITY;
+              }
               sr[q][i] = __float_as_uint(s);
               tm[i & 3] = fmaxf(tm[i & 3], s);
             }
@@ -826,8 +845,8 @@ static int resident_pairs() {
   attr.id = cudaLaunchAttributeClusterDimension;
   attr.val.clusterDim.x = 2; attr.val.clusterDim.y = 1; attr.val.clusterDim.z = 1;
   cfg.attrs = &attr; cfg.numAttrs = 1;
-  if (cudaFuncSetAttribute(attn_tc2_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, pair::SMEM_BYTES) != cudaSuccess ||
-      cudaOccupancyMaxActiveClusters(&n, attn_tc2_kernel, &cfg) != cudaSuccess || n <= 0) {
+  if (cudaFuncSetAttribute(attn_tc2_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, pair::SMEM_BYTES) != cudaSuccess ||
+      cudaOccupancyMaxActiveClusters(&n, attn_tc2_kernel<false>, &cfg) != cudaSuccess || n <= 0) {
     cudaGetLastError();
     int sms = 0;
     if (cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || sms < 2) sms = 148;   // no device: a B200
@@ -846,7 +865,8 @@ int attn_tc2_launch(const AttnProblem& a) {
   p.HB = H >= 128 ? 128 : H;
   p.TB = 128 / p.HB;
   p.B = a.batch; p.q_len = a.q_len; p.H = H; p.L = a.seq_len; p.g = a.group_size; p.w = a.window;
-  p.cap = a.cache_row_capacity; p.n_rep_bias = a.n_rep_bias; p.decode = a.decode;
+  p.cap = a.cache_row_capacity; p.decode = a.decode;
+  p.dl = DecodeLayout{a.cache_rows, a.ring_n_rep, a.ring_n_tok, a.cache_row_capacity, a.n_rep_bias, a.window + a.group_size, a.group_size};
   p.n_tok_tiles = (a.q_len + p.TB - 1) / p.TB;
   p.n_head_blocks = H >= 128 ? H / 128 : 1;
   p.n_items = (long long)p.n_tok_tiles * p.n_head_blocks * a.batch;
@@ -881,7 +901,7 @@ int attn_tc2_launch(const AttnProblem& a) {
   }
   p.scale_log2 = a.softmax_scale * 1.4426950408889634f;
   p.bias_log2 = a.rep_logit_bias * 1.4426950408889634f;
-  p.out = (bf16*)a.out; p.lse = a.lse; p.cache_rows = a.cache_rows;
+  p.out = (bf16*)a.out; p.lse = a.lse;
   p.out_wide = (reinterpret_cast<uintptr_t>(a.out) & 31u) == 0;
   const int hbc = p.HB >= 64 ? 64 : p.HB, tbc = 64 / hbc;
   bool ok = make_tensor_map_3d(&p.q_sem, a.q_sem, 512, H, qrows, hbc, tbc);
@@ -893,7 +913,9 @@ int attn_tc2_launch(const AttnProblem& a) {
   ok = ok && make_tensor_map_chunks(&p.k_val, a.kv_sem, 8, krows, 64, VBOX);
   ok = ok && make_tensor_map_chunks(&p.c_val, a.cache_sem, 8, crows, 64, VBOX);
   if (!ok) return LCA_ERR_CUDA;
-  if (cudaFuncSetAttribute(attn_tc2_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM_BYTES) != cudaSuccess)
+  const bool ring = a.decode && a.ring_n_tok != nullptr;
+  if (cudaFuncSetAttribute(ring ? attn_tc2_kernel<true> : attn_tc2_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                           SMEM_BYTES) != cudaSuccess)
     return LCA_ERR_CUDA;
   long long n_pairs = p.n_items < resident_pairs() ? p.n_items : resident_pairs();
   if (n_pairs <= 0) return LCA_OK;
@@ -905,7 +927,8 @@ int attn_tc2_launch(const AttnProblem& a) {
     n_pairs = resident_pairs();
   }
   dim3 grid((unsigned)(2 * n_pairs));
-  attn_tc2_kernel<<<grid, THREADS, SMEM_BYTES, a.stream>>>(p);
+  if (ring) attn_tc2_kernel<true><<<grid, THREADS, SMEM_BYTES, a.stream>>>(p);
+  else attn_tc2_kernel<false><<<grid, THREADS, SMEM_BYTES, a.stream>>>(p);
   note_launch();
   if (p.split) {
     decode_combine_kernel<<<dim3((unsigned)(a.batch * p.n_head_blocks * p.HB)), 128, 0, a.stream>>>(p, (int)n_pairs);

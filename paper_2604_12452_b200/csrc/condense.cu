@@ -60,8 +60,9 @@ __global__ void qbar_partial_kernel(const bf16* __restrict__ q_sem, const bf16* 
         const int rr = r + u * row_lanes;
         v[u] = make_uint4(0u, 0u, 0u, 0u);
         if (rr < r1) {
-          const int pos = rr / rep, head = hk * rep + rr % rep;
-          const size_t row = ((size_t)first_pos + pos) * Hq + head;
+          // one KV head: the rows of the tail are consecutive rows of the query arrays (no division per row)
+          const size_t row = Hkv == 1 ? (size_t)first_pos * Hq + rr
+                                      : ((size_t)first_pos + rr / rep) * Hq + hk * rep + rr % rep;
           const bf16* src = (pc < sem_pieces) ? q_sem + row * d_sem + 8 * pc : q_pos + row * d_pos + 8 * (pc - sem_pieces);
           v[u] = *reinterpret_cast<const uint4*>(src);
         }
@@ -1028,21 +1029,37 @@ int condense_launch(const CondenseLaunch& c) {
 // has grown to window + g rows, its earliest g tokens become one representative (Eq. 6-8 with the
 // summary query of the last g queries), stored right after the existing representatives, and the
 // remaining tokens move up by g - 1 rows, so the cache keeps the layout [representatives ; tokens].
+// Ring layout (n_tok != nullptr): the uncondensed tokens live in a ring of R = w + g rows (token n at row n % R), the
+// representatives from row R on; the new representative goes to row R + n_rep and nothing else moves.
 struct UpdateArgs {
   bf16* cache_sem; bf16* cache_pos; const double* qbar;
-  int32_t* n_rep; int32_t* n_rows; int32_t* anchor_out;
+  int32_t* n_rep; int32_t* n_rows; const int32_t* n_tok; int32_t* anchor_out;
   int cap, Hkv, d_sem, d_pos, g, w, sem_in_logit;
   double scale;
 };
+// Does sequence b condense a group now, and where: first row of the group, row of the new representative.
+__device__ __forceinline__ bool update_due(const UpdateArgs& a, int b, int& group_row, int& rep_row) {
+  const int nr = a.n_rep[b];
+  if (a.n_tok) {
+    const int R = a.w + a.g;
+    const long long first = (long long)nr * a.g;
+    if (nr < 0 || (long long)a.n_tok[b] - first < R || R + nr >= a.cap) return false;
+    group_row = (int)(first % R); rep_row = R + nr;
+    return true;
+  }
+  if (a.n_rows[b] - nr < a.w + a.g || nr + a.g > a.cap) return false;
+  group_row = nr; rep_row = nr;
+  return true;
+}
 
 // grid (Hkv, B), 256 threads: condense rows n_rep .. n_rep + g - 1 of one KV stream.  Same
 // arithmetic as the condense kernels: fp64 scores, arg-max on them, fp32 softmax and pooling.
 __global__ void __launch_bounds__(256) update_condense_kernel(UpdateArgs a) {
   extern __shared__ __align__(16) unsigned char smem_raw[];
   const int hk = blockIdx.x, b = blockIdx.y;
-  const int nr = a.n_rep[b], rows = a.n_rows[b];
   const int g = a.g, d_sem = a.d_sem, d_pos = a.d_pos;
-  if (rows - nr < a.w + g || nr + g > a.cap) {           // nothing to condense yet
+  int group_row, rep_row;
+  if (!update_due(a, b, group_row, rep_row)) {           // nothing to condense yet
     if (threadIdx.x == 0) a.anchor_out[b * a.Hkv + hk] = -1;
     return;
   }
@@ -1054,10 +1071,12 @@ __global__ void __launch_bounds__(256) update_condense_kernel(UpdateArgs a) {
   float* s_a = reinterpret_cast<float*>(s_s + g);
   __shared__ int s_anchor;
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5, nwarps = blockDim.x >> 5;
-  const size_t row0 = (size_t)b * a.cap + nr;
+  const size_t row0 = (size_t)b * a.cap + group_row, rowr = (size_t)b * a.cap + rep_row;
   const size_t rs_sem = (size_t)a.Hkv * d_sem, rs_pos = (size_t)a.Hkv * d_pos;
-  bf16* gs = a.cache_sem + row0 * rs_sem + (size_t)hk * d_sem;
-  bf16* gp = a.cache_pos + row0 * rs_pos + (size_t)hk * d_pos;
+  const bf16* gs = a.cache_sem + row0 * rs_sem + (size_t)hk * d_sem;
+  const bf16* gp = a.cache_pos + row0 * rs_pos + (size_t)hk * d_pos;
+  bf16* out_sem = a.cache_sem + rowr * rs_sem + (size_t)hk * d_sem;     // packed layout: the group's first row
+  bf16* out_pos = a.cache_pos + rowr * rs_pos + (size_t)hk * d_pos;
   const int cps = d_sem / 8, cpp = d_pos / 8;
   for (int x = tid; x < g * cps; x += blockDim.x) {
     const int i = x / cps, c = x % cps;
@@ -1101,10 +1120,10 @@ __global__ void __launch_bounds__(256) update_condense_kernel(UpdateArgs a) {
   for (int c = tid; c < d_sem; c += blockDim.x) {
     float acc = 0.f;
     for (int i = 0; i < g; ++i) acc = fmaf(s_a[i], __bfloat162float(t_sem[(size_t)i * d_sem + c]), acc);
-    gs[c] = __float2bfloat16_rn(acc);                    // row n_rep of this stream: the new representative
+    out_sem[c] = __float2bfloat16_rn(acc);               // the new representative
   }
   const int ia = s_anchor;
-  for (int c = tid; c < d_pos; c += blockDim.x) gp[c] = t_pos[(size_t)ia * d_pos + c];
+  for (int c = tid; c < d_pos; c += blockDim.x) out_pos[c] = t_pos[(size_t)ia * d_pos + c];
   if (tid == 0) a.anchor_out[b * a.Hkv + hk] = ia;
 }
 
@@ -1113,8 +1132,14 @@ __global__ void __launch_bounds__(256) update_condense_kernel(UpdateArgs a) {
 // ascending chunks that are loaded completely before any of their bytes is stored.
 __global__ void __launch_bounds__(1024) update_shift_kernel(UpdateArgs a) {
   const int b = blockIdx.x;
-  const int nr = a.n_rep[b], rows = a.n_rows[b];
-  if (rows - nr < a.w + a.g || nr + a.g > a.cap) return;
+  int group_row, rep_row;
+  if (!update_due(a, b, group_row, rep_row)) return;
+  const int nr = a.n_rep[b];
+  if (a.n_tok) {                                           // ring layout: only the counter changes
+    if (threadIdx.x == 0) a.n_rep[b] = nr + 1;
+    return;
+  }
+  const int rows = a.n_rows[b];
   const int n_move = rows - (nr + a.g);
   for (int pass = 0; pass < 2; ++pass) {
     const size_t row16 = (size_t)a.Hkv * (pass ? a.d_pos : a.d_sem) * sizeof(bf16) / 16;
@@ -1150,7 +1175,7 @@ size_t update_smem_bytes(const lca_params* p) {
 
 int update_launch(const lca_params* p, const void* q_tail_sem, const void* q_tail_pos, int64_t q_tail_batch_stride,
                   const float* qbar_opt, void* cache_sem, void* cache_pos, int cap, int32_t* n_rep, int32_t* n_rows,
-                  int32_t* anchor_out, void* ws, cudaStream_t stream) {
+                  const int32_t* n_tok, int32_t* anchor_out, void* ws, cudaStream_t stream) {
   const int dk = key_dim(p), B = p->batch, Hkv = p->n_kv_heads;
   const int sem_in_logit = p->variant == LCA_VARIANT_MLA;
   double* qbar = reinterpret_cast<double*>(ws);
@@ -1178,15 +1203,60 @@ int update_launch(const lca_params* p, const void* q_tail_sem, const void* q_tai
   }
   UpdateArgs a;
   a.cache_sem = (bf16*)cache_sem; a.cache_pos = (bf16*)cache_pos; a.qbar = qbar;
-  a.n_rep = n_rep; a.n_rows = n_rows; a.anchor_out = anchor_out;
+  a.n_rep = n_rep; a.n_rows = n_rows; a.n_tok = n_tok; a.anchor_out = anchor_out;
   a.cap = cap; a.Hkv = Hkv; a.d_sem = p->d_sem; a.d_pos = p->d_pos; a.g = p->group_size; a.w = p->window;
   a.sem_in_logit = sem_in_logit; a.scale = (double)p->softmax_scale;
   const size_t smem = update_smem_bytes(p);
   if (cudaFuncSetAttribute(update_condense_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) != cudaSuccess)
     return LCA_ERR_CUDA;
   update_condense_kernel<<<dim3(Hkv, B), 256, smem, stream>>>(a);
-  update_shift_kernel<<<dim3(B), 1024, 0, stream>>>(a);
+  update_shift_kernel<<<dim3(B), n_tok ? 32 : 1024, 0, stream>>>(a);
   note_launch(2);
+  return cudaGetLastError() == cudaSuccess ? LCA_OK : LCA_ERR_CUDA;
+}
+
+// Packed cache [representatives ; tokens in order] -> ring layout (see UpdateArgs): the step between the prefill
+// condensation and decoding on the ring.  grid (chunks, B, 2): z = 0 the semantic part, 1 the positional part.
+struct RingCopyArgs {
+  const uint4* src[2]; uint4* dst[2]; size_t row16[2];      // 16-byte pieces per row
+  const int32_t* packed_rows; const int32_t* n_rep; int32_t* n_tok_out;
+  int packed_cap, ring_cap, R, g;
+};
+__global__ void __launch_bounds__(256) ring_from_packed_kernel(RingCopyArgs a) {
+  const int b = blockIdx.y, z = blockIdx.z;
+  const int rows = min(max(a.packed_rows[b], 0), a.packed_cap);
+  const int nr = min(max(a.n_rep[b], 0), rows);
+  const int n_tok_rows = min(rows - nr, a.R);               // tokens beyond the ring's size cannot be placed
+  const int n_rep_rows = min(nr, max(a.ring_cap - a.R, 0));
+  const long long first = (long long)nr * a.g;
+  const size_t row16 = a.row16[z];
+  const uint4* src = a.src[z] + (size_t)b * a.packed_cap * row16;
+  uint4* dst = a.dst[z] + (size_t)b * a.ring_cap * row16;
+  const size_t n16 = (size_t)(n_rep_rows + n_tok_rows) * row16;
+  for (size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x; i < n16; i += (size_t)gridDim.x * blockDim.x) {
+    const int r = (int)(i / row16);
+    const size_t piece = i % row16;
+    int srow, drow;
+    if (r < n_rep_rows) { srow = r; drow = a.R + r; }
+    else { const int t = r - n_rep_rows; srow = nr + t; drow = (int)((first + t) % a.R); }
+    dst[(size_t)drow * row16 + piece] = src[(size_t)srow * row16 + piece];
+  }
+  if (z == 0 && blockIdx.x == 0 && threadIdx.x == 0) a.n_tok_out[b] = (int32_t)(first + (rows - nr));
+}
+
+int ring_from_packed_launch(const lca_params* p, const void* packed_sem, const void* packed_pos, const int32_t* packed_rows,
+                            const int32_t* n_rep, int packed_cap, void* ring_sem, void* ring_pos, int ring_cap,
+                            int32_t* n_tok_out, cudaStream_t stream) {
+  RingCopyArgs a;
+  a.src[0] = (const uint4*)packed_sem; a.src[1] = (const uint4*)packed_pos;
+  a.dst[0] = (uint4*)ring_sem; a.dst[1] = (uint4*)ring_pos;
+  a.row16[0] = (size_t)p->n_kv_heads * p->d_sem * sizeof(bf16) / 16;
+  a.row16[1] = (size_t)p->n_kv_heads * p->d_pos * sizeof(bf16) / 16;
+  a.packed_rows = packed_rows; a.n_rep = n_rep; a.n_tok_out = n_tok_out;
+  a.packed_cap = packed_cap; a.ring_cap = ring_cap; a.R = p->window + p->group_size; a.g = p->group_size;
+  const unsigned chunks = p->batch >= 148 ? 4 : (unsigned)((148 * 4 + p->batch - 1) / p->batch);
+  ring_from_packed_kernel<<<dim3(chunks, p->batch, 2), 256, 0, stream>>>(a);
+  note_launch();
   return cudaGetLastError() == cudaSuccess ? LCA_OK : LCA_ERR_CUDA;
 }
 

@@ -332,7 +332,82 @@ int lca_decode_update(const lca_params* p, const void* q_tail_sem, const void* q
   if (ws_bytes < update_workspace_bytes(p)) return LCA_ERR_WORKSPACE_TOO_SMALL;
   if (update_smem_bytes(p) > 227u * 1024u) return LCA_ERR_UNSUPPORTED_SHAPE;
   return update_launch(p, q_tail_sem, q_tail_pos, q_tail_batch_stride, qbar_opt, cache_sem, cache_pos,
-                       cache_row_capacity, n_rep, cache_rows, anchor_out, ws, (cudaStream_t)stream);
+                       cache_row_capacity, n_rep, cache_rows, nullptr, anchor_out, ws, (cudaStream_t)stream);
+}
+
+// The ring layout needs whole groups to leave the ring: window a multiple of group_size.
+static int check_ring(const lca_params* p, int32_t ring_row_capacity) {
+  if (p->group_size <= 0 || p->window < 0 || p->window % p->group_size != 0) return LCA_ERR_INVALID_ARG;
+  if ((int64_t)p->window + p->group_size > (int64_t)ring_row_capacity) return LCA_ERR_INVALID_ARG;
+  return LCA_OK;
+}
+
+int lca_ring_from_packed(const lca_params* p, const void* packed_sem, const void* packed_pos,
+                         const int32_t* packed_rows, const int32_t* n_rep, int32_t packed_row_capacity,
+                         void* ring_sem, void* ring_pos, int32_t ring_row_capacity, int32_t* n_tok_out,
+                         void* stream) {
+  int st = check_params(p, false);
+  if (st != LCA_OK) return st;
+  if (!packed_sem || !packed_pos || !packed_rows || !n_rep || !ring_sem || !ring_pos || !n_tok_out ||
+      packed_row_capacity <= 0)
+    return LCA_ERR_INVALID_ARG;
+  st = check_ring(p, ring_row_capacity);
+  if (st != LCA_OK) return st;
+  if (!aligned16(packed_sem) || !aligned16(packed_pos) || !aligned16(ring_sem) || !aligned16(ring_pos))
+    return LCA_ERR_MISALIGNED;
+  if (((size_t)p->n_kv_heads * p->d_sem * 2) % 16 || ((size_t)p->n_kv_heads * p->d_pos * 2) % 16) return LCA_ERR_UNSUPPORTED_SHAPE;
+  return ring_from_packed_launch(p, packed_sem, packed_pos, packed_rows, n_rep, packed_row_capacity, ring_sem, ring_pos,
+                                 ring_row_capacity, n_tok_out, (cudaStream_t)stream);
+}
+
+int lca_decode_attention_ring(const lca_params* p, const void* q_sem, const void* q_pos,
+                              const void* ring_sem, const void* ring_pos, const int32_t* n_rep,
+                              const int32_t* n_tok, int32_t ring_row_capacity, void* out, float* lse_opt,
+                              void* ws, size_t ws_bytes, void* stream) {
+  int st = check_params(p, false);
+  if (st != LCA_OK) return st;
+  if (!q_pos || !ring_sem || !ring_pos || !n_rep || !n_tok || !out) return LCA_ERR_INVALID_ARG;
+  if (p->variant == LCA_VARIANT_MLA && !q_sem) return LCA_ERR_INVALID_ARG;
+  st = check_ring(p, ring_row_capacity);
+  if (st != LCA_OK) return st;
+  if (!aligned16(q_pos) || !aligned16(ring_sem) || !aligned16(ring_pos) || !aligned16(out) || (q_sem && !aligned16(q_sem)))
+    return LCA_ERR_MISALIGNED;
+  if (!simt_shape_ok(p)) return LCA_ERR_UNSUPPORTED_SHAPE;
+  AttnProblem a = {};
+  a.variant = p->variant; a.batch = p->batch; a.q_len = 1; a.n_q_heads = p->n_q_heads;
+  a.n_kv_heads = p->n_kv_heads; a.d_sem = p->d_sem; a.d_pos = p->d_pos; a.decode = 1;
+  a.seq_len = 0; a.group_size = p->group_size; a.window = p->window;
+  a.cache_rows = nullptr; a.cache_row_capacity = ring_row_capacity; a.n_rep_bias = 0;
+  a.ring_n_rep = n_rep; a.ring_n_tok = n_tok;
+  a.softmax_scale = p->softmax_scale; a.rep_logit_bias = p->rep_logit_bias;
+  a.q_sem = q_sem; a.q_pos = q_pos; a.kv_sem = nullptr; a.kv_pos = nullptr;
+  a.cache_sem = ring_sem; a.cache_pos = ring_pos; a.out = out; a.lse = lse_opt;
+  a.ws = ws; a.ws_bytes = ws_bytes; a.stream = (cudaStream_t)stream;
+  return run_attention(a);
+}
+
+int lca_decode_update_ring(const lca_params* p, const void* q_tail_sem, const void* q_tail_pos,
+                           int64_t q_tail_batch_stride, const float* qbar_opt, void* ring_sem,
+                           void* ring_pos, int32_t ring_row_capacity, int32_t* n_rep, const int32_t* n_tok,
+                           int32_t* anchor_out, void* ws, size_t ws_bytes, void* stream) {
+  int st = check_params(p, false);
+  if (st != LCA_OK) return st;
+  if (p->n_summary_q < 0) return LCA_ERR_INVALID_ARG;
+  if (!ring_sem || !ring_pos || !n_rep || !n_tok || !anchor_out) return LCA_ERR_INVALID_ARG;
+  st = check_ring(p, ring_row_capacity);
+  if (st != LCA_OK) return st;
+  if (!qbar_opt) {
+    if (!q_tail_pos || (p->variant == LCA_VARIANT_MLA && !q_tail_sem)) return LCA_ERR_INVALID_ARG;
+    const int n = p->n_summary_q > 0 ? p->n_summary_q : p->group_size;
+    if (q_tail_batch_stride < n) return LCA_ERR_INVALID_ARG;
+    if (!aligned16(q_tail_pos) || (q_tail_sem && !aligned16(q_tail_sem))) return LCA_ERR_MISALIGNED;
+  }
+  if (!aligned16(ring_sem) || !aligned16(ring_pos)) return LCA_ERR_MISALIGNED;
+  if (!ws || !aligned16(ws)) return LCA_ERR_INVALID_ARG;
+  if (ws_bytes < update_workspace_bytes(p)) return LCA_ERR_WORKSPACE_TOO_SMALL;
+  if (update_smem_bytes(p) > 227u * 1024u) return LCA_ERR_UNSUPPORTED_SHAPE;
+  return update_launch(p, q_tail_sem, q_tail_pos, q_tail_batch_stride, qbar_opt, ring_sem, ring_pos,
+                       ring_row_capacity, n_rep, nullptr, n_tok, anchor_out, ws, (cudaStream_t)stream);
 }
 
 int lca_latent_to_value(const void* attn_latent, const void* w_uv, void* out_v, int64_t n_tokens,

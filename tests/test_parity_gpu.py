@@ -748,3 +748,158 @@ def test_random_shapes_match_oracle(B):
         np.testing.assert_allclose(lse[0].cpu().numpy(), ref["lse"], atol=2e-3, rtol=1e-4, err_msg=what)
         # decoding the last token against the final cache is the last prefill row (Sec. 4.3)
         Hh.check_outputs(dout[0], ref["out"][-1], what + " decode", vmax=ref["vmax"])
+
+
+# ------------------------------------------------------------------ ring layout of the decode cache
+def _ring_states(g, w, cap, specs, d_sem, d_pos, gen, heads=None):
+    """Random packed caches with (n_rep, uncondensed tokens) per sequence -> (packed sem, pos [B, cap_packed, ...],
+    packed_rows, n_rep).  heads = None: one KV stream ([.., 1, d]); else [.., heads, d]."""
+    hk = 1 if heads is None else heads
+    cap_packed = max(r + c for r, c in specs) + 1
+    sem = torch.zeros((len(specs), cap_packed, hk, d_sem), dtype=torch.bfloat16)
+    pos = torch.zeros((len(specs), cap_packed, hk, d_pos), dtype=torch.bfloat16)
+    for b, (r, c) in enumerate(specs):
+        sem[b, :r + c] = torch.randn((r + c, hk, d_sem), generator=gen).bfloat16()
+        pos[b, :r + c] = torch.randn((r + c, hk, d_pos), generator=gen).bfloat16()
+    return sem, pos, [r + c for r, c in specs], [r for r, _ in specs]
+
+
+@pytest.mark.parametrize("impl,bias", [(0, 0.0), (0, math.log(16.0)), (1, 0.3)])
+def test_ring_cache_streaming_matches_oracle_over_many_decode_steps(B, impl, bias):
+    # Ring of R = w + g = 192 rows (one and a half key tiles, so the representatives start in the middle of a tile).
+    # Three sequences in different phases, one of them so short that its ring has not wrapped; more than two trips
+    # round the ring.  Every step: append the token at its ring row, decode (device against the oracle on the rows
+    # that take part), update (device against the oracle: only the new representative's row may change).
+    cfg = I.scaled(I.CONFIGS["mla_decode"], batch=3, seq_len=0, n_q_heads=16, group_size=16, window=176)
+    g, w, H, Bsz = cfg.group_size, cfg.window, cfg.n_q_heads, 3
+    R = w + g
+    steps = 2 * R + g + 7
+    cap = R + 8 + steps // g + 4
+    gen = torch.Generator().manual_seed(29)
+    specs = [(3, w + g - 1), (5, w + 3), (0, 9)]                   # (representatives, uncondensed tokens)
+    psem, ppos, prow, prep = _ring_states(g, w, cap, specs, 512, 64, gen)
+    p = B.params_from_config(cfg, batch=Bsz, rep_logit_bias=bias)
+    d_rep = torch.tensor(prep, dtype=torch.int32, device=DEV)
+    d_sem, d_pos, d_tok = B.ring_from_packed(p, psem.to(DEV), ppos.to(DEV), torch.tensor(prow, dtype=torch.int32, device=DEV),
+                                             d_rep, cap)
+    o_sem, o_pos, o_tok, o_rep = [], [], [], list(prep)
+    for b in range(Bsz):
+        s, q, n = O.ring_from_packed(Hh.bits(psem[b, :, 0]), Hh.bits(ppos[b, :, 0]), prep[b], prow[b], g, w, cap)
+        o_sem.append(s); o_pos.append(q); o_tok.append(n)
+        assert np.array_equal(Hh.bits(d_sem[b, :, 0]), s) and np.array_equal(Hh.bits(d_pos[b, :, 0]), q)
+    assert d_tok.cpu().tolist() == o_tok
+    scale = Hh.f32(cfg.softmax_scale)
+    prev = B.lca_set_attention_impl(impl)
+    n_updates = 0
+    try:
+        for step in range(steps):
+            new_sem = torch.randn((Bsz, 512), generator=gen).bfloat16()
+            new_pos = torch.randn((Bsz, 64), generator=gen).bfloat16()
+            for b in range(Bsz):                       # the caller writes the new token at its ring row and counts it
+                d_sem[b, o_tok[b] % R, 0] = new_sem[b].to(DEV)
+                d_pos[b, o_tok[b] % R, 0] = new_pos[b].to(DEV)
+                o_sem[b][o_tok[b] % R] = Hh.bits(new_sem[b])
+                o_pos[b][o_tok[b] % R] = Hh.bits(new_pos[b])
+                o_tok[b] += 1
+            d_tok += 1
+            if step % 3 == 0 or step >= steps - 40:
+                q_sem = torch.randn((Bsz, H, 512), generator=gen).bfloat16()
+                q_pos = torch.randn((Bsz, H, 64), generator=gen).bfloat16()
+                out, lse = B.decode_attention_ring(p, q_sem.to(DEV), q_pos.to(DEV), d_sem, d_pos, d_rep, d_tok, want_lse=True)
+                torch.cuda.synchronize()
+                assert B.lca_last_device_status() == 0
+                for b in range(Bsz):
+                    cs, cp, n_rows = O.ring_to_packed(o_sem[b], o_pos[b], o_rep[b], o_tok[b], g, w)
+                    ro, rl = O.mla_decode(O.torch_bf16_to_f64(q_sem[b]), O.torch_bf16_to_f64(q_pos[b]), O.bits_to_f64(cs),
+                                          O.bits_to_f64(cp), o_rep[b], scale, bias)
+                    Hh.check_outputs(out[b], ro, f"ring decode step {step} seq {b}")
+                    np.testing.assert_allclose(lse[b].cpu().numpy(), rl, atol=2e-3, rtol=1e-4)
+            q_tail_sem = torch.randn((Bsz, g, H, 512), generator=gen).bfloat16()
+            q_tail_pos = torch.randn((Bsz, g, H, 64), generator=gen).bfloat16()
+            anchor = B.decode_update_ring(p, q_tail_sem.to(DEV), q_tail_pos.to(DEV), d_sem, d_pos, d_rep, d_tok)
+            torch.cuda.synchronize()
+            for b in range(Bsz):
+                qbar = O.mla_summary_query(O.torch_bf16_to_f64(q_tail_sem[b]), O.torch_bf16_to_f64(q_tail_pos[b]))
+                s2, p2, nr, ia = O.mla_decode_update_ring(o_sem[b], o_pos[b], o_rep[b], o_tok[b], qbar, g, w, scale)
+                assert int(anchor[b, 0]) == ia
+                if ia >= 0:
+                    n_updates += 1
+                    got_sem, got_pos = Hh.bits(d_sem[b, :, 0]), Hh.bits(d_pos[b, :, 0])
+                    row = R + o_rep[b]
+                    assert np.array_equal(got_pos, p2)                                   # anchor row: a bit copy; nothing else moved
+                    assert (Hh.bf16_ulp_distance(got_sem[row], s2[row]) <= 1).all()      # representative: fp32 pooling
+                    s2[row] = got_sem[row]                                               # carry the device's rounding forward
+                    assert np.array_equal(got_sem, s2)
+                o_sem[b], o_pos[b], o_rep[b] = s2, p2, nr
+            assert d_rep.cpu().tolist() == o_rep and d_tok.cpu().tolist() == o_tok
+    finally:
+        B.lca_set_attention_impl(prev)
+    assert n_updates >= 3 * (steps // g) - 12
+
+
+def test_ring_decode_without_key_range_split_and_full_representative_region(B):
+    # 40 sequences x 16 heads: more units than half the CTA pairs, so every unit is one work item (no partial results).
+    # States: ring exactly full, one token after an update (g - 1 stale rows), ring not wrapped, empty sequence.
+    cfg = I.scaled(I.CONFIGS["mla_decode"], batch=40, seq_len=0, n_q_heads=16, group_size=32, window=224)
+    g, w, H, Bsz = cfg.group_size, cfg.window, cfg.n_q_heads, 40
+    R = w + g
+    gen = torch.Generator().manual_seed(31)
+    specs = []
+    for b in range(Bsz):
+        kind = b % 5
+        specs.append([(b % 7 + 1, R), (b % 9 + 1, w + 1), (0, 1 + (b * 13) % (R - 1)), (0, 0), (b % 11 + 2, w + g // 2)][kind])
+    cap = R + 16
+    psem, ppos, prow, prep = _ring_states(g, w, cap, specs, 512, 64, gen)
+    p = B.params_from_config(cfg, batch=Bsz, rep_logit_bias=0.5)
+    d_rep = torch.tensor(prep, dtype=torch.int32, device=DEV)
+    d_sem, d_pos, d_tok = B.ring_from_packed(p, psem.to(DEV), ppos.to(DEV), torch.tensor(prow, dtype=torch.int32, device=DEV),
+                                             d_rep, cap)
+    q_sem = torch.randn((Bsz, H, 512), generator=gen).bfloat16()
+    q_pos = torch.randn((Bsz, H, 64), generator=gen).bfloat16()
+    out, lse = B.decode_attention_ring(p, q_sem.to(DEV), q_pos.to(DEV), d_sem, d_pos, d_rep, d_tok, want_lse=True)
+    torch.cuda.synchronize()
+    assert B.lca_last_device_status() == 0
+    tok = d_tok.cpu().tolist()
+    for b in range(Bsz):
+        r, c = specs[b]
+        assert tok[b] == r * g + c
+        if r + c == 0:
+            assert float(out[b].abs().max()) == 0.0 and bool(torch.isinf(lse[b]).all())
+            continue
+        cs, cp, n_rows = O.ring_to_packed(Hh.bits(d_sem[b, :, 0]), Hh.bits(d_pos[b, :, 0]), r, tok[b], g, w)
+        assert n_rows == r + c
+        assert np.array_equal(cs, Hh.bits(psem[b, :r + c, 0])) and np.array_equal(cp, Hh.bits(ppos[b, :r + c, 0]))
+        ro, rl = O.mla_decode(O.torch_bf16_to_f64(q_sem[b]), O.torch_bf16_to_f64(q_pos[b]), O.bits_to_f64(cs), O.bits_to_f64(cp),
+                              r, Hh.f32(cfg.softmax_scale), 0.5)
+        Hh.check_outputs(out[b], ro, f"ring decode seq {b}")
+        np.testing.assert_allclose(lse[b].cpu().numpy(), rl, atol=2e-3, rtol=1e-4)
+
+
+def test_gqa_ring_decode_matches_oracle(B):
+    # GQA cache in the ring layout (one ring per KV head, same rows): the one-tile tensor-core kernel and the scalar kernel
+    cfg = I.scaled(I.CONFIGS["gqa_64k"], batch=4, seq_len=0, n_q_heads=32, n_kv_heads=8, group_size=64, window=192)
+    g, w, Hq, Hkv, d = cfg.group_size, cfg.window, cfg.n_q_heads, cfg.n_kv_heads, cfg.d_sem
+    R = w + g
+    gen = torch.Generator().manual_seed(37)
+    specs = [(6, R), (2, w + 5), (0, 77), (9, w + g - 1)]
+    cap = R + 12
+    pv, pk, prow, prep = _ring_states(g, w, cap, specs, d, d, gen, heads=Hkv)
+    p = B.params_from_config(cfg, batch=4, rep_logit_bias=0.25)
+    d_rep = torch.tensor(prep, dtype=torch.int32, device=DEV)
+    ring_v, ring_k, d_tok = B.ring_from_packed(p, pv.to(DEV), pk.to(DEV), torch.tensor(prow, dtype=torch.int32, device=DEV), d_rep, cap)
+    q = torch.randn((4, Hq, d), generator=gen).bfloat16()
+    refs = []
+    for b, (r, c) in enumerate(specs):
+        refs.append(O.gqa_decode(O.torch_bf16_to_f64(q[b]), O.bits_to_f64(Hh.bits(pk[b, :r + c])), O.bits_to_f64(Hh.bits(pv[b, :r + c])),
+                                 r, Hh.f32(cfg.softmax_scale), 0.25))
+    for impl in (0, 1):
+        prev = B.lca_set_attention_impl(impl)
+        try:
+            out, lse = B.decode_attention_ring(p, None, q.to(DEV), ring_v, ring_k, d_rep, d_tok, want_lse=True)
+        finally:
+            B.lca_set_attention_impl(prev)
+        torch.cuda.synchronize()
+        assert B.lca_last_device_status() == 0
+        for b in range(4):
+            Hh.check_outputs(out[b], refs[b][0], f"gqa ring decode seq {b} impl {impl}")
+            np.testing.assert_allclose(lse[b].cpu().numpy(), refs[b][1], atol=2e-3, rtol=1e-4)
