@@ -462,6 +462,31 @@ def time_cuda(fn, warmup=3, iters=5):
     return e0.elapsed_time(e1) / iters
 
 
+def time_cuda_graph(fn, n=10):
+    """Device time per call of a short sequence of launches: n calls captured into one CUDA graph, replayed twice
+    (eager calls of a few microseconds each measure the host's launch rate instead)."""
+    side = torch.cuda.Stream()
+    side.wait_stream(torch.cuda.current_stream())
+    with torch.cuda.stream(side):
+        fn()
+        torch.cuda.synchronize()
+        graph = torch.cuda.CUDAGraph()
+        with torch.cuda.graph(graph, stream=side):
+            for _ in range(n):
+                fn()
+        torch.cuda.synchronize()
+        graph.replay()
+        torch.cuda.synchronize()
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record(side)
+        graph.replay()
+        graph.replay()
+        e1.record(side)
+        torch.cuda.synchronize()
+    torch.cuda.current_stream().wait_stream(side)
+    return e0.elapsed_time(e1) / (2 * n)
+
+
 def measure_decode_config(B, dev, batch, peaks, warmup=3, iters=5, parity=None):
     """Config 4: lca_condense over `batch` contexts of 65536 tokens (the HBM-bound figure), then
     lca_decode_attention of one new query per sequence over the condensed cache."""
@@ -548,9 +573,29 @@ def measure_decode_config(B, dev, batch, peaks, warmup=3, iters=5, parity=None):
         out_r = torch.empty_like(out)
         t_ring_dec = time_cuda(lambda: B.decode_attention_ring(p, q_new_sem, q_new_pos, rsem, rpos, n_rep_t, n_tok_t, out=out_r, ws=wsd),
                                warmup, iters)
+        # one call per decode step with a running summary query: a step in which no sequence is due, and one in which all are
+        qsum = torch.zeros((batch, 1, cfg.d_sem + cfg.d_pos), dtype=torch.float64, device=dev)
+        qcount = torch.zeros((batch,), dtype=torch.int32, device=dev)
+        anc = torch.empty((batch, 1), dtype=torch.int32, device=dev)
+        n_rep_idle = torch.full((batch,), m, dtype=torch.int32, device=dev)
+        n_tok_idle = torch.full((batch,), m * g + R - 1, dtype=torch.int32, device=dev)
+        t_step_idle = time_cuda_graph(lambda: B.decode_step_update_ring(p, q_new_sem, q_new_pos, qsum, qcount, rsem, rpos, n_rep_idle,
+                                                                        n_tok_idle, ws=wsu, anchor=anc))
+        n_rep_t = torch.full((batch,), m, dtype=torch.int32, device=dev)
+
+        def due_step():
+            n_rep_t.fill_(m)                                       # every sequence is due again (a 64-element fill)
+            B.decode_step_update_ring(p, q_new_sem, q_new_pos, qsum, qcount, rsem, rpos, n_rep_t, n_tok_full, ws=wsu, anchor=anc)
+        t_step_due = time_cuda_graph(due_step)
+        assert int(n_rep_t.min()) == m + 1 and int(qcount.max()) == 0 and int(anc.min()) >= 0
         upd["ring_layout"] = dict(us_per_update_all_sequences=ring["tails"], us_with_ready_summary_query=ring["ready_summary_query"],
-                                  amortised_us_per_token=ring["ready_summary_query"] / g, decode_us=t_ring_dec * 1e3,
-                                  note="lca_decode_update_ring / lca_decode_attention_ring: one new row per sequence, no row moves")
+                                  amortised_us_per_token_from_tails=ring["tails"] / g,
+                                  decode_us=t_ring_dec * 1e3, step_update_us_nobody_due=t_step_idle * 1e3,
+                                  step_update_us_all_due=t_step_due * 1e3,
+                                  step_update_amortised_us_per_token=(t_step_idle * (g - 1) + t_step_due) * 1e3 / g,
+                                  note="lca_decode_update_ring / lca_decode_attention_ring: one new row per sequence, no row moves; "
+                                       "step_update = lca_decode_step_update_ring, called at every decode step (running summary query), device time "
+                                       "from a CUDA graph of ten calls; its amortised figure = (g - 1) steps with nobody due + one with all due")
         del rsem, rpos
     except Exception as ex:
         upd = dict(error=str(ex)[:200])

@@ -270,6 +270,25 @@ int lca_decode_update_ring(const lca_params* p, const void* q_tail_sem, const vo
                            void* ring_pos, int32_t ring_row_capacity, int32_t* n_rep, const int32_t* n_tok,
                            int32_t* anchor_out, void* ws, size_t ws_bytes, void* stream);
 
+/* The update on the ring layout with a running summary query, called once per decode step after the
+ * step's token has been written and counted (Sec. 4.3: "the average query of the last g tokens"):
+ *   1. qsum[b, hk, :] += sum over the query heads of KV head hk of this step's [q_sem | q_pos] (fp64;
+ *      MLA: dk = d_sem + d_pos, GQA: dk = d_pos), qcount[b] += 1;
+ *   2. every sequence that is due (window + group_size uncondensed tokens) is condensed exactly as by
+ *      lca_decode_update_ring with the summary query qsum / (qcount * heads per KV head), i.e. the mean of
+ *      the queries of all steps since its previous update (the last group_size queries when this is
+ *      called at every step), and its qsum and qcount are cleared.
+ * No query tail is re-read: a step costs the bytes of that step's queries.
+ *   q_sem [B, H, d_sem] (NULL for GQA), q_pos [B, H, d_pos]: this step's queries
+ *   qsum [B, n_kv_heads, dk] fp64, qcount [B] int32 (device, in / out): zero them when a sequence
+ *        starts; to include queries of the prefill, call this with them before decoding starts (a
+ *        sequence that is not due only accumulates)
+ *   the other arguments as for lca_decode_update_ring; p->n_summary_q must be 0 or group_size. */
+int lca_decode_step_update_ring(const lca_params* p, const void* q_sem, const void* q_pos, double* qsum,
+                                int32_t* qcount, void* ring_sem, void* ring_pos, int32_t ring_row_capacity,
+                                int32_t* n_rep, const int32_t* n_tok, int32_t* anchor_out, void* ws,
+                                size_t ws_bytes, void* stream);
+
 /* Value up-projection of the latent attention output (Alg. 1: v = c W^UV; Sec. 4.3: in the absorbed
  * form the attention result lives in the latent space and W^UV is applied to it once per query and
  * head):   out_v[t, h, :] = attn_latent[t, h, :] . W^UV[h]

@@ -78,6 +78,8 @@ def _load() -> C.CDLL:
     lib.lca_decode_attention_ring.argtypes = [P, vp, vp, vp, vp, vp, vp, i32, vp, vp, vp, sz, vp]
     lib.lca_decode_update_ring.restype = C.c_int
     lib.lca_decode_update_ring.argtypes = [P, vp, vp, i64, vp, vp, vp, i32, vp, vp, vp, vp, sz, vp]
+    lib.lca_decode_step_update_ring.restype = C.c_int
+    lib.lca_decode_step_update_ring.argtypes = [P, vp, vp, vp, vp, vp, vp, i32, vp, vp, vp, vp, sz, vp]
     pi32, pi64 = C.POINTER(i32), C.POINTER(i64)
     lib.lca_varlen_layout.restype = C.c_int
     lib.lca_varlen_layout.argtypes = [P, pi32, pi64, pi64, pi64]
@@ -215,6 +217,14 @@ def lca_decode_update_ring(params, q_tail_sem, q_tail_pos, q_tail_batch_stride, 
     return int(_lib.lca_decode_update_ring(C.byref(params), _ptr(q_tail_sem), _ptr(q_tail_pos), int(q_tail_batch_stride),
                                            _ptr(qbar_opt), _ptr(ring_sem), _ptr(ring_pos), int(ring_row_capacity),
                                            _ptr(n_rep), _ptr(n_tok), _ptr(anchor_out), _ptr(ws), wsb, _stream(stream)))
+
+
+def lca_decode_step_update_ring(params, q_sem, q_pos, qsum, qcount, ring_sem, ring_pos, ring_row_capacity, n_rep, n_tok,
+                                anchor_out, ws, ws_bytes=None, stream=None) -> int:
+    wsb = _nbytes(ws) if ws_bytes is None else int(ws_bytes)
+    return int(_lib.lca_decode_step_update_ring(C.byref(params), _ptr(q_sem), _ptr(q_pos), _ptr(qsum), _ptr(qcount),
+                                                _ptr(ring_sem), _ptr(ring_pos), int(ring_row_capacity), _ptr(n_rep),
+                                                _ptr(n_tok), _ptr(anchor_out), _ptr(ws), wsb, _stream(stream)))
 
 
 def _lens(seq_lens):
@@ -443,4 +453,18 @@ def decode_update_ring(params: LcaParams, q_tail_sem, q_tail_pos, ring_sem, ring
     st = lca_decode_update_ring(params, q_tail_sem, q_tail_pos, n, qbar, ring_sem, ring_pos, ring_sem.shape[1], n_rep,
                                 n_tok, anchor, ws, stream=stream)
     _check(st, "lca_decode_update_ring")
+    return anchor
+
+
+def decode_step_update_ring(params: LcaParams, q_sem, q_pos, qsum, qcount, ring_sem, ring_pos, n_rep, n_tok, ws=None,
+                            anchor=None, stream=None):
+    """Run lca_decode_step_update_ring in place (qsum [B, Hkv, dk] float64, qcount [B] int32); returns anchor offsets."""
+    dev = ring_sem.device
+    if anchor is None:
+        anchor = torch.empty((params.batch, params.n_kv_heads), dtype=torch.int32, device=dev)
+    if ws is None:
+        ws = workspace(params, LCA_WS_UPDATE, dev)
+    st = lca_decode_step_update_ring(params, q_sem, q_pos, qsum, qcount, ring_sem, ring_pos, ring_sem.shape[1], n_rep, n_tok,
+                                     anchor, ws, stream=stream)
+    _check(st, "lca_decode_step_update_ring")
     return anchor

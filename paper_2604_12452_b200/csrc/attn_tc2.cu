@@ -753,7 +753,7 @@ __global__ void __launch_bounds__(128) decode_combine_kernel(const Tc2Params p, 
   int total = 0;
   for (int u0 = 0; u0 < n_units; u0 += 32) total += __reduce_add_sync(0xffffffffu, u0 + lane < n_units ? unit_tiles(p, u0 + lane) : 0);
   const int q = total > 0 ? (total + n_pairs - 1) / n_pairs : 1;
-  int off = 0, slot_base = 0, n = 0, my_slot = 0, n_seg = 0;
+  int off = 0, slot_base = 0, my_slot = 0, n_seg = 0;
   for (int u0 = 0; u0 <= u; u0 += 32) {
     const int nn = u0 + lane < n_units ? unit_tiles(p, u0 + lane) : 0;
     int incl = nn;
@@ -765,7 +765,6 @@ __global__ void __launch_bounds__(128) decode_combine_kernel(const Tc2Params p, 
     for (int o = 1; o < 32; o <<= 1) { const int t = __shfl_up_sync(0xffffffffu, rincl, o); if (lane >= o) rincl += t; }
     if (u < u0 + 32) {
       const int src = u - u0;
-      n = __shfl_sync(0xffffffffu, nn, src);
       n_seg = __shfl_sync(0xffffffffu, r, src);
       my_slot = slot_base + __shfl_sync(0xffffffffu, rincl - r, src);
     }
@@ -795,7 +794,6 @@ __global__ void __launch_bounds__(128) decode_combine_kernel(const Tc2Params p, 
   w.x = pack_bf16x2(acc.x * inv, acc.y * inv); w.y = pack_bf16x2(acc.z * inv, acc.w * inv);
   *reinterpret_cast<uint2*>(p.out + orow * 512 + 4 * c4) = w;
   if (p.lse && c4 == 0) p.lse[orow] = Lsum > 0.f ? (M + log2f(Lsum)) * 0.6931471805599453f : -INFINITY;
-  (void)n;
 }
 
 // ----------------------------------------------------------------------------------- host

@@ -1036,6 +1036,7 @@ struct UpdateArgs {
   int32_t* n_rep; int32_t* n_rows; const int32_t* n_tok; int32_t* anchor_out;
   int cap, Hkv, d_sem, d_pos, g, w, sem_in_logit;
   double scale;
+  int32_t* qcount;             // streaming summary query: positions summed so far per sequence (null otherwise)
 };
 // Does sequence b condense a group now, and where: first row of the group, row of the new representative.
 __device__ __forceinline__ bool update_due(const UpdateArgs& a, int b, int& group_row, int& rep_row) {
@@ -1054,8 +1055,7 @@ __device__ __forceinline__ bool update_due(const UpdateArgs& a, int b, int& grou
 
 // grid (Hkv, B), 256 threads: condense rows n_rep .. n_rep + g - 1 of one KV stream.  Same
 // arithmetic as the condense kernels: fp64 scores, arg-max on them, fp32 softmax and pooling.
-__global__ void __launch_bounds__(256) update_condense_kernel(UpdateArgs a) {
-  extern __shared__ __align__(16) unsigned char smem_raw[];
+__device__ __forceinline__ void update_condense_body(const UpdateArgs& a, unsigned char* smem_raw) {
   const int hk = blockIdx.x, b = blockIdx.y;
   const int g = a.g, d_sem = a.d_sem, d_pos = a.d_pos;
   int group_row, rep_row;
@@ -1126,6 +1126,10 @@ __global__ void __launch_bounds__(256) update_condense_kernel(UpdateArgs a) {
   for (int c = tid; c < d_pos; c += blockDim.x) out_pos[c] = t_pos[(size_t)ia * d_pos + c];
   if (tid == 0) a.anchor_out[b * a.Hkv + hk] = ia;
 }
+__global__ void __launch_bounds__(256) update_condense_kernel(UpdateArgs a) {
+  extern __shared__ __align__(16) unsigned char smem_raw[];
+  update_condense_body(a, smem_raw);
+}
 
 // grid (B), 1024 threads: move rows [n_rep + g, n_rows) up to [n_rep + 1, ...) and update the
 // counters.  Source and destination overlap (destination below source), so the rows are moved in
@@ -1135,8 +1139,11 @@ __global__ void __launch_bounds__(1024) update_shift_kernel(UpdateArgs a) {
   int group_row, rep_row;
   if (!update_due(a, b, group_row, rep_row)) return;
   const int nr = a.n_rep[b];
-  if (a.n_tok) {                                           // ring layout: only the counter changes
-    if (threadIdx.x == 0) a.n_rep[b] = nr + 1;
+  if (a.n_tok) {                                           // ring layout: only the counters change
+    if (threadIdx.x == 0) {
+      a.n_rep[b] = nr + 1;
+      if (a.qcount) a.qcount[b] = 0;                       // its running query sum has been used and cleared
+    }
     return;
   }
   const int rows = a.n_rows[b];
@@ -1203,7 +1210,7 @@ int update_launch(const lca_params* p, const void* q_tail_sem, const void* q_tai
   }
   UpdateArgs a;
   a.cache_sem = (bf16*)cache_sem; a.cache_pos = (bf16*)cache_pos; a.qbar = qbar;
-  a.n_rep = n_rep; a.n_rows = n_rows; a.n_tok = n_tok; a.anchor_out = anchor_out;
+  a.n_rep = n_rep; a.n_rows = n_rows; a.n_tok = n_tok; a.anchor_out = anchor_out; a.qcount = nullptr;
   a.cap = cap; a.Hkv = Hkv; a.d_sem = p->d_sem; a.d_pos = p->d_pos; a.g = p->group_size; a.w = p->window;
   a.sem_in_logit = sem_in_logit; a.scale = (double)p->softmax_scale;
   const size_t smem = update_smem_bytes(p);
@@ -1212,6 +1219,101 @@ int update_launch(const lca_params* p, const void* q_tail_sem, const void* q_tai
   update_condense_kernel<<<dim3(Hkv, B), 256, smem, stream>>>(a);
   update_shift_kernel<<<dim3(B), n_tok ? 32 : 1024, 0, stream>>>(a);
   note_launch(2);
+  return cudaGetLastError() == cudaSuccess ? LCA_OK : LCA_ERR_CUDA;
+}
+
+// Streaming summary query (ring layout, one call per decode step), fused with the condensation of the sequences that
+// are due.  grid (Hkv, B), 256 threads.  First qsum[b, hk, :] += sum over the query heads of KV head hk of this step's
+// [q_sem | q_pos] (fp64: sums of bf16 values are exact as long as their exponents span less than 2^30): a thread owns one
+// 16-byte piece of the key dimension and every eighth head, eight loads in flight, the eight head lanes are added through
+// shared memory in a fixed order.  A sequence that is not due keeps the sum and counts the position.  A sequence that is
+// due takes the mean over everything summed since its previous update as its summary query, clears the sum and runs the
+// condensation of its earliest group in the same CTA; its counters are advanced by that CTA when there is one KV head
+// (the CTA is then the only one that reads them), by update_shift_kernel afterwards otherwise.
+static const int QSUM_HEAD_LANES = 8;
+static const int RING_STEP_THREADS = 576;
+__global__ void __launch_bounds__(RING_STEP_THREADS) ring_step_kernel(const bf16* __restrict__ q_sem, const bf16* __restrict__ q_pos, int Hq,
+                                                        double* __restrict__ qsum, double* __restrict__ qbar, UpdateArgs a) {
+  extern __shared__ __align__(16) unsigned char smem_raw[];
+  const int hk = blockIdx.x, b = blockIdx.y;
+  const int rep = Hq / a.Hkv;
+  const int sem_cols = a.sem_in_logit ? a.d_sem : 0, dk = sem_cols + a.d_pos;
+  const int pieces = dk / 8, sem_pieces = sem_cols / 8;
+  int group_row, rep_row;
+  const bool due = update_due(a, b, group_row, rep_row);
+  const int n = a.qcount[b] + 1;                           // only used when due, and then no CTA of this launch writes qcount[b]
+  double* s_part = reinterpret_cast<double*>(smem_raw);    // [QSUM_HEAD_LANES][dk]
+  for (int x = threadIdx.x; x < pieces * QSUM_HEAD_LANES; x += blockDim.x) {
+    const int pc = x % pieces, hl = x / pieces;
+    double acc[8];
+#pragma unroll
+    for (int i = 0; i < 8; ++i) acc[i] = 0.0;
+    for (int h = hl; h < rep; h += 8 * QSUM_HEAD_LANES) {
+      uint4 v[8];
+#pragma unroll
+      for (int u = 0; u < 8; ++u) {
+        const int hh = h + u * QSUM_HEAD_LANES;
+        v[u] = make_uint4(0u, 0u, 0u, 0u);
+        if (hh < rep) {
+          const size_t row = (size_t)b * Hq + (size_t)hk * rep + hh;
+          const bf16* src = pc < sem_pieces ? q_sem + row * a.d_sem + 8 * pc : q_pos + row * a.d_pos + 8 * (pc - sem_pieces);
+          v[u] = *reinterpret_cast<const uint4*>(src);
+        }
+      }
+#pragma unroll
+      for (int u = 0; u < 8; ++u) {
+        const unsigned w[4] = {v[u].x, v[u].y, v[u].z, v[u].w};
+#pragma unroll
+        for (int i = 0; i < 4; ++i) {
+          acc[2 * i] += (double)__uint_as_float(w[i] << 16);
+          acc[2 * i + 1] += (double)__uint_as_float(w[i] & 0xffff0000u);
+        }
+      }
+    }
+#pragma unroll
+    for (int i = 0; i < 8; ++i) s_part[(size_t)hl * dk + 8 * pc + i] = acc[i];
+  }
+  __syncthreads();
+  double* acc_g = qsum + ((size_t)b * a.Hkv + hk) * dk;
+  double* out = qbar + ((size_t)b * a.Hkv + hk) * dk;
+  for (int c = threadIdx.x; c < dk; c += blockDim.x) {
+    double sum = acc_g[c];
+    for (int l = 0; l < QSUM_HEAD_LANES; ++l) sum += s_part[(size_t)l * dk + c];
+    if (due) { out[c] = sum / ((double)n * (double)rep); acc_g[c] = 0.0; }
+    else acc_g[c] = sum;
+  }
+  if (!due) {
+    if (hk == 0 && threadIdx.x == 0) a.qcount[b] = n;
+    if (threadIdx.x == 0) a.anchor_out[b * a.Hkv + hk] = -1;
+    return;
+  }
+  __syncthreads();                                         // the summary query written above is read back by the whole CTA
+  update_condense_body(a, smem_raw);
+  if (a.Hkv == 1 && threadIdx.x == 0) { a.n_rep[b] += 1; a.qcount[b] = 0; }
+}
+
+int update_step_launch(const lca_params* p, const void* q_sem, const void* q_pos, double* qsum, int32_t* qcount,
+                       void* ring_sem, void* ring_pos, int cap, int32_t* n_rep, const int32_t* n_tok,
+                       int32_t* anchor_out, void* ws, cudaStream_t stream) {
+  const int B = p->batch, Hkv = p->n_kv_heads;
+  UpdateArgs a;
+  a.cache_sem = (bf16*)ring_sem; a.cache_pos = (bf16*)ring_pos; a.qbar = reinterpret_cast<double*>(ws);
+  a.n_rep = n_rep; a.n_rows = nullptr; a.n_tok = n_tok; a.anchor_out = anchor_out;
+  a.cap = cap; a.Hkv = Hkv; a.d_sem = p->d_sem; a.d_pos = p->d_pos; a.g = p->group_size; a.w = p->window;
+  a.sem_in_logit = p->variant == LCA_VARIANT_MLA; a.scale = (double)p->softmax_scale;
+  a.qcount = qcount;
+  size_t smem = update_smem_bytes(p);
+  const size_t part = (size_t)QSUM_HEAD_LANES * key_dim(p) * sizeof(double);
+  if (smem < part) smem = part;
+  if (cudaFuncSetAttribute(ring_step_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) != cudaSuccess)
+    return LCA_ERR_CUDA;
+  ring_step_kernel<<<dim3(Hkv, B), RING_STEP_THREADS, smem, stream>>>((const bf16*)q_sem, (const bf16*)q_pos, p->n_q_heads, qsum,
+                                                                      reinterpret_cast<double*>(ws), a);
+  note_launch();
+  if (Hkv > 1) {
+    update_shift_kernel<<<dim3(B), 32, 0, stream>>>(a);
+    note_launch();
+  }
   return cudaGetLastError() == cudaSuccess ? LCA_OK : LCA_ERR_CUDA;
 }
 

@@ -410,6 +410,26 @@ int lca_decode_update_ring(const lca_params* p, const void* q_tail_sem, const vo
                        ring_row_capacity, n_rep, nullptr, n_tok, anchor_out, ws, (cudaStream_t)stream);
 }
 
+int lca_decode_step_update_ring(const lca_params* p, const void* q_sem, const void* q_pos, double* qsum,
+                                int32_t* qcount, void* ring_sem, void* ring_pos, int32_t ring_row_capacity,
+                                int32_t* n_rep, const int32_t* n_tok, int32_t* anchor_out, void* ws,
+                                size_t ws_bytes, void* stream) {
+  int st = check_params(p, false);
+  if (st != LCA_OK) return st;
+  if (!q_pos || !qsum || !qcount || !ring_sem || !ring_pos || !n_rep || !n_tok || !anchor_out) return LCA_ERR_INVALID_ARG;
+  if (p->variant == LCA_VARIANT_MLA && !q_sem) return LCA_ERR_INVALID_ARG;
+  if (p->n_summary_q != 0 && p->n_summary_q != p->group_size) return LCA_ERR_INVALID_ARG;   // the sum runs from update to update
+  st = check_ring(p, ring_row_capacity);
+  if (st != LCA_OK) return st;
+  if (!aligned16(q_pos) || (q_sem && !aligned16(q_sem)) || !aligned16(ring_sem) || !aligned16(ring_pos) || !aligned16(qsum))
+    return LCA_ERR_MISALIGNED;
+  if (!ws || !aligned16(ws)) return LCA_ERR_INVALID_ARG;
+  if (ws_bytes < update_workspace_bytes(p)) return LCA_ERR_WORKSPACE_TOO_SMALL;
+  if (update_smem_bytes(p) > 227u * 1024u) return LCA_ERR_UNSUPPORTED_SHAPE;
+  return update_step_launch(p, q_sem, q_pos, qsum, qcount, ring_sem, ring_pos, ring_row_capacity, n_rep, n_tok,
+                            anchor_out, ws, (cudaStream_t)stream);
+}
+
 int lca_latent_to_value(const void* attn_latent, const void* w_uv, void* out_v, int64_t n_tokens,
                         int32_t n_heads, int32_t d_latent, int32_t d_v, void* stream) {
   if (n_tokens < 0 || n_heads <= 0 || d_latent <= 0 || d_v <= 0) return LCA_ERR_INVALID_ARG;

@@ -125,6 +125,9 @@ size_t update_smem_bytes(const lca_params* p);
 int update_launch(const lca_params* p, const void* q_tail_sem, const void* q_tail_pos, int64_t q_tail_batch_stride,
                   const float* qbar_opt, void* cache_sem, void* cache_pos, int cap, int32_t* n_rep, int32_t* n_rows,
                   const int32_t* n_tok, int32_t* anchor_out, void* ws, cudaStream_t stream);
+int update_step_launch(const lca_params* p, const void* q_sem, const void* q_pos, double* qsum, int32_t* qcount,
+                       void* ring_sem, void* ring_pos, int cap, int32_t* n_rep, const int32_t* n_tok,
+                       int32_t* anchor_out, void* ws, cudaStream_t stream);
 int ring_from_packed_launch(const lca_params* p, const void* packed_sem, const void* packed_pos, const int32_t* packed_rows,
                             const int32_t* n_rep, int packed_cap, void* ring_sem, void* ring_pos, int ring_cap,
                             int32_t* n_tok_out, cudaStream_t stream);

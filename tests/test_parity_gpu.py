@@ -903,3 +903,62 @@ def test_gqa_ring_decode_matches_oracle(B):
         for b in range(4):
             Hh.check_outputs(out[b], refs[b][0], f"gqa ring decode seq {b} impl {impl}")
             np.testing.assert_allclose(lse[b].cpu().numpy(), refs[b][1], atol=2e-3, rtol=1e-4)
+
+
+def test_ring_cache_step_update_with_running_summary_query_matches_oracle(B):
+    # One call per decode step: the step's queries go into the running sum, sequences that are due are condensed with
+    # the mean of everything summed since their previous update.  Oracle: the same queries collected per sequence and
+    # averaged by mla_summary_query.  The sequences are in different phases, so the first updates use fewer than g queries.
+    cfg = I.scaled(I.CONFIGS["mla_decode"], batch=3, seq_len=0, n_q_heads=16, group_size=16, window=48)
+    g, w, H, Bsz = cfg.group_size, cfg.window, cfg.n_q_heads, 3
+    R = w + g
+    steps = 3 * g + 5
+    cap = R + 8 + steps // g + 2
+    gen = torch.Generator().manual_seed(41)
+    specs = [(2, w + g - 3), (4, w + 1), (0, 20)]
+    psem, ppos, prow, prep = _ring_states(g, w, cap, specs, 512, 64, gen)
+    p = B.params_from_config(cfg, batch=Bsz)
+    d_rep = torch.tensor(prep, dtype=torch.int32, device=DEV)
+    d_sem, d_pos, d_tok = B.ring_from_packed(p, psem.to(DEV), ppos.to(DEV), torch.tensor(prow, dtype=torch.int32, device=DEV),
+                                             d_rep, cap)
+    o_sem = [Hh.bits(d_sem[b, :, 0]) for b in range(Bsz)]
+    o_pos = [Hh.bits(d_pos[b, :, 0]) for b in range(Bsz)]
+    o_tok, o_rep = d_tok.cpu().tolist(), list(prep)
+    qsum = torch.zeros((Bsz, 1, 576), dtype=torch.float64, device=DEV)
+    qcount = torch.zeros((Bsz,), dtype=torch.int32, device=DEV)
+    seen = [[] for _ in range(Bsz)]
+    scale = Hh.f32(cfg.softmax_scale)
+    n_updates = 0
+    for step in range(steps):
+        new_sem = torch.randn((Bsz, 512), generator=gen).bfloat16()
+        new_pos = torch.randn((Bsz, 64), generator=gen).bfloat16()
+        for b in range(Bsz):
+            d_sem[b, o_tok[b] % R, 0] = new_sem[b].to(DEV)
+            d_pos[b, o_tok[b] % R, 0] = new_pos[b].to(DEV)
+            o_sem[b][o_tok[b] % R] = Hh.bits(new_sem[b])
+            o_pos[b][o_tok[b] % R] = Hh.bits(new_pos[b])
+            o_tok[b] += 1
+        d_tok += 1
+        q_sem = torch.randn((Bsz, H, 512), generator=gen).bfloat16()
+        q_pos = torch.randn((Bsz, H, 64), generator=gen).bfloat16()
+        anchor = B.decode_step_update_ring(p, q_sem.to(DEV), q_pos.to(DEV), qsum, qcount, d_sem, d_pos, d_rep, d_tok)
+        torch.cuda.synchronize()
+        for b in range(Bsz):
+            seen[b].append((q_sem[b], q_pos[b]))
+            qbar = O.mla_summary_query(O.torch_bf16_to_f64(torch.stack([s for s, _ in seen[b]])),
+                                       O.torch_bf16_to_f64(torch.stack([q for _, q in seen[b]])))
+            s2, p2, nr, ia = O.mla_decode_update_ring(o_sem[b], o_pos[b], o_rep[b], o_tok[b], qbar, g, w, scale)
+            assert int(anchor[b, 0]) == ia
+            if ia >= 0:
+                n_updates += 1
+                seen[b] = []
+                got_sem, got_pos = Hh.bits(d_sem[b, :, 0]), Hh.bits(d_pos[b, :, 0])
+                row = R + o_rep[b]
+                assert np.array_equal(got_pos, p2)
+                assert (Hh.bf16_ulp_distance(got_sem[row], s2[row]) <= 1).all()
+                s2[row] = got_sem[row]
+                assert np.array_equal(got_sem, s2)
+                assert float(qsum[b].abs().max()) == 0.0
+            o_sem[b], o_pos[b], o_rep[b] = s2, p2, nr
+        assert d_rep.cpu().tolist() == o_rep and qcount.cpu().tolist() == [len(x) for x in seen]
+    assert n_updates >= 8
