@@ -86,3 +86,24 @@ def test_invalid_calls_return_error_codes_without_launching(B):
     odd = B.make_params("mla", 1, 1024, 4, 1, 256, 32, 64, 128, 0.07)
     assert B.lca_prefill_attention(odd, 16, 16, 16, 16, 16, 16, 16, None, None, 0) == -2
     assert B.lca_launch_count() == before
+
+
+def test_ring_calls_reject_invalid_arguments_without_launching(B):
+    # the ring layout needs whole groups to leave the ring (window % group_size == 0) and a buffer that holds the ring
+    before = B.lca_launch_count()
+    good = B.make_params("mla", 2, 0, 16, 1, 512, 64, 16, 48, 0.07)
+    R = 48 + 16
+    assert B.lca_ring_from_packed(good, None, 16, 16, 16, 80, 16, 16, R + 4, 16) == -1            # NULL packed cache
+    assert B.lca_ring_from_packed(good, 16, 16, 16, 16, 80, 16, 16, R - 1, 16) == -1              # buffer smaller than the ring
+    assert B.lca_ring_from_packed(good, 16, 16, 16, 16, 80, 24, 16, R + 4, 16) == -3              # misaligned ring buffer
+    assert B.lca_decode_attention_ring(good, 16, 16, 16, 16, None, 16, R + 4, 16, None, None, 0) == -1   # NULL n_rep
+    assert B.lca_decode_update_ring(good, 16, 16, 16, None, 16, 16, R + 4, 16, None, 16, 16, 1 << 20) == -1   # NULL n_tok
+    assert B.lca_decode_update_ring(good, 16, 16, 16, None, 16, 16, R + 4, 16, 16, 16, 16, 8) == -4      # workspace too small
+    assert B.lca_decode_step_update_ring(good, 16, 16, None, 16, 16, 16, R + 4, 16, 16, 16, 16, 1 << 20) == -1   # NULL running sum
+    ragged_window = B.make_params("mla", 2, 0, 16, 1, 512, 64, 16, 40, 0.07)                      # 40 % 16 != 0
+    assert B.lca_decode_attention_ring(ragged_window, 16, 16, 16, 16, 16, 16, 80, 16, None, None, 0) == -1
+    assert B.lca_decode_update_ring(ragged_window, 16, 16, 16, None, 16, 16, 80, 16, 16, 16, 16, 1 << 20) == -1
+    few = B.make_params("mla", 2, 0, 16, 1, 512, 64, 16, 48, 0.07, )
+    few.n_summary_q = 4                                                                            # the running sum spans update to update
+    assert B.lca_decode_step_update_ring(few, 16, 16, 16, 16, 16, 16, R + 4, 16, 16, 16, 16, 1 << 20) == -1
+    assert B.lca_launch_count() == before
