@@ -19,6 +19,12 @@ static const int QBAR_ROWS_PER_CHUNK = 64;
 static const int CONDENSE_THREADS = 512;
 
 // ---------------------------------------------------------------------------- summary query
+// Row lanes of qbar_partial_kernel for a key of `pieces` 16-byte pieces: about 288 threads per CTA.  With the 72 pieces
+// of the MLA key that is four lanes, so that a chunk of 64 rows is two full rounds of eight rows per lane.
+static int qbar_row_lanes(int pieces) {
+  int lanes = 288 / pieces;
+  return lanes < 1 ? 1 : lanes > 16 ? 16 : lanes;
+}
 // Partial sums of the query tail.  Rows of one KV head = (position, query head in its group);
 // a chunk is QBAR_ROWS_PER_CHUNK rows and has its own partial sum; a CTA takes `chunks_per_cta` consecutive chunks one
 // after the other (the sums do not depend on that number).  grid (CTAs, Hkv, B).  A thread owns one 16-byte piece
@@ -31,7 +37,7 @@ __global__ void qbar_partial_kernel(const bf16* __restrict__ q_sem, const bf16* 
                                     int64_t batch_stride_rows, int n_pos, int Hq, int Hkv, int d_sem,
                                     int d_pos, int sem_in_logit, int row_lanes, double* __restrict__ partial, SeqTab tab,
                                     int nchunks, int chunks_per_cta) {
-  extern __shared__ double s_part[];                     // [row_lanes][dk]
+  extern __shared__ double s_part_all[];                 // [2][row_lanes][dk]: chunks alternate, one barrier per chunk
   const int hk = blockIdx.y, b = blockIdx.z;
   const int rep = Hq / Hkv;
   long long first_pos = (long long)b * batch_stride_rows;     // row (position) of the first averaged query
@@ -45,37 +51,56 @@ __global__ void qbar_partial_kernel(const bf16* __restrict__ q_sem, const bf16* 
   const int pieces = dk / 8, sem_pieces = sem_in_logit ? d_sem / 8 : 0;
   const int pc = threadIdx.x % pieces, rl = threadIdx.x / pieces;
   for (int chunk = blockIdx.x * chunks_per_cta; chunk < min(nchunks, (int)(blockIdx.x + 1) * chunks_per_cta); ++chunk) {
+  double* s_part = s_part_all + (size_t)(chunk & 1) * row_lanes * dk;
   const int r0 = chunk * QBAR_ROWS_PER_CHUNK;
   const int r1 = min(n_rows, r0 + QBAR_ROWS_PER_CHUNK);
   double acc[8];
 #pragma unroll
   for (int i = 0; i < 8; ++i) acc[i] = 0.0;
   if (rl < row_lanes) {
-    // eight rows per step: all eight loads are issued before the first one is used (the kernel is bound by memory
-    // latency otherwise); rows behind the end of the chunk contribute exact zeros, the order of the sums is fixed
-    for (int r = r0 + rl; r < r1; r += 8 * row_lanes) {
+    // Several rows per step: all loads of a step are issued before the first one is used (the kernel is bound by memory
+    // latency otherwise); rows behind the end of the chunk contribute exact zeros, the order of the sums is fixed.
+    // The piece of this thread lies in one of the two arrays, whose rows are d elements apart.
+    const bool in_sem = pc < sem_pieces;
+    const bf16* arr = in_sem ? q_sem + 8 * pc : q_pos + 8 * (pc - sem_pieces);
+    const size_t d = in_sem ? d_sem : d_pos;
+    auto add_row = [&](const uint4& x) {
+      const unsigned w[4] = {x.x, x.y, x.z, x.w};
+#pragma unroll
+      for (int i = 0; i < 4; ++i) {
+        acc[2 * i] += (double)__uint_as_float(w[i] << 16);
+        acc[2 * i + 1] += (double)__uint_as_float(w[i] & 0xffff0000u);
+      }
+    };
+    int r = r0 + rl;
+    if (Hkv == 1) {
+      // one KV head: the rows of the tail are consecutive rows of the query arrays, so the loads of a thread are a fixed
+      // stride apart (no per-row index arithmetic, no guards).  Eight rows per step: with sixteen the registers allow
+      // only two CTAs per SM and the kernel was slower.
+      const size_t step = (size_t)row_lanes * d / 8;
+      for (; r + 7 * row_lanes < r1; r += 8 * row_lanes) {
+        const uint4* src = reinterpret_cast<const uint4*>(arr + ((size_t)first_pos * Hq + r) * d);
+        uint4 v[8];
+#pragma unroll
+        for (int u = 0; u < 8; ++u) v[u] = src[u * step];
+#pragma unroll
+        for (int u = 0; u < 8; ++u) add_row(v[u]);
+      }
+    }
+    for (; r < r1; r += 8 * row_lanes) {
       uint4 v[8];
 #pragma unroll
       for (int u = 0; u < 8; ++u) {
         const int rr = r + u * row_lanes;
         v[u] = make_uint4(0u, 0u, 0u, 0u);
         if (rr < r1) {
-          // one KV head: the rows of the tail are consecutive rows of the query arrays (no division per row)
           const size_t row = Hkv == 1 ? (size_t)first_pos * Hq + rr
                                       : ((size_t)first_pos + rr / rep) * Hq + hk * rep + rr % rep;
-          const bf16* src = (pc < sem_pieces) ? q_sem + row * d_sem + 8 * pc : q_pos + row * d_pos + 8 * (pc - sem_pieces);
-          v[u] = *reinterpret_cast<const uint4*>(src);
+          v[u] = *reinterpret_cast<const uint4*>(arr + row * d);
         }
       }
 #pragma unroll
-      for (int u = 0; u < 8; ++u) {
-        const unsigned w[4] = {v[u].x, v[u].y, v[u].z, v[u].w};
-#pragma unroll
-        for (int i = 0; i < 4; ++i) {
-          acc[2 * i] += (double)__uint_as_float(w[i] << 16);
-          acc[2 * i + 1] += (double)__uint_as_float(w[i] & 0xffff0000u);
-        }
-      }
+      for (int u = 0; u < 8; ++u) add_row(v[u]);
     }
 #pragma unroll
     for (int i = 0; i < 8; ++i) s_part[(size_t)rl * dk + 8 * pc + i] = acc[i];
@@ -87,7 +112,8 @@ __global__ void qbar_partial_kernel(const bf16* __restrict__ q_sem, const bf16* 
     for (int l = 0; l < row_lanes; ++l) sum += s_part[(size_t)l * dk + c];
     dst[c] = sum;
   }
-  __syncthreads();                                       // s_part is reused by the next chunk
+  // no second barrier: the next chunk writes the other half of s_part_all, and the chunk after it passes the next
+  // chunk's barrier before it writes this half again
   }
 }
 
@@ -953,12 +979,10 @@ int condense_launch(const CondenseLaunch& c) {
       const int nch = (rows_q + QBAR_ROWS_PER_CHUNK - 1) / QBAR_ROWS_PER_CHUNK;
       dim3 grid((nch + cpc - 1) / cpc, Hkv, B);
       const int pieces = dk / 8;
-      int row_lanes = 256 / pieces;
-      if (row_lanes < 1) row_lanes = 1;
-      if (row_lanes > 16) row_lanes = 16;
+      const int row_lanes = qbar_row_lanes(pieces);
       const int threads = ((pieces * row_lanes + 31) / 32) * 32;
       const int n = n_req;
-      qbar_partial_kernel<<<grid, threads, (size_t)row_lanes * dk * sizeof(double), c.stream>>>(
+      qbar_partial_kernel<<<grid, threads, (size_t)2 * row_lanes * dk * sizeof(double), c.stream>>>(
           (const bf16*)c.q_tail_sem, (const bf16*)c.q_tail_pos, c.q_tail_batch_stride, n,
           p->n_q_heads, Hkv, p->d_sem, p->d_pos, sem_in_logit, row_lanes, partial, c.tab, nch, cpc);
       double count = (double)n * (double)(p->n_q_heads / Hkv);
@@ -1197,11 +1221,9 @@ int update_launch(const lca_params* p, const void* q_tail_sem, const void* q_tai
     const int cpc = qbar_chunks_per_cta((long long)rows * Hkv * B);
     const int nch = (rows + QBAR_ROWS_PER_CHUNK - 1) / QBAR_ROWS_PER_CHUNK;
     const int pieces = dk / 8;
-    int row_lanes = 256 / pieces;
-    if (row_lanes < 1) row_lanes = 1;
-    if (row_lanes > 16) row_lanes = 16;
+    const int row_lanes = qbar_row_lanes(pieces);
     const int threads = ((pieces * row_lanes + 31) / 32) * 32;
-    qbar_partial_kernel<<<dim3((nch + cpc - 1) / cpc, Hkv, B), threads, (size_t)row_lanes * dk * sizeof(double), stream>>>(
+    qbar_partial_kernel<<<dim3((nch + cpc - 1) / cpc, Hkv, B), threads, (size_t)2 * row_lanes * dk * sizeof(double), stream>>>(
         (const bf16*)q_tail_sem, (const bf16*)q_tail_pos, q_tail_batch_stride, n, p->n_q_heads, Hkv, p->d_sem, p->d_pos,
         sem_in_logit, row_lanes, partial, SeqTab{}, nch, cpc);
     qbar_final_kernel<<<dim3(Hkv, B), dk < 1024 ? ((dk + 31) / 32) * 32 : 1024, 0, stream>>>(
