@@ -232,7 +232,9 @@ int lca_decode_update(const lca_params* p, const void* q_tail_sem, const void* q
  *                (0-based, counted from the start of the sequence) is at row n % R
  *   rows [R, R + n_rep[b]): the representatives in group order
  * State per sequence: n_rep[b] and n_tok[b] (tokens of the sequence so far); the uncondensed tokens
- * are n_rep[b]*group_size .. n_tok[b]-1, at most R of them.  The caller writes the row of a new
+ * are n_rep[b]*group_size .. n_tok[b]-1, at most R of them (and, once a sequence has representatives,
+ * at least `window` of them: the state lca_ring_from_packed and every update leave; with fewer, ring rows
+ * of condensed tokens would be attended to).  The caller writes the row of a new
  * token at row n_tok[b] % R and then counts it in n_tok[b].  window must be a multiple of group_size
  * (groups leave the ring whole), ring_row_capacity >= R + the representatives the sequence will have;
  * buffers are [B, ring_row_capacity, n_kv_heads, d_sem | d_pos].  Rows that hold nothing yet must hold
