@@ -482,7 +482,7 @@ condense_mla64_kernel(CondenseArgs a) {
     }
   } else if (warp < SCORE_WARPS) {
     // ===================================================== fp32 product sums and max |k| of four tokens per warp
-    float q[18];
+    unsigned long long q2[9];                             // q_bar components of this lane, in pairs (two FMAs per instruction)
     long long cur_b = -1;
     for (long long it = 0; it < n_mine; ++it) {
       const int st = (int)(it % STAGES), p = (int)(it & 1);
@@ -492,8 +492,11 @@ condense_mla64_kernel(CondenseArgs a) {
         cur_b = b;
         const double* qb = a.qbar + (size_t)b * DK;
 #pragma unroll
-        for (int i = 0; i < 8; ++i) { q[i] = (float)qb[8 * lane + i]; q[8 + i] = (float)qb[256 + 8 * lane + i]; }
-        q[16] = (float)qb[DS + 2 * lane]; q[17] = (float)qb[DS + 2 * lane + 1];
+        for (int i = 0; i < 4; ++i) {
+          q2[i] = f32x2((float)qb[8 * lane + 2 * i], (float)qb[8 * lane + 2 * i + 1]);
+          q2[4 + i] = f32x2((float)qb[256 + 8 * lane + 2 * i], (float)qb[256 + 8 * lane + 2 * i + 1]);
+        }
+        q2[8] = f32x2((float)qb[DS + 2 * lane], (float)qb[DS + 2 * lane + 1]);
       }
       if (!cond_wait(BAR_FULL(st), (unsigned)((it / STAGES) & 1), s_abort)) break;
       if (it >= 2 && !cond_wait(BAR_AFREE(p), (unsigned)(((it >> 1) - 1) & 1), s_abort)) break;
@@ -507,14 +510,16 @@ condense_mla64_kernel(CondenseArgs a) {
         const uint4 v1 = *reinterpret_cast<const uint4*>(t_sem + (size_t)i * (DS * 2) + 512 + 16 * lane);
         const unsigned vp = *reinterpret_cast<const unsigned*>(t_pos + (size_t)i * (DP * 2) + 4 * lane);
         const unsigned w[9] = {v0.x, v0.y, v0.z, v0.w, v1.x, v1.y, v1.z, v1.w, vp};
-        float acc0 = 0.f, acc1 = 0.f, kmax = 0.f;
+        unsigned long long acc = f32x2(0.f, 0.f);        // even / odd components: the same two fp32 chains as scalar FMAs
+        float kmax = 0.f;
 #pragma unroll
         for (int k = 0; k < 9; ++k) {
           const float lo = __uint_as_float(w[k] << 16), hi = __uint_as_float(w[k] & 0xffff0000u);
-          acc0 = fmaf(q[2 * k], lo, acc0);
-          acc1 = fmaf(q[2 * k + 1], hi, acc1);
+          acc = fma_f32x2(q2[k], f32x2(lo, hi), acc);
           kmax = f32_max3_abs(kmax, lo, hi);
         }
+        float acc0, acc1;
+        asm("mov.b64 {%0, %1}, %2;" : "=f"(acc0), "=f"(acc1) : "l"(acc));
         v[tt] = acc0 + acc1;
         v[4 + tt] = kmax;
       }
