@@ -641,10 +641,28 @@ def measure_gqa_config(B, dev, peaks, warmup=3, iters=5, seq_len=None, parity=No
         parity[cfg.name] = parity_record(ref, out[0][idx], {kk: cond[kk][0] for kk in ("cache_sem", "cache_pos", "anchor_idx")}, kind="gqa")
     flops = attention_flops(cfg)
     cbytes = condense_bytes(cfg)
-    return dict(workload=f"gqa_64k: L={L}, {cfg.n_q_heads} q heads / {cfg.n_kv_heads} kv heads, d={cfg.d_sem}, g={g}, w={cfg.window}",
-                tokens_per_s=L / ((t_cond + t_attn) * 1e-3), condense_ms=t_cond, condense_gbs=cbytes / t_cond / 1e6,
-                attention_ms=t_attn, attention_tflops=flops / t_attn / 1e9,
-                attention_frac_of_measured_burst=flops / t_attn / 1e9 / peaks["tflops_burst"])
+    res = dict(workload=f"gqa_64k: L={L}, {cfg.n_q_heads} q heads / {cfg.n_kv_heads} kv heads, d={cfg.d_sem}, g={g}, w={cfg.window}",
+               tokens_per_s=L / ((t_cond + t_attn) * 1e-3), condense_ms=t_cond, condense_gbs=cbytes / t_cond / 1e6,
+               attention_ms=t_attn, attention_tflops=flops / t_attn / 1e9,
+               attention_frac_of_measured_burst=flops / t_attn / 1e9 / peaks["tflops_burst"])
+    if not seq_len:
+        # decode over condensed caches of this shape: 64 sequences, one new query each (HBM-bound: K and V of every row once)
+        m, k = B.lca_partition(p)
+        nb, cap = 64, m + k + 1
+        gen = torch.Generator(device=dev)
+        gen.manual_seed(cfg.seed + 7)
+        ck = torch.randn((nb, cap, cfg.n_kv_heads, cfg.d_sem), generator=gen, device=dev).bfloat16()
+        cv = torch.randn((nb, cap, cfg.n_kv_heads, cfg.d_sem), generator=gen, device=dev).bfloat16()
+        qn = torch.randn((nb, cfg.n_q_heads, cfg.d_sem), generator=gen, device=dev).bfloat16()
+        pd = B.params_from_config(cfg, batch=nb)
+        rows_t = torch.full((nb,), cap, dtype=torch.int32, device=dev)
+        od = torch.empty((nb, cfg.n_q_heads, cfg.d_sem), dtype=torch.bfloat16, device=dev)
+        wsd = B.workspace(pd, B.LCA_WS_DECODE, dev)
+        t_dec = time_cuda(lambda: B.decode_attention(pd, None, qn, cv, ck, rows_t, m, out=od, ws=wsd), warmup, iters)
+        kv_bytes = float(nb) * cap * cfg.n_kv_heads * cfg.d_sem * 2 * 2
+        res["decode"] = dict(batch=nb, rows_per_seq=cap, us=t_dec * 1e3, kv_gbs=kv_bytes / t_dec / 1e6,
+                             frac_of_measured_hbm=kv_bytes / t_dec / 1e6 / peaks["hbm_gbs"])
+    return res
 
 
 def measure_mla_small(B, dev, name, want_oracle, parity):
