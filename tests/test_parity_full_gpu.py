@@ -161,3 +161,55 @@ def test_attention_is_bit_reproducible_at_full_size(B):
     for t in range(0, L, step):
         assert torch.equal(Hh.bits_t(out1[0, t:t + step]), Hh.bits_t(out2[0, t:t + step])), f"tokens {t}..{t + step}"
     assert torch.equal(lse1, lse2)
+
+
+def test_config4_ring_cache_update_and_decode_full_size(B):
+    # The decode cache of config 4 in the ring layout (64 sequences, ring of w + g = 4160 rows, ~960 representatives):
+    # sequences in four phases (ring full and due for an update, one token after an update, one token short of an update,
+    # a few representatives fewer).  One update call with the query tails, then one decode call; four sequences against
+    # the oracle (every row of the ring buffers, every head of the decode output).
+    cfg = I.CONFIGS["mla_decode"]
+    Bsz, g, w, H = cfg.batch, cfg.group_size, cfg.window, cfg.n_q_heads
+    R = w + g
+    m0 = 960
+    cap = R + m0 + 8
+    gen = torch.Generator(device=DEV)
+    gen.manual_seed(91)
+    specs = [[(m0, R), (m0, w + 1), (m0, R - 1), (m0 - 3, w + 17)][b % 4] for b in range(Bsz)]
+    cap_packed = m0 + R
+    psem = torch.randn((Bsz, cap_packed, 1, 512), generator=gen, device=DEV).bfloat16()
+    ppos = torch.randn((Bsz, cap_packed, 1, 64), generator=gen, device=DEV).bfloat16()
+    p = B.params_from_config(cfg, batch=Bsz)
+    d_rep = torch.tensor([r for r, _ in specs], dtype=torch.int32, device=DEV)
+    prow = torch.tensor([r + c for r, c in specs], dtype=torch.int32, device=DEV)
+    rsem, rpos, d_tok = B.ring_from_packed(p, psem, ppos, prow, d_rep, cap)
+    qts = torch.randn((Bsz, g, H, 512), generator=gen, device=DEV).bfloat16()
+    qtp = torch.randn((Bsz, g, H, 64), generator=gen, device=DEV).bfloat16()
+    before = {b: (Hh.bits(rsem[b, :, 0]), Hh.bits(rpos[b, :, 0])) for b in (0, 1, 2, 63)}
+    anchor = B.decode_update_ring(p, qts, qtp, rsem, rpos, d_rep, d_tok)
+    qs = torch.randn((Bsz, H, 512), generator=gen, device=DEV).bfloat16()
+    qp = torch.randn((Bsz, H, 64), generator=gen, device=DEV).bfloat16()
+    out, lse = B.decode_attention_ring(p, qs, qp, rsem, rpos, d_rep, d_tok, want_lse=True)
+    torch.cuda.synchronize()
+    assert B.lca_last_device_status() == 0
+    n_rep_after, tok = d_rep.cpu().tolist(), d_tok.cpu().tolist()
+    scale = Hh.f32(cfg.softmax_scale)
+    for b in (0, 1, 2, 63):
+        r, c = specs[b]
+        assert tok[b] == r * g + c
+        o_sem, o_pos, n = O.ring_from_packed(Hh.bits(psem[b, :r + c, 0]), Hh.bits(ppos[b, :r + c, 0]), r, r + c, g, w, cap)
+        assert n == tok[b] and np.array_equal(before[b][0], o_sem) and np.array_equal(before[b][1], o_pos)
+        qbar = O.mla_summary_query(O.torch_bf16_to_f64(qts[b].cpu()), O.torch_bf16_to_f64(qtp[b].cpu()))
+        s2, p2, nr, ia = O.mla_decode_update_ring(o_sem, o_pos, r, tok[b], qbar, g, w, scale)
+        assert int(anchor[b, 0]) == ia and n_rep_after[b] == nr and (ia >= 0) == (c == R)
+        got_sem, got_pos = Hh.bits(rsem[b, :, 0]), Hh.bits(rpos[b, :, 0])
+        assert np.array_equal(got_pos, p2)
+        if ia >= 0:
+            assert (Hh.bf16_ulp_distance(got_sem[R + r], s2[R + r]) <= 1).all()
+            s2[R + r] = got_sem[R + r]
+        assert np.array_equal(got_sem, s2)
+        cs, cp, _ = O.ring_to_packed(s2, p2, nr, tok[b], g, w)
+        ro, rl = O.mla_decode(O.torch_bf16_to_f64(qs[b].cpu()), O.torch_bf16_to_f64(qp[b].cpu()), O.bits_to_f64(cs), O.bits_to_f64(cp),
+                              nr, scale)
+        Hh.check_outputs(out[b], ro, f"ring decode seq {b}")
+        np.testing.assert_allclose(lse[b].cpu().numpy(), rl, atol=2e-3, rtol=1e-4)
