@@ -63,7 +63,7 @@ enum { LCA_WS_CONDENSE = 0, LCA_WS_PREFILL = 1, LCA_WS_DECODE = 2, LCA_WS_UPDATE
  *   MLA: n_kv_heads = 1, d_sem = d_c (512), d_pos = d_R (64); logits use [sem | pos], values = sem.
  *   GQA: d_sem = d_pos = head_dim (128); logits use pos (= K) only, values = sem (= V);
  *        n_q_heads must be a multiple of n_kv_heads.
- *   n_summary_q: number of trailing queries averaged into the summary query (Alg. 1 line 1;
+ *   n_summary_q: number of trailing queries averaged into the summary query (Alg. 1, first step;
  *                Table 8 varies it); 0 means g; clamped to L.
  *   softmax_scale: 1/sqrt(d_h), used for the importance scores (Sec. 4.2) and the attention (Eq. 10).
  *   rep_logit_bias: added to the logit of every representative; 0 = Alg. 1 as printed,
@@ -94,7 +94,7 @@ int lca_partition(const lca_params* p, int32_t* m, int32_t* k);
  * Returns 0 for invalid parameters as well; the entry point then reports the error. */
 size_t lca_workspace_bytes(const lca_params* p, int32_t which);
 
-/* Condensation: Alg. 1 lines 1-10 (summary query, Eq. 6 group softmax, Eq. 7 pooling, Eq. 8
+/* Condensation: Alg. 1 up to the local window (summary query, Eq. 6 group softmax, Eq. 7 pooling, Eq. 8
  * anchors, Eq. 9 local window) for `batch` sequences.
  *   q_tail_sem [B, n, H, d_sem], q_tail_pos [B, n, H, d_pos]: the LAST n = n_summary_q query
  *       positions of each sequence (MLA: q_latent and q_rope; GQA: q_tail_sem = NULL and
@@ -273,7 +273,7 @@ int lca_decode_update_ring(const lca_params* p, const void* q_tail_sem, const vo
                            int32_t* anchor_out, void* ws, size_t ws_bytes, void* stream);
 
 /* The update on the ring layout with a running summary query, called once per decode step after the
- * step's token has been written and counted (Sec. 4.3: "the average query of the last g tokens"):
+ * step's token has been written and counted (Sec. 4.3: an update scores with the mean of the last g queries):
  *   1. qsum[b, hk, :] += sum over the query heads of KV head hk of this step's [q_sem | q_pos] (fp64;
  *      MLA: dk = d_sem + d_pos, GQA: dk = d_pos), qcount[b] += 1;
  *   2. every sequence that is due (window + group_size uncondensed tokens) is condensed exactly as by

@@ -7,12 +7,12 @@
 // Every function follows one passage of the paper, in the paper's order and notation
 // (1-based token/group indices in the comments, 0-based in the arrays):
 //
-//   summary query      Alg. 1 line 1, Sec. 4.2 ("average of the last g queries")
+//   summary query      Alg. 1 (first step), Sec. 4.2: the mean of the last g queries
 //   scores, alpha      Sec. 4.2 importance score s_i, Eq. 6
-//   weighted pooling   Eq. 7 (Alg. 1 line 5)
-//   anchor selection   Eq. 8 (Alg. 1 line 6)
+//   weighted pooling   Eq. 7
+//   anchor selection   Eq. 8
 //   local window       Sec. 4.2 "Preserving Fine-Grained Local Context", Eq. 9
-//   fused attention    Eq. 10 (Alg. 1 lines 11-12), evaluated at every prefix length t
+//   fused attention    Eq. 10 (the last steps of Alg. 1), evaluated at every prefix length t
 //   decode             Sec. 4.3 "Decoding and Online Cache Update"
 //   GQA variant        Sec. 5.4 "Extension to Other Attention Variants"
 //
@@ -89,7 +89,7 @@ void lca_oracle_partition(int64_t L, int64_t w, int64_t g, int64_t* m, int64_t* 
   *k = w + r;
 }
 
-// Alg. 1 line 1: q_bar = Avg(q_{L-n+1} .. q_L), n = n_summary_q (default g), here also
+// Summary query of Alg. 1: q_bar = Avg(q_{L-n+1} .. q_L), n = n_summary_q (default g), here also
 // averaged over the `heads` query heads that share the key/value stream.
 //   q: [n_rows, heads, d]  -- the LAST n_rows query positions only
 void lca_oracle_summary_query(const double* q, int64_t n_rows, int64_t heads, int64_t d,
@@ -102,7 +102,7 @@ void lca_oracle_summary_query(const double* q, int64_t n_rows, int64_t heads, in
   for (int64_t c = 0; c < d; ++c) qbar[c] /= cnt;
 }
 
-// Alg. 1 lines 2-8 for one key/value stream.
+// The condensation steps of Alg. 1 (scores, Eq. 6-8) for one key/value stream.
 //   key  [L, dk]  the vectors the score is taken against (MLA: k_i = [c_i | k^R_i], dk = 576;
 //                 GQA: the key of this KV head)
 //   pool [L, dp]  the vectors that are pooled (MLA: c_i^KV; GQA: the value of this KV head)

@@ -92,7 +92,7 @@ def partition(L: int, w: int, g: int):
 
 # ------------------------------------------------------------------------- generic streams
 def summary_query(q_tail: np.ndarray) -> np.ndarray:
-    """Alg. 1 line 1.  q_tail [n, heads, d] (the last n query positions) -> q_bar [d]."""
+    """Summary query of Alg. 1 (Sec. 4.2).  q_tail [n, heads, d] (the last n query positions) -> q_bar [d]."""
     q = _f64(q_tail)
     n, heads, d = q.shape
     out = np.empty(d, dtype=np.float64)
@@ -102,7 +102,7 @@ def summary_query(q_tail: np.ndarray) -> np.ndarray:
 
 def condense_stream(key: np.ndarray, pool: np.ndarray, qbar: np.ndarray, g: int, w: int,
                     scale: float):
-    """Alg. 1 lines 2-8 on one key/value stream.  Returns dict(scores, alpha, pooled, anchor, m, k)."""
+    """The condensation steps of Alg. 1 (scores, Eq. 6, Eq. 7, Eq. 8) on one key/value stream.  Returns dict(scores, alpha, pooled, anchor, m, k)."""
     key = _f64(key)
     pool = _f64(pool)
     qbar = _f64(qbar)
@@ -192,7 +192,7 @@ def mla_summary_query(q_sem_tail: np.ndarray, q_pos_tail: np.ndarray) -> np.ndar
 
 def mla_condense(qbar: np.ndarray, ckv: np.ndarray, kr: np.ndarray, g: int, w: int, scale: float,
                  sem_reducer: str = "weighted", pos_reducer: str = "maxsel"):
-    """Condensed MLA cache of one sequence (Alg. 1 lines 2-10).
+    """Condensed MLA cache of one sequence (the condensation and local-window steps of Alg. 1).
 
     Returns dict with
       scores, alpha [m*g]; c_rep [m, d_c] (unrounded); anchor [m] int32 (absolute 0-based);
@@ -335,7 +335,7 @@ def mla_decode_update(cache_sem_bits: np.ndarray, cache_pos_bits: np.ndarray, n_
 
 
 # ------------------------------------------------------- ring layout of the decode cache
-# Sec. 4.3 keeps "the m representatives ... together with the w most recent latent vectors" and says
+# Sec. 4.3 states what the cache holds while decoding (the m representatives and the most recent tokens) and says
 # nothing about where they live.  The packed layout above moves every buffered token when a group is
 # condensed; the ring layout moves none:
 #   rows [0, R), R = w + g : token number n of the sequence (0-based from its start) at row n % R;

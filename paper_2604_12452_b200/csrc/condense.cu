@@ -1,4 +1,4 @@
-// Condensation kernels: summary query (Alg. 1 line 1), group scores + softmax (Sec. 4.2, Eq. 6),
+// Condensation kernels: summary query (Alg. 1, first step), group scores + softmax (Sec. 4.2, Eq. 6),
 // weighted pooling (Eq. 7), anchor selection (Eq. 8) and the local-window copy (Eq. 9).
 //
 // The work is HBM-bound (about 2 flop per byte): every history token is read from global memory

@@ -260,7 +260,7 @@ def test_dominant_token_gives_one_hot_and_constant_group_is_preserved():
 
 
 def test_absorbed_form_equals_unabsorbed_form():
-    # Alg. 1 line 7 builds k_rep = [c_rep W^UK, k^R_I], v_rep = c_rep W^UV.  With
+    # Alg. 1 builds k_rep = [c_rep W^UK, k^R_I], v_rep = c_rep W^UV.  With
     # q_latent = q_nope W^UK^T the latent-space result times W^UV must equal it exactly.
     rng = RNG(9)
     L, H, dc, dr, dn, dv = 37, 2, 6, 4, 5, 3
