@@ -35,7 +35,7 @@ METRIC = "lca_prefill_tokens_per_s"
 UNIT = "tokens/s"
 # dram__bytes_read.sum + dram__bytes_write.sum of attn_tc2_kernel at mla_32k (L=32768, H=16) divided by
 # L*H: the kernel reads every query row and writes every output row once, the key/value stream stays in L2.
-ATTN_DRAM_BYTES_PER_TOKEN_HEAD = (642.909440e6 + 497.025536e6) / (32768 * 16)
+ATTN_DRAM_BYTES_PER_TOKEN_HEAD = (642.586880e6 + 497.310208e6) / (32768 * 16)
 
 
 # ---------------------------------------------------------------------------- work counts
