@@ -388,3 +388,27 @@ def mla_decode_update_ring(ring_sem_bits: np.ndarray, ring_pos_bits: np.ndarray,
     ring_sem[R + n_rep] = round_bf16_bits(r["pooled"])[0]
     ring_pos[R + n_rep] = ring_pos_bits[rows[ia]]
     return ring_sem, ring_pos, n_rep + 1, ia
+
+
+def gqa_decode_update_ring(ring_k_bits: np.ndarray, ring_v_bits: np.ndarray, n_rep: int, n_tok: int,
+                           qbar: np.ndarray, g: int, w: int, scale: float):
+    """The online update of Sec. 4.3 for the GQA variant (Sec. 5.4: select K, pool V, per KV head) on the
+    ring layout.  ring_*_bits [capacity, Hkv, d] bf16 bit patterns, qbar [Hkv, d].  Returns
+    (ring_k_bits, ring_v_bits, n_rep, anchors [Hkv] or None when nothing was condensed)."""
+    R = w + g
+    first = n_rep * g
+    if n_tok - first < R or R + n_rep >= ring_k_bits.shape[0]:
+        return ring_k_bits, ring_v_bits, n_rep, None
+    rows = [(first + i) % R for i in range(g)]
+    ring_k = ring_k_bits.copy()
+    ring_v = ring_v_bits.copy()
+    anchors = []
+    for h in range(ring_k_bits.shape[1]):
+        grp_k = bits_to_f64(ring_k_bits[rows, h])
+        grp_v = bits_to_f64(ring_v_bits[rows, h])
+        r = condense_stream(grp_k, grp_v, qbar[h], g, 0, scale)       # one group: scores on K, pooling of V
+        ia = int(r["anchor"][0])
+        ring_v[R + n_rep, h] = round_bf16_bits(r["pooled"])[0]
+        ring_k[R + n_rep, h] = ring_k_bits[rows[ia], h]
+        anchors.append(ia)
+    return ring_k, ring_v, n_rep + 1, np.array(anchors, dtype=np.int32)

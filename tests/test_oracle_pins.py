@@ -614,6 +614,40 @@ def test_ring_layout_streaming_reproduces_alg1_on_the_longer_sequence():
     assert n_updates == (L0 + T - w) // g - start["m"] and n_updates >= 4 * R // g
 
 
+def test_gqa_ring_streaming_reproduces_the_condensation_of_the_longer_sequence():
+    """GQA variant of the online update (Sec. 5.4 with Sec. 4.3) on the ring layout: per KV head the anchor key is selected
+    and the values are pooled.  Streaming token by token from the packed cache of a prefix must give, after every token, the
+    cache gqa_condense builds from scratch on the longer sequence (per head: its own scores, its own anchors)."""
+    rng = RNG(24)
+    g, w, d, hkv = 4, 8, 6, 3
+    R = w + g
+    L0, T = w + g + 2, 2 * R + 3
+    import torch
+    K = torch.from_numpy(rng.standard_normal((L0 + T, hkv, d))).bfloat16()
+    V = torch.from_numpy(rng.standard_normal((L0 + T, hkv, d))).bfloat16()
+    Kb, Vb = O.torch_bf16_to_bits(K), O.torch_bf16_to_bits(V)
+    qbar = rng.standard_normal((hkv, d))
+    scale = 0.4
+    start = O.gqa_condense(qbar, O.bits_to_f64(Kb[:L0]), O.bits_to_f64(Vb[:L0]), g, w, scale)
+    cap = R + (L0 + T) // g + 1
+    # ring_from_packed treats the trailing dimensions as one row: the same for [rows, Hkv, d]
+    rk, rv, n_tok = O.ring_from_packed(start["cache_k_bits"], start["cache_v_bits"], start["m"], start["m"] + start["k"], g, w, cap)
+    n_rep = start["m"]
+    n_updates = 0
+    for t in range(L0, L0 + T):
+        rk[t % R], rv[t % R] = Kb[t], Vb[t]
+        n_tok += 1
+        rk, rv, n_rep, anchors = O.gqa_decode_update_ring(rk, rv, n_rep, n_tok, qbar, g, w, scale)
+        whole = O.gqa_condense(qbar, O.bits_to_f64(Kb[:t + 1]), O.bits_to_f64(Vb[:t + 1]), g, w, scale)
+        pk, pv, n_rows = O.ring_to_packed(rk, rv, n_rep, n_tok, g, w)
+        assert n_rep == whole["m"] and n_rows == whole["m"] + whole["k"]
+        assert np.array_equal(pk, whole["cache_k_bits"]) and np.array_equal(pv, whole["cache_v_bits"])
+        if anchors is not None:
+            n_updates += 1
+            assert np.array_equal(anchors, whole["anchor"][-1] - (n_rep - 1) * g)     # offsets inside the newest group, per head
+    assert n_updates == (L0 + T - w) // g - start["m"] and n_updates >= 5
+
+
 def test_ablation_reducers_have_their_defining_properties():
     """Table 5 operators: the method's pair is the default; mean pooling is weighted pooling at a zero
     summary query; max selection returns a member of the group bit for bit; max pooling dominates every

@@ -962,3 +962,67 @@ def test_ring_cache_step_update_with_running_summary_query_matches_oracle(B):
             o_sem[b], o_pos[b], o_rep[b] = s2, p2, nr
         assert d_rep.cpu().tolist() == o_rep and qcount.cpu().tolist() == [len(x) for x in seen]
     assert n_updates >= 8
+
+
+def test_gqa_ring_cache_update_matches_oracle(B):
+    # GQA variant of the online update (pool V, select K, per KV head) on the ring layout: query tails, then the per-step
+    # form with the running summary query; three sequences in different phases, g + 3 steps.
+    cfg = I.scaled(I.CONFIGS["gqa_64k"], batch=3, seq_len=0, n_q_heads=16, n_kv_heads=4, group_size=16, window=48)
+    g, w, Hq, Hkv, d, Bsz = cfg.group_size, cfg.window, cfg.n_q_heads, cfg.n_kv_heads, cfg.d_sem, 3
+    R = w + g
+    steps = g + 3
+    cap = R + 8
+    gen = torch.Generator().manual_seed(43)
+    specs = [(2, w + g - 2), (4, w + 1), (0, w + g - 1)]
+    pv, pk, prow, prep = _ring_states(g, w, cap, specs, d, d, gen, heads=Hkv)
+    p = B.params_from_config(cfg, batch=Bsz)
+    scale = Hh.f32(cfg.softmax_scale)
+    for form in ("tails", "step"):
+        d_rep = torch.tensor(prep, dtype=torch.int32, device=DEV)
+        ring_v, ring_k, d_tok = B.ring_from_packed(p, pv.to(DEV), pk.to(DEV), torch.tensor(prow, dtype=torch.int32, device=DEV), d_rep, cap)
+        o_k = [Hh.bits(ring_k[b]) for b in range(Bsz)]
+        o_v = [Hh.bits(ring_v[b]) for b in range(Bsz)]
+        o_tok, o_rep = d_tok.cpu().tolist(), list(prep)
+        qsum = torch.zeros((Bsz, Hkv, d), dtype=torch.float64, device=DEV)
+        qcount = torch.zeros((Bsz,), dtype=torch.int32, device=DEV)
+        seen = [[] for _ in range(Bsz)]
+        n_updates = 0
+        for step in range(steps):
+            new_k = torch.randn((Bsz, Hkv, d), generator=gen).bfloat16()
+            new_v = torch.randn((Bsz, Hkv, d), generator=gen).bfloat16()
+            for b in range(Bsz):
+                ring_k[b, o_tok[b] % R] = new_k[b].to(DEV)
+                ring_v[b, o_tok[b] % R] = new_v[b].to(DEV)
+                o_k[b][o_tok[b] % R] = Hh.bits(new_k[b])
+                o_v[b][o_tok[b] % R] = Hh.bits(new_v[b])
+                o_tok[b] += 1
+            d_tok += 1
+            if form == "tails":
+                q_tail = torch.randn((Bsz, g, Hq, d), generator=gen).bfloat16()
+                anchor = B.decode_update_ring(p, None, q_tail.to(DEV), ring_v, ring_k, d_rep, d_tok)
+            else:
+                q_now = torch.randn((Bsz, Hq, d), generator=gen).bfloat16()
+                anchor = B.decode_step_update_ring(p, None, q_now.to(DEV), qsum, qcount, ring_v, ring_k, d_rep, d_tok)
+            torch.cuda.synchronize()
+            for b in range(Bsz):
+                if form == "tails":
+                    qbar = O.gqa_summary_query(O.torch_bf16_to_f64(q_tail[b]), Hkv)
+                else:
+                    seen[b].append(q_now[b])
+                    qbar = O.gqa_summary_query(O.torch_bf16_to_f64(torch.stack(seen[b])), Hkv)
+                k2, v2, nr, anc = O.gqa_decode_update_ring(o_k[b], o_v[b], o_rep[b], o_tok[b], qbar, g, w, scale)
+                if anc is None:
+                    assert (anchor[b].cpu().numpy() == -1).all()
+                else:
+                    n_updates += 1
+                    seen[b] = []
+                    assert np.array_equal(anchor[b].cpu().numpy(), anc)
+                    got_k, got_v = Hh.bits(ring_k[b]), Hh.bits(ring_v[b])
+                    row = R + o_rep[b]
+                    assert np.array_equal(got_k, k2)                                     # selected keys: bit copies, per head
+                    assert (Hh.bf16_ulp_distance(got_v[row], v2[row]) <= 1).all()        # pooled values: fp32 pooling
+                    v2[row] = got_v[row]
+                    assert np.array_equal(got_v, v2)
+                o_k[b], o_v[b], o_rep[b] = k2, v2, nr
+            assert d_rep.cpu().tolist() == o_rep
+        assert n_updates >= 3
