@@ -1026,3 +1026,38 @@ def test_gqa_ring_cache_update_matches_oracle(B):
                 o_k[b], o_v[b], o_rep[b] = k2, v2, nr
             assert d_rep.cpu().tolist() == o_rep
         assert n_updates >= 3
+
+
+def test_gqa_packed_cache_update_matches_oracle(B):
+    # lca_decode_update (packed layout, the window moves up) for the GQA variant: one call on three sequences, two of them
+    # due.  Expected state: the oracle's ring update read back in packed order (the two layouts hold the same rows).
+    cfg = I.scaled(I.CONFIGS["gqa_64k"], batch=3, seq_len=0, n_q_heads=16, n_kv_heads=4, group_size=16, window=48)
+    g, w, Hq, Hkv, d, Bsz = cfg.group_size, cfg.window, cfg.n_q_heads, cfg.n_kv_heads, cfg.d_sem, 3
+    R = w + g
+    gen = torch.Generator().manual_seed(47)
+    specs = [(2, R), (4, w + 5), (0, R)]
+    cap = R + 8
+    pv, pk, prow, prep = _ring_states(g, w, cap, specs, d, d, gen, heads=Hkv)
+    capacity = pv.shape[1]
+    p = B.params_from_config(cfg, batch=Bsz)
+    d_v, d_k = pv.to(DEV), pk.to(DEV)
+    d_rep = torch.tensor(prep, dtype=torch.int32, device=DEV)
+    d_rows = torch.tensor(prow, dtype=torch.int32, device=DEV)
+    q_tail = torch.randn((Bsz, g, Hq, d), generator=gen).bfloat16()
+    anchor = B.decode_update(p, None, q_tail.to(DEV), d_v, d_k, d_rep, d_rows)
+    torch.cuda.synchronize()
+    for b, (r, c) in enumerate(specs):
+        rk, rv, n_tok = O.ring_from_packed(Hh.bits(pk[b]), Hh.bits(pv[b]), r, r + c, g, w, cap)
+        qbar = O.gqa_summary_query(O.torch_bf16_to_f64(q_tail[b]), Hkv)
+        k2, v2, nr, anc = O.gqa_decode_update_ring(rk, rv, r, n_tok, qbar, g, w, Hh.f32(cfg.softmax_scale))
+        ek, ev, n_rows = O.ring_to_packed(k2, v2, nr, n_tok, g, w)
+        assert int(d_rep[b]) == nr and int(d_rows[b]) == n_rows and (anc is None) == (c < R)
+        got_k, got_v = Hh.bits(d_k[b, :n_rows]), Hh.bits(d_v[b, :n_rows])
+        if anc is None:
+            assert (anchor[b].cpu().numpy() == -1).all()
+        else:
+            assert np.array_equal(anchor[b].cpu().numpy(), anc)
+            assert (Hh.bf16_ulp_distance(got_v[nr - 1], ev[nr - 1]) <= 1).all()
+            ev[nr - 1] = got_v[nr - 1]
+        assert np.array_equal(got_k, ek) and np.array_equal(got_v, ev)
+    assert capacity >= max(prow)
