@@ -1061,3 +1061,44 @@ def test_gqa_packed_cache_update_matches_oracle(B):
             ev[nr - 1] = got_v[nr - 1]
         assert np.array_equal(got_k, ek) and np.array_equal(got_v, ev)
     assert capacity >= max(prow)
+
+
+@pytest.mark.parametrize("kind", ["mla_dc128", "gqa_d64"])
+def test_smaller_head_shapes_on_the_scalar_kernel_match_oracle(B, kind):
+    # Shapes without a tensor-core kernel (MLA with a 128-wide latent, GQA with 64-wide heads): generic condensation
+    # kernel and the scalar attention kernel; prefill on every row, decode over the packed cache and over the ring layout.
+    g, w, L = 16, 48, 333
+    if kind == "mla_dc128":
+        cfg = I.scaled(I.CONFIGS["mla_1k"], seq_len=L, n_q_heads=6, group_size=g, window=w, d_sem=128, n_needles=2)
+        inp = I.make_mla_inputs(cfg, "cpu")
+        d = to_dev(inp)
+        p = B.params_from_config(cfg, batch=1, rep_logit_bias=0.4)
+        cond = B.condense(p, d["q_sem"][L - g:], d["q_pos"][L - g:], d["ckv"], d["kr"])
+        out, lse = B.prefill_attention(p, d["q_sem"], d["q_pos"], d["ckv"], d["kr"], cond["cache_sem"], cond["cache_pos"], want_lse=True)
+        ref = Hh.oracle_mla(inp, g, w, cfg.softmax_scale, rows=np.arange(L), rep_logit_bias=0.4)
+        q_last = (d["q_sem"][L - 1].contiguous()[None], d["q_pos"][L - 1].contiguous()[None])
+        ckind = "mla"
+    else:
+        cfg = I.scaled(I.CONFIGS["gqa_64k"], seq_len=L, n_q_heads=6, n_kv_heads=3, group_size=g, window=w, d_sem=64, n_needles=2)
+        inp = I.make_gqa_inputs(cfg, "cpu")
+        d = to_dev(inp)
+        p = B.params_from_config(cfg, batch=1, rep_logit_bias=0.4)
+        cond = B.condense(p, None, d["q"][L - g:], d["v"], d["k"])
+        out, lse = B.prefill_attention(p, None, d["q"], d["v"], d["k"], cond["cache_sem"], cond["cache_pos"], want_lse=True)
+        ref = Hh.oracle_gqa(inp, g, w, cfg.softmax_scale, rows=np.arange(L), rep_logit_bias=0.4)
+        q_last = (None, d["q"][L - 1].contiguous()[None])
+        ckind = "gqa"
+    torch.cuda.synchronize()
+    Hh.check_condense(one_seq(cond), ref["cond"], kind=ckind)
+    Hh.check_outputs(out[0], ref, kind)
+    np.testing.assert_allclose(lse[0].cpu().numpy(), ref["lse"], atol=2e-3, rtol=1e-4)
+    m, k = cond["m"], cond["k"]
+    rows = torch.tensor([m + k], dtype=torch.int32, device=DEV)
+    dout, _ = B.decode_attention(p, q_last[0], q_last[1], cond["cache_sem"], cond["cache_pos"], rows, m)
+    Hh.check_outputs(dout[0], ref["out"][-1], kind + " decode", vmax=ref["vmax"])
+    n_rep = torch.tensor([m], dtype=torch.int32, device=DEV)
+    ring_sem, ring_pos, n_tok = B.ring_from_packed(p, cond["cache_sem"], cond["cache_pos"], rows, n_rep, w + g + m + 2)
+    assert int(n_tok[0]) == L
+    rout, _ = B.decode_attention_ring(p, q_last[0], q_last[1], ring_sem, ring_pos, n_rep, n_tok)
+    torch.cuda.synchronize()
+    Hh.check_outputs(rout[0], ref["out"][-1], kind + " ring decode", vmax=ref["vmax"])
