@@ -178,6 +178,13 @@ def gather_oracle_inputs(cfg, inp, n_rows, seed=0):
     """CPU copies of what the oracle sample needs (the K/V streams and the sampled query rows)."""
     L, g = cfg.seq_len, cfg.group_size
     rows = sample_rows(cfg, n_rows, seed)
+    if inp is None:
+        # no GPU and queries too large for host memory (timing only, nothing is compared): the keys / values of the whole
+        # sequence, the query tail, and as many further query rows as are sampled, drawn for the positions before the tail
+        n = len(rows)
+        part = I.make_mla_inputs(cfg, "cpu", q_positions=slice(L - g - n, L))
+        return dict(ckv=part["ckv"], kr=part["kr"], q_sem=part["q_sem"][n:], q_pos=part["q_pos"][n:],
+                    q_sem_rows=part["q_sem"][:n], q_pos_rows=part["q_pos"][:n])
     idx = torch.from_numpy(rows).to(inp["q_sem"].device)
     return dict(ckv=inp["ckv"].cpu(), kr=inp["kr"].cpu(), q_sem=inp["q_sem"][L - g:].cpu(), q_pos=inp["q_pos"][L - g:].cpu(),
                 q_sem_rows=inp["q_sem"][idx].cpu(), q_pos_rows=inp["q_pos"][idx].cpu())
