@@ -51,8 +51,9 @@ latent_to_value_kernel(const __grid_constant__ UvParams p) {
   volatile uint32_t* tmem_slot = reinterpret_cast<volatile uint32_t*>(base_ptr + OFF_MISC);
   volatile int* abort_flag = reinterpret_cast<volatile int*>(base_ptr + OFF_MISC + 4);
   const int warp = __shfl_sync(0xffffffffu, (int)(threadIdx.x >> 5), 0), lane = threadIdx.x & 31;
-  const int h = blockIdx.y;
-  const long long t0 = (long long)blockIdx.x * BM;
+  // heads vary fastest over the grid: CTAs that run at the same time read neighbouring 1 KB pieces of the same token rows
+  const int h = (int)(blockIdx.x % (unsigned)p.H);
+  const long long t0 = (long long)(blockIdx.x / (unsigned)p.H) * BM;
 
   if (threadIdx.x == 0) {
     for (int s = 0; s < STAGES; ++s) { mbar_init(BAR_FULL(s), 1); mbar_init(BAR_EMPTY(s), 1); }
@@ -161,7 +162,9 @@ int latent_to_value_launch(const void* latent, const void* w_uv, void* out, long
   if (!ok) return LCA_ERR_CUDA;
   if (cudaFuncSetAttribute(latent_to_value_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM_BYTES) != cudaSuccess)
     return LCA_ERR_CUDA;
-  dim3 grid((unsigned)((n_tokens + BM - 1) / BM), n_heads);
+  const long long n_ctas = ((n_tokens + BM - 1) / BM) * n_heads;
+  if (n_ctas > 0x7fffffffll) return LCA_ERR_UNSUPPORTED_SHAPE;
+  dim3 grid((unsigned)n_ctas);
   latent_to_value_kernel<<<grid, THREADS, SMEM_BYTES, stream>>>(p);
   note_launch();
   return cudaGetLastError() == cudaSuccess ? LCA_OK : LCA_ERR_CUDA;
