@@ -151,8 +151,10 @@ struct CondenseArgs {
   SeqTab tab;                  // ragged batch: L, m and cache_rows above are unused
 };
 
-// Where group `grp` of the launch lives: uniform batch grp = (b * Hkv + hk) * m + j; ragged batch: the groups of
-// sequence b are grp_off[b] * Hkv + hk * m_b + j.
+// Where group `grp` of the launch lives: the KV head varies fastest, grp = (b * m + j) * Hkv + hk (ragged batch: the groups
+// of sequence b start at grp_off[b] * Hkv), so that the CTAs of a persistent launch, which work on consecutive groups at any
+// one time, read all heads of the same token rows together (a token row holds the Hkv heads side by side; one head at a
+// time would touch an eighth of every DRAM page with Hkv = 8) and grp % Hkv is the head.
 struct GroupLoc { int b, hk, j; long long tok0, out_row, grp_row; };     // first token row, cache row, row of anchor_idx
 __device__ inline GroupLoc locate_group(const CondenseArgs& a, long long grp) {
   GroupLoc l;
@@ -165,14 +167,15 @@ __device__ inline GroupLoc locate_group(const CondenseArgs& a, long long grp) {
     l.b = lo;
     const int m_b = a.tab.grp_off[lo + 1] - a.tab.grp_off[lo];
     const long long local = grp - (long long)a.tab.grp_off[lo] * a.Hkv;
-    l.hk = (int)(local / m_b); l.j = (int)(local % m_b);
+    l.hk = (int)(local % a.Hkv); l.j = (int)(local / a.Hkv);
+    (void)m_b;
     l.tok0 = (long long)a.tab.tok_off[lo] + (long long)l.j * a.g;
     l.out_row = (long long)a.tab.cache_off[lo] + l.j;
     l.grp_row = (long long)a.tab.grp_off[lo] + l.j;
   } else {
-    l.j = (int)(grp % a.m);
-    const long long bh = grp / a.m;
-    l.hk = (int)(bh % a.Hkv); l.b = (int)(bh / a.Hkv);
+    l.hk = (int)(grp % a.Hkv);
+    const long long bj = grp / a.Hkv;
+    l.j = (int)(bj % a.m); l.b = (int)(bj / a.m);
     l.tok0 = (long long)l.b * a.L + (long long)l.j * a.g;
     l.out_row = (long long)l.b * a.cache_rows + l.j;
     l.grp_row = (long long)l.b * a.m + l.j;
@@ -1021,7 +1024,9 @@ int condense_launch(const CondenseLaunch& c) {
         return LCA_ERR_CUDA;
       if (cudaFuncSetAttribute(condense_gqa64_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, gfast::SMEM_BYTES) != cudaSuccess)
         return LCA_ERR_CUDA;
-      condense_gqa64_kernel<<<dim3((unsigned)ctas), gfast::THREADS, gfast::SMEM_BYTES, c.stream>>>(a, maps);
+      // a grid that is a multiple of the KV heads: every CTA then stays with one head (its summary query stays in registers)
+      const long long ctas_h = ctas >= Hkv ? ctas / Hkv * Hkv : ctas;
+      condense_gqa64_kernel<<<dim3((unsigned)ctas_h), gfast::THREADS, gfast::SMEM_BYTES, c.stream>>>(a, maps);
     } else {
       size_t smem = condense_smem_bytes(p);
       if (cudaFuncSetAttribute(condense_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) != cudaSuccess)
