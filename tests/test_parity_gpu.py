@@ -1102,3 +1102,70 @@ def test_smaller_head_shapes_on_the_scalar_kernel_match_oracle(B, kind):
     rout, _ = B.decode_attention_ring(p, q_last[0], q_last[1], ring_sem, ring_pos, n_rep, n_tok)
     torch.cuda.synchronize()
     Hh.check_outputs(rout[0], ref["out"][-1], kind + " ring decode", vmax=ref["vmax"])
+
+
+def test_prefill_then_ring_decode_loop_end_to_end(B):
+    # The calls composed as a serving loop would use them (MLA shape, tensor-core kernels): condense + prefill of a prompt,
+    # the packed cache moved into the ring layout, then decode steps of [append the token, attend, per-step update with the
+    # running summary query].  The running sum is primed with the prompt's queries after its last group boundary, so every
+    # update uses the last g queries.  Each step against the oracle's streaming state.
+    cfg = I.scaled(I.CONFIGS["mla_1k"], seq_len=700, n_q_heads=16, group_size=16, window=48, n_needles=3)
+    L, g, w, H = cfg.seq_len, cfg.group_size, cfg.window, cfg.n_q_heads
+    R = w + g
+    steps = 2 * g + 3
+    inp = I.make_mla_inputs(cfg, "cpu")
+    d = to_dev(inp)
+    p = B.params_from_config(cfg, batch=1)
+    scale = Hh.f32(cfg.softmax_scale)
+    cond = B.condense(p, d["q_sem"][L - g:], d["q_pos"][L - g:], d["ckv"], d["kr"])
+    out, _ = B.prefill_attention(p, d["q_sem"], d["q_pos"], d["ckv"], d["kr"], cond["cache_sem"], cond["cache_pos"])
+    ref = Hh.oracle_mla(inp, g, w, cfg.softmax_scale, rows=np.array([L - 1]))
+    Hh.check_condense(one_seq(cond), ref["cond"])
+    Hh.check_outputs(out[0, L - 1:], ref, "last prefill row")
+    m, k = cond["m"], cond["k"]
+    n_rep = torch.tensor([m], dtype=torch.int32, device=DEV)
+    cap = R + m + steps // g + 2
+    ring_sem, ring_pos, n_tok = B.ring_from_packed(p, cond["cache_sem"], cond["cache_pos"],
+                                                   torch.tensor([m + k], dtype=torch.int32, device=DEV), n_rep, cap)
+    o_sem, o_pos, o_tok = O.ring_from_packed(ref["cond"]["cache_sem_bits"], ref["cond"]["cache_pos_bits"], m, m + k, g, w, cap)
+    got = Hh.bits(ring_sem[0, :, 0])
+    assert (Hh.bf16_ulp_distance(got[R:R + m], o_sem[R:R + m]) <= 1).all()          # representatives: fp32 pooling on the device
+    o_sem[R:R + m] = got[R:R + m]
+    assert np.array_equal(got, o_sem) and np.array_equal(Hh.bits(ring_pos[0, :, 0]), o_pos) and int(n_tok[0]) == o_tok == L
+    # prime the running sum with the queries of the tokens behind the last group boundary (k - w of them)
+    qsum = torch.zeros((1, 1, 576), dtype=torch.float64, device=DEV)
+    qcount = torch.zeros((1,), dtype=torch.int32, device=DEV)
+    seen = []
+    for t in range(L - (k - w), L):
+        B.decode_step_update_ring(p, d["q_sem"][t][None].contiguous(), d["q_pos"][t][None].contiguous(), qsum, qcount,
+                                  ring_sem, ring_pos, n_rep, n_tok)
+        seen.append((inp["q_sem"][t], inp["q_pos"][t]))
+    assert int(qcount[0]) == k - w and int(n_rep[0]) == m
+    o_rep, gen, n_updates = m, torch.Generator().manual_seed(53), 0
+    for step in range(steps):
+        new_sem, new_pos = torch.randn((512,), generator=gen).bfloat16(), torch.randn((64,), generator=gen).bfloat16()
+        q_sem, q_pos = torch.randn((1, H, 512), generator=gen).bfloat16(), torch.randn((1, H, 64), generator=gen).bfloat16()
+        ring_sem[0, o_tok % R, 0], ring_pos[0, o_tok % R, 0] = new_sem.to(DEV), new_pos.to(DEV)
+        o_sem[o_tok % R], o_pos[o_tok % R] = Hh.bits(new_sem), Hh.bits(new_pos)
+        o_tok += 1
+        n_tok += 1
+        dout, _ = B.decode_attention_ring(p, q_sem.to(DEV), q_pos.to(DEV), ring_sem, ring_pos, n_rep, n_tok)
+        cs, cp, _ = O.ring_to_packed(o_sem, o_pos, o_rep, o_tok, g, w)
+        ro, _ = O.mla_decode(O.torch_bf16_to_f64(q_sem[0]), O.torch_bf16_to_f64(q_pos[0]), O.bits_to_f64(cs), O.bits_to_f64(cp), o_rep, scale)
+        Hh.check_outputs(dout[0], ro, f"decode step {step}")
+        anchor = B.decode_step_update_ring(p, q_sem.to(DEV), q_pos.to(DEV), qsum, qcount, ring_sem, ring_pos, n_rep, n_tok)
+        torch.cuda.synchronize()
+        seen.append((q_sem[0], q_pos[0]))
+        qbar = O.mla_summary_query(O.torch_bf16_to_f64(torch.stack([a for a, _ in seen])), O.torch_bf16_to_f64(torch.stack([c for _, c in seen])))
+        s2, p2, nr, ia = O.mla_decode_update_ring(o_sem, o_pos, o_rep, o_tok, qbar, g, w, scale)
+        assert int(anchor[0, 0]) == ia
+        if ia >= 0:
+            assert len(seen) == g                                      # the last g queries
+            n_updates, seen = n_updates + 1, []
+            got = Hh.bits(ring_sem[0, :, 0])
+            assert (Hh.bf16_ulp_distance(got[R + o_rep], s2[R + o_rep]) <= 1).all()
+            s2[R + o_rep] = got[R + o_rep]
+            assert np.array_equal(got, s2) and np.array_equal(Hh.bits(ring_pos[0, :, 0]), p2)
+        o_sem, o_pos, o_rep = s2, p2, nr
+        assert int(n_rep[0]) == o_rep
+    assert n_updates >= 2 and B.lca_last_device_status() == 0
