@@ -620,7 +620,7 @@ condense_mla64_kernel(CondenseArgs a) {
       unsigned long long acc01 = f32x2(0.f, 0.f), acc23 = f32x2(0.f, 0.f);
       const uint2* col = reinterpret_cast<const uint2*>(t_sem) + pt;
       const float* al_base = s_a + p * G;
-#pragma unroll 2
+#pragma unroll 4                                           // sixteen tokens' loads in flight: the one pooling warp of a scheduler waits for shared memory otherwise
       for (int i = 0; i < G; i += 4) {
         const float4 al = *reinterpret_cast<const float4*>(al_base + i);
         const float alv[4] = {al.x, al.y, al.z, al.w};
